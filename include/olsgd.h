@@ -1,0 +1,189 @@
+/*
+ * olsgd.h -- C ABI of the Overlap-Local-SGD hot path for m simulated workers
+ * stacked on one GPU (Wang, Liang, Joshi, "Overlap Local-SGD", arXiv
+ * 2002.09539, Section 2 "Proposed Algorithm").
+ *
+ * One context holds the m worker models x^(1..m), their local momentum
+ * buffers, the anchor z and the anchor momentum buffer v, all resident in
+ * device memory that the CALLER allocates and hands over as one workspace.
+ * The library owns host memory and CUDA events only.  It never allocates
+ * device memory, never throws, never aborts: every call returns a status and
+ * `olsgd_last_error` gives the reason as text.
+ *
+ * Conventions
+ *   - "device pointer": memory on the current CUDA device, 16-byte aligned.
+ *   - Flat parameter layout: for each layer in order, the weight matrix
+ *     W_l row-major as [out][in] followed by its bias b_l [out]; linear
+ *     regression is one weight vector w [d] without bias.
+ *   - Iterations k are 0-based.  Iteration k is a "sync step" when
+ *     (k + 1) mod tau == 0.
+ *   - Calls are asynchronous with respect to the host unless stated.  All
+ *     calls on one context must come from one host thread at a time.
+ */
+#ifndef OLSGD_H
+#define OLSGD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct olsgd_ctx olsgd_ctx; /* opaque, host side */
+
+typedef enum {
+  OLSGD_OK = 0,
+  OLSGD_EINVAL = 1,   /* bad argument; nothing was changed                */
+  OLSGD_ESTATE = 2,   /* call out of order; nothing was changed           */
+  OLSGD_ENOMEM = 3,   /* workspace too small / host allocation failed     */
+  OLSGD_ECUDA = 4,    /* a CUDA runtime or driver call failed             */
+  OLSGD_ETIMEOUT = 5  /* a bounded device-side wait gave up               */
+} olsgd_status;
+
+typedef enum {
+  OLSGD_LINREG = 0,   /* loss (1/2B) sum (x_s . w - y_s)^2, dims = {d}             */
+  OLSGD_SOFTMAX = 1,  /* softmax regression, dims = {d_in, n_classes}              */
+  OLSGD_MLP = 2,      /* ReLU MLP + mean cross-entropy, dims = {d_in, h.., classes} */
+  OLSGD_FLAT = 3      /* flat parameter vector, gradients supplied by the caller   */
+} olsgd_model;
+
+#define OLSGD_MAX_DIMS 8
+
+typedef struct {
+  int32_t kind;                 /* olsgd_model                                        */
+  int32_t n_dims;               /* entries used in dims (1 for LINREG, 0 for FLAT)    */
+  int32_t dims[OLSGD_MAX_DIMS]; /* e.g. {3072, 1024, 1024, 10}                        */
+  int32_t gemm_bf16;            /* MLP only: 1 = bf16 operands on the tensor cores,
+                                   fp32 accumulate, fp32 master weights; 0 = fp32    */
+  int32_t reserved;
+  int64_t flat_P;               /* FLAT only: number of parameters                    */
+} olsgd_model_spec;
+
+/* The paper's symbols (Section 2): m workers, tau local steps per period,
+ * gamma learning rate (Eq. 3), alpha pull-back rate (Eq. 4), beta anchor
+ * momentum factor (Eq. 10).  mu is the factor of the "common Nesterov
+ * momentum" of the local step (u <- mu u + g, x <- x - gamma (g + mu u));
+ * mu = 0 is plain SGD, beta = 0 is the vanilla anchor refresh of Eq. 5.     */
+typedef struct {
+  int32_t m, tau, batch, reserved;
+  float gamma, alpha, beta, mu;
+  uint64_t seed;                /* seeds the minibatch index rule                    */
+} olsgd_hparams;
+
+/* Worker i's data set D_i (Eq. 1).  Device pointers, borrowed for the life of
+ * the context, never written, never freed.
+ *   X  float32 [m][n_per_worker][dims[0]]
+ *   y  float32 [m][n_per_worker]  (LINREG targets)  or
+ *      int32   [m][n_per_worker]  (class labels in [0, dims[last]))         */
+typedef struct {
+  const void* X;
+  const void* y;
+  int64_t n_per_worker;
+} olsgd_data;
+
+/* Number of parameters P of one model copy in the flat layout.              */
+olsgd_status olsgd_param_count(const olsgd_model_spec* spec, int64_t* out_P);
+
+/* Bytes of device workspace `olsgd_init` needs for this model and these
+ * hyper-parameters (state, gradients, batch staging, activations).          */
+olsgd_status olsgd_workspace_bytes(const olsgd_model_spec* spec, const olsgd_hparams* hp,
+                                   size_t* out_bytes);
+
+/* Create a context.  Sets x_0^(i) = z_0 = x0 for every worker (the initial
+ * condition of Theorem 1), zeroes the momentum buffers u_i and v, k = 0.
+ *   x0_device        P floats, device; copied, not kept
+ *   workspace_device at least olsgd_workspace_bytes bytes, 256-byte aligned;
+ *                    owned by the caller, must outlive the context
+ *   main_stream      cudaStream_t on which the local steps run
+ *   side_stream      cudaStream_t on which the anchor refresh runs; may equal
+ *                    main_stream (then nothing overlaps)
+ *   data             may be NULL for OLSGD_FLAT
+ * Checks: m, tau, batch >= 1; gamma > 0; 0 <= alpha <= 1; 0 <= beta < 1;
+ * 0 <= mu < 1; pointers non-null and aligned.  On error *out is NULL.       */
+olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const olsgd_hparams* hp,
+                        const olsgd_data* data, const float* x0_device, void* workspace_device,
+                        size_t workspace_bytes, void* main_stream, void* side_stream);
+
+/* One iteration k -> k+1 for all m workers on the main stream: draw the
+ * minibatches xi_k^(i), evaluate g_i(x_k^(i); xi_k^(i)), apply Eq. 3 (with
+ * the local Nesterov buffer when mu > 0) and, on a sync step, Eq. 4 against
+ * the anchor produced by the previous period (the one-period lag stated after
+ * Eq. 5), all on the device.
+ *   loss_device  m floats, device: mean minibatch loss per worker at x_k; or NULL
+ * Returns OLSGD_ESTATE if a period ended and olsgd_period_sync has not been
+ * called since.                                                             */
+olsgd_status olsgd_local_step(olsgd_ctx* ctx, float* loss_device);
+
+/* Same iteration for OLSGD_FLAT: the stacked gradients G_k (Eq. 7 without its
+ * zero column) come from the caller.
+ *   g_device  float32 [m][P], device, row stride P; read on the main stream */
+olsgd_status olsgd_local_step_with_grads(olsgd_ctx* ctx, const float* g_device);
+
+/* Anchor refresh at the end of a period: Eq. 5 (beta = 0) or Eq. 10-11, as a
+ * reduction over the worker dimension launched on the side stream after the
+ * pull-back that closed the period.  Returns at once; the next period's local
+ * steps overlap with it and its result is first read by the next pull-back.
+ * Legal exactly once per period, when k > 0 and k mod tau == 0; otherwise
+ * OLSGD_ESTATE.                                                             */
+olsgd_status olsgd_period_sync(olsgd_ctx* ctx);
+
+/* n_iters iterations in one call: olsgd_local_step, followed by
+ * olsgd_period_sync whenever a period ends.  Not for OLSGD_FLAT.
+ *   loss_device  n_iters * m floats ([iteration][worker]), device; or NULL  */
+olsgd_status olsgd_run(olsgd_ctx* ctx, int64_t n_iters, float* loss_device);
+
+/* Copy one vector of the state to the caller.  Joins both streams (blocks
+ * the host).  which: 0..m-1 worker model x^(i); -1 anchor z; -2 anchor
+ * momentum v; -3 virtual sequence y = (1-alpha) mean_i x^(i) + alpha z
+ * (Appendix A); -4 mean model mean_i x^(i); -5 - i local momentum u_i.
+ *   dst       host or device memory
+ *   n_floats  must equal P                                                   */
+olsgd_status olsgd_get_params(olsgd_ctx* ctx, int32_t which, float* dst, size_t n_floats);
+
+/* The minibatch indices xi_k^(i) that iteration k uses (or used): slot j of
+ * worker i is floor(w * n / 2^32) with w word (j mod 4) of the Philox4x32-10
+ * block (Salmon et al., SC'11) of counter (j div 4, k, i, 1) and key
+ * (seed mod 2^32, seed div 2^32).  Computed on the device; blocks the host.
+ *   dst  int32 [m][batch], host or device                                   */
+olsgd_status olsgd_get_indices(olsgd_ctx* ctx, int64_t k, int32_t* dst);
+
+/* Non-IID partition table: the two classes (of ten) each worker samples
+ * from.  Class slots are concatenated seeded Fisher-Yates permutations of
+ * 0..9 (permutation t, position p from 9 down to 1, swaps with
+ * floor(w (p+1) / 2^32), w = word 0 of the Philox block of counter
+ * (p, t, 0, 2)); worker i takes slots 2i and 2i+1.  Stand-in for the skewed
+ * partitions of the paper's non-IID experiment (Section 4).  Computed on the
+ * device on `stream`; blocks the host.
+ *   dst  int32 [m][2], host or device                                       */
+olsgd_status olsgd_class_pairs(uint64_t seed, int32_t m, int32_t* dst, void* stream);
+
+/* Iteration counter k.                                                      */
+int64_t olsgd_iteration(const olsgd_ctx* ctx);
+
+/* Number of kernels this context has launched so far.                       */
+int64_t olsgd_launch_count(const olsgd_ctx* ctx);
+
+/* Device-time profile of the kernel classes.  When enabled, every launch is
+ * bracketed by CUDA events on its own stream.  olsgd_profile_read joins both
+ * streams and returns, per class c in 0..OLSGD_N_KERNEL_CLASSES-1, the launch
+ * count and the summed duration in milliseconds since the last reset.       */
+#define OLSGD_N_KERNEL_CLASSES 8
+enum { OLSGD_KC_INDEX = 0, OLSGD_KC_GATHER = 1, OLSGD_KC_FORWARD = 2, OLSGD_KC_BACKWARD = 3,
+       OLSGD_KC_UPDATE = 4, OLSGD_KC_ANCHOR = 5, OLSGD_KC_LOSS = 6, OLSGD_KC_OTHER = 7 };
+olsgd_status olsgd_profile_enable(olsgd_ctx* ctx, int32_t on);
+olsgd_status olsgd_profile_read(olsgd_ctx* ctx, int64_t* launches, double* millis, int32_t reset);
+
+/* Text of the last error on this context ("" if none).  ctx may be NULL, in
+ * which case the last error of a failed olsgd_init / context-free call in this
+ * thread is returned.                                                       */
+const char* olsgd_last_error(const olsgd_ctx* ctx);
+
+/* Join both streams, destroy events, free host memory.  Device memory stays
+ * with the caller.                                                          */
+olsgd_status olsgd_destroy(olsgd_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OLSGD_H */

@@ -1,0 +1,279 @@
+// Forward/backward orchestration of the model families: which kernels run, in
+// which order, on which staging buffers.  Host code only.
+#include <cstdio>
+#include <cstring>
+
+#include "olsgd_internal.h"
+
+namespace olsgd {
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Scope {
+  const ProfHook& h;
+  void* handle;
+  Scope(const ProfHook& hook, int cls, cudaStream_t s) : h(hook), handle(hook.begin(hook.ctx, cls, s)) {}
+  ~Scope() { if (handle) h.end(handle); }
+};
+
+#define OLSGD_TRY(call)                    \
+  do {                                     \
+    cudaError_t e_ = (call);               \
+    if (e_ != cudaSuccess) return e_;      \
+  } while (0)
+
+inline int n_layers(const olsgd_model_spec& s) { return s.n_dims - 1; }
+
+// gemm_bf16: 0 = fp32 CUDA cores, 1 = tcgen05 tensor cores, 2 = the same bf16
+// data flow on CUDA cores (validation of the tensor-core kernels)
+inline bool bf16_path(const olsgd_model_spec& s) { return s.kind == OLSGD_MLP && s.gemm_bf16 != 0; }
+
+cudaError_t run_gemm(const olsgd_model_spec& spec, const GemmArgs& ga, cudaStream_t s) {
+  if (spec.gemm_bf16 == 1) return launch_gemm_tc(ga, s);
+  return launch_gemm_simt(ga, s);
+}
+
+}  // namespace
+
+bool plan_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, ModelPlan* mp) {
+  const size_t m = hp.m, B = hp.batch;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, 256);
+    return o;
+  };
+  mp->off_loss = take(m * sizeof(float));
+  if (spec.kind == OLSGD_LINREG) {
+    mp->bytes = off;
+    return true;
+  }
+  const int L = n_layers(spec);
+  const size_t d0 = spec.dims[0], C = spec.dims[L];
+  mp->off_yb = take(m * B * sizeof(int32_t));
+  mp->off_dlogits = take(m * B * C * sizeof(float));
+  mp->off_rowloss = take(m * B * sizeof(float));
+  if (!bf16_path(spec)) {
+    if (L != 1) {
+      snprintf(mp->error, sizeof mp->error,
+               "hidden layers need gemm_bf16 = 1 (tensor cores) or 2 (CUDA-core check)");
+      return false;
+    }
+    mp->off_xb32 = take(m * B * d0 * sizeof(float));
+    mp->bytes = off;
+    return true;
+  }
+  if (L < 2) {
+    snprintf(mp->error, sizeof mp->error, "gemm_bf16 needs at least one hidden layer");
+    return false;
+  }
+  if (B % 8 != 0) {
+    snprintf(mp->error, sizeof mp->error, "the bf16 path needs batch %% 8 == 0");
+    return false;
+  }
+  for (int l = 0; l < L; ++l) {
+    // every hidden width is a GEMM M dimension, every layer input a GEMM K
+    if (l < L - 1 && spec.dims[l + 1] % 128 != 0) {
+      snprintf(mp->error, sizeof mp->error, "hidden width dims[%d] must be a multiple of 128", l + 1);
+      return false;
+    }
+    if (l < L - 1 && spec.dims[l] % 64 != 0) {
+      snprintf(mp->error, sizeof mp->error, "dims[%d] must be a multiple of 64", l);
+      return false;
+    }
+  }
+  if (spec.gemm_bf16 == 1 && (B % 64 != 0 || B > 256)) {
+    snprintf(mp->error, sizeof mp->error, "the tensor-core path needs batch in {64, 128, 192, 256}");
+    return false;
+  }
+  const size_t e = sizeof(__nv_bfloat16);
+  mp->off_xb16 = take(m * B * d0 * e);
+  mp->off_xb16t = take(m * B * d0 * e);
+  for (int l = 1; l < L; ++l) {
+    const size_t w = spec.dims[l];
+    mp->off_h[l] = take(m * B * w * e);
+    mp->off_ht[l] = take(m * B * w * e);
+    mp->off_da[l] = take(m * B * w * e);
+    mp->off_dat[l] = take(m * B * w * e);
+  }
+  for (int l = 1; l < L - 1; ++l)  // layers whose input gradient is a GEMM
+    mp->off_wt[l] = take(m * (size_t)spec.dims[l + 1] * spec.dims[l] * e);
+  mp->bytes = off;
+  return true;
+}
+
+bool bind_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, const ModelPlan& mp,
+                char* base, ModelBuffers* mb) {
+  (void)hp;
+  mb->loss = reinterpret_cast<float*>(base + mp.off_loss);
+  if (spec.kind == OLSGD_LINREG) return true;
+  const int L = n_layers(spec);
+  int64_t off = 0;
+  for (int l = 0; l < L; ++l) {
+    mb->w_off[l] = off;
+    off += (int64_t)spec.dims[l + 1] * spec.dims[l];
+    mb->b_off[l] = off;
+    off += spec.dims[l + 1];
+  }
+  mb->yb = reinterpret_cast<int32_t*>(base + mp.off_yb);
+  mb->dlogits = reinterpret_cast<float*>(base + mp.off_dlogits);
+  mb->rowloss = reinterpret_cast<float*>(base + mp.off_rowloss);
+  if (!bf16_path(spec)) {
+    mb->xb32 = reinterpret_cast<float*>(base + mp.off_xb32);
+    return true;
+  }
+  auto bp = [&](size_t o) { return reinterpret_cast<__nv_bfloat16*>(base + o); };
+  mb->xb16 = bp(mp.off_xb16);
+  mb->xb16t = bp(mp.off_xb16t);
+  for (int l = 1; l < L; ++l) {
+    mb->h[l] = bp(mp.off_h[l]);
+    mb->ht[l] = bp(mp.off_ht[l]);
+    mb->da[l] = bp(mp.off_da[l]);
+    mb->dat[l] = bp(mp.off_dat[l]);
+  }
+  for (int l = 1; l < L - 1; ++l) mb->wt[l] = bp(mp.off_wt[l]);
+  return true;
+}
+
+cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hparams& hp,
+                                   const olsgd_data& data, const ModelBuffers& mb,
+                                   const StepIO& io, cudaStream_t s, const ProfHook& hook) {
+  const int m = hp.m, B = hp.batch;
+  const int64_t n = data.n_per_worker;
+  float* loss = io.loss ? io.loss : mb.loss;
+  const float* X = static_cast<const float*>(data.X);
+
+  if (spec.kind == OLSGD_LINREG) {
+    Scope sc(hook, OLSGD_KC_FORWARD, s);
+    return launch_linreg(X, static_cast<const float*>(data.y), io.idx, io.x, io.g, loss, m, B, n,
+                         spec.dims[0], io.ld, s);
+  }
+
+  const int L = n_layers(spec);
+  const int d0 = spec.dims[0], C = spec.dims[L];
+  const bool bf = bf16_path(spec);
+  {
+    Scope sc(hook, OLSGD_KC_GATHER, s);
+    OLSGD_TRY(launch_gather(X, static_cast<const int32_t*>(data.y), io.idx, bf ? nullptr : mb.xb32,
+                            bf ? mb.xb16 : nullptr, bf ? mb.xb16t : nullptr, mb.yb, m, B, n, d0,
+                            s));
+  }
+
+  // hidden layers, forward: H_l^T [d_l][B] = relu(W_l [d_l][d_{l-1}] * H_{l-1} [B][d_{l-1}]^T + b)
+  for (int l = 1; l < L; ++l) {
+    GemmArgs ga{};
+    ga.A = io.shadow + mb.w_off[l - 1];
+    ga.lda = spec.dims[l - 1];
+    ga.a_batch = io.ld;
+    ga.B = (l == 1) ? mb.xb16 : mb.h[l - 1];
+    ga.ldb = spec.dims[l - 1];
+    ga.b_batch = (int64_t)B * spec.dims[l - 1];
+    ga.m = m;
+    ga.Ma = spec.dims[l];
+    ga.Nb = B;
+    ga.K = spec.dims[l - 1];
+    ga.epilogue = GEMM_EPI_BIAS_RELU;
+    ga.bias = io.x + mb.b_off[l - 1];
+    ga.bias_batch = io.ld;
+    ga.out_t = mb.ht[l];
+    ga.out_n = mb.h[l];
+    Scope sc(hook, OLSGD_KC_FORWARD, s);
+    OLSGD_TRY(run_gemm(spec, ga, s));
+  }
+
+  // output layer: forward, loss, and backward to its input
+  HeadArgs ha{};
+  ha.in32 = bf ? nullptr : mb.xb32;
+  ha.in16 = bf ? mb.h[L - 1] : nullptr;
+  ha.x = io.x;
+  ha.ld = io.ld;
+  ha.w_off = mb.w_off[L - 1];
+  ha.b_off = mb.b_off[L - 1];
+  ha.yb = mb.yb;
+  ha.dlogits = mb.dlogits;
+  ha.rowloss = mb.rowloss;
+  ha.din32 = nullptr;
+  ha.din16 = bf ? mb.da[L - 1] : nullptr;
+  ha.din16t = bf ? mb.dat[L - 1] : nullptr;
+  ha.m = m;
+  ha.batch = B;
+  ha.K = spec.dims[L - 1];
+  ha.C = C;
+  ha.round_w_bf16 = bf;
+  {
+    Scope sc(hook, OLSGD_KC_LOSS, s);
+    OLSGD_TRY(launch_head_forward(ha, s));
+  }
+  {
+    Scope sc(hook, OLSGD_KC_BACKWARD, s);
+    OLSGD_TRY(launch_head_wgrad(ha, io.g, loss, s));
+  }
+
+  // hidden layers, backward
+  for (int l = L - 1; l >= 1; --l) {
+    // dW_l [d_l][d_{l-1}] = dA_l^T [d_l][B] * (H_{l-1}^T [d_{l-1}][B])^T
+    GemmArgs gw{};
+    gw.A = mb.dat[l];
+    gw.lda = B;
+    gw.a_batch = (int64_t)spec.dims[l] * B;
+    gw.B = (l == 1) ? mb.xb16t : mb.ht[l - 1];
+    gw.ldb = B;
+    gw.b_batch = (int64_t)spec.dims[l - 1] * B;
+    gw.m = m;
+    gw.Ma = spec.dims[l];
+    gw.Nb = spec.dims[l - 1];
+    gw.K = B;
+    gw.epilogue = GEMM_EPI_STORE_F32;
+    gw.out_f = io.g + mb.w_off[l - 1];
+    gw.ldo = spec.dims[l - 1];
+    gw.out_batch = io.ld;
+    {
+      Scope sc(hook, OLSGD_KC_BACKWARD, s);
+      OLSGD_TRY(run_gemm(spec, gw, s));
+    }
+    {
+      Scope sc(hook, OLSGD_KC_BACKWARD, s);
+      OLSGD_TRY(launch_bias_grad(mb.dat[l], io.g, io.ld, mb.b_off[l - 1], m, spec.dims[l], B, s));
+    }
+    if (l >= 2) {
+      // dA_{l-1}^T [d_{l-1}][B] = (W_l^T [d_{l-1}][d_l] * dA_l [B][d_l]^T) .* (H_{l-1}^T > 0)
+      GemmArgs gd{};
+      gd.A = mb.wt[l - 1];
+      gd.lda = spec.dims[l];
+      gd.a_batch = (int64_t)spec.dims[l] * spec.dims[l - 1];
+      gd.B = mb.da[l];
+      gd.ldb = spec.dims[l];
+      gd.b_batch = (int64_t)B * spec.dims[l];
+      gd.m = m;
+      gd.Ma = spec.dims[l - 1];
+      gd.Nb = B;
+      gd.K = spec.dims[l];
+      gd.epilogue = GEMM_EPI_RELU_MASK;
+      gd.mask = mb.ht[l - 1];
+      gd.out_t = mb.dat[l - 1];
+      gd.out_n = mb.da[l - 1];
+      Scope sc(hook, OLSGD_KC_BACKWARD, s);
+      OLSGD_TRY(run_gemm(spec, gd, s));
+    }
+  }
+  return cudaSuccess;
+}
+
+cudaError_t model_post_update(const olsgd_model_spec& spec, const olsgd_hparams& hp,
+                              const ModelBuffers& mb, const __nv_bfloat16* shadow, int64_t ld,
+                              cudaStream_t s, const ProfHook& hook) {
+  if (!bf16_path(spec)) return cudaSuccess;
+  const int L = n_layers(spec);
+  // layer index l here is 0-based in the parameter layout: weights of the
+  // (l+1)-th layer map dims[l] -> dims[l+1]; its transposed copy feeds dgrad
+  for (int l = 1; l < L - 1; ++l) {
+    Scope sc(hook, OLSGD_KC_OTHER, s);
+    OLSGD_TRY(launch_transpose_bf16(shadow, ld, mb.w_off[l], mb.wt[l],
+                                    (int64_t)spec.dims[l + 1] * spec.dims[l], hp.m,
+                                    spec.dims[l + 1], spec.dims[l], s));
+  }
+  return cudaSuccess;
+}
+
+}  // namespace olsgd

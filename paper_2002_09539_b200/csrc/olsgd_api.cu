@@ -1,0 +1,578 @@
+// C ABI of libolsgd: context, argument checks, workspace carving, stream and
+// event choreography of one Overlap-Local-SGD period.  No arithmetic of the
+// method happens on the host; every step is a kernel launch.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "olsgd_internal.h"
+
+using namespace olsgd;
+
+namespace {
+
+thread_local std::string g_last_error;
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct ProfRec {
+  int cls;
+  cudaEvent_t start, stop;
+};
+
+}  // namespace
+
+struct olsgd_ctx {
+  olsgd_model_spec spec;
+  olsgd_hparams hp;
+  olsgd_data data;
+  int64_t P = 0, ld = 0;
+
+  // device state, carved from the caller's workspace
+  float* x[2] = {nullptr, nullptr};  // ping-pong worker models [m][ld]
+  int cur = 0;                       // x[cur] holds x_k
+  float* u = nullptr;                // local momentum [m][ld]
+  float* g = nullptr;                // stacked gradients [m][ld] (model modes)
+  float* z = nullptr;                // anchor [ld]
+  float* v = nullptr;                // anchor momentum [ld]
+  float* tmp = nullptr;              // [ld] scratch for olsgd_get_params
+  __nv_bfloat16* shadow = nullptr;   // bf16 copy of x_k [m][ld] (tensor-core path)
+  int32_t* idx = nullptr;            // [m][batch]
+  ModelBuffers mb;
+
+  cudaStream_t main = nullptr, side = nullptr;
+  cudaEvent_t pullback_done = nullptr, reduce_done = nullptr;
+  bool reduce_pending = false;  // an anchor refresh was launched and not yet waited for
+  int reduce_reads = -1;        // which x buffer that refresh reads
+  bool need_sync = false;       // a period ended; olsgd_period_sync is due
+
+  int64_t k = 0;
+  int64_t launches = 0;
+  bool prof = false;
+  std::vector<ProfRec> prof_pending;
+  std::vector<cudaEvent_t> prof_pool;
+  int64_t prof_launches[OLSGD_N_KERNEL_CLASSES] = {0};
+  double prof_ms[OLSGD_N_KERNEL_CLASSES] = {0};
+  std::string err;
+};
+
+namespace {
+
+olsgd_status fail(olsgd_ctx* ctx, olsgd_status st, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (ctx) ctx->err = buf;
+  g_last_error = buf;
+  return st;
+}
+
+#define OLSGD_CUDA(ctx, call)                                                             \
+  do {                                                                                    \
+    cudaError_t e_ = (call);                                                              \
+    if (e_ != cudaSuccess)                                                                \
+      return fail(ctx, OLSGD_ECUDA, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(e_), \
+                  __FILE__, __LINE__);                                                    \
+  } while (0)
+
+// Brackets one kernel launch: counts it and, when profiling, times it with
+// events on the launching stream.
+struct Launch {
+  olsgd_ctx* c;
+  cudaStream_t s;
+  ProfRec rec{};
+  bool timed = false;
+  Launch(olsgd_ctx* ctx, int cls, cudaStream_t stream) : c(ctx), s(stream) {
+    c->launches++;
+    if (!c->prof) return;
+    auto get = [&]() {
+      cudaEvent_t e = nullptr;
+      if (!c->prof_pool.empty()) {
+        e = c->prof_pool.back();
+        c->prof_pool.pop_back();
+      } else if (cudaEventCreate(&e) != cudaSuccess) {
+        e = nullptr;
+      }
+      return e;
+    };
+    rec.cls = cls;
+    rec.start = get();
+    rec.stop = get();
+    if (rec.start && rec.stop) {
+      timed = true;
+      cudaEventRecord(rec.start, s);
+    }
+  }
+  ~Launch() {
+    if (timed) {
+      cudaEventRecord(rec.stop, s);
+      c->prof_pending.push_back(rec);
+    }
+  }
+};
+
+ProfHook make_hook(olsgd_ctx* c) {
+  ProfHook hook;
+  hook.ctx = c;
+  hook.begin = [](void* ctx, int cls, cudaStream_t s) -> void* {
+    return new (std::nothrow) Launch(static_cast<olsgd_ctx*>(ctx), cls, s);
+  };
+  hook.end = [](void* h) { delete static_cast<Launch*>(h); };
+  return hook;
+}
+
+struct Plan {
+  int64_t P = 0, ld = 0;
+  size_t off_x0 = 0, off_x1 = 0, off_u = 0, off_g = 0, off_z = 0, off_v = 0, off_tmp = 0,
+         off_shadow = 0, off_idx = 0, off_model = 0, total = 0;
+  bool has_u = false, has_g = false, has_shadow = false;
+  ModelPlan mp;
+};
+
+olsgd_status check_spec(const olsgd_model_spec* spec, int64_t* P) {
+  if (!spec) return fail(nullptr, OLSGD_EINVAL, "model spec is NULL");
+  switch (spec->kind) {
+    case OLSGD_FLAT:
+      if (spec->flat_P < 1) return fail(nullptr, OLSGD_EINVAL, "flat_P must be >= 1");
+      *P = spec->flat_P;
+      return OLSGD_OK;
+    case OLSGD_LINREG:
+      if (spec->n_dims != 1 || spec->dims[0] < 1)
+        return fail(nullptr, OLSGD_EINVAL, "LINREG needs n_dims == 1 and dims[0] >= 1");
+      *P = spec->dims[0];
+      return OLSGD_OK;
+    case OLSGD_SOFTMAX:
+    case OLSGD_MLP: {
+      if (spec->kind == OLSGD_SOFTMAX && spec->n_dims != 2)
+        return fail(nullptr, OLSGD_EINVAL, "SOFTMAX needs n_dims == 2");
+      if (spec->n_dims < 2 || spec->n_dims > OLSGD_MAX_DIMS)
+        return fail(nullptr, OLSGD_EINVAL, "MLP needs 2 <= n_dims <= %d", OLSGD_MAX_DIMS);
+      int64_t p = 0;
+      for (int l = 0; l < spec->n_dims; ++l)
+        if (spec->dims[l] < 1) return fail(nullptr, OLSGD_EINVAL, "dims[%d] must be >= 1", l);
+      for (int l = 0; l + 1 < spec->n_dims; ++l)
+        p += (int64_t)spec->dims[l + 1] * spec->dims[l] + spec->dims[l + 1];
+      if (spec->dims[spec->n_dims - 1] > kMaxClasses)
+        return fail(nullptr, OLSGD_EINVAL, "at most %d classes are supported", kMaxClasses);
+      *P = p;
+      return OLSGD_OK;
+    }
+    default:
+      return fail(nullptr, OLSGD_EINVAL, "unknown model kind %d", spec->kind);
+  }
+}
+
+olsgd_status check_hp(const olsgd_hparams* hp) {
+  if (!hp) return fail(nullptr, OLSGD_EINVAL, "hyper-parameters are NULL");
+  if (hp->m < 1 || hp->m > 65535) return fail(nullptr, OLSGD_EINVAL, "m must be in [1, 65535]");
+  if (hp->tau < 1) return fail(nullptr, OLSGD_EINVAL, "tau must be >= 1");
+  if (hp->batch < 1) return fail(nullptr, OLSGD_EINVAL, "batch must be >= 1");
+  if (!(hp->gamma > 0.f)) return fail(nullptr, OLSGD_EINVAL, "gamma must be > 0");
+  if (!(hp->alpha >= 0.f && hp->alpha <= 1.f))
+    return fail(nullptr, OLSGD_EINVAL, "alpha must be in [0, 1]");
+  if (!(hp->beta >= 0.f && hp->beta < 1.f))
+    return fail(nullptr, OLSGD_EINVAL, "beta must be in [0, 1)");
+  if (!(hp->mu >= 0.f && hp->mu < 1.f)) return fail(nullptr, OLSGD_EINVAL, "mu must be in [0, 1)");
+  return OLSGD_OK;
+}
+
+olsgd_status make_plan(const olsgd_model_spec* spec, const olsgd_hparams* hp, Plan* pl) {
+  olsgd_status st = check_spec(spec, &pl->P);
+  if (st != OLSGD_OK) return st;
+  st = check_hp(hp);
+  if (st != OLSGD_OK) return st;
+  const int64_t m = hp->m;
+  pl->ld = (int64_t)align_up((size_t)pl->P, 64);  // rows start on 256-byte boundaries
+  const size_t row = (size_t)pl->ld * sizeof(float);
+  pl->has_u = hp->mu != 0.f;
+  pl->has_g = spec->kind != OLSGD_FLAT;
+  pl->has_shadow = spec->kind == OLSGD_MLP && spec->gemm_bf16 != 0;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, kAlign);
+    return o;
+  };
+  pl->off_x0 = take(row * m);
+  pl->off_x1 = take(row * m);
+  pl->off_u = pl->has_u ? take(row * m) : 0;
+  pl->off_g = pl->has_g ? take(row * m) : 0;
+  pl->off_z = take(row);
+  pl->off_v = take(row);
+  pl->off_tmp = take(row);
+  pl->off_shadow = pl->has_shadow ? take((size_t)pl->ld * m * sizeof(__nv_bfloat16)) : 0;
+  pl->off_idx = pl->has_g ? take((size_t)m * hp->batch * sizeof(int32_t)) : 0;
+  pl->off_model = off;
+  if (pl->has_g) {
+    if (!plan_model(*spec, *hp, &pl->mp)) return fail(nullptr, OLSGD_EINVAL, "%s", pl->mp.error);
+    off = align_up(off + pl->mp.bytes, kAlign);
+  }
+  pl->total = off;
+  return OLSGD_OK;
+}
+
+olsgd_status drain_profile(olsgd_ctx* c) {
+  OLSGD_CUDA(c, cudaStreamSynchronize(c->main));
+  OLSGD_CUDA(c, cudaStreamSynchronize(c->side));
+  for (auto& r : c->prof_pending) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, r.start, r.stop) == cudaSuccess) {
+      c->prof_ms[r.cls] += ms;
+      c->prof_launches[r.cls] += 1;
+    }
+    c->prof_pool.push_back(r.start);
+    c->prof_pool.push_back(r.stop);
+  }
+  c->prof_pending.clear();
+  return OLSGD_OK;
+}
+
+// Eq. 3 / Eq. 4 for all workers: reads x[cur], writes x[1-cur], flips.
+olsgd_status apply_update(olsgd_ctx* c, const float* g, int64_t ldg) {
+  const bool sync = (c->k + 1) % c->hp.tau == 0;
+  const int nxt = 1 - c->cur;
+  // The anchor refresh of the previous period runs on the side stream.  It must
+  // have finished before a pull-back reads z, and before its input buffer is
+  // overwritten.
+  if (c->reduce_pending && (sync || c->reduce_reads == nxt)) {
+    OLSGD_CUDA(c, cudaStreamWaitEvent(c->main, c->reduce_done, 0));
+    c->reduce_pending = false;
+  }
+  UpdateArgs a;
+  a.x_in = c->x[c->cur];
+  a.x_out = c->x[nxt];
+  a.g = g;
+  a.u = c->u;
+  a.z = c->z;
+  a.shadow = c->shadow;
+  a.P = c->P;
+  a.ld = c->ld;
+  a.ldg = ldg;
+  a.m = c->hp.m;
+  a.gamma = c->hp.gamma;
+  a.mu = c->hp.mu;
+  a.alpha = c->hp.alpha;
+  a.sync = sync;
+  {
+    Launch l(c, OLSGD_KC_UPDATE, c->main);
+    OLSGD_CUDA(c, launch_fused_update(a, c->main));
+  }
+  c->cur = nxt;
+  c->k += 1;
+  if (sync) c->need_sync = true;
+  return OLSGD_OK;
+}
+
+olsgd_status copy_out(olsgd_ctx* c, void* dst, const void* src, size_t bytes) {
+  OLSGD_CUDA(c, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDefault, c->main));
+  OLSGD_CUDA(c, cudaStreamSynchronize(c->main));
+  return OLSGD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+olsgd_status olsgd_param_count(const olsgd_model_spec* spec, int64_t* out_P) {
+  if (!out_P) return fail(nullptr, OLSGD_EINVAL, "out_P is NULL");
+  return check_spec(spec, out_P);
+}
+
+olsgd_status olsgd_workspace_bytes(const olsgd_model_spec* spec, const olsgd_hparams* hp,
+                                   size_t* out_bytes) {
+  if (!out_bytes) return fail(nullptr, OLSGD_EINVAL, "out_bytes is NULL");
+  Plan pl;
+  olsgd_status st = make_plan(spec, hp, &pl);
+  if (st != OLSGD_OK) return st;
+  *out_bytes = pl.total;
+  return OLSGD_OK;
+}
+
+olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const olsgd_hparams* hp,
+                        const olsgd_data* data, const float* x0_device, void* workspace_device,
+                        size_t workspace_bytes, void* main_stream, void* side_stream) {
+  if (!out) return fail(nullptr, OLSGD_EINVAL, "out is NULL");
+  *out = nullptr;
+  Plan pl;
+  olsgd_status st = make_plan(spec, hp, &pl);
+  if (st != OLSGD_OK) return st;
+  if (!x0_device || (reinterpret_cast<uintptr_t>(x0_device) & 15))
+    return fail(nullptr, OLSGD_EINVAL, "x0_device must be non-null and 16-byte aligned");
+  if (!workspace_device || (reinterpret_cast<uintptr_t>(workspace_device) & (kAlign - 1)))
+    return fail(nullptr, OLSGD_EINVAL, "workspace_device must be non-null and 256-byte aligned");
+  if (workspace_bytes < pl.total)
+    return fail(nullptr, OLSGD_ENOMEM, "workspace too small: %zu bytes given, %zu needed",
+                workspace_bytes, pl.total);
+  if (spec->kind != OLSGD_FLAT) {
+    if (!data || !data->X || !data->y) return fail(nullptr, OLSGD_EINVAL, "data is required");
+    if (data->n_per_worker < 1 || data->n_per_worker > 0x7FFFFFFF)
+      return fail(nullptr, OLSGD_EINVAL, "n_per_worker must be in [1, 2^31)");
+    if ((reinterpret_cast<uintptr_t>(data->X) & 15) || (reinterpret_cast<uintptr_t>(data->y) & 3))
+      return fail(nullptr, OLSGD_EINVAL, "data pointers are misaligned");
+  }
+  olsgd_ctx* c = new (std::nothrow) olsgd_ctx();
+  if (!c) return fail(nullptr, OLSGD_ENOMEM, "host allocation failed");
+  c->spec = *spec;
+  c->hp = *hp;
+  if (data) c->data = *data; else memset(&c->data, 0, sizeof c->data);
+  c->P = pl.P;
+  c->ld = pl.ld;
+  c->main = static_cast<cudaStream_t>(main_stream);
+  c->side = static_cast<cudaStream_t>(side_stream);
+  char* ws = static_cast<char*>(workspace_device);
+  c->x[0] = reinterpret_cast<float*>(ws + pl.off_x0);
+  c->x[1] = reinterpret_cast<float*>(ws + pl.off_x1);
+  c->u = pl.has_u ? reinterpret_cast<float*>(ws + pl.off_u) : nullptr;
+  c->g = pl.has_g ? reinterpret_cast<float*>(ws + pl.off_g) : nullptr;
+  c->z = reinterpret_cast<float*>(ws + pl.off_z);
+  c->v = reinterpret_cast<float*>(ws + pl.off_v);
+  c->tmp = reinterpret_cast<float*>(ws + pl.off_tmp);
+  c->shadow = pl.has_shadow ? reinterpret_cast<__nv_bfloat16*>(ws + pl.off_shadow) : nullptr;
+  c->idx = pl.has_g ? reinterpret_cast<int32_t*>(ws + pl.off_idx) : nullptr;
+
+  auto bail = [&](olsgd_status s) {
+    if (c->pullback_done) cudaEventDestroy(c->pullback_done);
+    if (c->reduce_done) cudaEventDestroy(c->reduce_done);
+    g_last_error = c->err;
+    delete c;
+    return s;
+  };
+#define OLSGD_INIT_CUDA(call)                                                               \
+  do {                                                                                      \
+    cudaError_t e_ = (call);                                                                \
+    if (e_ != cudaSuccess)                                                                  \
+      return bail(fail(c, OLSGD_ECUDA, "%s failed: %s", #call, cudaGetErrorString(e_)));    \
+  } while (0)
+
+  OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->pullback_done, cudaEventDisableTiming));
+  OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->reduce_done, cudaEventDisableTiming));
+  // zero everything once (padding, momentum buffers, gradient padding), then
+  // x_0^(i) = z_0 = x0
+  OLSGD_INIT_CUDA(cudaMemsetAsync(ws, 0, pl.total, c->main));
+  const size_t pbytes = (size_t)c->P * sizeof(float);
+  for (int i = 0; i < c->hp.m; ++i)
+    OLSGD_INIT_CUDA(cudaMemcpyAsync(c->x[0] + (int64_t)i * c->ld, x0_device, pbytes,
+                                    cudaMemcpyDeviceToDevice, c->main));
+  OLSGD_INIT_CUDA(cudaMemcpyAsync(c->z, x0_device, pbytes, cudaMemcpyDeviceToDevice, c->main));
+  if (pl.has_g) {
+    if (!bind_model(c->spec, c->hp, pl.mp, ws + pl.off_model, &c->mb)) {
+      return bail(fail(c, OLSGD_EINVAL, "%s", c->mb.error));
+    }
+    if (c->shadow) {
+      Launch l(c, OLSGD_KC_OTHER, c->main);
+      OLSGD_INIT_CUDA(launch_cast_bf16(c->x[0], c->shadow, (int64_t)c->hp.m * c->ld, c->main));
+    }
+    cudaError_t e = model_post_update(c->spec, c->hp, c->mb, c->shadow, c->ld, c->main,
+                                      make_hook(c));
+    if (e != cudaSuccess)
+      return bail(fail(c, OLSGD_ECUDA, "model set-up failed: %s", cudaGetErrorString(e)));
+  }
+  OLSGD_INIT_CUDA(cudaStreamSynchronize(c->main));
+#undef OLSGD_INIT_CUDA
+  *out = c;
+  return OLSGD_OK;
+}
+
+olsgd_status olsgd_local_step_with_grads(olsgd_ctx* c, const float* g_device) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  if (c->spec.kind != OLSGD_FLAT)
+    return fail(c, OLSGD_ESTATE, "olsgd_local_step_with_grads is for OLSGD_FLAT contexts");
+  if (!g_device || (reinterpret_cast<uintptr_t>(g_device) & 3))
+    return fail(c, OLSGD_EINVAL, "g_device must be non-null and 4-byte aligned");
+  if (c->need_sync) return fail(c, OLSGD_ESTATE, "a period ended: call olsgd_period_sync first");
+  return apply_update(c, g_device, c->P);
+}
+
+olsgd_status olsgd_local_step(olsgd_ctx* c, float* loss_device) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  if (c->spec.kind == OLSGD_FLAT)
+    return fail(c, OLSGD_ESTATE, "OLSGD_FLAT contexts take olsgd_local_step_with_grads");
+  if (c->need_sync) return fail(c, OLSGD_ESTATE, "a period ended: call olsgd_period_sync first");
+  // S1: minibatch indices xi_k^(i)
+  {
+    Launch l(c, OLSGD_KC_INDEX, c->main);
+    OLSGD_CUDA(c, launch_minibatch_indices(c->idx, c->hp.seed, c->hp.m, c->k, c->hp.batch,
+                                           c->data.n_per_worker, c->main));
+  }
+  // S2-S4: gather, forward, loss, backward -> g [m][ld]
+  StepIO io;
+  io.x = c->x[c->cur];
+  io.shadow = c->shadow;
+  io.g = c->g;
+  io.ld = c->ld;
+  io.idx = c->idx;
+  io.loss = loss_device;
+  const ProfHook hook = make_hook(c);
+  cudaError_t e = model_forward_backward(c->spec, c->hp, c->data, c->mb, io, c->main, hook);
+  if (e != cudaSuccess)
+    return fail(c, OLSGD_ECUDA, "forward/backward failed: %s", cudaGetErrorString(e));
+  // S5-S6
+  olsgd_status st = apply_update(c, c->g, c->ld);
+  if (st != OLSGD_OK) return st;
+  e = model_post_update(c->spec, c->hp, c->mb, c->shadow, c->ld, c->main, hook);
+  if (e != cudaSuccess)
+    return fail(c, OLSGD_ECUDA, "post-update failed: %s", cudaGetErrorString(e));
+  return OLSGD_OK;
+}
+
+olsgd_status olsgd_period_sync(olsgd_ctx* c) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  if (!c->need_sync)
+    return fail(c, OLSGD_ESTATE, "olsgd_period_sync is legal once, right after a period ends (k=%lld, tau=%d)",
+                (long long)c->k, c->hp.tau);
+  // S7 on the side stream, ordered after the pull-back that closed the period
+  OLSGD_CUDA(c, cudaEventRecord(c->pullback_done, c->main));
+  OLSGD_CUDA(c, cudaStreamWaitEvent(c->side, c->pullback_done, 0));
+  AnchorArgs a;
+  a.x = c->x[c->cur];
+  a.z = c->z;
+  a.v = c->v;
+  a.P = c->P;
+  a.ld = c->ld;
+  a.m = c->hp.m;
+  a.beta = c->hp.beta;
+  {
+    Launch l(c, OLSGD_KC_ANCHOR, c->side);
+    OLSGD_CUDA(c, launch_worker_mean_anchor(a, c->side));
+  }
+  OLSGD_CUDA(c, cudaEventRecord(c->reduce_done, c->side));
+  c->reduce_pending = true;
+  c->reduce_reads = c->cur;
+  c->need_sync = false;
+  return OLSGD_OK;
+}
+
+olsgd_status olsgd_run(olsgd_ctx* c, int64_t n_iters, float* loss_device) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  if (n_iters < 0) return fail(c, OLSGD_EINVAL, "n_iters must be >= 0");
+  for (int64_t t = 0; t < n_iters; ++t) {
+    olsgd_status st = olsgd_local_step(c, loss_device ? loss_device + t * c->hp.m : nullptr);
+    if (st != OLSGD_OK) return st;
+    if (c->need_sync) {
+      st = olsgd_period_sync(c);
+      if (st != OLSGD_OK) return st;
+    }
+  }
+  return OLSGD_OK;
+}
+
+olsgd_status olsgd_get_params(olsgd_ctx* c, int32_t which, float* dst, size_t n_floats) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  if (!dst) return fail(c, OLSGD_EINVAL, "dst is NULL");
+  if (n_floats != (size_t)c->P)
+    return fail(c, OLSGD_EINVAL, "n_floats is %zu but P is %lld", n_floats, (long long)c->P);
+  const int m = c->hp.m;
+  if (which >= m || which < -5 - (m - 1))
+    return fail(c, OLSGD_EINVAL, "which = %d is out of range", which);
+  if (which <= -5 && !c->u) return fail(c, OLSGD_EINVAL, "no local momentum buffer (mu = 0)");
+  OLSGD_CUDA(c, cudaStreamSynchronize(c->side));
+  c->reduce_pending = false;
+  OLSGD_CUDA(c, cudaStreamSynchronize(c->main));
+  const size_t bytes = (size_t)c->P * sizeof(float);
+  const float* xk = c->x[c->cur];
+  if (which >= 0) return copy_out(c, dst, xk + (int64_t)which * c->ld, bytes);
+  if (which == -1) return copy_out(c, dst, c->z, bytes);
+  if (which == -2) return copy_out(c, dst, c->v, bytes);
+  if (which <= -5) return copy_out(c, dst, c->u + (int64_t)(-5 - which) * c->ld, bytes);
+  {
+    Launch l(c, OLSGD_KC_OTHER, c->main);
+    OLSGD_CUDA(c, launch_virtual_sequence(xk, c->z, c->tmp, c->P, c->ld, m,
+                                          which == -3 ? c->hp.alpha : 0.f, c->main));
+  }
+  return copy_out(c, dst, c->tmp, bytes);
+}
+
+olsgd_status olsgd_get_indices(olsgd_ctx* c, int64_t k, int32_t* dst) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  if (!dst) return fail(c, OLSGD_EINVAL, "dst is NULL");
+  if (c->spec.kind == OLSGD_FLAT) return fail(c, OLSGD_ESTATE, "OLSGD_FLAT draws no minibatches");
+  if (k < 0) return fail(c, OLSGD_EINVAL, "k must be >= 0");
+  OLSGD_CUDA(c, cudaStreamSynchronize(c->main));
+  {
+    Launch l(c, OLSGD_KC_INDEX, c->main);
+    OLSGD_CUDA(c, launch_minibatch_indices(c->idx, c->hp.seed, c->hp.m, k, c->hp.batch,
+                                           c->data.n_per_worker, c->main));
+  }
+  return copy_out(c, dst, c->idx, (size_t)c->hp.m * c->hp.batch * sizeof(int32_t));
+}
+
+olsgd_status olsgd_class_pairs(uint64_t seed, int32_t m, int32_t* dst, void* stream) {
+  if (m < 1 || m > 65535) return fail(nullptr, OLSGD_EINVAL, "m must be in [1, 65535]");
+  if (!dst) return fail(nullptr, OLSGD_EINVAL, "dst is NULL");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaPointerAttributes attr;
+  OLSGD_CUDA(nullptr, cudaPointerGetAttributes(&attr, dst));
+  if (attr.type == cudaMemoryTypeDevice || attr.type == cudaMemoryTypeManaged) {
+    OLSGD_CUDA(nullptr, launch_class_pairs(dst, seed, m, s));
+    OLSGD_CUDA(nullptr, cudaStreamSynchronize(s));
+    return OLSGD_OK;
+  }
+  // host destination: the table is tiny, stage it through pinned host memory
+  // that the device writes directly
+  int32_t* pinned = nullptr;
+  OLSGD_CUDA(nullptr, cudaHostAlloc(reinterpret_cast<void**>(&pinned), sizeof(int32_t) * 2 * m,
+                                    cudaHostAllocMapped));
+  int32_t* dev_view = nullptr;
+  cudaError_t e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&dev_view), pinned, 0);
+  if (e == cudaSuccess) e = launch_class_pairs(dev_view, seed, m, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e == cudaSuccess) memcpy(dst, pinned, sizeof(int32_t) * 2 * m);
+  cudaFreeHost(pinned);
+  if (e != cudaSuccess)
+    return fail(nullptr, OLSGD_ECUDA, "class-pair kernel failed: %s", cudaGetErrorString(e));
+  return OLSGD_OK;
+}
+
+int64_t olsgd_iteration(const olsgd_ctx* c) { return c ? c->k : -1; }
+int64_t olsgd_launch_count(const olsgd_ctx* c) { return c ? c->launches : -1; }
+
+olsgd_status olsgd_profile_enable(olsgd_ctx* c, int32_t on) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  olsgd_status st = drain_profile(c);
+  if (st != OLSGD_OK) return st;
+  c->prof = on != 0;
+  return OLSGD_OK;
+}
+
+olsgd_status olsgd_profile_read(olsgd_ctx* c, int64_t* launches, double* millis, int32_t reset) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  if (!launches || !millis) return fail(c, OLSGD_EINVAL, "output arrays are NULL");
+  olsgd_status st = drain_profile(c);
+  if (st != OLSGD_OK) return st;
+  for (int i = 0; i < OLSGD_N_KERNEL_CLASSES; ++i) {
+    launches[i] = c->prof_launches[i];
+    millis[i] = c->prof_ms[i];
+    if (reset) {
+      c->prof_launches[i] = 0;
+      c->prof_ms[i] = 0.0;
+    }
+  }
+  return OLSGD_OK;
+}
+
+const char* olsgd_last_error(const olsgd_ctx* c) {
+  return c ? c->err.c_str() : g_last_error.c_str();
+}
+
+olsgd_status olsgd_destroy(olsgd_ctx* c) {
+  if (!c) return OLSGD_OK;
+  cudaStreamSynchronize(c->side);
+  cudaStreamSynchronize(c->main);
+  for (auto& r : c->prof_pending) {
+    cudaEventDestroy(r.start);
+    cudaEventDestroy(r.stop);
+  }
+  for (auto e : c->prof_pool) cudaEventDestroy(e);
+  if (c->pullback_done) cudaEventDestroy(c->pullback_done);
+  if (c->reduce_done) cudaEventDestroy(c->reduce_done);
+  delete c;
+  return OLSGD_OK;
+}
+
+}  // extern "C"

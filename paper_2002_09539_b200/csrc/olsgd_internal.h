@@ -1,0 +1,189 @@
+// Internal declarations shared by the translation units of libolsgd.
+// Host-side launch wrappers only; every kernel lives in its own .cu file.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "olsgd.h"
+
+namespace olsgd {
+
+// ---- update_kernels.cu ------------------------------------------------------
+// Eq. 3 (+ local Nesterov buffer) and, when `sync`, Eq. 4, for all m workers.
+// x_in/x_out/u/shadow rows have stride `ld` floats (multiple of 4, 16-byte
+// aligned rows); g rows have stride `ldg`.  z may be null unless `sync`.
+struct UpdateArgs {
+  const float* x_in;
+  float* x_out;
+  const float* g;
+  float* u;              // null when mu == 0
+  const float* z;        // anchor, read on sync steps
+  __nv_bfloat16* shadow; // bf16 copy of x_out, or null
+  int64_t P, ld, ldg;
+  int m;
+  float gamma, mu, alpha;
+  bool sync;
+};
+cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t s);
+
+// Eq. 5 (beta == 0) or Eq. 10-11: worker mean in a fixed order, then z (and v).
+struct AnchorArgs {
+  const float* x;
+  float* z;
+  float* v;
+  int64_t P, ld;
+  int m;
+  float beta;
+};
+cudaError_t launch_worker_mean_anchor(const AnchorArgs& a, cudaStream_t s);
+
+// dst[j] = (1-alpha) * mean_i x_i[j] + alpha * z[j]   (alpha = 0: mean model)
+cudaError_t launch_virtual_sequence(const float* x, const float* z, float* dst, int64_t P,
+                                    int64_t ld, int m, float alpha, cudaStream_t s);
+
+// ---- sampling_kernels.cu ----------------------------------------------------
+cudaError_t launch_minibatch_indices(int32_t* idx, uint64_t seed, int m, int64_t k, int batch,
+                                     int64_t n, cudaStream_t s);
+cudaError_t launch_class_pairs(int32_t* dst, uint64_t seed, int m, cudaStream_t s);
+
+// ---- simt_kernels.cu --------------------------------------------------------
+constexpr int kMaxClasses = 32;  // the output layer is handled by one warp per row
+
+cudaError_t launch_cast_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t s);
+
+// Linear regression, one block per worker: r = X_b w - y_b, loss = sum r^2 / 2B,
+// g = X_b^T r / B, reading the batch rows straight from the worker's partition.
+cudaError_t launch_linreg(const float* X, const float* y, const int32_t* idx, const float* x,
+                          float* g, float* loss, int m, int batch, int64_t n, int d, int64_t ld,
+                          cudaStream_t s);
+
+// S2: copy the minibatch rows of every worker into contiguous staging.
+//   xb32  float [m][B][d]   (or null)
+//   xb16  bf16  [m][B][d]   (or null), xb16t bf16 [m][d][B] (or null)
+//   yb    int32 [m][B]
+cudaError_t launch_gather(const float* X, const int32_t* y, const int32_t* idx, float* xb32,
+                          __nv_bfloat16* xb16, __nv_bfloat16* xb16t, int32_t* yb, int m, int batch,
+                          int64_t n, int d, cudaStream_t s);
+
+// Output layer, forward + loss + backward to its input, one warp per batch row.
+//   in32 / in16   the layer's input [m][B][K], exactly one non-null
+//   W, b          this layer's fp32 weights [C][K] and bias [C] inside row i of x (stride ld)
+//   dlogits       float [m][B][C]  (p - onehot) / B
+//   rowloss       float [m][B]
+//   din32 / din16 / din16t   gradient w.r.t. the layer's input, already multiplied by the
+//                 ReLU mask (input > 0); any may be null ([m][B][K], [m][B][K], [m][K][B])
+struct HeadArgs {
+  const float* in32;
+  const __nv_bfloat16* in16;
+  const float* x;        // parameters [m][ld]
+  int64_t ld, w_off, b_off;
+  const int32_t* yb;
+  float* dlogits;
+  float* rowloss;
+  float* din32;
+  __nv_bfloat16* din16;
+  __nv_bfloat16* din16t;
+  int m, batch, K, C;
+  bool round_w_bf16;     // round W to bf16 before use (tensor-core path's operand rule)
+};
+cudaError_t launch_head_forward(const HeadArgs& a, cudaStream_t s);
+
+// Output layer weight/bias gradient and the mean loss:
+//   g[i][w_off + c*K + j] = sum_b dlogits[i][b][c] * in[i][b][j];  g[i][b_off + c] = sum_b dlogits
+//   loss[i] = mean_b rowloss[i][b]   (loss may be null)
+cudaError_t launch_head_wgrad(const HeadArgs& a, float* g, float* loss, cudaStream_t s);
+
+// g[i][b_off + r] = sum_c dat[i][r][c]   (bias gradient of a hidden layer from dA^T [m][R][B])
+cudaError_t launch_bias_grad(const __nv_bfloat16* dat, float* g, int64_t ld, int64_t b_off, int m,
+                             int R, int batch, cudaStream_t s);
+
+// dst[i][c][r] = src[i][r][c] for a [R][C] bf16 matrix inside every row of a [m][ld] array
+cudaError_t launch_transpose_bf16(const __nv_bfloat16* src, int64_t src_ld, int64_t src_off,
+                                  __nv_bfloat16* dst, int64_t dst_batch, int m, int R, int C,
+                                  cudaStream_t s);
+
+// ---- gemm --------------------------------------------------------------------
+// Worker-batched D[i] = A[i] * B[i]^T with both operands K-major bf16:
+//   A [m][Ma][K] (row pitch lda, batch pitch a_batch, in elements)
+//   B [m][Nb][K] (row pitch ldb, batch pitch b_batch)
+// D is [Ma][Nb] per worker, fp32 accumulate, consumed by one of three epilogues.
+enum GemmEpilogue {
+  // out = relu(D + bias[row]); written bf16 as [Ma][Nb] (out_t) and [Nb][Ma] (out_n)
+  GEMM_EPI_BIAS_RELU = 0,
+  // out = D * (mask[row][col] > 0); written bf16 as [Ma][Nb] (out_t) and [Nb][Ma] (out_n)
+  GEMM_EPI_RELU_MASK = 1,
+  // out = D, written fp32 to out_f [row * ldo + col]
+  GEMM_EPI_STORE_F32 = 2
+};
+struct GemmArgs {
+  const __nv_bfloat16* A;
+  const __nv_bfloat16* B;
+  int64_t lda, a_batch, ldb, b_batch;
+  int m, Ma, Nb, K;
+  int epilogue;
+  const float* bias;         // BIAS_RELU: bias[i * bias_batch + row]
+  int64_t bias_batch;
+  const __nv_bfloat16* mask; // RELU_MASK: [m][Ma][Nb], same layout as out_t
+  __nv_bfloat16* out_t;      // [m][Ma][Nb]
+  __nv_bfloat16* out_n;      // [m][Nb][Ma]
+  float* out_f;              // STORE_F32: out_f[i * out_batch + row * ldo + col]
+  int64_t ldo, out_batch;
+};
+// Plain CUDA-core version, used to validate the tensor-core kernel.
+cudaError_t launch_gemm_simt(const GemmArgs& a, cudaStream_t s);
+// tcgen05 / TMEM / TMA version.  Needs Ma % 128 == 0, K % 64 == 0, Nb % 16 == 0.
+bool gemm_tc_supported(const GemmArgs& a);
+cudaError_t launch_gemm_tc(const GemmArgs& a, cudaStream_t s);
+
+// ---- model.cu ------------------------------------------------------------------
+struct ModelPlan {
+  size_t bytes = 0;
+  char error[160] = {0};
+  // offsets inside the model area
+  size_t off_yb = 0, off_xb32 = 0, off_xb16 = 0, off_xb16t = 0, off_dlogits = 0, off_rowloss = 0,
+         off_loss = 0;
+  size_t off_h[OLSGD_MAX_DIMS] = {0}, off_ht[OLSGD_MAX_DIMS] = {0};    // hidden activations
+  size_t off_da[OLSGD_MAX_DIMS] = {0}, off_dat[OLSGD_MAX_DIMS] = {0};  // their gradients
+  size_t off_wt[OLSGD_MAX_DIMS] = {0};  // transposed bf16 weights of layer l (for dgrad)
+};
+struct ModelBuffers {
+  char error[160] = {0};
+  int32_t* yb = nullptr;
+  float* xb32 = nullptr;
+  __nv_bfloat16 *xb16 = nullptr, *xb16t = nullptr;
+  float *dlogits = nullptr, *rowloss = nullptr, *loss = nullptr;
+  __nv_bfloat16* h[OLSGD_MAX_DIMS] = {nullptr};
+  __nv_bfloat16* ht[OLSGD_MAX_DIMS] = {nullptr};
+  __nv_bfloat16* da[OLSGD_MAX_DIMS] = {nullptr};
+  __nv_bfloat16* dat[OLSGD_MAX_DIMS] = {nullptr};
+  __nv_bfloat16* wt[OLSGD_MAX_DIMS] = {nullptr};
+  int64_t w_off[OLSGD_MAX_DIMS] = {0}, b_off[OLSGD_MAX_DIMS] = {0};
+};
+struct StepIO {
+  const float* x;                // x_k, [m][ld]
+  const __nv_bfloat16* shadow;   // bf16 copy of x_k or null
+  float* g;                      // out: [m][ld]
+  int64_t ld;
+  const int32_t* idx;            // [m][batch]
+  float* loss;                   // out: [m] or null
+};
+// Lets model.cu count and time its launches without knowing the context type.
+struct ProfHook {
+  void* ctx;
+  void* (*begin)(void* ctx, int cls, cudaStream_t s);
+  void (*end)(void* handle);
+};
+bool plan_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, ModelPlan* mp);
+bool bind_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, const ModelPlan& mp,
+                char* base, ModelBuffers* mb);
+cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hparams& hp,
+                                   const olsgd_data& data, const ModelBuffers& mb,
+                                   const StepIO& io, cudaStream_t s, const ProfHook& hook);
+// Work that must follow every parameter update (transposed bf16 weights for dgrad).
+cudaError_t model_post_update(const olsgd_model_spec& spec, const olsgd_hparams& hp,
+                              const ModelBuffers& mb, const __nv_bfloat16* shadow, int64_t ld,
+                              cudaStream_t s, const ProfHook& hook);
+
+}  // namespace olsgd

@@ -1,0 +1,90 @@
+// Minibatch index rule and the non-IID class-pair table, on the device.
+//
+// Philox4x32-10 is implemented here from its published definition (Salmon,
+// Moraes, Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3", SC'11,
+// Section 3.3 and the Philox4x32 row of its constants table): ten rounds of
+//   (c0, c1, c2, c3) <- (hi(M1 c2) ^ c1 ^ k0, lo(M1 c2), hi(M0 c0) ^ c3 ^ k1, lo(M0 c0))
+// with the key bumped by the two Weyl constants before every round but the first.
+#include "olsgd_internal.h"
+
+namespace olsgd {
+namespace {
+
+struct U4 { uint32_t w[4]; };
+
+__device__ __forceinline__ U4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                            uint32_t k0, uint32_t k1) {
+  constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+  constexpr uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    if (r > 0) { k0 += W0; k1 += W1; }
+    const uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
+    const uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+  }
+  U4 r; r.w[0] = c0; r.w[1] = c1; r.w[2] = c2; r.w[3] = c3;
+  return r;
+}
+
+constexpr uint32_t kStreamMinibatch = 1;
+constexpr uint32_t kStreamPartition = 2;
+
+// One thread per Philox block: four consecutive slots of one worker.
+__global__ void minibatch_indices_kernel(int32_t* __restrict__ idx, uint32_t k0, uint32_t k1,
+                                         int m, uint32_t k, int batch, uint32_t n) {
+  const int blocks_per_worker = (batch + 3) / 4;
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= m * blocks_per_worker) return;
+  const int i = t / blocks_per_worker, q = t % blocks_per_worker;
+  const U4 r = philox4x32_10((uint32_t)q, k, (uint32_t)i, kStreamMinibatch, k0, k1);
+#pragma unroll
+  for (int lane = 0; lane < 4; ++lane) {
+    const int j = q * 4 + lane;
+    if (j < batch) idx[(int64_t)i * batch + j] = (int32_t)__umulhi(r.w[lane], n);
+  }
+}
+
+// One thread per permutation of the ten classes (ten slots = five workers).
+__global__ void class_pairs_kernel(int32_t* __restrict__ dst, uint32_t k0, uint32_t k1, int m) {
+  const int n_perm = (2 * m + 9) / 10;
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n_perm) return;
+  int perm[10];
+#pragma unroll
+  for (int c = 0; c < 10; ++c) perm[c] = c;
+  for (int p = 9; p >= 1; --p) {
+    const U4 r = philox4x32_10((uint32_t)p, (uint32_t)t, 0u, kStreamPartition, k0, k1);
+    const int q = (int)__umulhi(r.w[0], (uint32_t)(p + 1));
+    const int a = perm[p];
+    perm[p] = perm[q];
+    perm[q] = a;
+  }
+  for (int c = 0; c < 10; ++c) {
+    const int slot = t * 10 + c;
+    if (slot < 2 * m) dst[slot] = perm[c];
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_minibatch_indices(int32_t* idx, uint64_t seed, int m, int64_t k, int batch,
+                                     int64_t n, cudaStream_t s) {
+  const int total = m * ((batch + 3) / 4);
+  const int threads = 128;
+  minibatch_indices_kernel<<<(total + threads - 1) / threads, threads, 0, s>>>(
+      idx, (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), m, (uint32_t)k, batch,
+      (uint32_t)n);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_class_pairs(int32_t* dst, uint64_t seed, int m, cudaStream_t s) {
+  const int n_perm = (2 * m + 9) / 10;
+  const int threads = 64;
+  class_pairs_kernel<<<(n_perm + threads - 1) / threads, threads, 0, s>>>(
+      dst, (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), m);
+  return cudaGetLastError();
+}
+
+}  // namespace olsgd

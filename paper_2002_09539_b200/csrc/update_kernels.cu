@@ -1,0 +1,236 @@
+// Fused parameter update (Eq. 3 with the local Nesterov buffer, Eq. 4 on sync
+// steps) and the worker-mean / anchor kernel (Eq. 5, Eq. 10-11).
+//
+// Both are pure streaming kernels bound by HBM bandwidth: every byte is read
+// once and written once, all accesses are 128-bit and coalesced along the
+// parameter dimension, and each thread keeps several independent loads in
+// flight by unrolling over the worker dimension.
+#include "olsgd_internal.h"
+
+namespace olsgd {
+namespace {
+
+constexpr int kUpdateThreads = 256;
+constexpr int kUnroll = 4;
+
+__device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
+
+__device__ __forceinline__ float4 load_g(const float* g_row, int64_t col4, int64_t P, bool vec) {
+  if (vec) return ld_stream(reinterpret_cast<const float4*>(g_row) + col4);
+  // unaligned rows (row stride not a multiple of 4 floats): scalar, bounds-checked
+  const int64_t j = col4 * 4;
+  float4 r;
+  r.x = (j + 0 < P) ? __ldcs(g_row + j + 0) : 0.f;
+  r.y = (j + 1 < P) ? __ldcs(g_row + j + 1) : 0.f;
+  r.z = (j + 2 < P) ? __ldcs(g_row + j + 2) : 0.f;
+  r.w = (j + 3 < P) ? __ldcs(g_row + j + 3) : 0.f;
+  return r;
+}
+
+// One thread owns a 16-byte column strip and walks over `wpt` workers, so the
+// anchor strip is read once per thread on sync steps.
+template <bool MOM, bool SYNC, bool SHADOW>
+__global__ void __launch_bounds__(kUpdateThreads)
+fused_update_kernel(const float* __restrict__ x_in, float* __restrict__ x_out,
+                    const float* __restrict__ g, float* __restrict__ u,
+                    const float* __restrict__ z, __nv_bfloat16* __restrict__ shadow, int64_t P,
+                    int64_t n4, int64_t ld, int64_t ldg, int m, int wpt, bool gvec, float gamma,
+                    float mu, float alpha) {
+  const int64_t col4 = (int64_t)blockIdx.x * kUpdateThreads + threadIdx.x;
+  if (col4 >= n4) return;
+  const int i0 = blockIdx.y * wpt;
+  const int i1 = min(m, i0 + wpt);
+
+  float4 zz = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (SYNC) zz = reinterpret_cast<const float4*>(z)[col4];
+
+  for (int ib = i0; ib < i1; ib += kUnroll) {
+    float4 xv[kUnroll], gv[kUnroll], uv[kUnroll];
+#pragma unroll
+    for (int t = 0; t < kUnroll; ++t) {
+      const int i = ib + t;
+      if (i < i1) {
+        xv[t] = reinterpret_cast<const float4*>(x_in + (int64_t)i * ld)[col4];
+        gv[t] = load_g(g + (int64_t)i * ldg, col4, P, gvec);
+        if (MOM) uv[t] = reinterpret_cast<const float4*>(u + (int64_t)i * ld)[col4];
+      }
+    }
+#pragma unroll
+    for (int t = 0; t < kUnroll; ++t) {
+      const int i = ib + t;
+      if (i < i1) {
+        float4 x = xv[t];
+        const float4 gg = gv[t];
+        if (MOM) {
+          // u <- mu u + g ;  x <- x - gamma (g + mu u)
+          float4 uu = uv[t];
+          uu.x = fmaf(mu, uu.x, gg.x);
+          uu.y = fmaf(mu, uu.y, gg.y);
+          uu.z = fmaf(mu, uu.z, gg.z);
+          uu.w = fmaf(mu, uu.w, gg.w);
+          reinterpret_cast<float4*>(u + (int64_t)i * ld)[col4] = uu;
+          x.x -= gamma * fmaf(mu, uu.x, gg.x);
+          x.y -= gamma * fmaf(mu, uu.y, gg.y);
+          x.z -= gamma * fmaf(mu, uu.z, gg.z);
+          x.w -= gamma * fmaf(mu, uu.w, gg.w);
+        } else {
+          x.x -= gamma * gg.x;  // Eq. 3
+          x.y -= gamma * gg.y;
+          x.z -= gamma * gg.z;
+          x.w -= gamma * gg.w;
+        }
+        if (SYNC) {  // Eq. 4
+          x.x -= alpha * (x.x - zz.x);
+          x.y -= alpha * (x.y - zz.y);
+          x.z -= alpha * (x.z - zz.z);
+          x.w -= alpha * (x.w - zz.w);
+        }
+        reinterpret_cast<float4*>(x_out + (int64_t)i * ld)[col4] = x;
+        if (SHADOW) {
+          __nv_bfloat162 lo = __floats2bfloat162_rn(x.x, x.y);
+          __nv_bfloat162 hi = __floats2bfloat162_rn(x.z, x.w);
+          uint2 pk;
+          pk.x = *reinterpret_cast<uint32_t*>(&lo);
+          pk.y = *reinterpret_cast<uint32_t*>(&hi);
+          reinterpret_cast<uint2*>(shadow + (int64_t)i * ld)[col4] = pk;
+        }
+      }
+    }
+  }
+}
+
+constexpr int kMeanCols = 32;   // float4 columns per block: 512 contiguous bytes per row
+constexpr int kMeanSlices = 8;  // worker slices per block, combined through shared memory
+
+// Column sums over the worker dimension in a fixed order: slice s adds workers
+// s, s + S, s + 2S, ... sequentially, then slice 0 adds the S partial sums in
+// slice order.  The result does not depend on launch shape or timing.
+template <bool MOM>
+__global__ void __launch_bounds__(kMeanCols* kMeanSlices)
+worker_mean_anchor_kernel(const float* __restrict__ x, float* __restrict__ z,
+                          float* __restrict__ v, int64_t n4, int64_t ld, int m, float beta,
+                          float m_f) {
+  __shared__ float4 part[kMeanSlices][kMeanCols];
+  const int64_t col4 = (int64_t)blockIdx.x * kMeanCols + threadIdx.x;
+  const int slice = threadIdx.y;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (col4 < n4) {
+    for (int ib = slice; ib < m; ib += kMeanSlices * kUnroll) {
+      float4 xv[kUnroll];
+#pragma unroll
+      for (int t = 0; t < kUnroll; ++t) {
+        const int i = ib + t * kMeanSlices;
+        if (i < m) xv[t] = ld_stream(reinterpret_cast<const float4*>(x + (int64_t)i * ld) + col4);
+      }
+#pragma unroll
+      for (int t = 0; t < kUnroll; ++t) {
+        const int i = ib + t * kMeanSlices;
+        if (i < m) {
+          acc.x += xv[t].x;
+          acc.y += xv[t].y;
+          acc.z += xv[t].z;
+          acc.w += xv[t].w;
+        }
+      }
+    }
+  }
+  part[slice][threadIdx.x] = acc;
+  __syncthreads();
+  if (slice != 0 || col4 >= n4) return;
+  float4 s = part[0][threadIdx.x];
+#pragma unroll
+  for (int t = 1; t < kMeanSlices; ++t) {
+    const float4 p = part[t][threadIdx.x];
+    s.x += p.x;
+    s.y += p.y;
+    s.z += p.z;
+    s.w += p.w;
+  }
+  s.x /= m_f;
+  s.y /= m_f;
+  s.z /= m_f;
+  s.w /= m_f;
+  float4* z4 = reinterpret_cast<float4*>(z) + col4;
+  if (MOM) {
+    // Eq. 10: v <- beta v + (mean - z);  Eq. 11: z <- z + v
+    float4* v4 = reinterpret_cast<float4*>(v) + col4;
+    float4 zz = *z4, vv = *v4;
+    vv.x = fmaf(beta, vv.x, s.x - zz.x);
+    vv.y = fmaf(beta, vv.y, s.y - zz.y);
+    vv.z = fmaf(beta, vv.z, s.z - zz.z);
+    vv.w = fmaf(beta, vv.w, s.w - zz.w);
+    zz.x += vv.x;
+    zz.y += vv.y;
+    zz.z += vv.z;
+    zz.w += vv.w;
+    *v4 = vv;
+    *z4 = zz;
+  } else {
+    *z4 = s;  // Eq. 5
+  }
+}
+
+__global__ void virtual_sequence_kernel(const float* __restrict__ x, const float* __restrict__ z,
+                                        float* __restrict__ dst, int64_t P, int64_t ld, int m,
+                                        float alpha, float m_f) {
+  const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= P) return;
+  float s = 0.f;
+  for (int i = 0; i < m; ++i) s += x[(int64_t)i * ld + j];
+  s /= m_f;
+  dst[j] = (alpha == 0.f) ? s : (1.f - alpha) * s + alpha * z[j];
+}
+
+}  // namespace
+
+cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t s) {
+  const int64_t n4 = (a.P + 3) / 4;
+  const int64_t gx = (n4 + kUpdateThreads - 1) / kUpdateThreads;
+  // enough blocks for a few waves over 148 SMs; the rest of the worker
+  // dimension is walked inside the thread so the anchor strip is reused
+  const int64_t target_blocks = 148 * 16;
+  int gy = (int)((target_blocks + gx - 1) / gx);
+  if (gy < 1) gy = 1;
+  if (gy > a.m) gy = a.m;
+  const int wpt = (a.m + gy - 1) / gy;
+  gy = (a.m + wpt - 1) / wpt;
+  const bool gvec = (a.ldg % 4 == 0) && ((reinterpret_cast<uintptr_t>(a.g) & 15) == 0);
+  const bool mom = a.u != nullptr && a.mu != 0.f;
+  const bool shadow = a.shadow != nullptr;
+  dim3 grid((unsigned)gx, (unsigned)gy), block(kUpdateThreads);
+#define OLSGD_LAUNCH_UPD(MOM, SYNC, SH)                                                        \
+  fused_update_kernel<MOM, SYNC, SH><<<grid, block, 0, s>>>(a.x_in, a.x_out, a.g, a.u, a.z,    \
+                                                           a.shadow, a.P, n4, a.ld, a.ldg,    \
+                                                           a.m, wpt, gvec, a.gamma, a.mu,     \
+                                                           a.alpha)
+  if (mom) {
+    if (a.sync) { if (shadow) OLSGD_LAUNCH_UPD(true, true, true); else OLSGD_LAUNCH_UPD(true, true, false); }
+    else        { if (shadow) OLSGD_LAUNCH_UPD(true, false, true); else OLSGD_LAUNCH_UPD(true, false, false); }
+  } else {
+    if (a.sync) { if (shadow) OLSGD_LAUNCH_UPD(false, true, true); else OLSGD_LAUNCH_UPD(false, true, false); }
+    else        { if (shadow) OLSGD_LAUNCH_UPD(false, false, true); else OLSGD_LAUNCH_UPD(false, false, false); }
+  }
+#undef OLSGD_LAUNCH_UPD
+  return cudaGetLastError();
+}
+
+cudaError_t launch_worker_mean_anchor(const AnchorArgs& a, cudaStream_t s) {
+  const int64_t n4 = (a.P + 3) / 4;
+  dim3 grid((unsigned)((n4 + kMeanCols - 1) / kMeanCols)), block(kMeanCols, kMeanSlices);
+  const float m_f = (float)a.m;
+  if (a.beta != 0.f)
+    worker_mean_anchor_kernel<true><<<grid, block, 0, s>>>(a.x, a.z, a.v, n4, a.ld, a.m, a.beta, m_f);
+  else
+    worker_mean_anchor_kernel<false><<<grid, block, 0, s>>>(a.x, a.z, a.v, n4, a.ld, a.m, a.beta, m_f);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_virtual_sequence(const float* x, const float* z, float* dst, int64_t P,
+                                    int64_t ld, int m, float alpha, cudaStream_t s) {
+  const int threads = 256;
+  virtual_sequence_kernel<<<(unsigned)((P + threads - 1) / threads), threads, 0, s>>>(
+      x, z, dst, P, ld, m, alpha, (float)m);
+  return cudaGetLastError();
+}
+
+}  // namespace olsgd

@@ -1,0 +1,124 @@
+"""Fused update (Eq. 3-4) and worker-mean anchor (Eq. 5, 10-11) kernels against
+the oracle on external gradients: element by element, sizes that span several
+tiles with a ragged tail, all four momentum combinations."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+import synth_inputs as si
+from oracle import runner
+from helpers import max_rel_err, state_err, to_dev
+
+TOL = 1e-5   # max relative parameter error of the fp32 path
+
+
+def _run_pair(P, m, tau, gamma, alpha, beta, mu, iters, seed=0, overlap=True, std=0.1):
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    x0 = si.flat_init(seed, P)
+    grads = [si.flat_grads(seed, k, m, P, std) for k in range(iters)]
+    st = runner.run_flat(x0, grads, m=m, tau=tau, gamma=gamma, alpha=alpha, beta=beta, mu=mu)
+    opt = OverlapLocalSGD("flat", m=m, tau=tau, gamma=gamma, alpha=alpha, beta=beta, mu=mu,
+                          flat_P=P, x0=x0, overlap=overlap)
+    for k in range(iters):
+        opt.local_step_with_grads(to_dev(grads[k]))
+        if (k + 1) % tau == 0:
+            opt.period_sync()
+    return opt, st
+
+
+@pytest.mark.parametrize("beta,mu", [(0.0, 0.0), (0.9, 0.0), (0.0, 0.9), (0.9, 0.9)])
+@pytest.mark.parametrize("P,m,tau", [(4 * 256 * 3 + 7, 8, 4), (1, 1, 1), (5, 3, 2), (1000003, 16, 4),
+                                     (70001, 37, 3), (4096, 64, 1)])
+def test_flat_parity(P, m, tau, beta, mu):
+    opt, st = _run_pair(P, m, tau, 0.05, 0.5, beta, mu, iters=3 * tau + 1)
+    assert state_err(opt, st) <= TOL
+    v = opt.get_params(-2)
+    if beta:
+        assert max_rel_err([v], [st.v]) <= 1e-4
+    if mu:
+        u0 = opt.get_params(-5)
+        assert max_rel_err([u0], [st.u[0]]) <= TOL
+        ul = opt.get_params(-5 - (m - 1))
+        assert max_rel_err([ul], [st.u[m - 1]]) <= TOL
+    y = opt.get_params(-3)
+    assert max_rel_err([y], [st.virtual_sequence()]) <= TOL
+    xbar = opt.get_params(-4)
+    assert max_rel_err([xbar], [st.mean_model()]) <= TOL
+
+
+def test_hundred_iterations_stay_within_tolerance():
+    opt, st = _run_pair(50021, 16, 4, 0.05, 0.5, 0.9, 0.9, iters=100)
+    assert state_err(opt, st) <= TOL
+
+
+def test_anchor_is_exact_mean_and_frozen_between_syncs():
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    P, m, tau = 3000, 8, 3
+    x0 = si.flat_init(1, P)
+    opt = OverlapLocalSGD("flat", m=m, tau=tau, gamma=0.1, alpha=0.6, flat_P=P, x0=x0)
+    z_prev = opt.get_params(-1).copy()
+    assert np.array_equal(z_prev, x0)
+    for k in range(2 * tau):
+        opt.local_step_with_grads(to_dev(si.flat_grads(1, k, m, P)))
+        if (k + 1) % tau == 0:
+            opt.period_sync()
+            x, z, _ = opt.state()
+            assert np.abs(z - x.astype(np.float64).mean(0)).max() <= 2e-7 * np.abs(z).max()
+            z_prev = z
+        else:
+            assert np.array_equal(opt.get_params(-1), z_prev)
+
+
+def test_alpha_zero_and_alpha_one():
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    P, m, tau = 2049, 4, 2
+    x0 = si.flat_init(2, P)
+    grads = [si.flat_grads(2, k, m, P) for k in range(4)]
+    a0 = OverlapLocalSGD("flat", m=m, tau=tau, gamma=0.1, alpha=0.0, flat_P=P, x0=x0)
+    a1 = OverlapLocalSGD("flat", m=m, tau=tau, gamma=0.1, alpha=1.0, flat_P=P, x0=x0)
+    for k, g in enumerate(grads):
+        for o in (a0, a1):
+            o.local_step_with_grads(to_dev(g))
+            if (k + 1) % tau == 0:
+                o.period_sync()
+    x, _, _ = a0.state()
+    want = x0[None, :].astype(np.float64) - 0.1 * np.sum(grads, axis=0, dtype=np.float64)
+    assert max_rel_err(list(x), list(want)) <= TOL       # m independent SGD runs
+    x, z, _ = a1.state()
+    assert np.array_equal(z, x0) and all(np.array_equal(x[i], x0) for i in range(m))
+
+
+def test_overlapped_and_serial_streams_give_identical_bits():
+    a, _ = _run_pair(123457, 8, 2, 0.05, 0.5, 0.9, 0.9, iters=9, overlap=True)
+    b, _ = _run_pair(123457, 8, 2, 0.05, 0.5, 0.9, 0.9, iters=9, overlap=False)
+    xa, za, va = a.state()
+    xb, zb, vb = b.state()
+    assert np.array_equal(xa, xb) and np.array_equal(za, zb) and np.array_equal(va, vb)
+
+
+def test_call_order_is_enforced():
+    from paper_2002_09539_b200 import OverlapLocalSGD, OlsgdError
+    P, m = 64, 2
+    opt = OverlapLocalSGD("flat", m=m, tau=2, gamma=0.1, alpha=0.5, flat_P=P, x0=np.zeros(P, np.float32))
+    g = torch.zeros((m, P), device="cuda")
+    with pytest.raises(OlsgdError) as e:
+        opt.period_sync()                       # no period has ended
+    assert e.value.status == 2
+    opt.local_step_with_grads(g)
+    with pytest.raises(OlsgdError):
+        opt.period_sync()                       # mid-period
+    opt.local_step_with_grads(g)
+    with pytest.raises(OlsgdError):
+        opt.local_step_with_grads(g)            # sync is due
+    opt.period_sync()
+    with pytest.raises(OlsgdError):
+        opt.period_sync()                       # only once per period
+    with pytest.raises(OlsgdError):
+        opt.local_step()                        # wrong entry point for FLAT
+    with pytest.raises(OlsgdError):
+        opt.get_params(m)
+    assert opt.iteration == 2
+    opt.local_step_with_grads(g)
+    assert opt.iteration == 3 and opt.launch_count >= 4

@@ -1,0 +1,93 @@
+"""End-to-end parity of the model configurations against the oracle on the
+same seeded data and minibatch indices."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+import synth_inputs as si
+from oracle import models, runner, sampling
+from helpers import max_rel_err, state_err, to_dev
+
+TOL_FP32 = 1e-5
+
+
+def _pair(kind, dims, X, y, x0, *, m, tau, batch, gamma, alpha, beta, mu, seed, iters,
+          gemm_bf16=0, bf16_oracle=False, overlap=True):
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    st, losses, _ = runner.run_model(kind, dims, X, y, x0, m=m, tau=tau, batch=batch, gamma=gamma,
+                                     alpha=alpha, beta=beta, mu=mu, seed=seed, iters=iters,
+                                     bf16_operands=bf16_oracle)
+    opt = OverlapLocalSGD(kind, m=m, tau=tau, gamma=gamma, alpha=alpha, beta=beta, mu=mu,
+                          batch=batch, seed=seed, dims=dims, gemm_bf16=gemm_bf16, x0=x0,
+                          X=to_dev(X), y=to_dev(y), overlap=overlap)
+    loss_dev = torch.zeros((iters, m), device="cuda")
+    opt.run(iters, loss_dev)
+    return opt, st, loss_dev.cpu().numpy(), losses
+
+
+def test_config1_linear_regression_full():
+    c = si.CONFIGS["c1"]
+    X, y, _ = si.linreg_data(0, c["m"], c["n"], c["dims"][0])
+    x0 = si.model_init(0, "linreg", c["dims"])
+    opt, st, lg, lo = _pair("linreg", c["dims"], X, y, x0, m=c["m"], tau=c["tau"], batch=c["batch"],
+                            gamma=c["gamma"], alpha=c["alpha"], beta=0.0, mu=0.0, seed=0,
+                            iters=c["iters"])
+    assert state_err(opt, st) <= TOL_FP32
+    assert np.abs(lg - lo).max() <= 1e-5 * np.abs(lo).max()
+    assert lo[-1].mean() < 0.05 * lo[0].mean()          # it actually trains
+
+
+@pytest.mark.parametrize("m,n,d,batch,tau,beta,mu", [(3, 40, 5, 7, 2, 0.0, 0.0),
+                                                     (2, 64, 130, 33, 3, 0.7, 0.9),
+                                                     (1, 9, 1, 1, 1, 0.0, 0.0)])
+def test_linear_regression_ragged_shapes(m, n, d, batch, tau, beta, mu):
+    X, y, _ = si.linreg_data(3, m, n, d)
+    x0 = np.zeros(d, np.float32)
+    opt, st, lg, lo = _pair("linreg", [d], X, y, x0, m=m, tau=tau, batch=batch, gamma=0.02,
+                            alpha=0.5, beta=beta, mu=mu, seed=4, iters=3 * tau + 1)
+    assert state_err(opt, st) <= TOL_FP32
+    assert np.abs(lg - lo).max() <= 1e-5 * np.abs(lo).max()
+
+
+def test_config2_softmax_regression_100_iterations():
+    c = si.CONFIGS["c2"]
+    X, y = si.mixture_data(0, c["m"], c["n"], c["dims"][0])
+    x0 = si.model_init(0, "softmax", c["dims"])
+    opt, st, lg, lo = _pair("softmax", c["dims"], X, y, x0, m=c["m"], tau=c["tau"],
+                            batch=c["batch"], gamma=c["gamma"], alpha=c["alpha"], beta=0.0, mu=0.0,
+                            seed=0, iters=100)
+    assert state_err(opt, st) <= TOL_FP32
+    assert np.abs(lg - lo).max() <= 2e-5 * np.abs(lo).max()
+
+
+@pytest.mark.parametrize("m,n,d,C,batch,tau,beta,mu", [(3, 50, 100, 7, 20, 2, 0.0, 0.0),
+                                                       (2, 300, 515, 32, 130, 3, 0.5, 0.9),
+                                                       (5, 10, 3, 2, 1, 1, 0.0, 0.0)])
+def test_softmax_regression_ragged_shapes(m, n, d, C, batch, tau, beta, mu):
+    rng = np.random.default_rng(5)
+    X = rng.standard_normal((m, n, d)).astype(np.float32)
+    y = rng.integers(0, C, size=(m, n)).astype(np.int32)
+    x0 = (0.1 * rng.standard_normal(models.n_params("softmax", [d, C]))).astype(np.float32)
+    opt, st, lg, lo = _pair("softmax", [d, C], X, y, x0, m=m, tau=tau, batch=batch, gamma=0.05,
+                            alpha=0.6, beta=beta, mu=mu, seed=6, iters=3 * tau + 1)
+    assert state_err(opt, st) <= TOL_FP32
+    assert np.abs(lg - lo).max() <= 2e-5 * np.abs(lo).max()
+
+
+def test_local_step_and_period_sync_equal_run():
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    X, y, _ = si.linreg_data(1, 2, 50, 6)
+    args = dict(m=2, tau=2, gamma=0.05, alpha=0.5, batch=4, seed=1, dims=[6],
+                x0=np.zeros(6, np.float32), X=to_dev(X), y=to_dev(y))
+    a = OverlapLocalSGD("linreg", **args)
+    b = OverlapLocalSGD("linreg", **args)
+    a.run(6)
+    for k in range(6):
+        b.local_step()
+        if (k + 1) % 2 == 0:
+            b.period_sync()
+    xa, za, _ = a.state()
+    xb, zb, _ = b.state()
+    assert np.array_equal(xa, xb) and np.array_equal(za, zb)
