@@ -36,7 +36,8 @@ def test_flat_parity(P, m, tau, beta, mu):
     assert state_err(opt, st) <= TOL
     v = opt.get_params(-2)
     if beta:
-        assert max_rel_err([v], [st.v]) <= 1e-4
+        # v is a difference of nearly equal vectors: its error is measured on the scale of z
+        assert np.abs(v - st.v).max() <= TOL * max(np.abs(st.z).max(), np.abs(st.v).max())
     if mu:
         u0 = opt.get_params(-5)
         assert max_rel_err([u0], [st.u[0]]) <= TOL
@@ -87,7 +88,8 @@ def test_alpha_zero_and_alpha_one():
     want = x0[None, :].astype(np.float64) - 0.1 * np.sum(grads, axis=0, dtype=np.float64)
     assert max_rel_err(list(x), list(want)) <= TOL       # m independent SGD runs
     x, z, _ = a1.state()
-    assert np.array_equal(z, x0) and all(np.array_equal(x[i], x0) for i in range(m))
+    # x - 1.0 * (x - z) returns z up to one rounding of the difference
+    assert max_rel_err([z] + list(x), [x0] * (m + 1)) <= 1e-6
 
 
 def test_overlapped_and_serial_streams_give_identical_bits():
