@@ -1,0 +1,464 @@
+#!/usr/bin/env python
+"""Benchmark of the Overlap-Local-SGD hot path: simulated worker-steps per second.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c1|c5]
+                    [--impl ours|reference]
+
+One "step" is one iteration k -> k+1 for all m workers: minibatch indices,
+gather, forward, loss, backward, fused update (+ pull-back on sync steps) and,
+every tau steps, the anchor refresh on the side stream.  Prints one JSON line.
+
+With N > 1 (launched by torchrun, one rank per GPU) every rank runs an
+independent replica of the whole m-worker job on its own seed; there is no
+collective on the data path.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import synth_inputs as si  # noqa: E402
+
+METRIC = "simulated_worker_steps_per_sec"
+UNIT = "worker-steps/s"
+L2_BYTES = 126 * 2 ** 20
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained"), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0,
+                source="fallback")
+
+
+# ------------------------------------------------------------------ inputs
+
+def make_inputs(name, seed, class_table=None):
+    c = si.CONFIGS[name]
+    if c["kind"] == "linreg":
+        X, y, _ = si.linreg_data(seed, c["m"], c["n"], c["dims"][0])
+    else:
+        X, y = si.mixture_data(seed, c["m"], c["n"], c["dims"][0], class_table)
+    x0 = si.model_init(seed, c["kind"], c["dims"])
+    return X, y, x0
+
+
+def n_params(c):
+    d = c["dims"]
+    if c["kind"] == "linreg":
+        return d[0]
+    return sum(d[l + 1] * d[l] + d[l + 1] for l in range(len(d) - 1))
+
+
+# ------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.QUERY,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            f = [t.strip() for t in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None,
+                    sm_max_mhz=float(np.max(mx)) if mx else None, reasons=sorted(reasons),
+                    samples=len(sm))
+
+
+# ------------------------------------------------------------------ roofline accounting
+
+def algorithmic_bytes(c, kernel_class, P, sync_fraction):
+    """Algorithmic HBM bytes of ONE launch of the given kernel class (averaged over
+    sync and ordinary steps for the update kernel)."""
+    m = c["m"]
+    mom = c["mu"] != 0.0
+    shadow = 2 if c.get("gemm_bf16") else 0
+    if kernel_class == "update":
+        per = (20 if mom else 12) + shadow
+        return m * P * per + sync_fraction * 4 * P
+    if kernel_class == "anchor":
+        return 4 * m * P + (16 if c["beta"] != 0.0 else 4) * P
+    return None
+
+
+# ------------------------------------------------------------------ our arm
+
+def run_ours(args, rank, world):
+    import torch
+    import torch.distributed as dist
+    from paper_2002_09539_b200 import OverlapLocalSGD, class_pairs
+    from paper_2002_09539_b200.build import build
+
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        build()
+    if world > 1:
+        dist.barrier()
+
+    name = args.workload
+    c = si.CONFIGS[name]
+    seed = rank                      # every rank is an independent replica
+    table = None
+    if c.get("non_iid"):
+        table = class_pairs(seed, c["m"], device="cpu").numpy()
+    X, y, x0 = make_inputs(name, seed, table)
+    P = n_params(c)
+    Xd, yd = torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda()
+    opt = OverlapLocalSGD(c["kind"], m=c["m"], tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"],
+                          beta=c["beta"], mu=c["mu"], batch=c["batch"], seed=seed, dims=c["dims"],
+                          gemm_bf16=c["gemm_bf16"], x0=x0, X=Xd, y=yd)
+    m, K, W = c["m"], args.steps, args.warmup
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        opt.main.wait_stream(opt.side)
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    # ---- device-resident throughput
+    opt.run(W)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches0 = opt.launch_count
+    ms = timed(lambda: opt.run(K))
+    launches = opt.launch_count - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    value = world * m * K / (ms * 1e-3)
+
+    # ---- per-kernel-class device time (second pass, every launch bracketed by events)
+    opt.profile_enable(True)
+    opt.run(K)
+    prof = opt.profile_read()
+    opt.profile_enable(False)
+    busy = {k: v for k, v in prof.items() if v[0] > 0}
+    total_ms = sum(v[1] for v in busy.values())
+    dominant = max(busy, key=lambda k: busy[k][1])
+    peaks = measured_peaks()
+    n_sync = sum(1 for k in range(K) if (k + 1) % c["tau"] == 0)
+    roof_class = dominant if algorithmic_bytes(c, dominant, P, 0) is not None else "update"
+    ab = algorithmic_bytes(c, roof_class, P, n_sync / K)
+    avg_ms = busy[roof_class][1] / busy[roof_class][0]
+    achieved = ab / (avg_ms * 1e-3) / 1e9
+    roofline = dict(bound="hbm", kernel=roof_class, achieved=round(achieved, 1),
+                    peak=peaks["hbm_gbs"], unit="GB/s", frac=round(achieved / peaks["hbm_gbs"], 4),
+                    frac_of_8000=round(achieved / 8000.0, 4), traffic=None,
+                    peak_source=peaks["source"], avg_launch_us=round(avg_ms * 1e3, 2),
+                    algorithmic_bytes_per_launch=int(ab),
+                    dominant_class=dominant,
+                    class_share={k: round(v[1] / total_ms, 4) for k, v in busy.items()},
+                    class_us_per_step={k: round(v[1] * 1e3 / K, 2) for k, v in busy.items()})
+
+    # ---- end to end: host minibatches in, host losses out, through the C ABI
+    pool = 4
+    n, B, d0 = c["n"], c["batch"], c["dims"][0]
+    rng = np.random.default_rng(seed + 77)
+    Xh, yh = [], []
+    for _ in range(pool):
+        idx = rng.integers(0, n, size=(m, B))
+        Xh.append(torch.from_numpy(np.stack([X[i][idx[i]] for i in range(m)])).pin_memory())
+        yh.append(torch.from_numpy(np.stack([y[i][idx[i]] for i in range(m)])).pin_memory())
+    loss_h = torch.zeros((K + W, m), dtype=torch.float32).pin_memory()
+
+    def e2e_steps(k0, count):
+        for t in range(k0, k0 + count):
+            opt.local_step_host(Xh[t % pool], yh[t % pool], loss_h[t])
+            if (opt.iteration) % c["tau"] == 0:
+                opt.period_sync()
+
+    e2e_steps(0, W)
+    opt.join()
+    barrier()
+    t0 = time.perf_counter()
+    e2e_steps(W, K)
+    opt.join()                      # host sees the last losses here
+    t1 = time.perf_counter()
+    e2e_ms = (t1 - t0) * 1e3
+    if world > 1:
+        t = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    assert np.isfinite(loss_h[W:].numpy()).all()
+    e2e = dict(value=round(world * m * K / (e2e_ms * 1e-3), 1), unit=UNIT,
+               h2d_bytes_per_step=int(m * B * d0 * 4 + m * B * 4), d2h_bytes_per_step=int(m * 4),
+               ms_per_step=round(e2e_ms / K, 4),
+               api="olsgd_local_step_host + olsgd_period_sync, pinned host minibatches")
+
+    out = None
+    if rank == 0:
+        cpu = cpu_baseline(name, c, X, y, x0, seed)
+        resident = X.nbytes + (2 + (1 if c["mu"] else 0) + 1) * m * P * 4
+        out = {
+            "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world,
+            "steps": K, "warmup": W, "ms_per_step": round(ms / K, 4), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if c["gemm_bf16"] else "f32", "data": "synthetic",
+            "config": {"workload": workload_name(name, c), "m": m, "tau": c["tau"],
+                       "batch": B, "dims": c["dims"], "P": P, "gamma": c["gamma"],
+                       "alpha": c["alpha"], "beta": c["beta"], "mu": c["mu"],
+                       "l2": "no flush: resident inputs+state %.0f MB exceed the %d MB L2"
+                             % (resident / 1e6, L2_BYTES >> 20) if resident > L2_BYTES else
+                             "state fits in L2 (%.1f MB): steady-state training keeps it there"
+                             % (resident / 1e6),
+                       "replicas": world},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+            "roofline": roofline, "cpu_baseline": cpu,
+        }
+    opt.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return out
+
+
+def run_flat_sweep(args, rank, world):
+    """Config 5: fused update and worker-mean kernels on flat parameter vectors with
+    external gradients, P x m sweep.  One JSON line; `value` is the largest point."""
+    import torch
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    from paper_2002_09539_b200.build import build
+
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if rank == 0:
+        build()
+    c = si.CONFIGS["c5"]
+    K, W = args.steps, args.warmup
+    peaks = measured_peaks()
+    points = []
+    Ps = [args.P] if args.P else c["P"]
+    ms_ = [args.m] if args.m else c["m"]
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    for P in Ps:
+        for m in ms_:
+            x0 = torch.randn(P, device="cuda")
+            g = torch.randn((m, P), device="cuda") * c["grad_std"]
+            opt = OverlapLocalSGD("flat", m=m, tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"],
+                                  beta=c["beta"], mu=c["mu"], flat_P=P, x0=x0)
+
+            def steps(count):
+                for _ in range(count):
+                    opt.local_step_with_grads(g)
+                    if opt.iteration % c["tau"] == 0:
+                        opt.period_sync()
+
+            steps(W)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n0 = opt.launch_count
+            e0.record()
+            steps(K)
+            opt.main.wait_stream(opt.side)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            launches = opt.launch_count - n0
+            opt.profile_enable(True)
+            steps(K)
+            prof = opt.profile_read()
+            opt.profile_enable(False)
+            cc = dict(c, m=m)
+            n_sync = K // c["tau"]
+            upd_b = algorithmic_bytes(cc, "update", P, n_sync / K)
+            anc_b = algorithmic_bytes(cc, "anchor", P, 0)
+            upd_ms = prof["update"][1] / prof["update"][0]
+            anc_ms = prof["anchor"][1] / max(1, prof["anchor"][0])
+            state_mb = (3 * m * P + 2 * P + m * P) * 4 / 1e6
+            points.append(dict(
+                P=P, m=m, worker_steps_per_s=round(m * K / (ms * 1e-3), 1),
+                ms_per_step=round(ms / K, 4), gpu_launches=int(launches),
+                update_gbs=round(upd_b / upd_ms / 1e6, 1), anchor_gbs=round(anc_b / anc_ms / 1e6, 1),
+                update_us=round(upd_ms * 1e3, 2), anchor_us=round(anc_ms * 1e3, 2),
+                update_frac_measured=round(upd_b / upd_ms / 1e6 / peaks["hbm_gbs"], 4),
+                anchor_frac_measured=round(anc_b / anc_ms / 1e6 / peaks["hbm_gbs"], 4),
+                update_frac_8000=round(upd_b / upd_ms / 1e6 / 8000.0, 4),
+                anchor_frac_8000=round(anc_b / anc_ms / 1e6 / 8000.0, 4),
+                resident_mb=round(state_mb, 1), in_l2=bool(state_mb * 1e6 < L2_BYTES)))
+            opt.close()
+            del opt, g, x0
+            torch.cuda.empty_cache()
+    clocks = sampler.stop() if rank == 0 else None
+    big = points[-1]
+    return {
+        "metric": METRIC, "value": big["worker_steps_per_s"], "unit": UNIT, "n_gpus": world,
+        "steps": K, "warmup": W, "ms_per_step": big["ms_per_step"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "config 5: update/anchor kernel sweep, flat fp32 parameters, "
+                               "external gradients, tau=4, momentum",
+                   "value_point": {"P": big["P"], "m": big["m"]},
+                   "l2": "no flush; points whose state fits the L2 are flagged in_l2"},
+        "clocks": clocks, "e2e": None, "gpu_launches": big["gpu_launches"],
+        "roofline": dict(bound="hbm", kernel="update", achieved=big["update_gbs"],
+                         peak=peaks["hbm_gbs"], unit="GB/s", frac=big["update_frac_measured"],
+                         frac_of_8000=big["update_frac_8000"], traffic=None,
+                         peak_source=peaks["source"]),
+        "sweep": points,
+    }
+
+
+def workload_name(name, c):
+    return {"c1": "config 1: linear regression d=64, m=4",
+            "c2": "config 2: softmax regression 3072->10, m=16, batch 128",
+            "c3": "config 3: MLP 3072-1024-1024-10 bf16, m=16, batch 128, momentum",
+            "c4": "config 4: non-IID MLP 3072-512-10 bf16, m=64, batch 64, momentum"}[name]
+
+
+# ------------------------------------------------------------------ oracle arms (CPU)
+
+def oracle_steps(c, X, y, x0, seed, workers, iters):
+    """Run `iters` oracle iterations on the first `workers` workers; returns seconds."""
+    from oracle import runner
+    t0 = time.perf_counter()
+    runner.run_model(c["kind"], c["dims"], X[:workers], y[:workers], x0, m=workers, tau=c["tau"],
+                     batch=c["batch"], gamma=c["gamma"], alpha=c["alpha"], beta=c["beta"],
+                     mu=c["mu"], seed=seed, iters=iters)
+    return time.perf_counter() - t0
+
+
+def cpu_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count()
+
+
+def cpu_baseline(name, c, X, y, x0, seed, budget_s=15.0):
+    """The oracle as it stands, timed on a bounded sample of the same workload."""
+    m = c["m"]
+    t1 = oracle_steps(c, X, y, x0, seed, m, 1)              # one full iteration, all workers
+    iters = int(max(1, min(c["iters"], budget_s / max(t1, 1e-6))))
+    t = oracle_steps(c, X, y, x0, seed, m, iters)
+    return dict(value=round(m * iters / t, 2), unit=UNIT, cores=cpu_cores(), kind="oracle",
+                sample="%d iterations of all %d workers (%.1f s)" % (iters, m, t))
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return None
+    name = args.workload
+    c = si.CONFIGS[name]
+    table = None
+    if c.get("non_iid"):
+        from oracle import sampling
+        table = sampling.class_pairs(0, c["m"])
+    X, y, x0 = make_inputs(name, 0, table)
+    K, W = args.steps, args.warmup
+    m = c["m"]
+    # bounded sample: a subset of the workers per step, sized so the run ends in minutes
+    t1 = oracle_steps(c, X, y, x0, 0, 1, 1)
+    budget = 150.0
+    workers = int(max(1, min(m, budget / ((K + W) * max(t1, 1e-6)))))
+    oracle_steps(c, X, y, x0, 0, workers, W)
+    t = oracle_steps(c, X, y, x0, 0, workers, K)
+    value = workers * K / t
+    sample = "%d of %d workers per step, %d steps" % (workers, m, K)
+    return {
+        "impl": "reference", "metric": METRIC, "value": round(value, 2), "unit": UNIT,
+        "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": round(t / K * 1e3, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": workload_name(name, c), "m": m, "tau": c["tau"],
+                   "batch": c["batch"], "dims": c["dims"], "sample": sample},
+        "cpu_baseline": dict(value=round(value, 2), unit=UNIT, cores=cpu_cores(), kind="oracle",
+                             sample=sample),
+        "e2e": dict(value=round(value, 2), unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+        "gpu_launches": 0,
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--P", type=int, default=0, help="c5 only: one parameter count")
+    ap.add_argument("--m", type=int, default=0, help="c5 only: one worker count")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        out = run_reference(args, rank, world)
+    elif args.workload == "c5":
+        out = run_flat_sweep(args, rank, world) if rank == 0 else None
+    else:
+        out = run_ours(args, rank, world)
+    if out is not None:
+        print(json.dumps(out), flush=True)
+
+
+if __name__ == "__main__":
+    main()

@@ -115,6 +115,24 @@ olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const ols
  * called since.                                                             */
 olsgd_status olsgd_local_step(olsgd_ctx* ctx, float* loss_device);
 
+/* The same iteration, with this step's minibatches supplied from HOST memory
+ * instead of being drawn from the resident data set: for a caller whose data
+ * loader lives on the host.  The rows are copied to the device on a copy stream
+ * owned by the context (double-buffered, so the copy of step k+1 overlaps the
+ * kernels of step k), then the step runs exactly as olsgd_local_step does.
+ *   Xb_host    float32 [m][batch][dims[0]], host (pinned memory for a truly
+ *              asynchronous copy); must stay valid and unchanged until a later
+ *              call has joined the streams (olsgd_get_params, olsgd_join)
+ *   yb_host    float32 [m][batch] (LINREG) or int32 [m][batch]
+ *   loss_host  m floats, host: written asynchronously with the per-worker
+ *              minibatch losses, valid after the streams are joined; or NULL
+ * The minibatch index rule is not used by this call.                         */
+olsgd_status olsgd_local_step_host(olsgd_ctx* ctx, const float* Xb_host, const void* yb_host,
+                                   float* loss_host);
+
+/* Block the host until every stream of the context is idle.                 */
+olsgd_status olsgd_join(olsgd_ctx* ctx);
+
 /* Same iteration for OLSGD_FLAT: the stacked gradients G_k (Eq. 7 without its
  * zero column) come from the caller.
  *   g_device  float32 [m][P], device, row stride P; read on the main stream */

@@ -61,6 +61,8 @@ def load_library():
                              C.POINTER(_Data), vp, vp, C.c_size_t, vp, vp]),
         "olsgd_local_step": (i32, [vp, vp]),
         "olsgd_local_step_with_grads": (i32, [vp, vp]),
+        "olsgd_local_step_host": (i32, [vp, vp, vp, vp]),
+        "olsgd_join": (i32, [vp]),
         "olsgd_period_sync": (i32, [vp]),
         "olsgd_run": (i32, [vp, i64, vp]),
         "olsgd_get_params": (i32, [vp, i32, vp, C.c_size_t]),
@@ -154,6 +156,18 @@ class OverlapLocalSGD:
         assert g.is_cuda and g.dtype == torch.float32 and g.is_contiguous()
         assert g.numel() == self.m * self.P
         _check(self.lib, self.lib.olsgd_local_step_with_grads(self.ctx, g.data_ptr()), self.ctx)
+
+    def local_step_host(self, Xb, yb, loss=None):
+        """Xb, yb (and loss) are HOST tensors, ideally pinned."""
+        assert not Xb.is_cuda and not yb.is_cuda and Xb.is_contiguous() and yb.is_contiguous()
+        assert Xb.dtype == torch.float32 and Xb.numel() == self.m * self.batch * self.spec.dims[0]
+        assert yb.numel() == self.m * self.batch and yb.element_size() == 4
+        _check(self.lib, self.lib.olsgd_local_step_host(
+            self.ctx, Xb.data_ptr(), yb.data_ptr(), loss.data_ptr() if loss is not None else None),
+            self.ctx)
+
+    def join(self):
+        _check(self.lib, self.lib.olsgd_join(self.ctx), self.ctx)
 
     def period_sync(self):
         _check(self.lib, self.lib.olsgd_period_sync(self.ctx), self.ctx)

@@ -42,10 +42,16 @@ struct olsgd_ctx {
   float* tmp = nullptr;              // [ld] scratch for olsgd_get_params
   __nv_bfloat16* shadow = nullptr;   // bf16 copy of x_k [m][ld] (tensor-core path)
   int32_t* idx = nullptr;            // [m][batch]
+  int32_t* ident = nullptr;          // [m][batch], ident[i][j] = j
+  float* stage_x[2] = {nullptr, nullptr};  // host-fed minibatches [m][batch][d_in]
+  void* stage_y[2] = {nullptr, nullptr};   // [m][batch] targets / labels
   ModelBuffers mb;
 
   cudaStream_t main = nullptr, side = nullptr;
+  cudaStream_t copy = nullptr;       // owned: host-to-device staging copies
   cudaEvent_t pullback_done = nullptr, reduce_done = nullptr;
+  cudaEvent_t h2d_done[2] = {nullptr, nullptr}, stage_free[2] = {nullptr, nullptr};
+  int host_slot = 0;
   bool reduce_pending = false;  // an anchor refresh was launched and not yet waited for
   int reduce_reads = -1;        // which x buffer that refresh reads
   bool need_sync = false;       // a period ended; olsgd_period_sync is due
@@ -117,6 +123,22 @@ struct Launch {
   }
 };
 
+void free_host_side(olsgd_ctx* c) {
+  for (auto& r : c->prof_pending) {
+    cudaEventDestroy(r.start);
+    cudaEventDestroy(r.stop);
+  }
+  for (auto e : c->prof_pool) cudaEventDestroy(e);
+  if (c->pullback_done) cudaEventDestroy(c->pullback_done);
+  if (c->reduce_done) cudaEventDestroy(c->reduce_done);
+  for (int b = 0; b < 2; ++b) {
+    if (c->h2d_done[b]) cudaEventDestroy(c->h2d_done[b]);
+    if (c->stage_free[b]) cudaEventDestroy(c->stage_free[b]);
+  }
+  if (c->copy) cudaStreamDestroy(c->copy);
+  delete c;
+}
+
 ProfHook make_hook(olsgd_ctx* c) {
   ProfHook hook;
   hook.ctx = c;
@@ -130,7 +152,8 @@ ProfHook make_hook(olsgd_ctx* c) {
 struct Plan {
   int64_t P = 0, ld = 0;
   size_t off_x0 = 0, off_x1 = 0, off_u = 0, off_g = 0, off_z = 0, off_v = 0, off_tmp = 0,
-         off_shadow = 0, off_idx = 0, off_model = 0, total = 0;
+         off_shadow = 0, off_idx = 0, off_ident = 0, off_stage_x[2] = {0, 0},
+         off_stage_y[2] = {0, 0}, off_model = 0, total = 0;
   bool has_u = false, has_g = false, has_shadow = false;
   ModelPlan mp;
 };
@@ -208,6 +231,13 @@ olsgd_status make_plan(const olsgd_model_spec* spec, const olsgd_hparams* hp, Pl
   pl->off_tmp = take(row);
   pl->off_shadow = pl->has_shadow ? take((size_t)pl->ld * m * sizeof(__nv_bfloat16)) : 0;
   pl->off_idx = pl->has_g ? take((size_t)m * hp->batch * sizeof(int32_t)) : 0;
+  if (pl->has_g) {
+    pl->off_ident = take((size_t)m * hp->batch * sizeof(int32_t));
+    for (int b = 0; b < 2; ++b) {
+      pl->off_stage_x[b] = take((size_t)m * hp->batch * spec->dims[0] * sizeof(float));
+      pl->off_stage_y[b] = take((size_t)m * hp->batch * sizeof(int32_t));
+    }
+  }
   pl->off_model = off;
   if (pl->has_g) {
     if (!plan_model(*spec, *hp, &pl->mp)) return fail(nullptr, OLSGD_EINVAL, "%s", pl->mp.error);
@@ -266,6 +296,31 @@ olsgd_status apply_update(olsgd_ctx* c, const float* g, int64_t ldg) {
   c->cur = nxt;
   c->k += 1;
   if (sync) c->need_sync = true;
+  return OLSGD_OK;
+}
+
+// S2-S6 of one iteration on the main stream, reading the minibatch rows
+// idx[i][:] of `data`.  stage_slot >= 0 marks a host-fed staging slot to release.
+olsgd_status step_body(olsgd_ctx* c, const olsgd_data& data, const int32_t* idx,
+                       float* loss_device, int stage_slot) {
+  StepIO io;
+  io.x = c->x[c->cur];
+  io.shadow = c->shadow;
+  io.g = c->g;
+  io.ld = c->ld;
+  io.idx = idx;
+  io.loss = loss_device;
+  const ProfHook hook = make_hook(c);
+  cudaError_t e = model_forward_backward(c->spec, c->hp, data, c->mb, io, c->main, hook);
+  if (e != cudaSuccess)
+    return fail(c, OLSGD_ECUDA, "forward/backward failed: %s", cudaGetErrorString(e));
+  if (stage_slot >= 0) OLSGD_CUDA(c, cudaEventRecord(c->stage_free[stage_slot], c->main));
+  // S5-S6
+  olsgd_status st = apply_update(c, c->g, c->ld);
+  if (st != OLSGD_OK) return st;
+  e = model_post_update(c->spec, c->hp, c->mb, c->shadow, c->ld, c->main, hook);
+  if (e != cudaSuccess)
+    return fail(c, OLSGD_ECUDA, "post-update failed: %s", cudaGetErrorString(e));
   return OLSGD_OK;
 }
 
@@ -335,12 +390,17 @@ olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const ols
   c->tmp = reinterpret_cast<float*>(ws + pl.off_tmp);
   c->shadow = pl.has_shadow ? reinterpret_cast<__nv_bfloat16*>(ws + pl.off_shadow) : nullptr;
   c->idx = pl.has_g ? reinterpret_cast<int32_t*>(ws + pl.off_idx) : nullptr;
+  if (pl.has_g) {
+    c->ident = reinterpret_cast<int32_t*>(ws + pl.off_ident);
+    for (int b = 0; b < 2; ++b) {
+      c->stage_x[b] = reinterpret_cast<float*>(ws + pl.off_stage_x[b]);
+      c->stage_y[b] = ws + pl.off_stage_y[b];
+    }
+  }
 
   auto bail = [&](olsgd_status s) {
-    if (c->pullback_done) cudaEventDestroy(c->pullback_done);
-    if (c->reduce_done) cudaEventDestroy(c->reduce_done);
     g_last_error = c->err;
-    delete c;
+    free_host_side(c);
     return s;
   };
 #define OLSGD_INIT_CUDA(call)                                                               \
@@ -352,6 +412,13 @@ olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const ols
 
   OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->pullback_done, cudaEventDisableTiming));
   OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->reduce_done, cudaEventDisableTiming));
+  if (pl.has_g) {
+    OLSGD_INIT_CUDA(cudaStreamCreateWithFlags(&c->copy, cudaStreamNonBlocking));
+    for (int b = 0; b < 2; ++b) {
+      OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->h2d_done[b], cudaEventDisableTiming));
+      OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->stage_free[b], cudaEventDisableTiming));
+    }
+  }
   // zero everything once (padding, momentum buffers, gradient padding), then
   // x_0^(i) = z_0 = x0
   OLSGD_INIT_CUDA(cudaMemsetAsync(ws, 0, pl.total, c->main));
@@ -361,6 +428,10 @@ olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const ols
                                     cudaMemcpyDeviceToDevice, c->main));
   OLSGD_INIT_CUDA(cudaMemcpyAsync(c->z, x0_device, pbytes, cudaMemcpyDeviceToDevice, c->main));
   if (pl.has_g) {
+    {
+      Launch l(c, OLSGD_KC_INDEX, c->main);
+      OLSGD_INIT_CUDA(launch_identity_indices(c->ident, c->hp.m, c->hp.batch, c->main));
+    }
     if (!bind_model(c->spec, c->hp, pl.mp, ws + pl.off_model, &c->mb)) {
       return bail(fail(c, OLSGD_EINVAL, "%s", c->mb.error));
     }
@@ -400,24 +471,44 @@ olsgd_status olsgd_local_step(olsgd_ctx* c, float* loss_device) {
     OLSGD_CUDA(c, launch_minibatch_indices(c->idx, c->hp.seed, c->hp.m, c->k, c->hp.batch,
                                            c->data.n_per_worker, c->main));
   }
-  // S2-S4: gather, forward, loss, backward -> g [m][ld]
-  StepIO io;
-  io.x = c->x[c->cur];
-  io.shadow = c->shadow;
-  io.g = c->g;
-  io.ld = c->ld;
-  io.idx = c->idx;
-  io.loss = loss_device;
-  const ProfHook hook = make_hook(c);
-  cudaError_t e = model_forward_backward(c->spec, c->hp, c->data, c->mb, io, c->main, hook);
-  if (e != cudaSuccess)
-    return fail(c, OLSGD_ECUDA, "forward/backward failed: %s", cudaGetErrorString(e));
-  // S5-S6
-  olsgd_status st = apply_update(c, c->g, c->ld);
+  return step_body(c, c->data, c->idx, loss_device, -1);
+}
+
+olsgd_status olsgd_local_step_host(olsgd_ctx* c, const float* Xb_host, const void* yb_host,
+                                   float* loss_host) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  if (c->spec.kind == OLSGD_FLAT)
+    return fail(c, OLSGD_ESTATE, "OLSGD_FLAT contexts take olsgd_local_step_with_grads");
+  if (!Xb_host || !yb_host) return fail(c, OLSGD_EINVAL, "host minibatch pointers are NULL");
+  if (c->need_sync) return fail(c, OLSGD_ESTATE, "a period ended: call olsgd_period_sync first");
+  const int slot = c->host_slot;
+  c->host_slot ^= 1;
+  const size_t rows = (size_t)c->hp.m * c->hp.batch;
+  // the kernels that read this slot two steps ago must be done before it is refilled
+  OLSGD_CUDA(c, cudaStreamWaitEvent(c->copy, c->stage_free[slot], 0));
+  OLSGD_CUDA(c, cudaMemcpyAsync(c->stage_x[slot], Xb_host, rows * c->spec.dims[0] * sizeof(float),
+                                cudaMemcpyHostToDevice, c->copy));
+  OLSGD_CUDA(c, cudaMemcpyAsync(c->stage_y[slot], yb_host, rows * 4, cudaMemcpyHostToDevice, c->copy));
+  OLSGD_CUDA(c, cudaEventRecord(c->h2d_done[slot], c->copy));
+  OLSGD_CUDA(c, cudaStreamWaitEvent(c->main, c->h2d_done[slot], 0));
+  olsgd_data staged;
+  staged.X = c->stage_x[slot];
+  staged.y = c->stage_y[slot];
+  staged.n_per_worker = c->hp.batch;
+  olsgd_status st = step_body(c, staged, c->ident, nullptr, slot);
   if (st != OLSGD_OK) return st;
-  e = model_post_update(c->spec, c->hp, c->mb, c->shadow, c->ld, c->main, hook);
-  if (e != cudaSuccess)
-    return fail(c, OLSGD_ECUDA, "post-update failed: %s", cudaGetErrorString(e));
+  if (loss_host)
+    OLSGD_CUDA(c, cudaMemcpyAsync(loss_host, c->mb.loss, (size_t)c->hp.m * sizeof(float),
+                                  cudaMemcpyDeviceToHost, c->main));
+  return OLSGD_OK;
+}
+
+olsgd_status olsgd_join(olsgd_ctx* c) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  if (c->copy) OLSGD_CUDA(c, cudaStreamSynchronize(c->copy));
+  OLSGD_CUDA(c, cudaStreamSynchronize(c->side));
+  OLSGD_CUDA(c, cudaStreamSynchronize(c->main));
+  c->reduce_pending = false;
   return OLSGD_OK;
 }
 
@@ -562,16 +653,10 @@ const char* olsgd_last_error(const olsgd_ctx* c) {
 
 olsgd_status olsgd_destroy(olsgd_ctx* c) {
   if (!c) return OLSGD_OK;
+  if (c->copy) cudaStreamSynchronize(c->copy);
   cudaStreamSynchronize(c->side);
   cudaStreamSynchronize(c->main);
-  for (auto& r : c->prof_pending) {
-    cudaEventDestroy(r.start);
-    cudaEventDestroy(r.stop);
-  }
-  for (auto e : c->prof_pool) cudaEventDestroy(e);
-  if (c->pullback_done) cudaEventDestroy(c->pullback_done);
-  if (c->reduce_done) cudaEventDestroy(c->reduce_done);
-  delete c;
+  free_host_side(c);
   return OLSGD_OK;
 }
 

@@ -47,6 +47,8 @@ cudaError_t launch_virtual_sequence(const float* x, const float* z, float* dst, 
 cudaError_t launch_minibatch_indices(int32_t* idx, uint64_t seed, int m, int64_t k, int batch,
                                      int64_t n, cudaStream_t s);
 cudaError_t launch_class_pairs(int32_t* dst, uint64_t seed, int m, cudaStream_t s);
+// idx[i][j] = j: the "indices" of a minibatch that is already contiguous
+cudaError_t launch_identity_indices(int32_t* idx, int m, int batch, cudaStream_t s);
 
 // ---- simt_kernels.cu --------------------------------------------------------
 constexpr int kMaxClasses = 32;  // the output layer is handled by one warp per row

@@ -67,7 +67,18 @@ __global__ void class_pairs_kernel(int32_t* __restrict__ dst, uint32_t k0, uint3
   }
 }
 
+__global__ void identity_indices_kernel(int32_t* __restrict__ idx, int total, int batch) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < total) idx[t] = t % batch;
+}
+
 }  // namespace
+
+cudaError_t launch_identity_indices(int32_t* idx, int m, int batch, cudaStream_t s) {
+  const int total = m * batch, threads = 256;
+  identity_indices_kernel<<<(total + threads - 1) / threads, threads, 0, s>>>(idx, total, batch);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_minibatch_indices(int32_t* idx, uint64_t seed, int m, int64_t k, int batch,
                                      int64_t n, cudaStream_t s) {

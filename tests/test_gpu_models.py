@@ -91,3 +91,40 @@ def test_local_step_and_period_sync_equal_run():
     xa, za, _ = a.state()
     xb, zb, _ = b.state()
     assert np.array_equal(xa, xb) and np.array_equal(za, zb)
+
+
+# ------------------------------------------------------------------ bf16 MLP path
+# gemm_bf16 = 1: tcgen05 tensor-core GEMMs; 2: the same bf16 data flow on CUDA cores.
+# The oracle runs with bf16-rounded GEMM operands, so what is left is fp32-vs-fp64
+# accumulation and the occasional operand that rounds to the neighbouring bf16
+# value (2^-8 relative) on one side only.
+TOL_BF16_PARAM = 5e-3
+TOL_BF16_LOSS = 2e-2
+
+
+def _mlp_case(dims, m, n, batch, tau, iters, gemm_bf16, seed=8):
+    X, y = si.mixture_data(seed, m, n, dims[0])
+    y = (y % dims[-1]).astype(np.int32)
+    x0 = si.model_init(seed, "mlp", dims)
+    return _pair("mlp", dims, X, y, x0, m=m, tau=tau, batch=batch, gamma=0.05, alpha=0.6,
+                 beta=0.9, mu=0.9, seed=seed, iters=iters, gemm_bf16=gemm_bf16, bf16_oracle=True)
+
+
+MLP_SHAPES = [([64, 128, 10], 2, 40, 64, 2, 5),
+              ([192, 256, 128, 7], 3, 100, 64, 2, 5),
+              ([128, 128, 128, 128, 10], 2, 150, 128, 3, 7)]
+
+
+@pytest.mark.parametrize("dims,m,n,batch,tau,iters", MLP_SHAPES)
+@pytest.mark.parametrize("gemm_bf16", [2, 1])
+def test_mlp_bf16_small(dims, m, n, batch, tau, iters, gemm_bf16):
+    opt, st, lg, lo = _mlp_case(dims, m, n, batch, tau, iters, gemm_bf16)
+    assert np.isfinite(lg).all()
+    assert np.abs(lg - lo).max() <= TOL_BF16_LOSS * np.abs(lo).max()
+    assert state_err(opt, st) <= TOL_BF16_PARAM
+
+
+def test_mlp_cuda_core_path_accepts_small_batches():
+    opt, st, lg, lo = _mlp_case([64, 128, 10], 2, 40, 8, 2, 4, 2)
+    assert np.abs(lg - lo).max() <= TOL_BF16_LOSS * np.abs(lo).max()
+    assert state_err(opt, st) <= TOL_BF16_PARAM
