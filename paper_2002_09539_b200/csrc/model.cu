@@ -29,7 +29,8 @@ inline int n_layers(const olsgd_model_spec& s) { return s.n_dims - 1; }
 // data flow on CUDA cores (validation of the tensor-core kernels)
 inline bool bf16_path(const olsgd_model_spec& s) { return s.kind == OLSGD_MLP && s.gemm_bf16 != 0; }
 
-cudaError_t run_gemm(const olsgd_model_spec& spec, const GemmArgs& ga, cudaStream_t s) {
+cudaError_t run_gemm(const olsgd_model_spec& spec, GemmArgs ga, int* status, cudaStream_t s) {
+  ga.status = status;
   if (spec.gemm_bf16 == 1) return launch_gemm_tc(ga, s);
   return launch_gemm_simt(ga, s);
 }
@@ -179,7 +180,7 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
     ga.out_t = mb.ht[l];
     ga.out_n = mb.h[l];
     Scope sc(hook, OLSGD_KC_FORWARD, s);
-    OLSGD_TRY(run_gemm(spec, ga, s));
+    OLSGD_TRY(run_gemm(spec, ga, io.status, s));
   }
 
   // output layer: forward, loss, and backward to its input
@@ -230,7 +231,7 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
     gw.out_batch = io.ld;
     {
       Scope sc(hook, OLSGD_KC_BACKWARD, s);
-      OLSGD_TRY(run_gemm(spec, gw, s));
+      OLSGD_TRY(run_gemm(spec, gw, io.status, s));
     }
     {
       Scope sc(hook, OLSGD_KC_BACKWARD, s);
@@ -254,7 +255,7 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
       gd.out_t = mb.dat[l - 1];
       gd.out_n = mb.da[l - 1];
       Scope sc(hook, OLSGD_KC_BACKWARD, s);
-      OLSGD_TRY(run_gemm(spec, gd, s));
+      OLSGD_TRY(run_gemm(spec, gd, io.status, s));
     }
   }
   return cudaSuccess;

@@ -43,6 +43,7 @@ struct olsgd_ctx {
   __nv_bfloat16* shadow = nullptr;   // bf16 copy of x_k [m][ld] (tensor-core path)
   int32_t* idx = nullptr;            // [m][batch]
   int32_t* ident = nullptr;          // [m][batch], ident[i][j] = j
+  int* dev_status = nullptr;         // one word: a kernel's bounded wait gave up
   float* stage_x[2] = {nullptr, nullptr};  // host-fed minibatches [m][batch][d_in]
   void* stage_y[2] = {nullptr, nullptr};   // [m][batch] targets / labels
   ModelBuffers mb;
@@ -152,7 +153,7 @@ ProfHook make_hook(olsgd_ctx* c) {
 struct Plan {
   int64_t P = 0, ld = 0;
   size_t off_x0 = 0, off_x1 = 0, off_u = 0, off_g = 0, off_z = 0, off_v = 0, off_tmp = 0,
-         off_shadow = 0, off_idx = 0, off_ident = 0, off_stage_x[2] = {0, 0},
+         off_shadow = 0, off_idx = 0, off_ident = 0, off_status = 0, off_stage_x[2] = {0, 0},
          off_stage_y[2] = {0, 0}, off_model = 0, total = 0;
   bool has_u = false, has_g = false, has_shadow = false;
   ModelPlan mp;
@@ -229,6 +230,7 @@ olsgd_status make_plan(const olsgd_model_spec* spec, const olsgd_hparams* hp, Pl
   pl->off_z = take(row);
   pl->off_v = take(row);
   pl->off_tmp = take(row);
+  pl->off_status = take(sizeof(int));
   pl->off_shadow = pl->has_shadow ? take((size_t)pl->ld * m * sizeof(__nv_bfloat16)) : 0;
   pl->off_idx = pl->has_g ? take((size_t)m * hp->batch * sizeof(int32_t)) : 0;
   if (pl->has_g) {
@@ -310,6 +312,7 @@ olsgd_status step_body(olsgd_ctx* c, const olsgd_data& data, const int32_t* idx,
   io.ld = c->ld;
   io.idx = idx;
   io.loss = loss_device;
+  io.status = c->dev_status;
   const ProfHook hook = make_hook(c);
   cudaError_t e = model_forward_backward(c->spec, c->hp, data, c->mb, io, c->main, hook);
   if (e != cudaSuccess)
@@ -327,6 +330,15 @@ olsgd_status step_body(olsgd_ctx* c, const olsgd_data& data, const int32_t* idx,
 olsgd_status copy_out(olsgd_ctx* c, void* dst, const void* src, size_t bytes) {
   OLSGD_CUDA(c, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDefault, c->main));
   OLSGD_CUDA(c, cudaStreamSynchronize(c->main));
+  return OLSGD_OK;
+}
+
+// Reads the device status word; both streams must be idle.
+olsgd_status check_device_status(olsgd_ctx* c) {
+  int st = 0;
+  OLSGD_CUDA(c, cudaMemcpy(&st, c->dev_status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (st != 0)
+    return fail(c, (olsgd_status)st, "a kernel gave up waiting on a barrier (status %d)", st);
   return OLSGD_OK;
 }
 
@@ -388,6 +400,7 @@ olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const ols
   c->z = reinterpret_cast<float*>(ws + pl.off_z);
   c->v = reinterpret_cast<float*>(ws + pl.off_v);
   c->tmp = reinterpret_cast<float*>(ws + pl.off_tmp);
+  c->dev_status = reinterpret_cast<int*>(ws + pl.off_status);
   c->shadow = pl.has_shadow ? reinterpret_cast<__nv_bfloat16*>(ws + pl.off_shadow) : nullptr;
   c->idx = pl.has_g ? reinterpret_cast<int32_t*>(ws + pl.off_idx) : nullptr;
   if (pl.has_g) {
@@ -509,7 +522,7 @@ olsgd_status olsgd_join(olsgd_ctx* c) {
   OLSGD_CUDA(c, cudaStreamSynchronize(c->side));
   OLSGD_CUDA(c, cudaStreamSynchronize(c->main));
   c->reduce_pending = false;
-  return OLSGD_OK;
+  return check_device_status(c);
 }
 
 olsgd_status olsgd_period_sync(olsgd_ctx* c) {
@@ -565,6 +578,10 @@ olsgd_status olsgd_get_params(olsgd_ctx* c, int32_t which, float* dst, size_t n_
   OLSGD_CUDA(c, cudaStreamSynchronize(c->side));
   c->reduce_pending = false;
   OLSGD_CUDA(c, cudaStreamSynchronize(c->main));
+  {
+    olsgd_status ds = check_device_status(c);
+    if (ds != OLSGD_OK) return ds;
+  }
   const size_t bytes = (size_t)c->P * sizeof(float);
   const float* xk = c->x[c->cur];
   if (which >= 0) return copy_out(c, dst, xk + (int64_t)which * c->ld, bytes);

@@ -132,6 +132,7 @@ struct GemmArgs {
   __nv_bfloat16* out_n;      // [m][Nb][Ma]
   float* out_f;              // STORE_F32: out_f[i * out_batch + row * ldo + col]
   int64_t ldo, out_batch;
+  int* status;               // device word that receives OLSGD_ETIMEOUT if a bounded wait gives up
 };
 // Plain CUDA-core version, used to validate the tensor-core kernel.
 cudaError_t launch_gemm_simt(const GemmArgs& a, cudaStream_t s);
@@ -170,6 +171,7 @@ struct StepIO {
   int64_t ld;
   const int32_t* idx;            // [m][batch]
   float* loss;                   // out: [m] or null
+  int* status;                   // device status word (see GemmArgs::status)
 };
 // Lets model.cu count and time its launches without knowing the context type.
 struct ProfHook {

@@ -1,6 +1,455 @@
-// Placeholder until the tcgen05 kernel lands.
+// Worker-batched bf16 GEMM on the fifth-generation tensor cores (sm_100a):
+//   D[i] = A[i] * B[i]^T,  A [Ma][K] and B [Nb][K] both K-major, fp32 accumulate.
+//
+// One CTA computes one 128 x BN tile of one worker's D.  Operand tiles of 64 K
+// elements (128 bytes per row) are brought in by TMA with the 128-byte swizzle
+// into a ring of shared-memory stages; one elected thread issues tcgen05.mma
+// (M = 128, N = BN, K = 16 per instruction) with the accumulator in tensor
+// memory; four warps read the accumulator back with tcgen05.ld and run the
+// epilogue (bias + ReLU, ReLU mask, or fp32 store).
+//
+// Warp roles (192 threads): warp 0 TMA producer, warp 1 MMA issuer and owner
+// of the tensor-memory allocation, warps 2-5 epilogue (warp w reads the 32
+// TMEM lanes of group w % 4).
+//
+// Every wait on an mbarrier is bounded.  A wait that runs out raises a flag in
+// shared memory that all roles poll, records OLSGD_ETIMEOUT in the status word
+// the host reads, and the CTA drains its own copies, frees its tensor memory
+// and returns.
+#include <cuda.h>
+
+#include <mutex>
+
 #include "olsgd_internal.h"
+
 namespace olsgd {
-bool gemm_tc_supported(const GemmArgs&) { return false; }
-cudaError_t launch_gemm_tc(const GemmArgs&, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+constexpr int kBM = 128;          // rows of A per tile = MMA M = TMEM lanes
+constexpr int kBK = 64;           // K elements per stage = one 128-byte swizzle row
+constexpr int kUmmaK = 16;        // K per tcgen05.mma for 16-bit operands
+constexpr int kThreads = 192;
+constexpr uint32_t kSpinLimit = 1u << 22;          // iterations, for the drain loops
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // wall-clock bound of one barrier wait
+
+// ------------------------------------------------------------------ PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t"
+      "}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded wait.  Returns false when it gave up or another role already did.
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  uint64_t t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 63u) {
+      if (*abort_flag) return false;
+      const uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) break;
+    }
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                            int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t holder, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder),
+               "r"(cols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols)
+               : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+
+// Arrives on the mbarrier once every MMA issued so far by this thread is done.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
+      "}" ::"r"(tmem_d),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes
+// (64 bf16) with the 128-byte swizzle: rows 128 B apart, groups of eight rows
+// 1024 B apart (stride byte offset), descriptor version 1, layout type 2.
+__device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);   // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                    // leading byte offset (unused for this layout)
+  d |= (uint64_t)(1024 >> 4) << 32;          // stride byte offset
+  d |= (uint64_t)1 << 46;                    // descriptor version
+  d |= (uint64_t)2 << 61;                    // SWIZZLE_128B
+  return d;
+}
+
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = bn.
+__host__ __device__ constexpr uint32_t instr_desc_bf16(int bn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) |
+         ((uint32_t)(kBM >> 4) << 24);
+}
+
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+        "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
+        "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+}
+
+struct EpiArgs {
+  int epilogue;
+  int Ma, Nb;
+  const float* bias;
+  int64_t bias_batch;
+  const __nv_bfloat16* mask;
+  __nv_bfloat16* out_t;
+  __nv_bfloat16* out_n;
+  float* out_f;
+  int64_t ldo, out_batch;
+  int* status;
+};
+
+struct SharedCtl {
+  uint64_t full[8];
+  uint64_t empty[8];
+  uint64_t tmem_full;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+template <int BN, int STAGES>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               int num_kb, EpiArgs ea) {
+  constexpr uint32_t kABytes = kBM * kBK * 2;
+  constexpr uint32_t kBBytes = BN * kBK * 2;
+  constexpr uint32_t kStageBytes = kABytes + kBBytes;
+  constexpr uint32_t kTmemCols = BN < 32 ? 32 : BN;  // power of two for BN in {64,128,256}
+
+  extern __shared__ uint8_t smem_raw[];
+  // operand tiles need 1024-byte alignment for the 128-byte swizzle
+  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                              ~static_cast<uintptr_t>(1023));
+  SharedCtl* ctl = reinterpret_cast<SharedCtl*>(tiles + STAGES * kStageBytes);
+  volatile int* abort_flag = &ctl->abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * BN, m0 = blockIdx.y * kBM, worker = blockIdx.z;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&ctl->full[s]), 1);
+      mbar_init(smem_u32(&ctl->empty[s]), 1);
+    }
+    mbar_init(smem_u32(&ctl->tmem_full), 1);
+    ctl->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+
+  if (warp == 0 && lane == 0) {
+    // ---------------- TMA producer
+    int issued = 0;
+    for (int kb = 0; kb < num_kb; ++kb) {
+      const int s = kb % STAGES;
+      const uint32_t ph = (kb / STAGES) & 1;
+      if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1, abort_flag)) break;
+      const uint32_t full = smem_u32(&ctl->full[s]);
+      mbar_expect_tx(full, kStageBytes);
+      const uint32_t a_dst = smem_u32(tiles + s * kStageBytes);
+      tma_load_3d(a_dst, &map_a, full, kb * kBK, m0, worker);
+      tma_load_3d(a_dst + kABytes, &map_b, full, kb * kBK, n0, worker);
+      issued = kb + 1;
+    }
+    if (*abort_flag) {
+      // drain: wait (bounded) for the copies this thread still has in flight
+      for (int kb = max(0, issued - STAGES); kb < issued; ++kb) {
+        const uint32_t full = smem_u32(&ctl->full[kb % STAGES]);
+        const uint32_t ph = (kb / STAGES) & 1;
+        for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(full, ph); ++it) {
+          if ((it & 1023u) == 1023u && global_ns() == 0) break;  // keeps the loop observable
+        }
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---------------- MMA issuer
+    constexpr uint32_t idesc = instr_desc_bf16(BN);
+    bool ok = true;
+    for (int kb = 0; kb < num_kb && ok; ++kb) {
+      const int s = kb % STAGES;
+      const uint32_t ph = (kb / STAGES) & 1;
+      ok = mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t a_addr = smem_u32(tiles + s * kStageBytes);
+      const uint64_t a_desc = smem_desc_k_sw128(a_addr);
+      const uint64_t b_desc = smem_desc_k_sw128(a_addr + kABytes);
+#pragma unroll
+      for (int k = 0; k < kBK / kUmmaK; ++k) {
+        // 16 K elements = 32 bytes = 2 units of the descriptor's start address
+        umma_bf16(tmem_base, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                  (kb > 0 || k > 0) ? 1u : 0u);
+      }
+      umma_commit(smem_u32(&ctl->empty[s]));  // stage reusable once these MMAs retire
+    }
+    umma_commit(smem_u32(&ctl->tmem_full));   // accumulator complete
+  } else if (warp >= 2) {
+    // ---------------- epilogue: TMEM lane r <-> row m0 + r, column j <-> col n0 + j
+    if (mbar_wait(smem_u32(&ctl->tmem_full), 0, abort_flag) && !*abort_flag) {
+      tc_fence_after();
+      const int lane_group = warp & 3;
+      const int row = m0 + lane_group * 32 + lane;
+      const int64_t wk = worker;
+      float bias = 0.f;
+      if (ea.epilogue == GEMM_EPI_BIAS_RELU) bias = ea.bias[wk * ea.bias_batch + row];
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        float v[32];
+        tmem_ld32(tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)(c * 32), v);
+        const int col0 = n0 + c * 32;
+        if (ea.epilogue == GEMM_EPI_STORE_F32) {
+          float4* dst = reinterpret_cast<float4*>(ea.out_f + wk * ea.out_batch +
+                                                  (int64_t)row * ea.ldo + col0);
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+        } else {
+          const int64_t t_off = (wk * ea.Ma + row) * ea.Nb + col0;
+          if (ea.epilogue == GEMM_EPI_BIAS_RELU) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j] + bias, 0.f);
+          } else {
+            const uint4* mk = reinterpret_cast<const uint4*>(ea.mask + t_off);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const uint4 w = mk[q];
+              const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                // a bf16 is positive iff its sign bit is clear and it is not zero
+                const uint32_t lo = ws[e] & 0xFFFFu, hi = ws[e] >> 16;
+                if (!(lo != 0 && lo < 0x8000u)) v[q * 8 + e * 2] = 0.f;
+                if (!(hi != 0 && hi < 0x8000u)) v[q * 8 + e * 2 + 1] = 0.f;
+              }
+            }
+          }
+          uint32_t pk[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+            pk[j] = *reinterpret_cast<uint32_t*>(&b2);
+          }
+          if (ea.out_t) {
+            uint4* dst = reinterpret_cast<uint4*>(ea.out_t + t_off);
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              dst[q] = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+          }
+          if (ea.out_n) {
+            // [Nb][Ma]: for a fixed column the 32 lanes of the warp write 32 consecutive rows
+            __nv_bfloat16* dst = ea.out_n + (wk * ea.Nb + col0) * ea.Ma + row;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const uint32_t w = pk[j >> 1];
+              const uint16_t h = (j & 1) ? (uint16_t)(w >> 16) : (uint16_t)(w & 0xFFFFu);
+              *reinterpret_cast<uint16_t*>(dst + (int64_t)j * ea.Ma) = h;
+            }
+          }
+        }
+      }
+    }
+  }
+
+  // ---------------- teardown: every role arrives here, all waits above are bounded
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    if (lane == 0 && *abort_flag) {
+      // let the MMAs that were issued retire before the tensor memory is released
+      for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(smem_u32(&ctl->tmem_full), 0); ++it) {
+      }
+    }
+    __syncwarp();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+  if (threadIdx.x == 0 && *abort_flag && ea.status) atomicExch(ea.status, (int)OLSGD_ETIMEOUT);
+}
+
+// ------------------------------------------------------------------ host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+// [m][rows][K] bf16, K contiguous, as a 3-D tensor map with a (64, box_rows, 1) box.
+bool make_map(CUtensorMap* map, const __nv_bfloat16* base, int64_t K, int64_t rows, int64_t m,
+              int64_t ld, int64_t batch, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)m};
+  cuuint64_t strides[2] = {(cuuint64_t)ld * 2, (cuuint64_t)batch * 2};
+  cuuint32_t box[3] = {(cuuint32_t)kBK, (cuuint32_t)box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(base), dims,
+            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int pick_bn(int Nb) {
+  if (Nb % 256 == 0) return 256;
+  if (Nb % 128 == 0) return 128;
+  if (Nb % 64 == 0) return 64;
+  return 0;
+}
+
+template <int BN, int STAGES>
+cudaError_t launch_one(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMap& mb,
+                       cudaStream_t s) {
+  constexpr size_t smem = (size_t)STAGES * (kBM * kBK * 2 + BN * kBK * 2) + sizeof(SharedCtl) + 1024;
+  static bool configured = false;
+  auto kern = gemm_tc_kernel<BN, STAGES>;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  EpiArgs ea;
+  ea.epilogue = a.epilogue;
+  ea.Ma = a.Ma;
+  ea.Nb = a.Nb;
+  ea.bias = a.bias;
+  ea.bias_batch = a.bias_batch;
+  ea.mask = a.mask;
+  ea.out_t = a.out_t;
+  ea.out_n = a.out_n;
+  ea.out_f = a.out_f;
+  ea.ldo = a.ldo;
+  ea.out_batch = a.out_batch;
+  ea.status = a.status;
+  dim3 grid(a.Nb / BN, a.Ma / kBM, a.m);
+  kern<<<grid, kThreads, smem, s>>>(ma, mb, a.K / kBK, ea);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool gemm_tc_supported(const GemmArgs& a) {
+  auto al16 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; };
+  if (a.Ma % kBM != 0 || a.K % kBK != 0 || a.K < kBK || pick_bn(a.Nb) == 0) return false;
+  if (a.lda % 8 || a.ldb % 8 || a.a_batch % 8 || a.b_batch % 8) return false;
+  if (!al16(a.A) || !al16(a.B)) return false;
+  if (a.epilogue == GEMM_EPI_STORE_F32) {
+    if (!al16(a.out_f) || a.ldo % 4 || a.out_batch % 4) return false;
+  } else {
+    if ((a.out_t && !al16(a.out_t)) || a.Nb % 8) return false;
+    if (a.epilogue == GEMM_EPI_RELU_MASK && !al16(a.mask)) return false;
+  }
+  return true;
+}
+
+cudaError_t launch_gemm_tc(const GemmArgs& a, cudaStream_t s) {
+  if (!gemm_tc_supported(a)) return cudaErrorInvalidValue;
+  const int bn = pick_bn(a.Nb);
+  CUtensorMap ma, mb;
+  if (!make_map(&ma, a.A, a.K, a.Ma, a.m, a.lda, a.a_batch, kBM)) return cudaErrorInvalidValue;
+  if (!make_map(&mb, a.B, a.K, a.Nb, a.m, a.ldb, a.b_batch, bn)) return cudaErrorInvalidValue;
+  // short K (weight gradients, K = batch): few stages so several CTAs share an SM
+  const bool short_k = a.K / kBK <= 2;
+  switch (bn) {
+    case 256: return short_k ? launch_one<256, 2>(a, ma, mb, s) : launch_one<256, 4>(a, ma, mb, s);
+    case 128: return short_k ? launch_one<128, 2>(a, ma, mb, s) : launch_one<128, 6>(a, ma, mb, s);
+    default:  return short_k ? launch_one<64, 2>(a, ma, mb, s) : launch_one<64, 8>(a, ma, mb, s);
+  }
+}
+
 }  // namespace olsgd
