@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libolsgd.so")
 SOURCES = ["olsgd_api.cu", "update_kernels.cu", "sampling_kernels.cu", "simt_kernels.cu",
-           "model.cu", "tc_gemm.cu"]
+           "model.cu", "tc_gemm.cu", "tc_wgrad.cu"]
 
 
 def _stale():

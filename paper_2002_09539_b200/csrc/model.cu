@@ -31,7 +31,8 @@ inline bool bf16_path(const olsgd_model_spec& s) { return s.kind == OLSGD_MLP &&
 
 cudaError_t run_gemm(const olsgd_model_spec& spec, GemmArgs ga, int* status, cudaStream_t s) {
   ga.status = status;
-  if (spec.gemm_bf16 == 1) return launch_gemm_tc(ga, s);
+  if (spec.gemm_bf16 == 1)
+    return wgrad_tc_supported(ga) ? launch_wgrad_tc(ga, s) : launch_gemm_tc(ga, s);
   return launch_gemm_simt(ga, s);
 }
 

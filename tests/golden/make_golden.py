@@ -2,6 +2,10 @@
 
 Calls only the CPU oracle and the seeded input generators.  Usage:
     python tests/golden/make_golden.py c3 [c4 ...]
+    python tests/golden/make_golden.py c3 --perturb     (writes c3_perturbed.json)
+With --perturb the run starts from x0 with 1e-7 added to its first entry: the
+difference to the unperturbed result measures how far two correct fp64 runs of
+the same configuration drift apart, i.e. what no parity tolerance can beat.
 Each run takes tens of minutes (fp64, full data set, every iteration) and
 writes tests/golden/<name>_final.json with the final objective F of Eq. 1
 evaluated on every worker's whole partition at the mean model and at the
@@ -24,11 +28,15 @@ SEED = 0
 
 
 def main(names):
+    perturb = "--perturb" in names
+    names = [n for n in names if not n.startswith("--")]
     for name in names:
         c = si.CONFIGS[name]
         table = sampling.class_pairs(SEED, c["m"]) if c["non_iid"] else None
         X, y = si.mixture_data(SEED, c["m"], c["n"], c["dims"][0], table)
         x0 = si.model_init(SEED, c["kind"], c["dims"])
+        if perturb:
+            x0[0] += 1e-7
         t0 = time.time()
         st, losses, _ = runner.run_model(
             c["kind"], c["dims"], X, y, x0, m=c["m"], tau=c["tau"], batch=c["batch"],
@@ -37,7 +45,7 @@ def main(names):
         xbar = st.mean_model()
         probe = np.linspace(0, xbar.size - 1, 16).astype(np.int64)
         out = {
-            "config": name, "seed": SEED, "iters": c["iters"],
+            "config": name, "seed": SEED, "iters": c["iters"], "x0_perturbation": 1e-7 if perturb else 0.0,
             "oracle_seconds": round(time.time() - t0, 1),
             "F_mean_model": models.full_objective(c["kind"], c["dims"], xbar, X, y),
             "F_anchor": models.full_objective(c["kind"], c["dims"], st.z, X, y),
@@ -50,7 +58,7 @@ def main(names):
             "probe_mean_model": [float(v) for v in xbar[probe]],
             "probe_anchor": [float(v) for v in st.z[probe]],
         }
-        with open(os.path.join(HERE, name + "_final.json"), "w") as f:
+        with open(os.path.join(HERE, name + ("_perturbed.json" if perturb else "_final.json")), "w") as f:
             json.dump(out, f, indent=1)
             f.write("\n")
         print(name, "done in", out["oracle_seconds"], "s", flush=True)

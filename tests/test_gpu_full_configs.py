@@ -1,0 +1,141 @@
+"""The benchmark configurations at full size, in the launch configuration that
+bench.py times (tensor-core GEMMs, overlapped anchor refresh, olsgd_run)."""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+import synth_inputs as si
+from oracle import models, olsgd, runner, sampling
+from conftest import GOLDEN
+from helpers import max_rel_err, state_err, to_dev
+
+TOL_BF16_LOSS = 2e-2      # acceptance bar of the bf16-GEMM paths, relative, on the loss
+
+
+def _gpu(name, iters, table=None, seed=0):
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    c = si.CONFIGS[name]
+    if c["kind"] == "linreg":
+        X, y, _ = si.linreg_data(seed, c["m"], c["n"], c["dims"][0])
+    else:
+        X, y = si.mixture_data(seed, c["m"], c["n"], c["dims"][0], table)
+    x0 = si.model_init(seed, c["kind"], c["dims"])
+    opt = OverlapLocalSGD(c["kind"], m=c["m"], tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"],
+                          beta=c["beta"], mu=c["mu"], batch=c["batch"], seed=seed, dims=c["dims"],
+                          gemm_bf16=c["gemm_bf16"], x0=x0, X=to_dev(X), y=to_dev(y))
+    loss = torch.zeros((iters, c["m"]), device="cuda")
+    opt.run(iters, loss)
+    return c, X, y, x0, opt, loss.cpu().numpy()
+
+
+def _oracle(c, X, y, x0, iters, seed=0):
+    return runner.run_model(c["kind"], c["dims"], X, y, x0, m=c["m"], tau=c["tau"],
+                            batch=c["batch"], gamma=c["gamma"], alpha=c["alpha"], beta=c["beta"],
+                            mu=c["mu"], seed=seed, iters=iters)
+
+
+def test_config2_full_length():
+    c, X, y, x0, opt, lg = _gpu("c2", 500)
+    st, lo, _ = _oracle(c, X, y, x0, 500)
+    err = state_err(opt, st)
+    assert err <= 5e-5, err                       # the 1e-5 bar is stated at 100 iterations
+    assert np.abs(lg - lo).max() <= 1e-4 * np.abs(lo).max()
+    F_gpu = models.full_objective("softmax", c["dims"], opt.get_params(-4), X, y)
+    F_or = models.full_objective("softmax", c["dims"], st.mean_model(), X, y)
+    assert abs(F_gpu - F_or) <= 1e-5 * F_or
+
+
+@pytest.mark.parametrize("name,iters", [("c3", 12), ("c4", 16)])
+def test_mlp_configs_first_iterations_against_exact_oracle(name, iters):
+    table = None
+    if name == "c4":
+        from paper_2002_09539_b200 import class_pairs
+        table = class_pairs(0, si.CONFIGS[name]["m"], device="cpu").numpy()
+        assert np.array_equal(table, sampling.class_pairs(0, si.CONFIGS[name]["m"]))
+    c, X, y, x0, opt, lg = _gpu(name, iters, table)
+    st, lo, _ = _oracle(c, X, y, x0, iters)       # exact fp64, no operand rounding
+    assert np.isfinite(lg).all()
+    assert np.abs(lg - lo).max() <= TOL_BF16_LOSS * np.abs(lo).max()
+    # parameters: bf16 operand rounding perturbs each gradient by O(2^-8) relative
+    assert state_err(opt, st) <= 2e-2
+    xbar = opt.get_params(-4)
+    idx = np.random.default_rng(0).integers(0, X.shape[1], size=(c["m"], 256))
+    Xs = np.stack([X[i][idx[i]] for i in range(c["m"])])
+    ys = np.stack([y[i][idx[i]] for i in range(c["m"])])
+    F_gpu = models.full_objective("mlp", c["dims"], xbar, Xs, ys)
+    F_or = models.full_objective("mlp", c["dims"], st.mean_model(), Xs, ys)
+    assert abs(F_gpu - F_or) <= TOL_BF16_LOSS * F_or
+
+
+@pytest.mark.parametrize("name", ["c3", "c4"])
+def test_mlp_configs_full_length_final_loss(name):
+    path = os.path.join(GOLDEN, name + "_final.json")
+    if not os.path.exists(path):
+        pytest.skip("stored oracle result %s has not been generated yet" % path)
+    gold = json.load(open(path))
+    table = sampling.class_pairs(0, si.CONFIGS[name]["m"]) if name == "c4" else None
+    c, X, y, x0, opt, lg = _gpu(name, gold["iters"], table)
+    assert np.isfinite(lg).all()
+    xbar, z = opt.get_params(-4).copy(), opt.get_params(-1).copy()
+    F_mean = models.full_objective("mlp", c["dims"], xbar, X, y)
+    F_anchor = models.full_objective("mlp", c["dims"], z, X, y)
+    assert abs(F_mean - gold["F_mean_model"]) <= TOL_BF16_LOSS * gold["F_mean_model"]
+    assert abs(F_anchor - gold["F_anchor"]) <= TOL_BF16_LOSS * gold["F_anchor"]
+    tail = float(lg[-10:].mean())
+    assert abs(tail - gold["minibatch_loss_last10_mean"]) <= 5e-2 * gold["minibatch_loss_last10_mean"]
+
+
+@pytest.mark.parametrize("m", [8, 16, 64])
+def test_config5_parity_size_point(m):
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    c = si.CONFIGS["c5"]
+    P, iters = 1_000_000, 2 * c["tau"] + 1
+    x0 = si.flat_init(0, P)
+    grads = [si.flat_grads(0, k, m, P, c["grad_std"]) for k in range(iters)]
+    st = runner.run_flat(x0, grads, m=m, tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"],
+                         beta=c["beta"], mu=c["mu"])
+    opt = OverlapLocalSGD("flat", m=m, tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"],
+                          beta=c["beta"], mu=c["mu"], flat_P=P, x0=x0)
+    for k in range(iters):
+        opt.local_step_with_grads(to_dev(grads[k]))
+        if (k + 1) % c["tau"] == 0:
+            opt.period_sync()
+    assert state_err(opt, st) <= 1e-5
+
+
+def test_config5_largest_point_on_sampled_columns():
+    # P = 50M, m = 64 as bench.py runs it.  The update is separable per parameter,
+    # so the oracle runs exactly on a random sample of columns.
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    c = si.CONFIGS["c5"]
+    P, m, iters = 50_000_000, 64, 2 * c["tau"] + 1
+    gen = torch.Generator(device="cuda").manual_seed(1)
+    x0 = torch.randn(P, device="cuda", generator=gen)
+    cols = torch.from_numpy(np.sort(np.random.default_rng(2).choice(P, 4096, replace=False))).cuda()
+    cols[0], cols[-1] = 0, P - 1
+    opt = OverlapLocalSGD("flat", m=m, tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"],
+                          beta=c["beta"], mu=c["mu"], flat_P=P, x0=x0)
+    st = olsgd.OverlapLocalSGD(x0[cols].cpu().numpy(), m, c["tau"], c["gamma"], c["alpha"],
+                               c["beta"], c["mu"])
+    g = torch.empty((m, P), device="cuda")
+    for k in range(iters):
+        g.normal_(0.0, c["grad_std"], generator=gen)
+        st.step(g[:, cols].cpu().numpy())
+        opt.local_step_with_grads(g)
+        if (k + 1) % c["tau"] == 0:
+            opt.period_sync()
+    out = torch.empty(P, device="cuda")
+    got = []
+    for which in list(range(0, m, 9)) + [m - 1, -1]:
+        opt.get_params(which, out)
+        got.append(out[cols].cpu().numpy())
+    want = [st.x[i] for i in list(range(0, m, 9)) + [m - 1]] + [st.z]
+    assert max_rel_err(got, want) <= 1e-5
+    opt.get_params(-2, out)
+    v = out[cols].cpu().numpy()
+    assert np.abs(v - st.v).max() <= 1e-5 * np.abs(st.z).max()
