@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libolsgd.so")
-SOURCES = ["olsgd_api.cu", "update_kernels.cu", "sampling_kernels.cu", "simt_kernels.cu",
+SOURCES = ["olsgd_api.cu", "update_kernels.cu", "sampling_kernels.cu", "simt_kernels.cu", "head_kernels.cu",
            "model.cu", "tc_gemm.cu", "tc_wgrad.cu"]
 
 

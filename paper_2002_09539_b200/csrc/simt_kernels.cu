@@ -1,6 +1,5 @@
 // CUDA-core kernels of the forward/backward path: minibatch gather, linear
-// regression, the (skinny) output layer with softmax cross-entropy, bias
-// gradients, bf16 casts and transposes, and a plain reference GEMM.
+// regression, bias gradients, bf16 casts and transposes, and a plain reference GEMM.
 //
 // Every reduction runs in a fixed order (no floating-point atomics), so a step
 // is reproducible bit for bit from run to run.
@@ -76,6 +75,58 @@ gather_kernel(const float* __restrict__ X, const int32_t* __restrict__ y,
   }
 }
 
+// Same copy for the common aligned case (d % 128 == 0, batch % 32 == 0): 128-bit
+// loads of 512 contiguous bytes per row segment, 16-byte stores in both layouts.
+constexpr int kGvRows = 32, kGvCols = 128;
+
+__global__ void __launch_bounds__(256)
+gather_vec_kernel(const float* __restrict__ X, const int32_t* __restrict__ y,
+                  const int32_t* __restrict__ idx, float* __restrict__ xb32,
+                  __nv_bfloat16* __restrict__ xb16, __nv_bfloat16* __restrict__ xb16t,
+                  int32_t* __restrict__ yb, int batch, int64_t n, int d) {
+  __shared__ __align__(16) __nv_bfloat16 tile[kGvRows][kGvCols + 8];
+  __shared__ int32_t rows[kGvRows];
+  const int i = blockIdx.z;
+  const int b0 = blockIdx.y * kGvRows, j0 = blockIdx.x * kGvCols;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x < kGvRows) {
+    const int32_t r = idx[(int64_t)i * batch + b0 + threadIdx.x];
+    rows[threadIdx.x] = r;
+    if (blockIdx.x == 0) yb[(int64_t)i * batch + b0 + threadIdx.x] = y[(int64_t)i * n + r];
+  }
+  __syncthreads();
+#pragma unroll
+  for (int t = 0; t < kGvRows / 8; ++t) {
+    const int bl = warp + 8 * t;
+    const float4 v = __ldcs(reinterpret_cast<const float4*>(
+        X + ((int64_t)i * n + rows[bl]) * d + j0) + lane);
+    const int64_t o = ((int64_t)i * batch + b0 + bl) * d + j0 + lane * 4;
+    if (xb32) *reinterpret_cast<float4*>(xb32 + o) = v;
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&lo);
+    pk.y = *reinterpret_cast<uint32_t*>(&hi);
+    if (xb16) *reinterpret_cast<uint2*>(xb16 + o) = pk;
+    *reinterpret_cast<uint2*>(&tile[bl][lane * 4]) = pk;
+  }
+  if (!xb16t) return;
+  __syncthreads();
+  // [d][B] layout: each thread writes eight consecutive batch entries of one column
+#pragma unroll
+  for (int pass = 0; pass < 2; ++pass) {
+    const int jl = pass * 64 + (threadIdx.x >> 2), bq = threadIdx.x & 3;
+    uint32_t w[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const uint16_t lo = *reinterpret_cast<const uint16_t*>(&tile[bq * 8 + 2 * e][jl]);
+      const uint16_t hi = *reinterpret_cast<const uint16_t*>(&tile[bq * 8 + 2 * e + 1][jl]);
+      w[e] = (uint32_t)lo | ((uint32_t)hi << 16);
+    }
+    *reinterpret_cast<uint4*>(xb16t + ((int64_t)i * d + j0 + jl) * batch + b0 + bq * 8) =
+        make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
 // ------------------------------------------------------------------ linear regression
 
 __global__ void __launch_bounds__(128)
@@ -112,194 +163,6 @@ linreg_kernel(const float* __restrict__ X, const float* __restrict__ y,
   }
 }
 
-// ------------------------------------------------------------------ output layer
-
-constexpr int kHeadWarps = 8;     // rows per block
-constexpr int kHeadChunk = 256;   // K elements of W staged in shared memory at a time
-
-template <typename InT>
-__device__ __forceinline__ float load_in(const InT* p);
-template <>
-__device__ __forceinline__ float load_in<float>(const float* p) { return *p; }
-template <>
-__device__ __forceinline__ float load_in<__nv_bfloat16>(const __nv_bfloat16* p) {
-  return __bfloat162float(*p);
-}
-
-// One warp per batch row: logits, stable log-softmax, loss, d loss / d logits
-// and, if asked, the gradient with respect to the layer's input.
-template <typename InT, int CMAX>
-__global__ void __launch_bounds__(kHeadWarps * 32)
-head_forward_kernel(HeadArgs a) {
-  __shared__ float wsm[CMAX][kHeadChunk + 1];
-  __shared__ __align__(16) __nv_bfloat16 tsm[kHeadChunk][kHeadWarps];
-  const int i = blockIdx.y;
-  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  const int b = blockIdx.x * kHeadWarps + warp;
-  const bool live = b < a.batch;
-  const int K = a.K, C = a.C;
-  const InT* in = (sizeof(InT) == 4 ? reinterpret_cast<const InT*>(a.in32)
-                                    : reinterpret_cast<const InT*>(a.in16)) +
-                  ((int64_t)i * a.batch + (live ? b : 0)) * K;
-  const float* W = a.x + (int64_t)i * a.ld + a.w_off;
-  const float* bias = a.x + (int64_t)i * a.ld + a.b_off;
-
-  float acc[CMAX];
-#pragma unroll
-  for (int c = 0; c < CMAX; ++c) acc[c] = 0.f;
-
-  for (int k0 = 0; k0 < K; k0 += kHeadChunk) {
-    const int kc = min(kHeadChunk, K - k0);
-    __syncthreads();
-    for (int e = threadIdx.x; e < C * kHeadChunk; e += blockDim.x) {
-      const int c = e / kHeadChunk, kk = e % kHeadChunk;
-      float w = (kk < kc) ? W[(int64_t)c * K + k0 + kk] : 0.f;
-      if (a.round_w_bf16) w = bf16_round(w);
-      wsm[c][kk] = w;
-    }
-    __syncthreads();
-    if (live) {
-      for (int kk = lane; kk < kc; kk += 32) {
-        const float xv = load_in<InT>(in + k0 + kk);
-#pragma unroll
-        for (int c = 0; c < CMAX; ++c)
-          if (c < C) acc[c] = fmaf(xv, wsm[c][kk], acc[c]);
-      }
-    }
-  }
-  // every lane ends up with every logit
-  float mx = -INFINITY;
-#pragma unroll
-  for (int c = 0; c < CMAX; ++c) {
-    if (c < C) {
-      acc[c] = warp_sum(acc[c]) + bias[c];
-      mx = fmaxf(mx, acc[c]);
-    }
-  }
-  float se = 0.f;
-#pragma unroll
-  for (int c = 0; c < CMAX; ++c)
-    if (c < C) se += expf(acc[c] - mx);
-  const float lse = mx + logf(se);
-  const int label = live ? a.yb[(int64_t)i * a.batch + b] : 0;
-  const float inv_b = 1.0f / (float)a.batch;
-  float picked = 0.f;
-#pragma unroll
-  for (int c = 0; c < CMAX; ++c) {
-    if (c < C) {
-      if (c == label) picked = acc[c];
-      acc[c] = (expf(acc[c] - lse) - (c == label ? 1.f : 0.f)) * inv_b;  // d loss / d logit
-    }
-  }
-  if (live) {
-    float* dl = a.dlogits + ((int64_t)i * a.batch + b) * C;
-#pragma unroll
-    for (int c = 0; c < CMAX; ++c)
-      if (c < C && lane == (c & 31)) dl[c] = acc[c];
-    if (lane == 0) a.rowloss[(int64_t)i * a.batch + b] = lse - picked;
-  }
-  if (!a.din32 && !a.din16 && !a.din16t) return;
-
-  // gradient w.r.t. the input: din[k] = (sum_c dl[c] W[c][k]) * (in[k] > 0); the
-  // operand that goes on to the tensor cores is the bf16-rounded dl
-  if (a.round_w_bf16) {
-#pragma unroll
-    for (int c = 0; c < CMAX; ++c) acc[c] = bf16_round(acc[c]);
-  }
-  const int b0 = blockIdx.x * kHeadWarps;
-  for (int k0 = 0; k0 < K; k0 += kHeadChunk) {
-    const int kc = min(kHeadChunk, K - k0);
-    __syncthreads();
-    for (int e = threadIdx.x; e < C * kHeadChunk; e += blockDim.x) {
-      const int c = e / kHeadChunk, kk = e % kHeadChunk;
-      float w = (kk < kc) ? W[(int64_t)c * K + k0 + kk] : 0.f;
-      if (a.round_w_bf16) w = bf16_round(w);
-      wsm[c][kk] = w;
-    }
-    __syncthreads();
-    for (int kk = lane; kk < kHeadChunk; kk += 32) {
-      float d = 0.f;
-      if (live && kk < kc) {
-#pragma unroll
-        for (int c = 0; c < CMAX; ++c)
-          if (c < C) d = fmaf(acc[c], wsm[c][kk], d);
-        if (!(load_in<InT>(in + k0 + kk) > 0.f)) d = 0.f;
-        const int64_t o = ((int64_t)i * a.batch + b) * K + k0 + kk;
-        if (a.din32) a.din32[o] = d;
-        if (a.din16) a.din16[o] = __float2bfloat16_rn(d);
-      }
-      tsm[kk][warp] = __float2bfloat16_rn(d);
-    }
-    if (a.din16t) {
-      __syncthreads();
-      // [K][B] layout: eight consecutive batch entries (16 bytes) per K index
-      for (int kk = threadIdx.x; kk < kc; kk += blockDim.x) {
-        __nv_bfloat16* dst = a.din16t + ((int64_t)i * K + k0 + kk) * a.batch + b0;
-        if (b0 + kHeadWarps <= a.batch && (a.batch % kHeadWarps) == 0) {
-          *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(&tsm[kk][0]);
-        } else {
-          for (int r = 0; r < kHeadWarps; ++r)
-            if (b0 + r < a.batch) dst[r] = tsm[kk][r];
-        }
-      }
-    }
-  }
-}
-
-constexpr int kWgradCols = 128;
-constexpr int kWgradRows = 128;
-
-template <typename InT, int CMAX>
-__global__ void __launch_bounds__(kWgradCols)
-head_wgrad_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ loss) {
-  __shared__ float dsm[kWgradRows][CMAX + 1];
-  const int i = blockIdx.y;
-  const int j = blockIdx.x * kWgradCols + threadIdx.x;
-  const int K = a.K, C = a.C, B = a.batch;
-  const InT* in = (sizeof(InT) == 4 ? reinterpret_cast<const InT*>(a.in32)
-                                    : reinterpret_cast<const InT*>(a.in16)) +
-                  (int64_t)i * B * K;
-  const float* dl = a.dlogits + (int64_t)i * B * C;
-  float acc[CMAX];
-#pragma unroll
-  for (int c = 0; c < CMAX; ++c) acc[c] = 0.f;
-  float bsum = 0.f;  // thread c < C of block 0 also sums the bias gradient
-  for (int r0 = 0; r0 < B; r0 += kWgradRows) {
-    const int rc = min(kWgradRows, B - r0);
-    __syncthreads();
-    for (int e = threadIdx.x; e < rc * C; e += blockDim.x) {
-      float d = dl[(int64_t)r0 * C + e];
-      if (a.round_w_bf16) d = bf16_round(d);
-      dsm[e / C][e % C] = d;
-    }
-    __syncthreads();
-    if (j < K) {
-      for (int r = 0; r < rc; ++r) {
-        const float xv = load_in<InT>(in + (int64_t)(r0 + r) * K + j);
-#pragma unroll
-        for (int c = 0; c < CMAX; ++c)
-          if (c < C) acc[c] = fmaf(dsm[r][c], xv, acc[c]);
-      }
-    }
-    if (blockIdx.x == 0 && threadIdx.x < C)
-      for (int r = 0; r < rc; ++r) bsum += dl[(int64_t)(r0 + r) * C + threadIdx.x];
-  }
-  float* gi = g + (int64_t)i * a.ld;
-  if (j < K) {
-#pragma unroll
-    for (int c = 0; c < CMAX; ++c)
-      if (c < C) gi[a.w_off + (int64_t)c * K + j] = acc[c];
-  }
-  if (blockIdx.x == 0) {
-    if (threadIdx.x < C) gi[a.b_off + threadIdx.x] = bsum;
-    if (loss && threadIdx.x == kWgradCols - 1) {
-      float s = 0.f;
-      for (int r = 0; r < B; ++r) s += a.rowloss[(int64_t)i * B + r];
-      loss[i] = s / (float)B;
-    }
-  }
-}
-
 // ------------------------------------------------------------------ hidden-layer bias gradient
 
 __global__ void bias_grad_kernel(const __nv_bfloat16* __restrict__ dat, float* __restrict__ g,
@@ -317,22 +180,34 @@ __global__ void bias_grad_kernel(const __nv_bfloat16* __restrict__ dat, float* _
 
 // ------------------------------------------------------------------ bf16 transpose
 
-__global__ void transpose_bf16_kernel(const __nv_bfloat16* __restrict__ src, int64_t src_ld,
-                                      int64_t src_off, __nv_bfloat16* __restrict__ dst,
-                                      int64_t dst_batch, int R, int C) {
-  __shared__ __nv_bfloat16 tile[32][34];
+// 64 x 64 tiles, two bf16 per global access (128 bytes per row segment both ways).
+__global__ void __launch_bounds__(256)
+transpose_bf16_kernel(const __nv_bfloat16* __restrict__ src, int64_t src_ld, int64_t src_off,
+                      __nv_bfloat16* __restrict__ dst, int64_t dst_batch, int R, int C) {
+  __shared__ __nv_bfloat16 tile[64][66];
   const int i = blockIdx.z;
   const __nv_bfloat16* s = src + (int64_t)i * src_ld + src_off;
   __nv_bfloat16* d = dst + (int64_t)i * dst_batch;
-  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
-  for (int rr = threadIdx.y; rr < 32; rr += blockDim.y) {
-    const int r = r0 + rr, c = c0 + threadIdx.x;
-    if (r < R && c < C) tile[rr][threadIdx.x] = s[(int64_t)r * C + c];
+  const int c0 = blockIdx.x * 64, r0 = blockIdx.y * 64;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t w[8];
+#pragma unroll
+  for (int t = 0; t < 8; ++t) {
+    const int r = r0 + warp + 8 * t, c = c0 + 2 * lane;
+    w[t] = 0;
+    if (r < R && c < C) w[t] = __ldcs(reinterpret_cast<const uint32_t*>(s + (int64_t)r * C + c));
   }
+#pragma unroll
+  for (int t = 0; t < 8; ++t)
+    *reinterpret_cast<uint32_t*>(&tile[warp + 8 * t][2 * lane]) = w[t];
   __syncthreads();
-  for (int cc = threadIdx.y; cc < 32; cc += blockDim.y) {
-    const int c = c0 + cc, r = r0 + threadIdx.x;
-    if (r < R && c < C) d[(int64_t)c * R + r] = tile[threadIdx.x][cc];
+  for (int cc = warp; cc < 64; cc += 8) {
+    const int c = c0 + cc, r = r0 + 2 * lane;
+    if (r < R && c < C) {
+      const uint16_t lo = *reinterpret_cast<const uint16_t*>(&tile[2 * lane][cc]);
+      const uint16_t hi = *reinterpret_cast<const uint16_t*>(&tile[2 * lane + 1][cc]);
+      *reinterpret_cast<uint32_t*>(d + (int64_t)c * R + r) = (uint32_t)lo | ((uint32_t)hi << 16);
+    }
   }
 }
 
@@ -388,6 +263,11 @@ cudaError_t launch_cast_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cu
 cudaError_t launch_gather(const float* X, const int32_t* y, const int32_t* idx, float* xb32,
                           __nv_bfloat16* xb16, __nv_bfloat16* xb16t, int32_t* yb, int m, int batch,
                           int64_t n, int d, cudaStream_t s) {
+  if (d % kGvCols == 0 && batch % kGvRows == 0) {
+    dim3 grid(d / kGvCols, batch / kGvRows, m);
+    gather_vec_kernel<<<grid, 256, 0, s>>>(X, y, idx, xb32, xb16, xb16t, yb, batch, n, d);
+    return cudaGetLastError();
+  }
   dim3 grid((d + kGatherCols - 1) / kGatherCols, (batch + kGatherRows - 1) / kGatherRows, m);
   dim3 block(kGatherCols, 4);
   gather_kernel<<<grid, block, 0, s>>>(X, y, idx, xb32, xb16, xb16t, yb, batch, n, d);
@@ -398,32 +278,6 @@ cudaError_t launch_linreg(const float* X, const float* y, const int32_t* idx, co
                           float* g, float* loss, int m, int batch, int64_t n, int d, int64_t ld,
                           cudaStream_t s) {
   linreg_kernel<<<m, 128, (size_t)batch * sizeof(float), s>>>(X, y, idx, x, g, loss, batch, n, d, ld);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_head_forward(const HeadArgs& a, cudaStream_t s) {
-  dim3 grid((a.batch + kHeadWarps - 1) / kHeadWarps, a.m), block(kHeadWarps * 32);
-  const bool f32 = a.in32 != nullptr;
-  if (a.C <= 16) {
-    if (f32) head_forward_kernel<float, 16><<<grid, block, 0, s>>>(a);
-    else head_forward_kernel<__nv_bfloat16, 16><<<grid, block, 0, s>>>(a);
-  } else {
-    if (f32) head_forward_kernel<float, 32><<<grid, block, 0, s>>>(a);
-    else head_forward_kernel<__nv_bfloat16, 32><<<grid, block, 0, s>>>(a);
-  }
-  return cudaGetLastError();
-}
-
-cudaError_t launch_head_wgrad(const HeadArgs& a, float* g, float* loss, cudaStream_t s) {
-  dim3 grid((a.K + kWgradCols - 1) / kWgradCols, a.m), block(kWgradCols);
-  const bool f32 = a.in32 != nullptr;
-  if (a.C <= 16) {
-    if (f32) head_wgrad_kernel<float, 16><<<grid, block, 0, s>>>(a, g, loss);
-    else head_wgrad_kernel<__nv_bfloat16, 16><<<grid, block, 0, s>>>(a, g, loss);
-  } else {
-    if (f32) head_wgrad_kernel<float, 32><<<grid, block, 0, s>>>(a, g, loss);
-    else head_wgrad_kernel<__nv_bfloat16, 32><<<grid, block, 0, s>>>(a, g, loss);
-  }
   return cudaGetLastError();
 }
 
@@ -438,8 +292,9 @@ cudaError_t launch_bias_grad(const __nv_bfloat16* dat, float* g, int64_t ld, int
 cudaError_t launch_transpose_bf16(const __nv_bfloat16* src, int64_t src_ld, int64_t src_off,
                                   __nv_bfloat16* dst, int64_t dst_batch, int m, int R, int C,
                                   cudaStream_t s) {
-  dim3 grid((C + 31) / 32, (R + 31) / 32, m), block(32, 8);
-  transpose_bf16_kernel<<<grid, block, 0, s>>>(src, src_ld, src_off, dst, dst_batch, R, C);
+  if (R % 2 || C % 2 || src_off % 2 || src_ld % 2 || dst_batch % 2) return cudaErrorInvalidValue;
+  dim3 grid((C + 63) / 64, (R + 63) / 64, m);
+  transpose_bf16_kernel<<<grid, 256, 0, s>>>(src, src_ld, src_off, dst, dst_batch, R, C);
   return cudaGetLastError();
 }
 

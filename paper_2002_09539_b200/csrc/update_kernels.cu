@@ -99,17 +99,20 @@ fused_update_kernel(const float* __restrict__ x_in, float* __restrict__ x_out,
   }
 }
 
-constexpr int kMeanCols = 32;   // float4 columns per block: 512 contiguous bytes per row
-constexpr int kMeanSlices = 8;  // worker slices per block, combined through shared memory
+constexpr int kMeanThreads = 256;
 
-// Column sums over the worker dimension in a fixed order: slice s adds workers
-// s, s + S, s + 2S, ... sequentially, then slice 0 adds the S partial sums in
-// slice order.  The result does not depend on launch shape or timing.
-template <bool MOM>
-__global__ void __launch_bounds__(kMeanCols* kMeanSlices)
+// Column sums over the worker dimension in a fixed order.  A block covers
+// 256 / SLICES float4 columns; slice s adds workers s, s + S, s + 2S, ...
+// sequentially (four loads in flight), the partial sums are staged in shared
+// memory and slice 0 adds them in slice order.  SLICES depends on m only, so the
+// result does not depend on P, on the launch shape or on timing.
+template <bool MOM, int SLICES>
+__global__ void __launch_bounds__(kMeanThreads)
 worker_mean_anchor_kernel(const float* __restrict__ x, float* __restrict__ z,
                           float* __restrict__ v, int64_t n4, int64_t ld, int m, float beta,
                           float m_f) {
+  constexpr int kMeanCols = kMeanThreads / SLICES;
+  constexpr int kMeanSlices = SLICES;
   __shared__ float4 part[kMeanSlices][kMeanCols];
   const int64_t col4 = (int64_t)blockIdx.x * kMeanCols + threadIdx.x;
   const int slice = threadIdx.y;
@@ -214,15 +217,25 @@ cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t s) {
   return cudaGetLastError();
 }
 
-cudaError_t launch_worker_mean_anchor(const AnchorArgs& a, cudaStream_t s) {
+template <int SLICES>
+cudaError_t launch_mean(const AnchorArgs& a, cudaStream_t s) {
   const int64_t n4 = (a.P + 3) / 4;
-  dim3 grid((unsigned)((n4 + kMeanCols - 1) / kMeanCols)), block(kMeanCols, kMeanSlices);
+  constexpr int cols = kMeanThreads / SLICES;
+  dim3 grid((unsigned)((n4 + cols - 1) / cols)), block(cols, SLICES);
   const float m_f = (float)a.m;
   if (a.beta != 0.f)
-    worker_mean_anchor_kernel<true><<<grid, block, 0, s>>>(a.x, a.z, a.v, n4, a.ld, a.m, a.beta, m_f);
+    worker_mean_anchor_kernel<true, SLICES><<<grid, block, 0, s>>>(a.x, a.z, a.v, n4, a.ld, a.m, a.beta, m_f);
   else
-    worker_mean_anchor_kernel<false><<<grid, block, 0, s>>>(a.x, a.z, a.v, n4, a.ld, a.m, a.beta, m_f);
+    worker_mean_anchor_kernel<false, SLICES><<<grid, block, 0, s>>>(a.x, a.z, a.v, n4, a.ld, a.m, a.beta, m_f);
   return cudaGetLastError();
+}
+
+cudaError_t launch_worker_mean_anchor(const AnchorArgs& a, cudaStream_t s) {
+  // about four workers per slice, so that every thread has four loads in flight
+  if (a.m >= 32) return launch_mean<8>(a, s);
+  if (a.m >= 16) return launch_mean<4>(a, s);
+  if (a.m >= 8) return launch_mean<2>(a, s);
+  return launch_mean<1>(a, s);
 }
 
 cudaError_t launch_virtual_sequence(const float* x, const float* z, float* dst, int64_t P,
