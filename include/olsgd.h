@@ -176,6 +176,39 @@ olsgd_status olsgd_get_indices(olsgd_ctx* ctx, int64_t k, int32_t* dst);
  *   dst  int32 [m][2], host or device                                       */
 olsgd_status olsgd_class_pairs(uint64_t seed, int32_t m, int32_t* dst, void* stream);
 
+/* The same table for callers that must not allocate.  (The paper has no
+ * counterpart to this entry point; it exists for the library's users.)
+ *
+ * olsgd_class_pairs stages a host destination through pinned memory that it
+ * allocates and frees on every call.  Some callers cannot do that: code that
+ * runs between cudaStreamBeginCapture and cudaStreamEndCapture on another
+ * stream of the same thread (an allocation call there invalidates the
+ * capture), a process whose memory has been handed in full to a pool or to
+ * another framework, or a latency-critical thread that is not allowed to take
+ * the allocator's locks.  This variant calls no cudaMalloc, cudaFree,
+ * cudaHostAlloc or any other allocating routine.  The kernel writes the table
+ * into a fixed array that lives in the library's device image, and the result
+ * is copied from there to `dst`.
+ *
+ *   m       at most OLSGD_NOALLOC_MAX_WORKERS; larger values are rejected with
+ *           OLSGD_EINVAL and a message, nothing is launched
+ *   dst     int32 [m][2], host or device
+ *   stream  cudaStream_t the kernel and the copy run on; the call blocks the
+ *           host until both are done
+ *
+ * Cost and rules of the fixed array:
+ *   - every GPU on which the library is loaded holds it (128 KB) until the
+ *     process exits, whether or not this entry point is ever called;
+ *   - the first call on each device looks the array's device address up once
+ *     (with that device current); make that first call before starting any
+ *     stream capture;
+ *   - all calls share the one array, which keeps what the last call wrote.
+ *     Each call overwrites every entry it returns, so nothing has to be
+ *     cleared, but two calls whose GPU work overlaps (different streams or
+ *     threads on the same device) race on it: serialise them.                 */
+#define OLSGD_NOALLOC_MAX_WORKERS 16384
+olsgd_status olsgd_class_pairs_noalloc(uint64_t seed, int32_t m, int32_t* dst, void* stream);
+
 /* Iteration counter k.                                                      */
 int64_t olsgd_iteration(const olsgd_ctx* ctx);
 

@@ -68,6 +68,7 @@ def load_library():
         "olsgd_get_params": (i32, [vp, i32, vp, C.c_size_t]),
         "olsgd_get_indices": (i32, [vp, i64, vp]),
         "olsgd_class_pairs": (i32, [u64, i32, vp, vp]),
+        "olsgd_class_pairs_noalloc": (i32, [u64, i32, vp, vp]),
         "olsgd_iteration": (i64, [vp]),
         "olsgd_launch_count": (i64, [vp]),
         "olsgd_profile_enable": (i32, [vp, i32]),
@@ -104,6 +105,21 @@ def class_pairs(seed, m, device="cuda"):
     out = torch.empty((m, 2), dtype=torch.int32, device=device)
     stream = torch.cuda.current_stream().cuda_stream
     _check(lib, lib.olsgd_class_pairs(int(seed), int(m), out.data_ptr(), stream))
+    return out
+
+
+NOALLOC_MAX_WORKERS = 16384
+
+
+def class_pairs_noalloc(seed, m, device="cpu"):
+    """olsgd_class_pairs_noalloc: the same table, for callers that must not allocate
+    (the library stages it in a fixed device array instead of fresh pinned memory).
+    The output tensor here is still created by torch; pass your own memory to the C
+    entry point if even that is not allowed."""
+    lib = load_library()
+    out = torch.empty((max(m, 0), 2), dtype=torch.int32, device=device)
+    stream = torch.cuda.current_stream().cuda_stream
+    _check(lib, lib.olsgd_class_pairs_noalloc(int(seed), int(m), out.data_ptr(), stream))
     return out
 
 

@@ -344,6 +344,10 @@ olsgd_status check_device_status(olsgd_ctx* c) {
 
 }  // namespace
 
+namespace olsgd {
+void set_thread_error(const char* text) { g_last_error = text ? text : ""; }
+}  // namespace olsgd
+
 extern "C" {
 
 olsgd_status olsgd_param_count(const olsgd_model_spec* spec, int64_t* out_P) {

@@ -10,6 +10,10 @@
 
 namespace olsgd {
 
+// ---- olsgd_api.cu -------------------------------------------------------------
+// Records the text olsgd_last_error(NULL) returns for context-free calls of this thread.
+void set_thread_error(const char* text);
+
 // ---- update_kernels.cu ------------------------------------------------------
 // Eq. 3 (+ local Nesterov buffer) and, when `sync`, Eq. 4, for all m workers.
 // x_in/x_out/u/shadow rows have stride `ld` floats (multiple of 4, 16-byte

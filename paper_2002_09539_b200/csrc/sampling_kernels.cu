@@ -5,6 +5,9 @@
 // Section 3.3 and the Philox4x32 row of its constants table): ten rounds of
 //   (c0, c1, c2, c3) <- (hi(M1 c2) ^ c1 ^ k0, lo(M1 c2), hi(M0 c0) ^ c3 ^ k1, lo(M0 c0))
 // with the key bumped by the two Weyl constants before every round but the first.
+#include <cstdio>
+#include <mutex>
+
 #include "olsgd_internal.h"
 
 namespace olsgd {
@@ -99,3 +102,71 @@ cudaError_t launch_class_pairs(int32_t* dst, uint64_t seed, int m, cudaStream_t 
 }
 
 }  // namespace olsgd
+
+// ---------------------------------------------------------------------------
+// olsgd_class_pairs_noalloc: the partition table without any allocation.
+//
+// The staging buffer is a file-scope array in the library's device image.  In
+// host code the name `g_pair_scratch` is only a handle for the runtime, not a
+// device address, so it is never passed to a kernel: its address on the current
+// device is looked up once per device with cudaGetSymbolAddress and that
+// pointer is what the kernel and the copy receive.
+namespace {
+
+static __device__ __align__(256) int32_t g_pair_scratch[2 * OLSGD_NOALLOC_MAX_WORKERS];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+int32_t* g_scratch_addr[kMaxDevices] = {nullptr};
+
+// Device address of the scratch array on the current device (set-up on first use).
+cudaError_t scratch_address(int32_t** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_addr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_pair_scratch);
+    if (e != cudaSuccess) return e;
+    g_scratch_addr[dev] = static_cast<int32_t*>(p);
+  }
+  *out = g_scratch_addr[dev];
+  return cudaSuccess;
+}
+
+olsgd_status noalloc_fail(olsgd_status st, const char* what, cudaError_t e) {
+  char buf[256];
+  if (e != cudaSuccess)
+    snprintf(buf, sizeof buf, "olsgd_class_pairs_noalloc: %s: %s", what, cudaGetErrorString(e));
+  else
+    snprintf(buf, sizeof buf, "olsgd_class_pairs_noalloc: %s", what);
+  olsgd::set_thread_error(buf);
+  return st;
+}
+
+}  // namespace
+
+extern "C" olsgd_status olsgd_class_pairs_noalloc(uint64_t seed, int32_t m, int32_t* dst,
+                                                  void* stream) {
+  if (m < 1) return noalloc_fail(OLSGD_EINVAL, "m must be >= 1", cudaSuccess);
+  if (m > OLSGD_NOALLOC_MAX_WORKERS) {
+    char buf[128];
+    snprintf(buf, sizeof buf, "m = %d exceeds the fixed scratch array (at most %d workers)", m,
+             OLSGD_NOALLOC_MAX_WORKERS);
+    return noalloc_fail(OLSGD_EINVAL, buf, cudaSuccess);
+  }
+  if (!dst) return noalloc_fail(OLSGD_EINVAL, "dst is NULL", cudaSuccess);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int32_t* scratch = nullptr;
+  cudaError_t e = scratch_address(&scratch);
+  if (e != cudaSuccess) return noalloc_fail(OLSGD_ECUDA, "looking up the scratch array failed", e);
+  e = olsgd::launch_class_pairs(scratch, seed, m, s);
+  if (e != cudaSuccess) return noalloc_fail(OLSGD_ECUDA, "kernel launch failed", e);
+  e = cudaMemcpyAsync(dst, scratch, sizeof(int32_t) * 2 * (size_t)m, cudaMemcpyDefault, s);
+  if (e != cudaSuccess) return noalloc_fail(OLSGD_ECUDA, "copy to dst failed", e);
+  e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return noalloc_fail(OLSGD_ECUDA, "stream synchronisation failed", e);
+  return OLSGD_OK;
+}
