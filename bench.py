@@ -118,6 +118,21 @@ class ClockSampler:
 
 # ------------------------------------------------------------------ roofline accounting
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the ncu capture
+# summarised in profiles/, keyed by (workload, kernel class); (ordinary step, sync step).
+# An entry must be removed when its kernel changes.
+NCU_TRAFFIC = {
+    ("c3", "update"): (1426.5e6, 1445.6e6),      # profiles/fused_update_c3_mlp.txt
+}
+
+
+def ncu_traffic(name, kernel_class, sync_fraction):
+    t = NCU_TRAFFIC.get((name, kernel_class))
+    if t is None:
+        return None
+    return int((1.0 - sync_fraction) * t[0] + sync_fraction * t[1])
+
+
 def algorithmic_bytes(c, kernel_class, P, sync_fraction):
     """Algorithmic HBM bytes of ONE launch of the given kernel class (averaged over
     sync and ordinary steps for the update kernel)."""
@@ -210,7 +225,8 @@ def run_ours(args, rank, world):
     achieved = ab / (avg_ms * 1e-3) / 1e9
     roofline = dict(bound="hbm", kernel=roof_class, achieved=round(achieved, 1),
                     peak=peaks["hbm_gbs"], unit="GB/s", frac=round(achieved / peaks["hbm_gbs"], 4),
-                    frac_of_8000=round(achieved / 8000.0, 4), traffic=None,
+                    frac_of_8000=round(achieved / 8000.0, 4),
+                    traffic=ncu_traffic(name, roof_class, n_sync / K),
                     peak_source=peaks["source"], avg_launch_us=round(avg_ms * 1e3, 2),
                     algorithmic_bytes_per_launch=int(ab),
                     dominant_class=dominant,
@@ -439,9 +455,9 @@ def run_reference(args, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4", "c5"])
     ap.add_argument("--P", type=int, default=0, help="c5 only: one parameter count")
     ap.add_argument("--m", type=int, default=0, help="c5 only: one worker count")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
