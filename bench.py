@@ -122,15 +122,28 @@ class ClockSampler:
 # summarised in profiles/, keyed by (workload, kernel class); (ordinary step, sync step).
 # An entry must be removed when its kernel changes.
 NCU_TRAFFIC = {
-    ("c3", "update"): (1426.5e6, 1445.6e6),      # profiles/fused_update_c3_mlp.txt
+    # (workload, gemm mode, kernel class)
+    ("c3", 3, "update"): (1426.5e6, 1445.6e6),      # profiles/fused_update_c3_mlp.txt
 }
 
 
-def ncu_traffic(name, kernel_class, sync_fraction):
-    t = NCU_TRAFFIC.get((name, kernel_class))
+def ncu_traffic(name, mode, kernel_class, sync_fraction):
+    t = NCU_TRAFFIC.get((name, mode, kernel_class))
     if t is None:
         return None
     return int((1.0 - sync_fraction) * t[0] + sync_fraction * t[1])
+
+
+def layer_is_fused(c, p):
+    """Does the weight-gradient GEMM of parameter layer p apply the update in its epilogue?"""
+    d = c["dims"]
+    return (c.get("gemm_bf16") == 1 and p < len(d) - 2 and d[p + 1] % 128 == 0 and
+            d[p] % 128 == 0 and c["batch"] % 64 == 0 and c["batch"] <= 128)
+
+
+def fused_weight_count(c):
+    d = c.get("dims", [])
+    return sum(d[p + 1] * d[p] for p in range(len(d) - 2) if layer_is_fused(c, p))
 
 
 def algorithmic_bytes(c, kernel_class, P, sync_fraction):
@@ -139,9 +152,21 @@ def algorithmic_bytes(c, kernel_class, P, sync_fraction):
     m = c["m"]
     mom = c["mu"] != 0.0
     shadow = 2 if c.get("gemm_bf16") else 0
+    fused = fused_weight_count(c)
+    if kernel_class == "wgrad_update":
+        # per launch, averaged over the fused layers: x read+write, u read+write, bf16 shadow
+        # write per parameter per worker, the anchor once on sync steps, the bf16 operands once
+        if not fused:
+            return None
+        d, B = c["dims"], c["batch"]
+        layers = [p for p in range(len(d) - 2) if layer_is_fused(c, p)]
+        per = (16 if mom else 8) + 2
+        operands = sum(m * B * 2 * (d[p + 1] + d[p]) for p in layers)
+        return (m * fused * per + sync_fraction * 4 * fused + operands) / len(layers)
     if kernel_class == "update":
         per = (20 if mom else 12) + shadow
-        return m * P * per + sync_fraction * 4 * P
+        rest = P - fused
+        return m * rest * per + sync_fraction * 4 * rest
     if kernel_class == "anchor":
         return 4 * m * P + (16 if c["beta"] != 0.0 else 4) * P
     return None
@@ -165,7 +190,9 @@ def run_ours(args, rank, world):
         dist.barrier()
 
     name = args.workload
-    c = si.CONFIGS[name]
+    c = dict(si.CONFIGS[name])
+    if c["gemm_bf16"] and args.gemm_mode:
+        c["gemm_bf16"] = args.gemm_mode
     seed = rank                      # every rank is an independent replica
     table = None
     if c.get("non_iid"):
@@ -226,7 +253,7 @@ def run_ours(args, rank, world):
     roofline = dict(bound="hbm", kernel=roof_class, achieved=round(achieved, 1),
                     peak=peaks["hbm_gbs"], unit="GB/s", frac=round(achieved / peaks["hbm_gbs"], 4),
                     frac_of_8000=round(achieved / 8000.0, 4),
-                    traffic=ncu_traffic(name, roof_class, n_sync / K),
+                    traffic=ncu_traffic(name, c["gemm_bf16"], roof_class, n_sync / K),
                     peak_source=peaks["source"], avg_launch_us=round(avg_ms * 1e3, 2),
                     algorithmic_bytes_per_launch=int(ab),
                     dominant_class=dominant,
@@ -280,6 +307,7 @@ def run_ours(args, rank, world):
             "config": {"workload": workload_name(name, c), "m": m, "tau": c["tau"],
                        "batch": B, "dims": c["dims"], "P": P, "gamma": c["gamma"],
                        "alpha": c["alpha"], "beta": c["beta"], "mu": c["mu"],
+                       "gemm_mode": c["gemm_bf16"],
                        "l2": "no flush: resident inputs+state %.0f MB exceed the %d MB L2"
                              % (resident / 1e6, L2_BYTES >> 20) if resident > L2_BYTES else
                              "state fits in L2 (%.1f MB): steady-state training keeps it there"
@@ -458,6 +486,9 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--gemm-mode", type=int, default=0, choices=[0, 1, 2, 3],
+                    help="MLP workloads: 1 tensor cores + update fused into the weight-gradient "
+                         "GEMM (default), 3 tensor cores + separate update kernel, 2 CUDA cores")
     ap.add_argument("--P", type=int, default=0, help="c5 only: one parameter count")
     ap.add_argument("--m", type=int, default=0, help="c5 only: one worker count")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

@@ -54,8 +54,13 @@ typedef struct {
   int32_t kind;                 /* olsgd_model                                        */
   int32_t n_dims;               /* entries used in dims (1 for LINREG, 0 for FLAT)    */
   int32_t dims[OLSGD_MAX_DIMS]; /* e.g. {3072, 1024, 1024, 10}                        */
-  int32_t gemm_bf16;            /* MLP only: 1 = bf16 operands on the tensor cores,
-                                   fp32 accumulate, fp32 master weights; 0 = fp32    */
+  int32_t gemm_bf16;            /* MLP only.  1 = bf16 operands on the tensor cores, fp32
+                                   accumulate, fp32 master weights, the parameter update
+                                   of the hidden-layer weights fused into the weight-
+                                   gradient GEMM; 3 = the same GEMMs with the update as a
+                                   separate kernel; 2 = the same bf16 data flow on CUDA
+                                   cores (a check of the tensor-core kernels); 0 = fp32
+                                   (models without hidden layers)                     */
   int32_t reserved;
   int64_t flat_P;               /* FLAT only: number of parameters                    */
 } olsgd_model_spec;
@@ -219,9 +224,10 @@ int64_t olsgd_launch_count(const olsgd_ctx* ctx);
  * bracketed by CUDA events on its own stream.  olsgd_profile_read joins both
  * streams and returns, per class c in 0..OLSGD_N_KERNEL_CLASSES-1, the launch
  * count and the summed duration in milliseconds since the last reset.       */
-#define OLSGD_N_KERNEL_CLASSES 8
+#define OLSGD_N_KERNEL_CLASSES 9
 enum { OLSGD_KC_INDEX = 0, OLSGD_KC_GATHER = 1, OLSGD_KC_FORWARD = 2, OLSGD_KC_BACKWARD = 3,
-       OLSGD_KC_UPDATE = 4, OLSGD_KC_ANCHOR = 5, OLSGD_KC_LOSS = 6, OLSGD_KC_OTHER = 7 };
+       OLSGD_KC_UPDATE = 4, OLSGD_KC_ANCHOR = 5, OLSGD_KC_LOSS = 6, OLSGD_KC_OTHER = 7,
+       OLSGD_KC_WGRAD_UPDATE = 8 /* weight-gradient GEMM with the update fused in */ };
 olsgd_status olsgd_profile_enable(olsgd_ctx* ctx, int32_t on);
 olsgd_status olsgd_profile_read(olsgd_ctx* ctx, int64_t* launches, double* millis, int32_t reset);
 

@@ -13,7 +13,8 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB = None
 
-KERNEL_CLASSES = ("index", "gather", "forward", "backward", "update", "anchor", "loss", "other")
+KERNEL_CLASSES = ("index", "gather", "forward", "backward", "update", "anchor", "loss", "other",
+                  "wgrad_update")
 _KINDS = {"linreg": 0, "softmax": 1, "mlp": 2, "flat": 3}
 MAX_DIMS = 8
 

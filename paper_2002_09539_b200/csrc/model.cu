@@ -28,10 +28,13 @@ inline int n_layers(const olsgd_model_spec& s) { return s.n_dims - 1; }
 // gemm_bf16: 0 = fp32 CUDA cores, 1 = tcgen05 tensor cores, 2 = the same bf16
 // data flow on CUDA cores (validation of the tensor-core kernels)
 inline bool bf16_path(const olsgd_model_spec& s) { return s.kind == OLSGD_MLP && s.gemm_bf16 != 0; }
+inline bool tensor_path(const olsgd_model_spec& s) {
+  return s.kind == OLSGD_MLP && (s.gemm_bf16 == 1 || s.gemm_bf16 == 3);
+}
 
 cudaError_t run_gemm(const olsgd_model_spec& spec, GemmArgs ga, int* status, cudaStream_t s) {
   ga.status = status;
-  if (spec.gemm_bf16 == 1)
+  if (tensor_path(spec))
     return wgrad_tc_supported(ga) ? launch_wgrad_tc(ga, s) : launch_gemm_tc(ga, s);
   return launch_gemm_simt(ga, s);
 }
@@ -85,7 +88,7 @@ bool plan_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, ModelPlan
       return false;
     }
   }
-  if (spec.gemm_bf16 == 1 && (B % 64 != 0 || B > 256)) {
+  if (tensor_path(spec) && (B % 64 != 0 || B > 256)) {
     snprintf(mp->error, sizeof mp->error, "the tensor-core path needs batch in {64, 128, 192, 256}");
     return false;
   }
@@ -107,9 +110,13 @@ bool plan_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, ModelPlan
 
 bool bind_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, const ModelPlan& mp,
                 char* base, ModelBuffers* mb) {
-  (void)hp;
   mb->loss = reinterpret_cast<float*>(base + mp.off_loss);
-  if (spec.kind == OLSGD_LINREG) return true;
+  mb->n_ranges = 1;
+  mb->range_off[0] = 0;
+  if (spec.kind == OLSGD_LINREG) {
+    mb->range_len[0] = spec.dims[0];
+    return true;
+  }
   const int L = n_layers(spec);
   int64_t off = 0;
   for (int l = 0; l < L; ++l) {
@@ -121,6 +128,7 @@ bool bind_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, const Mod
   mb->yb = reinterpret_cast<int32_t*>(base + mp.off_yb);
   mb->dlogits = reinterpret_cast<float*>(base + mp.off_dlogits);
   mb->rowloss = reinterpret_cast<float*>(base + mp.off_rowloss);
+  mb->range_len[0] = off;
   if (!bf16_path(spec)) {
     mb->xb32 = reinterpret_cast<float*>(base + mp.off_xb32);
     return true;
@@ -135,6 +143,28 @@ bool bind_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, const Mod
     mb->dat[l] = bp(mp.off_dat[l]);
   }
   for (int l = 1; l < L - 1; ++l) mb->wt[l] = bp(mp.off_wt[l]);
+  // gemm_bf16 == 1: hidden-layer weight matrices whose shape the weight-gradient kernel
+  // takes are updated in its epilogue; everything else goes to the update kernel
+  int64_t P = off;
+  for (int p = 0; p < L - 1; ++p)
+    mb->fused_layer[p] = spec.gemm_bf16 == 1 && spec.dims[p + 1] % 128 == 0 &&
+                         spec.dims[p] % 128 == 0 && hp.batch % 64 == 0 && hp.batch <= 128;
+  int64_t start = 0;
+  mb->n_ranges = 0;
+  auto close_range = [&](int64_t end) {
+    if (end > start) {
+      mb->range_off[mb->n_ranges] = start;
+      mb->range_len[mb->n_ranges] = end - start;
+      mb->n_ranges++;
+    }
+  };
+  for (int p = 0; p < L - 1; ++p) {
+    if (mb->fused_layer[p]) {
+      close_range(mb->w_off[p]);
+      start = mb->b_off[p];
+    }
+  }
+  close_range(P);
   return true;
 }
 
@@ -213,6 +243,7 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
   }
 
   // hidden layers, backward
+  bool waited = false;
   for (int l = L - 1; l >= 1; --l) {
     // dW_l [d_l][d_{l-1}] = dA_l^T [d_l][B] * (H_{l-1}^T [d_{l-1}][B])^T
     GemmArgs gw{};
@@ -230,7 +261,17 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
     gw.out_f = io.g + mb.w_off[l - 1];
     gw.ldo = spec.dims[l - 1];
     gw.out_batch = io.ld;
-    {
+    if (io.upd.enabled && mb.fused_layer[l - 1]) {
+      // the update of W_l happens in this GEMM's epilogue: no gradient is stored
+      gw.upd = io.upd;
+      gw.upd.w_off = mb.w_off[l - 1];
+      if (io.wait_before_update && !waited) {
+        OLSGD_TRY(cudaStreamWaitEvent(s, io.wait_before_update, 0));
+        waited = true;
+      }
+      Scope sc(hook, OLSGD_KC_WGRAD_UPDATE, s);
+      OLSGD_TRY(run_gemm(spec, gw, io.status, s));
+    } else {
       Scope sc(hook, OLSGD_KC_BACKWARD, s);
       OLSGD_TRY(run_gemm(spec, gw, io.status, s));
     }

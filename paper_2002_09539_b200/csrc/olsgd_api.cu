@@ -276,22 +276,27 @@ olsgd_status apply_update(olsgd_ctx* c, const float* g, int64_t ldg) {
     OLSGD_CUDA(c, cudaStreamWaitEvent(c->main, c->reduce_done, 0));
     c->reduce_pending = false;
   }
-  UpdateArgs a;
-  a.x_in = c->x[c->cur];
-  a.x_out = c->x[nxt];
-  a.g = g;
-  a.u = c->u;
-  a.z = c->z;
-  a.shadow = c->shadow;
-  a.P = c->P;
-  a.ld = c->ld;
-  a.ldg = ldg;
-  a.m = c->hp.m;
-  a.gamma = c->hp.gamma;
-  a.mu = c->hp.mu;
-  a.alpha = c->hp.alpha;
-  a.sync = sync;
-  {
+  // the whole row, or (when hidden-layer weights were updated inside their weight-gradient
+  // GEMM) the ranges that are left: biases and the output layer
+  const bool model = c->spec.kind != OLSGD_FLAT;
+  const int n_ranges = model ? c->mb.n_ranges : 1;
+  for (int r = 0; r < n_ranges; ++r) {
+    const int64_t off = model ? c->mb.range_off[r] : 0;
+    UpdateArgs a;
+    a.x_in = c->x[c->cur] + off;
+    a.x_out = c->x[nxt] + off;
+    a.g = g + off;
+    a.u = c->u ? c->u + off : nullptr;
+    a.z = c->z + off;
+    a.shadow = c->shadow ? c->shadow + off : nullptr;
+    a.P = model ? c->mb.range_len[r] : c->P;
+    a.ld = c->ld;
+    a.ldg = ldg;
+    a.m = c->hp.m;
+    a.gamma = c->hp.gamma;
+    a.mu = c->hp.mu;
+    a.alpha = c->hp.alpha;
+    a.sync = sync;
     Launch l(c, OLSGD_KC_UPDATE, c->main);
     OLSGD_CUDA(c, launch_fused_update(a, c->main));
   }
@@ -313,6 +318,28 @@ olsgd_status step_body(olsgd_ctx* c, const olsgd_data& data, const int32_t* idx,
   io.idx = idx;
   io.loss = loss_device;
   io.status = c->dev_status;
+  memset(&io.upd, 0, sizeof io.upd);
+  io.wait_before_update = nullptr;
+  if (c->spec.kind == OLSGD_MLP && c->spec.gemm_bf16 == 1) {
+    const bool sync = (c->k + 1) % c->hp.tau == 0;
+    const int nxt = 1 - c->cur;
+    io.upd.enabled = 1;
+    io.upd.x_in = c->x[c->cur];
+    io.upd.x_out = c->x[nxt];
+    io.upd.u = c->u;
+    io.upd.z = c->z;
+    io.upd.shadow = c->shadow;
+    io.upd.ld = c->ld;
+    io.upd.gamma = c->hp.gamma;
+    io.upd.mu = c->hp.mu;
+    io.upd.alpha = c->hp.alpha;
+    io.upd.sync = sync ? 1 : 0;
+    // same rule as in apply_update, applied before the first kernel that writes x[nxt]
+    if (c->reduce_pending && (sync || c->reduce_reads == nxt)) {
+      io.wait_before_update = c->reduce_done;
+      c->reduce_pending = false;
+    }
+  }
   const ProfHook hook = make_hook(c);
   cudaError_t e = model_forward_backward(c->spec, c->hp, data, c->mb, io, c->main, hook);
   if (e != cudaSuccess)

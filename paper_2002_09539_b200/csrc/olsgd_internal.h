@@ -123,6 +123,20 @@ enum GemmEpilogue {
   // out = D, written fp32 to out_f [row * ldo + col]
   GEMM_EPI_STORE_F32 = 2
 };
+// Parameter update applied inside the weight-gradient GEMM's epilogue instead of
+// storing the gradient: the tile D[row][col] updates parameter w_off + row * Nb + col
+// of every worker row (stride ld) of x_in/x_out/u/shadow.
+struct FusedUpdateArgs {
+  int enabled;
+  const float* x_in;
+  float* x_out;
+  float* u;               // null or mu == 0: plain SGD
+  const float* z;
+  __nv_bfloat16* shadow;
+  int64_t ld, w_off;
+  float gamma, mu, alpha;
+  int sync;
+};
 struct GemmArgs {
   const __nv_bfloat16* A;
   const __nv_bfloat16* B;
@@ -137,6 +151,7 @@ struct GemmArgs {
   float* out_f;              // STORE_F32: out_f[i * out_batch + row * ldo + col]
   int64_t ldo, out_batch;
   int* status;               // device word that receives OLSGD_ETIMEOUT if a bounded wait gives up
+  FusedUpdateArgs upd;       // weight-gradient kernel only
 };
 // Plain CUDA-core version, used to validate the tensor-core kernel.
 cudaError_t launch_gemm_simt(const GemmArgs& a, cudaStream_t s);
@@ -171,6 +186,11 @@ struct ModelBuffers {
   __nv_bfloat16* dat[OLSGD_MAX_DIMS] = {nullptr};
   __nv_bfloat16* wt[OLSGD_MAX_DIMS] = {nullptr};
   int64_t w_off[OLSGD_MAX_DIMS] = {0}, b_off[OLSGD_MAX_DIMS] = {0};
+  // weights of parameter layer p are updated inside their weight-gradient GEMM
+  bool fused_layer[OLSGD_MAX_DIMS] = {false};
+  // what is left for the stand-alone update kernel: ranges [off, off + len) of a worker row
+  int n_ranges = 0;
+  int64_t range_off[OLSGD_MAX_DIMS + 1] = {0}, range_len[OLSGD_MAX_DIMS + 1] = {0};
 };
 struct StepIO {
   const float* x;                // x_k, [m][ld]
@@ -180,6 +200,8 @@ struct StepIO {
   const int32_t* idx;            // [m][batch]
   float* loss;                   // out: [m] or null
   int* status;                   // device status word (see GemmArgs::status)
+  FusedUpdateArgs upd;           // state pointers and factors for the fused epilogue (w_off unset)
+  cudaEvent_t wait_before_update;  // if non-null, the stream waits for it before x_out is written
 };
 // Lets model.cu count and time its launches without knowing the context type.
 struct ProfHook {

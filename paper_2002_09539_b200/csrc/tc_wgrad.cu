@@ -13,7 +13,17 @@
 //
 // Warp roles (192 threads): warp 0 TMA loads, warp 1 MMA issue + TMEM owner,
 // warps 2-5 epilogue.  Every mbarrier wait is bounded (see tc_common.cuh).
+//
+// FUSED variant (320 threads, eight epilogue warps): the gradient never goes to
+// memory.  Each 32 x 32 block of dW is turned, through a swizzled shared-memory
+// buffer, from "one accumulator row per thread" into "one 16-byte row segment
+// per thread", and the same thread then applies the parameter update to that
+// segment: Eq. 3 with the local Nesterov buffer, Eq. 4 on sync steps, the new
+// fp32 weights into the other half of the ping-pong pair and their bf16 copy for
+// the next forward pass.  All global accesses are whole 128-byte row segments.
+// That removes the 4-byte write and the 4-byte read of G_k per parameter.
 #include "tc_common.cuh"
+#include "update_math.cuh"
 
 namespace olsgd {
 namespace {
@@ -24,20 +34,79 @@ constexpr int kWN = 128;            // columns per tile = MMA N
 constexpr int kWStages = 4;         // upper bound of the B ring (one k-block of one tile per stage)
 constexpr int kMaxKB = 4;           // K <= 256
 
+struct WgradUpd {
+  const float* x_in;
+  float* x_out;
+  float* u;
+  const float* z;
+  __nv_bfloat16* shadow;
+  int64_t ld, w_off;
+  float gamma, mu, alpha;
+  int mom, sync;
+};
+
+// Update of one 32 x 32 block held as v[32] = row `lane` of the block.
+//   stage    this warp's 4 KB shared buffer for the gradient block
+//   xt, ut   the block's tiles of x_k and of the momentum buffer, brought into shared
+//            memory by TMA with the 128-byte swizzle (row r, 16-byte chunk q at q ^ (r % 8))
+//   blk_off  element offset of the block's corner inside a worker row
+//   ldw      row pitch of the weight matrix (its input width)
+template <bool MOM, bool SYNC>
+__device__ __forceinline__ void fused_block(const float (&v)[32], float* stage, const float* xt,
+                                            const float* ut, uint32_t xu_bar, uint32_t xu_parity,
+                                            volatile int* abort_flag, int lane, const WgradUpd& up,
+                                            int64_t wk_off, int64_t blk_off, int ldw, bool* ok) {
+  const int q = lane & 7, rsub = lane >> 3;
+  // the anchor strip comes straight from global memory (it is shared by all workers and
+  // mostly served by L2); issued first so that it is in flight during the staging
+  float4 zs[8];
+#pragma unroll
+  for (int t = 0; t < 8; ++t) {
+    zs[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (SYNC) zs[t] = *reinterpret_cast<const float4*>(up.z + blk_off + (int64_t)(t * 4 + rsub) * ldw + q * 4);
+  }
+  __syncwarp();   // the previous block's reads of the staging buffer are done
+  float4* mine = reinterpret_cast<float4*>(stage + lane * 32);
+#pragma unroll
+  for (int c = 0; c < 8; ++c)
+    mine[c ^ (lane & 7)] = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+  __syncwarp();
+  *ok = mbar_wait(xu_bar, xu_parity, abort_flag);
+  if (!*ok) return;
+#pragma unroll
+  for (int t = 0; t < 8; ++t) {
+    const int row = t * 4 + rsub, slot = q ^ (row & 7);
+    const int64_t off = blk_off + (int64_t)row * ldw + q * 4;
+    float4 x = reinterpret_cast<const float4*>(xt + row * 32)[slot];
+    float4 u = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (MOM) u = reinterpret_cast<const float4*>(ut + row * 32)[slot];
+    const float4 g = reinterpret_cast<const float4*>(stage + row * 32)[slot];
+    update4<MOM, SYNC>(x, u, g, zs[t], up.gamma, up.mu, up.alpha);
+    *reinterpret_cast<float4*>(up.x_out + wk_off + off) = x;
+    if (MOM) *reinterpret_cast<float4*>(up.u + wk_off + off) = u;
+    *reinterpret_cast<uint2*>(up.shadow + wk_off + off) = pack_bf16x4(x);
+  }
+}
+
 struct WgradCtl {
   uint64_t a_full;
   uint64_t b_full[kWStages];
   uint64_t b_empty[kWStages];
   uint64_t tmem_full[2];
   uint64_t tmem_empty[2];
+  uint64_t xu_full[8][2];   // fused variant: per epilogue warp, x/u tile pair landed
   uint32_t tmem_base;
   int abort_flag;
 };
 
-__global__ void __launch_bounds__(kThreads, 1)
+constexpr uint32_t kXuTile = 32 * 32 * 4;        // one fp32 tile of x or u
+constexpr uint32_t kXuPerWarp = 2 * 2 * kXuTile; // two buffers of (x, u)
+
+template <bool FUSED>
+__global__ void __launch_bounds__(FUSED ? 320 : kThreads, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                const __grid_constant__ CUtensorMap map_out, int num_kb, int n_stages,
-                int tiles_per_cta, int* status) {
+                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_u,
+                int num_kb, int n_stages, int tiles_per_cta, int ldw, WgradUpd up, int* status) {
   constexpr uint32_t kABlock = kBM * kBK * 2;   // one k-block of the A slab, 16 KB
   constexpr uint32_t kBBlock = kWN * kBK * 2;   // one k-block of a B tile, 16 KB
   constexpr uint32_t kEpiBuf = 32 * 32 * 4;     // one 32 x 32 fp32 block, 4 KB
@@ -48,7 +117,8 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   uint8_t* a_smem = base;                                   // num_kb blocks
   uint8_t* b_smem = a_smem + num_kb * kABlock;              // n_stages blocks
   uint8_t* e_smem = b_smem + n_stages * kBBlock;            // 4 warps x 2 buffers
-  WgradCtl* ctl = reinterpret_cast<WgradCtl*>(e_smem + 8 * kEpiBuf);
+  uint8_t* xu_smem = e_smem + 8 * kEpiBuf;                  // fused: 8 warps x 2 x (x, u) tiles
+  WgradCtl* ctl = reinterpret_cast<WgradCtl*>(xu_smem + (FUSED ? 8 * kXuPerWarp : 0));
   volatile int* abort_flag = &ctl->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -63,8 +133,11 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&ctl->tmem_full[b]), 1);
-      mbar_init(smem_u32(&ctl->tmem_empty[b]), 4);   // one arrival per epilogue warp
+      mbar_init(smem_u32(&ctl->tmem_empty[b]), FUSED ? 8 : 4);   // one arrival per epilogue warp
     }
+    if (FUSED)
+      for (int w = 0; w < 8; ++w)
+        for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&ctl->xu_full[w][b]), 1);
     ctl->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -129,6 +202,70 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         umma_commit(smem_u32(&ctl->b_empty[s]));
       }
       if (ok) umma_commit(smem_u32(&ctl->tmem_full[buf]));
+    }
+  } else if (FUSED && warp >= 2) {
+    // ---------------- epilogue with the parameter update fused in: eight warps, two per
+    // TMEM lane group, taking alternate 32-column blocks of every tile.  In the fused
+    // variant map_out covers x_k and map_u the momentum buffer; each warp prefetches the
+    // tiles of its next two blocks with TMA while it works on the current one.
+    const int ew = warp - 2, lane_group = warp & 3, half = ew >> 2;
+    float* stage = reinterpret_cast<float*>(e_smem + ew * kEpiBuf);
+    uint8_t* xu = xu_smem + ew * kXuPerWarp;
+    const int64_t wk_off = (int64_t)worker * up.ld;
+    const int n_blocks = tiles_per_cta * 2;
+    const int row0 = m0 + lane_group * 32;
+    int issued = 0;
+    auto issue = [&](int n) {
+      const int b = n & 1, col = (tile0 + (n >> 1)) * kWN + (half + 2 * (n & 1)) * 32;
+      const uint32_t bar = smem_u32(&ctl->xu_full[ew][b]);
+      mbar_expect_tx(bar, up.mom ? 2 * kXuTile : kXuTile);
+      tma_load_3d(smem_u32(xu + b * 2 * kXuTile), &map_out, bar, col, row0, worker);
+      if (up.mom) tma_load_3d(smem_u32(xu + b * 2 * kXuTile + kXuTile), &map_u, bar, col, row0, worker);
+      issued = n + 1;
+    };
+    if (lane == 0) {
+      issue(0);
+      if (n_blocks > 1) issue(1);
+    }
+    bool ok = true;
+    int n = 0;
+    for (; n < n_blocks && ok; ++n) {
+      const int j = n >> 1, c = half + 2 * (n & 1), buf = j & 1, use = j >> 1, b = n & 1;
+      if ((n & 1) == 0) {
+        ok = mbar_wait(smem_u32(&ctl->tmem_full[buf]), use & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+      }
+      float v[32];
+      tmem_ld32(tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)(buf * kWN + c * 32), v);
+      const int64_t blk_off = up.w_off + (int64_t)row0 * ldw + (tile0 + j) * kWN + c * 32;
+      const float* xt = reinterpret_cast<const float*>(xu + b * 2 * kXuTile);
+      const float* ut = xt + kXuTile / 4;
+      const uint32_t bar = smem_u32(&ctl->xu_full[ew][b]);
+      const uint32_t par = (uint32_t)(n >> 1) & 1u;
+      if (up.mom) {
+        if (up.sync) fused_block<true, true>(v, stage, xt, ut, bar, par, abort_flag, lane, up, wk_off, blk_off, ldw, &ok);
+        else fused_block<true, false>(v, stage, xt, ut, bar, par, abort_flag, lane, up, wk_off, blk_off, ldw, &ok);
+      } else {
+        if (up.sync) fused_block<false, true>(v, stage, xt, ut, bar, par, abort_flag, lane, up, wk_off, blk_off, ldw, &ok);
+        else fused_block<false, false>(v, stage, xt, ut, bar, par, abort_flag, lane, up, wk_off, blk_off, ldw, &ok);
+      }
+      if (!ok) break;
+      __syncwarp();   // every lane has read this buffer's tiles: it may be refilled
+      if (lane == 0 && n + 2 < n_blocks) issue(n + 2);
+      if (n & 1) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[buf]));
+      }
+    }
+    if (lane == 0 && n < issued) {
+      // gave up early: wait (bounded) for the tiles that are still on their way
+      for (int t = n; t < issued; ++t) {
+        const uint32_t bar = smem_u32(&ctl->xu_full[ew][t & 1]);
+        for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar, (uint32_t)(t >> 1) & 1u); ++it) {
+        }
+      }
     }
   } else if (warp >= 2) {
     // ---------------- epilogue
@@ -197,21 +334,42 @@ bool wgrad_tc_supported(const GemmArgs& a) {
   if (a.Ma % kBM != 0 || a.Nb % kWN != 0 || a.K % kBK != 0 || a.K < kBK || a.K > kMaxKB * kBK)
     return false;
   if (a.lda % 8 || a.ldb % 8 || a.a_batch % 8 || a.b_batch % 8) return false;
-  if (!al16(a.A) || !al16(a.B) || !al16(a.out_f) || a.ldo % 4 || a.out_batch % 4) return false;
+  if (!al16(a.A) || !al16(a.B)) return false;
+  if (a.upd.enabled) {
+    const FusedUpdateArgs& u = a.upd;
+    if (a.K > 2 * kBK) return false;   // the x/u tile ring needs the shared memory
+    if (!al16(u.x_in) || !al16(u.x_out) || !al16(u.shadow) || (u.u && !al16(u.u)) ||
+        (u.sync && !al16(u.z)))
+      return false;
+    if (u.ld % 8 || u.w_off % 8) return false;
+  } else if (!al16(a.out_f) || a.ldo % 4 || a.out_batch % 4) {
+    return false;
+  }
   return true;
 }
 
 cudaError_t launch_wgrad_tc(const GemmArgs& a, cudaStream_t s) {
   if (!wgrad_tc_supported(a)) return cudaErrorInvalidValue;
+  const bool fused = a.upd.enabled != 0;
   CUtensorMap ma, mb, mo;
   if (!make_map(&ma, a.A, a.K, a.Ma, a.m, a.lda, a.a_batch, kBM)) return cudaErrorInvalidValue;
   if (!make_map(&mb, a.B, a.K, a.Nb, a.m, a.ldb, a.b_batch, kWN)) return cudaErrorInvalidValue;
-  if (!make_map_f32(&mo, a.out_f, a.Nb, a.Ma, a.m, a.ldo, a.out_batch, 32)) return cudaErrorInvalidValue;
+  CUtensorMap mu = ma;
+  if (fused) {
+    // map_out covers x_k, map_u the momentum buffer: [m][Ma][Nb] fp32 views of the weight matrix
+    if (!make_map_f32(&mo, a.upd.x_in + a.upd.w_off, a.Nb, a.Ma, a.m, a.Nb, a.upd.ld, 32))
+      return cudaErrorInvalidValue;
+    if (a.upd.u && a.upd.mu != 0.f &&
+        !make_map_f32(&mu, a.upd.u + a.upd.w_off, a.Nb, a.Ma, a.m, a.Nb, a.upd.ld, 32))
+      return cudaErrorInvalidValue;
+  } else if (!make_map_f32(&mo, a.out_f, a.Nb, a.Ma, a.m, a.ldo, a.out_batch, 32)) {
+    return cudaErrorInvalidValue;
+  }
   const int num_kb = a.K / kBK;
   const int n_tiles = a.Nb / kWN;
   // about two CTAs per SM in one wave: split the tile range of a slab over `chunks` CTAs
   const int slabs = (a.Ma / kBM) * a.m;
-  int chunks = (2 * 148) / slabs;
+  int chunks = ((fused ? 1 : 2) * 148) / slabs;
   if (chunks < 1) chunks = 1;
   if (chunks > n_tiles) chunks = n_tiles;
   while (n_tiles % chunks) --chunks;
@@ -221,17 +379,39 @@ cudaError_t launch_wgrad_tc(const GemmArgs& a, cudaStream_t s) {
   int n_stages = fixed < per_cta ? (int)((per_cta - fixed) / (kWN * kBK * 2)) : 0;
   if (n_stages > kWStages) n_stages = kWStages;
   if (n_stages < 2) n_stages = 2;
-  const size_t smem = fixed + (size_t)n_stages * kWN * kBK * 2;
-  static size_t configured = 0;
-  if (smem > configured) {
-    cudaError_t e = cudaFuncSetAttribute(wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
+  if (fused) n_stages = 2;   // one CTA per SM: the rest of the shared memory holds x/u tiles
+  const size_t smem = fixed + (size_t)n_stages * kWN * kBK * 2 + (fused ? 8 * kXuPerWarp : 0);
+  static size_t configured[2] = {0, 0};
+  if (smem > configured[fused]) {
+    cudaError_t e = fused ? cudaFuncSetAttribute(wgrad_tc_kernel<true>,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                          : cudaFuncSetAttribute(wgrad_tc_kernel<false>,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    configured = smem;
+    configured[fused] = smem;
+  }
+  WgradUpd up{};
+  if (fused) {
+    up.x_in = a.upd.x_in;
+    up.x_out = a.upd.x_out;
+    up.u = a.upd.u;
+    up.z = a.upd.z;
+    up.shadow = a.upd.shadow;
+    up.ld = a.upd.ld;
+    up.w_off = a.upd.w_off;
+    up.gamma = a.upd.gamma;
+    up.mu = a.upd.mu;
+    up.alpha = a.upd.alpha;
+    up.mom = (a.upd.u != nullptr && a.upd.mu != 0.f) ? 1 : 0;
+    up.sync = a.upd.sync;
   }
   dim3 grid(chunks, a.Ma / kBM, a.m);
-  wgrad_tc_kernel<<<grid, kThreads, smem, s>>>(ma, mb, mo, num_kb, n_stages, n_tiles / chunks,
-                                               a.status);
+  if (fused)
+    wgrad_tc_kernel<true><<<grid, 320, smem, s>>>(ma, mb, mo, mu, num_kb, n_stages,
+                                                  n_tiles / chunks, a.Nb, up, a.status);
+  else
+    wgrad_tc_kernel<false><<<grid, kThreads, smem, s>>>(ma, mb, mo, mu, num_kb, n_stages,
+                                                        n_tiles / chunks, a.Nb, up, a.status);
   return cudaGetLastError();
 }
 

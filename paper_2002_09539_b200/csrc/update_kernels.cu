@@ -6,6 +6,7 @@
 // parameter dimension, and each thread keeps several independent loads in
 // flight by unrolling over the worker dimension.
 #include "olsgd_internal.h"
+#include "update_math.cuh"
 
 namespace olsgd {
 namespace {
@@ -60,40 +61,12 @@ fused_update_kernel(const float* __restrict__ x_in, float* __restrict__ x_out,
       const int i = ib + t;
       if (i < i1) {
         float4 x = xv[t];
-        const float4 gg = gv[t];
-        if (MOM) {
-          // u <- mu u + g ;  x <- x - gamma (g + mu u)
-          float4 uu = uv[t];
-          uu.x = fmaf(mu, uu.x, gg.x);
-          uu.y = fmaf(mu, uu.y, gg.y);
-          uu.z = fmaf(mu, uu.z, gg.z);
-          uu.w = fmaf(mu, uu.w, gg.w);
-          reinterpret_cast<float4*>(u + (int64_t)i * ld)[col4] = uu;
-          x.x -= gamma * fmaf(mu, uu.x, gg.x);
-          x.y -= gamma * fmaf(mu, uu.y, gg.y);
-          x.z -= gamma * fmaf(mu, uu.z, gg.z);
-          x.w -= gamma * fmaf(mu, uu.w, gg.w);
-        } else {
-          x.x -= gamma * gg.x;  // Eq. 3
-          x.y -= gamma * gg.y;
-          x.z -= gamma * gg.z;
-          x.w -= gamma * gg.w;
-        }
-        if (SYNC) {  // Eq. 4
-          x.x -= alpha * (x.x - zz.x);
-          x.y -= alpha * (x.y - zz.y);
-          x.z -= alpha * (x.z - zz.z);
-          x.w -= alpha * (x.w - zz.w);
-        }
+        float4 uu = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (MOM) uu = uv[t];
+        update4<MOM, SYNC>(x, uu, gv[t], zz, gamma, mu, alpha);
+        if (MOM) reinterpret_cast<float4*>(u + (int64_t)i * ld)[col4] = uu;
         reinterpret_cast<float4*>(x_out + (int64_t)i * ld)[col4] = x;
-        if (SHADOW) {
-          __nv_bfloat162 lo = __floats2bfloat162_rn(x.x, x.y);
-          __nv_bfloat162 hi = __floats2bfloat162_rn(x.z, x.w);
-          uint2 pk;
-          pk.x = *reinterpret_cast<uint32_t*>(&lo);
-          pk.y = *reinterpret_cast<uint32_t*>(&hi);
-          reinterpret_cast<uint2*>(shadow + (int64_t)i * ld)[col4] = pk;
-        }
+        if (SHADOW) reinterpret_cast<uint2*>(shadow + (int64_t)i * ld)[col4] = pack_bf16x4(x);
       }
     }
   }

@@ -94,7 +94,8 @@ def test_local_step_and_period_sync_equal_run():
 
 
 # ------------------------------------------------------------------ bf16 MLP path
-# gemm_bf16 = 1: tcgen05 tensor-core GEMMs; 2: the same bf16 data flow on CUDA cores.
+# gemm_bf16 = 1: tcgen05 tensor-core GEMMs with the update fused into the weight-gradient
+# epilogue; 3: the same GEMMs, separate update kernel; 2: the same data flow on CUDA cores.
 # The oracle runs with bf16-rounded GEMM operands, so what is left is fp32-vs-fp64
 # accumulation and the occasional operand that rounds to the neighbouring bf16
 # value (2^-8 relative) on one side only.
@@ -116,7 +117,7 @@ MLP_SHAPES = [([64, 128, 10], 2, 40, 64, 2, 5),
 
 
 @pytest.mark.parametrize("dims,m,n,batch,tau,iters", MLP_SHAPES)
-@pytest.mark.parametrize("gemm_bf16", [2, 1])
+@pytest.mark.parametrize("gemm_bf16", [2, 3, 1])
 def test_mlp_bf16_small(dims, m, n, batch, tau, iters, gemm_bf16):
     opt, st, lg, lo = _mlp_case(dims, m, n, batch, tau, iters, gemm_bf16)
     assert np.isfinite(lg).all()
@@ -128,3 +129,18 @@ def test_mlp_cuda_core_path_accepts_small_batches():
     opt, st, lg, lo = _mlp_case([64, 128, 10], 2, 40, 8, 2, 4, 2)
     assert np.abs(lg - lo).max() <= TOL_BF16_LOSS * np.abs(lo).max()
     assert state_err(opt, st) <= TOL_BF16_PARAM
+
+
+@pytest.mark.parametrize("dims,m,n,batch,tau,iters", MLP_SHAPES[1:])
+def test_fused_weight_gradient_update_gives_the_bits_of_the_separate_kernel(dims, m, n, batch, tau,
+                                                                            iters):
+    # same GEMM accumulators, same update arithmetic: fusing only removes the round trip
+    # of the gradient through memory
+    a, _, la, _ = _mlp_case(dims, m, n, batch, tau, iters, 1)
+    b, _, lb, _ = _mlp_case(dims, m, n, batch, tau, iters, 3)
+    xa, za, va = a.state()
+    xb, zb, vb = b.state()
+    assert np.array_equal(la, lb)
+    assert np.array_equal(xa, xb) and np.array_equal(za, zb) and np.array_equal(va, vb)
+    for i in (0, m - 1):
+        assert np.array_equal(a.get_params(-5 - i), b.get_params(-5 - i))
