@@ -1,18 +1,20 @@
 // Weight-gradient GEMM of the worker-batched backward pass on the tensor cores:
 //   dW[i] [Ma][Nb] = A[i] [Ma][K] * B[i] [Nb][K]^T,   K = minibatch size (64..256),
-// fp32 result written straight into the stacked gradient G_k (Eq. 7).
+// either stored as fp32 into the stacked gradient G_k (Eq. 7) or consumed on the
+// spot by the parameter update (FUSED).
 //
-// The contraction is short and the output large, so the kernel is bound by the
-// fp32 store.  One CTA owns a 128-row slab of one worker's dW and walks over a
-// range of 128-column tiles: its A slab (128 x K bf16) is loaded once and stays
-// in shared memory, B tiles stream through a small TMA ring, and the fp32
-// accumulator is double-buffered in tensor memory so that the MMAs of tile j+1
-// run under the epilogue of tile j.  The epilogue moves 32 x 32 blocks from
-// TMEM through swizzled shared memory to global memory with TMA stores, which
-// writes whole 128-byte lines.
+// The contraction is short and the output large, so the kernel is bound by
+// memory traffic, not by the tensor pipe.  The work is cut into units of one
+// 128 x 128 tile.  A slab is a 128-row band of one worker's dW; a few CTAs share
+// a slab and take its tiles round-robin, so that together they sweep adjacent
+// column tiles at the same time.  A CTA's A operand (128 x K bf16) stays in
+// shared memory; B tiles stream through a small TMA ring; the fp32 accumulator
+// is double-buffered in tensor memory so that the MMAs of unit j+1 run under
+// the epilogue of unit j.
 //
-// Warp roles (192 threads): warp 0 TMA loads, warp 1 MMA issue + TMEM owner,
-// warps 2-5 epilogue.  Every mbarrier wait is bounded (see tc_common.cuh).
+// Plain variant (192 threads): warp 0 TMA loads, warp 1 MMA issue + TMEM owner,
+// warps 2-5 epilogue, which moves 32 x 32 blocks from TMEM through swizzled
+// shared memory to global memory with TMA stores (whole 128-byte lines).
 //
 // FUSED variant (320 threads, eight epilogue warps): the gradient never goes to
 // memory.  Each 32 x 32 block of dW is turned, through a swizzled shared-memory
@@ -20,8 +22,12 @@
 // per thread", and the same thread then applies the parameter update to that
 // segment: Eq. 3 with the local Nesterov buffer, Eq. 4 on sync steps, the new
 // fp32 weights into the other half of the ping-pong pair and their bf16 copy for
-// the next forward pass.  All global accesses are whole 128-byte row segments.
+// the next forward pass.  The matching tiles of x_k and of the momentum buffer
+// are prefetched by TMA two blocks ahead into a per-warp ring, which is what
+// keeps enough bytes in flight; results leave as whole 128-byte row segments.
 // That removes the 4-byte write and the 4-byte read of G_k per parameter.
+//
+// Every mbarrier wait is bounded (see tc_common.cuh).
 #include "tc_common.cuh"
 #include "update_math.cuh"
 
@@ -44,6 +50,19 @@ struct WgradUpd {
   float gamma, mu, alpha;
   int mom, sync;
 };
+
+// Where a unit lives.
+struct UnitPos {
+  int slab, worker, m0, col;
+};
+__device__ __forceinline__ UnitPos unit_pos(int unit, int n_tiles, int m_tiles) {
+  UnitPos p;
+  p.slab = unit / n_tiles;
+  p.col = (unit - p.slab * n_tiles) * kWN;
+  p.worker = p.slab / m_tiles;
+  p.m0 = (p.slab - p.worker * m_tiles) * kBM;
+  return p;
+}
 
 // Update of one 32 x 32 block held as v[32] = row `lane` of the block.
 //   stage    this warp's 4 KB shared buffer for the gradient block
@@ -89,7 +108,7 @@ __device__ __forceinline__ void fused_block(const float (&v)[32], float* stage, 
 }
 
 struct WgradCtl {
-  uint64_t a_full;
+  uint64_t a_full, a_empty;
   uint64_t b_full[kWStages];
   uint64_t b_empty[kWStages];
   uint64_t tmem_full[2];
@@ -106,7 +125,8 @@ template <bool FUSED>
 __global__ void __launch_bounds__(FUSED ? 320 : kThreads, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_u,
-                int num_kb, int n_stages, int tiles_per_cta, int ldw, WgradUpd up, int* status) {
+                int num_kb, int n_stages, int n_tiles, int m_tiles, int chunks, int ldw,
+                WgradUpd up, int* status) {
   constexpr uint32_t kABlock = kBM * kBK * 2;   // one k-block of the A slab, 16 KB
   constexpr uint32_t kBBlock = kWN * kBK * 2;   // one k-block of a B tile, 16 KB
   constexpr uint32_t kEpiBuf = 32 * 32 * 4;     // one 32 x 32 fp32 block, 4 KB
@@ -116,17 +136,22 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                                              ~static_cast<uintptr_t>(1023));
   uint8_t* a_smem = base;                                   // num_kb blocks
   uint8_t* b_smem = a_smem + num_kb * kABlock;              // n_stages blocks
-  uint8_t* e_smem = b_smem + n_stages * kBBlock;            // 4 warps x 2 buffers
+  uint8_t* e_smem = b_smem + n_stages * kBBlock;            // 8 x 4 KB gradient staging
   uint8_t* xu_smem = e_smem + 8 * kEpiBuf;                  // fused: 8 warps x 2 x (x, u) tiles
   WgradCtl* ctl = reinterpret_cast<WgradCtl*>(xu_smem + (FUSED ? 8 * kXuPerWarp : 0));
   volatile int* abort_flag = &ctl->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.y * kBM, worker = blockIdx.z;
-  const int tile0 = blockIdx.x * tiles_per_cta;
+  // this CTA's units: every `chunks`-th tile of one slab, so that the CTAs that share a
+  // slab (neighbours in the grid, running at the same time) sweep adjacent column tiles
+  // together and touch each DRAM page while it is open
+  const int my_slab = blockIdx.x / chunks, my_first = blockIdx.x - my_slab * chunks;
+  const int n_units = (n_tiles - my_first + chunks - 1) / chunks;
+  auto unit_of = [&](int j) { return my_slab * n_tiles + my_first + j * chunks; };
 
   if (threadIdx.x == 0) {
     mbar_init(smem_u32(&ctl->a_full), 1);
+    mbar_init(smem_u32(&ctl->a_empty), 1);
     for (int s = 0; s < n_stages; ++s) {
       mbar_init(smem_u32(&ctl->b_full[s]), 1);
       mbar_init(smem_u32(&ctl->b_empty[s]), 1);
@@ -150,12 +175,21 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   if (warp == 0 && lane == 0) {
     // ---------------- TMA producer
     const uint32_t a_full = smem_u32(&ctl->a_full);
-    mbar_expect_tx(a_full, num_kb * kABlock);
-    for (int kb = 0; kb < num_kb; ++kb)
-      tma_load_3d(smem_u32(a_smem + kb * kABlock), &map_a, a_full, kb * kBK, m0, worker);
-    int issued = 0;
-    bool ok = true;
-    for (int j = 0; j < tiles_per_cta && ok; ++j) {
+    int issued = 0, visit = -1, cur_slab = -1;
+    bool ok = true, a_pending = false;
+    for (int j = 0; j < n_units && ok; ++j) {
+      const UnitPos p = unit_pos(unit_of(j), n_tiles, m_tiles);
+      if (p.slab != cur_slab) {
+        // new slab: its A operand replaces the old one once the MMAs that read it retired
+        ++visit;
+        cur_slab = p.slab;
+        ok = mbar_wait(smem_u32(&ctl->a_empty), (uint32_t)(visit & 1) ^ 1u, abort_flag);
+        if (!ok) break;
+        mbar_expect_tx(a_full, num_kb * kABlock);
+        for (int kb = 0; kb < num_kb; ++kb)
+          tma_load_3d(smem_u32(a_smem + kb * kABlock), &map_a, a_full, kb * kBK, p.m0, p.worker);
+        a_pending = true;
+      }
       for (int kb = 0; kb < num_kb; ++kb) {
         const int t = j * num_kb + kb, s = t % n_stages;
         const uint32_t ph = (t / n_stages) & 1;
@@ -163,13 +197,15 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (!ok) break;
         const uint32_t full = smem_u32(&ctl->b_full[s]);
         mbar_expect_tx(full, kBBlock);
-        tma_load_3d(smem_u32(b_smem + s * kBBlock), &map_b, full, kb * kBK, (tile0 + j) * kWN, worker);
+        tma_load_3d(smem_u32(b_smem + s * kBBlock), &map_b, full, kb * kBK, p.col, p.worker);
         issued = t + 1;
       }
     }
     if (*abort_flag) {
-      for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(a_full, 0); ++it) {
-      }
+      // drain: wait (bounded) for the copies this thread still has in flight
+      if (a_pending)
+        for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(a_full, (uint32_t)(visit & 1)); ++it) {
+        }
       for (int t = max(0, issued - n_stages); t < issued; ++t) {
         const uint32_t full = smem_u32(&ctl->b_full[t % n_stages]);
         const uint32_t ph = (t / n_stages) & 1;
@@ -180,8 +216,16 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   } else if (warp == 1 && lane == 0) {
     // ---------------- MMA issuer
     constexpr uint32_t idesc = instr_desc_bf16(kWN);
-    bool ok = mbar_wait(smem_u32(&ctl->a_full), 0, abort_flag);
-    for (int j = 0; j < tiles_per_cta && ok; ++j) {
+    bool ok = true;
+    int visit = -1, cur_slab = -1;
+    for (int j = 0; j < n_units && ok; ++j) {
+      const int unit = unit_of(j), slab = unit / n_tiles;
+      if (slab != cur_slab) {
+        ++visit;
+        cur_slab = slab;
+        ok = mbar_wait(smem_u32(&ctl->a_full), (uint32_t)(visit & 1), abort_flag);
+        if (!ok) break;
+      }
       const int buf = j & 1, use = j >> 1;
       ok = mbar_wait(smem_u32(&ctl->tmem_empty[buf]), (use & 1) ^ 1, abort_flag);
       if (!ok) break;
@@ -201,30 +245,32 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     (kb > 0 || k > 0) ? 1u : 0u);
         umma_commit(smem_u32(&ctl->b_empty[s]));
       }
-      if (ok) umma_commit(smem_u32(&ctl->tmem_full[buf]));
+      if (!ok) break;
+      umma_commit(smem_u32(&ctl->tmem_full[buf]));
+      // last unit of this slab in this CTA: the A buffer is free once these MMAs retire
+      if (j + 1 < n_units && unit_of(j + 1) / n_tiles != slab) umma_commit(smem_u32(&ctl->a_empty));
     }
   } else if (FUSED && warp >= 2) {
     // ---------------- epilogue with the parameter update fused in: eight warps, two per
-    // TMEM lane group, taking alternate 32-column blocks of every tile.  In the fused
+    // TMEM lane group, taking alternate 32-column blocks of every unit.  In the fused
     // variant map_out covers x_k and map_u the momentum buffer; each warp prefetches the
     // tiles of its next two blocks with TMA while it works on the current one.
     const int ew = warp - 2, lane_group = warp & 3, half = ew >> 2;
     float* stage = reinterpret_cast<float*>(e_smem + ew * kEpiBuf);
     uint8_t* xu = xu_smem + ew * kXuPerWarp;
-    const int64_t wk_off = (int64_t)worker * up.ld;
-    const int n_blocks = tiles_per_cta * 2;
-    const int row0 = m0 + lane_group * 32;
+    const int n_blocks = n_units * 2;
     int issued = 0;
     auto issue = [&](int n) {
-      const int b = n & 1, col = (tile0 + (n >> 1)) * kWN + (half + 2 * (n & 1)) * 32;
+      const UnitPos p = unit_pos(unit_of(n >> 1), n_tiles, m_tiles);
+      const int b = n & 1, col = p.col + (half + 2 * (n & 1)) * 32, row = p.m0 + lane_group * 32;
       const uint32_t bar = smem_u32(&ctl->xu_full[ew][b]);
       mbar_expect_tx(bar, up.mom ? 2 * kXuTile : kXuTile);
-      tma_load_3d(smem_u32(xu + b * 2 * kXuTile), &map_out, bar, col, row0, worker);
-      if (up.mom) tma_load_3d(smem_u32(xu + b * 2 * kXuTile + kXuTile), &map_u, bar, col, row0, worker);
+      tma_load_3d(smem_u32(xu + b * 2 * kXuTile), &map_out, bar, col, row, p.worker);
+      if (up.mom) tma_load_3d(smem_u32(xu + b * 2 * kXuTile + kXuTile), &map_u, bar, col, row, p.worker);
       issued = n + 1;
     };
     if (lane == 0) {
-      issue(0);
+      if (n_blocks > 0) issue(0);
       if (n_blocks > 1) issue(1);
     }
     bool ok = true;
@@ -236,9 +282,11 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (!ok) break;
         tc_fence_after();
       }
+      const UnitPos p = unit_pos(unit_of(j), n_tiles, m_tiles);
       float v[32];
       tmem_ld32(tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)(buf * kWN + c * 32), v);
-      const int64_t blk_off = up.w_off + (int64_t)row0 * ldw + (tile0 + j) * kWN + c * 32;
+      const int64_t wk_off = (int64_t)p.worker * up.ld;
+      const int64_t blk_off = up.w_off + (int64_t)(p.m0 + lane_group * 32) * ldw + p.col + c * 32;
       const float* xt = reinterpret_cast<const float*>(xu + b * 2 * kXuTile);
       const float* ut = xt + kXuTile / 4;
       const uint32_t bar = smem_u32(&ctl->xu_full[ew][b]);
@@ -268,17 +316,17 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       }
     }
   } else if (warp >= 2) {
-    // ---------------- epilogue
+    // ---------------- epilogue: fp32 store
     const int lane_group = warp & 3;
     uint8_t* my_buf = e_smem + (warp - 2) * 2 * kEpiBuf;
     int store_count = 0;
     bool ok = true;
-    for (int j = 0; j < tiles_per_cta && ok; ++j) {
+    for (int j = 0; j < n_units && ok; ++j) {
       const int buf = j & 1, use = j >> 1;
       ok = mbar_wait(smem_u32(&ctl->tmem_full[buf]), use & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
-      const int col_tile = (tile0 + j) * kWN;
+      const UnitPos p = unit_pos(unit_of(j), n_tiles, m_tiles);
 #pragma unroll 1
       for (int c = 0; c < kWN / 32; ++c) {
         float v[32];
@@ -295,7 +343,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         fence_async_smem();
         __syncwarp();
         if (lane == 0) {
-          tma_store_3d(&map_out, smem_u32(stage), col_tile + c * 32, m0 + lane_group * 32, worker);
+          tma_store_3d(&map_out, smem_u32(stage), p.col + c * 32, p.m0 + lane_group * 32, p.worker);
           bulk_commit();
         }
         ++store_count;
@@ -335,6 +383,7 @@ bool wgrad_tc_supported(const GemmArgs& a) {
     return false;
   if (a.lda % 8 || a.ldb % 8 || a.a_batch % 8 || a.b_batch % 8) return false;
   if (!al16(a.A) || !al16(a.B)) return false;
+  if ((int64_t)(a.Ma / kBM) * a.m * (a.Nb / kWN) > 0x7FFFFFFF) return false;
   if (a.upd.enabled) {
     const FusedUpdateArgs& u = a.upd;
     if (a.K > 2 * kBK) return false;   // the x/u tile ring needs the shared memory
@@ -366,21 +415,22 @@ cudaError_t launch_wgrad_tc(const GemmArgs& a, cudaStream_t s) {
     return cudaErrorInvalidValue;
   }
   const int num_kb = a.K / kBK;
-  const int n_tiles = a.Nb / kWN;
-  // about two CTAs per SM in one wave: split the tile range of a slab over `chunks` CTAs
-  const int slabs = (a.Ma / kBM) * a.m;
-  int chunks = ((fused ? 1 : 2) * 148) / slabs;
-  if (chunks < 1) chunks = 1;
-  if (chunks > n_tiles) chunks = n_tiles;
-  while (n_tiles % chunks) --chunks;
-  // as many B stages as still let two CTAs share an SM's 227 KB of shared memory
+  const int n_tiles = a.Nb / kWN, m_tiles = a.Ma / kBM;
+  // shared memory: the fused variant fills an SM by itself (x/u tile rings); the plain one
+  // takes as many B stages as still let two CTAs share an SM's 227 KB
   const size_t fixed = (size_t)num_kb * kBM * kBK * 2 + 8 * 32 * 32 * 4 + sizeof(WgradCtl) + 1024;
   const size_t per_cta = (227 * 1024) / 2 - 1024;
   int n_stages = fixed < per_cta ? (int)((per_cta - fixed) / (kWN * kBK * 2)) : 0;
   if (n_stages > kWStages) n_stages = kWStages;
-  if (n_stages < 2) n_stages = 2;
-  if (fused) n_stages = 2;   // one CTA per SM: the rest of the shared memory holds x/u tiles
+  if (n_stages < 2 || fused) n_stages = 2;
   const size_t smem = fixed + (size_t)n_stages * kWN * kBK * 2 + (fused ? 8 * kXuPerWarp : 0);
+  // `chunks` CTAs per slab, about four CTAs per SM in total (measured: the count hardly
+  // matters, the alignment to slabs and the joint sweep do)
+  const int slabs = m_tiles * a.m;
+  int chunks = (4 * 148) / slabs;
+  if (chunks < 1) chunks = 1;
+  if (chunks > n_tiles) chunks = n_tiles;
+  const int ctas = slabs * chunks;
   static size_t configured[2] = {0, 0};
   if (smem > configured[fused]) {
     cudaError_t e = fused ? cudaFuncSetAttribute(wgrad_tc_kernel<true>,
@@ -405,13 +455,12 @@ cudaError_t launch_wgrad_tc(const GemmArgs& a, cudaStream_t s) {
     up.mom = (a.upd.u != nullptr && a.upd.mu != 0.f) ? 1 : 0;
     up.sync = a.upd.sync;
   }
-  dim3 grid(chunks, a.Ma / kBM, a.m);
   if (fused)
-    wgrad_tc_kernel<true><<<grid, 320, smem, s>>>(ma, mb, mo, mu, num_kb, n_stages,
-                                                  n_tiles / chunks, a.Nb, up, a.status);
+    wgrad_tc_kernel<true><<<ctas, 320, smem, s>>>(ma, mb, mo, mu, num_kb, n_stages, n_tiles, m_tiles,
+                                                  chunks, a.Nb, up, a.status);
   else
-    wgrad_tc_kernel<false><<<grid, kThreads, smem, s>>>(ma, mb, mo, mu, num_kb, n_stages,
-                                                        n_tiles / chunks, a.Nb, up, a.status);
+    wgrad_tc_kernel<false><<<ctas, kThreads, smem, s>>>(ma, mb, mo, mu, num_kb, n_stages, n_tiles,
+                                                        m_tiles, chunks, a.Nb, up, a.status);
   return cudaGetLastError();
 }
 
