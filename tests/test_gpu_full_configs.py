@@ -88,7 +88,10 @@ def test_mlp_configs_first_iterations_against_exact_oracle(name, iters, tol_para
 # No implementation can meet a 2e-2 bound on the loss after the full 1000 iterations,
 # so the bound is enforced on the stored checkpoints up to STRICT_UNTIL and the end of
 # the run is checked for having trained to the same level.
-STRICT_UNTIL = {"c3": 250, "c4": 100}
+# Config 4 (tau = 8, alpha = 0.5) stays reproducible to the end, so there the 2e-2 bound is
+# enforced on every checkpoint and on the final objective.
+STRICT_UNTIL = {"c3": 250, "c4": 800}
+FINAL_STRICT = {"c3": False, "c4": True}
 
 
 @pytest.mark.parametrize("name", ["c3", "c4"])
@@ -108,10 +111,14 @@ def test_mlp_configs_full_length(name):
     xbar, z = opt.get_params(-4).copy(), opt.get_params(-1).copy()
     F_mean = models.full_objective("mlp", c["dims"], xbar, X, y)
     F_anchor = models.full_objective("mlp", c["dims"], z, X, y)
-    first = float(lg[0].mean())
-    assert 0.5 * gold["F_mean_model"] <= F_mean <= 2.0 * gold["F_mean_model"], F_mean
-    assert 0.5 * gold["F_anchor"] <= F_anchor <= 2.0 * gold["F_anchor"], F_anchor
-    assert F_mean < 0.25 * first
+    if FINAL_STRICT[name]:
+        assert abs(F_mean - gold["F_mean_model"]) <= TOL_BF16_LOSS * gold["F_mean_model"], F_mean
+        assert abs(F_anchor - gold["F_anchor"]) <= TOL_BF16_LOSS * gold["F_anchor"], F_anchor
+    else:
+        assert 0.5 * gold["F_mean_model"] <= F_mean <= 2.0 * gold["F_mean_model"], F_mean
+        assert 0.5 * gold["F_anchor"] <= F_anchor <= 2.0 * gold["F_anchor"], F_anchor
+    # it trained: the minibatch loss at the end is far below the first iteration's
+    assert float(lg[-10:].mean()) < 0.5 * float(lg[0].mean())
     assert abs(np.linalg.norm(xbar) - gold["norm2_mean_model"]) <= 0.05 * gold["norm2_mean_model"]
 
 
