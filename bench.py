@@ -220,12 +220,7 @@ def run_ours(args, rank, world):
         opt.main.wait_stream(opt.side)
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), world, "cuda")
 
     # ---- device-resident throughput
     opt.run(W)
@@ -287,10 +282,7 @@ def run_ours(args, rank, world):
     opt.join()                      # host sees the last losses here
     t1 = time.perf_counter()
     e2e_ms = (t1 - t0) * 1e3
-    if world > 1:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, world, "cuda")
     assert np.isfinite(loss_h[W:].numpy()).all()
     e2e = dict(value=round(world * m * K / (e2e_ms * 1e-3), 1), unit=UNIT,
                h2d_bytes_per_step=int(m * B * d0 * 4 + m * B * 4), d2h_bytes_per_step=int(m * 4),
@@ -423,6 +415,17 @@ def run_flat_sweep(args, rank, world):
                          peak_source=peaks["source"]),
         "sweep": points,
     }
+
+
+def max_over_ranks(value, world, device):
+    """The slowest rank's value (timings are reported as the max over ranks)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
 
 
 def workload_name(name, c):
