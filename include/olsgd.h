@@ -138,6 +138,16 @@ olsgd_status olsgd_local_step_host(olsgd_ctx* ctx, const float* Xb_host, const v
 /* Block the host until every stream of the context is idle.                 */
 olsgd_status olsgd_join(olsgd_ctx* ctx);
 
+/* Every wait a kernel of this library performs on a barrier is bounded; a wait that runs
+ * out makes the kernel return early and the next joining call (olsgd_join,
+ * olsgd_get_params) return OLSGD_ETIMEOUT.  olsgd_selftest_wait_timeout exercises that
+ * path without any fault: it launches a kernel whose one thread waits, for at most
+ * limit_ms milliseconds, on a barrier that nothing ever arrives on.  After it, olsgd_join
+ * returns OLSGD_ETIMEOUT until olsgd_clear_status is called; the context and the GPU
+ * stay usable throughout.  limit_ms must be in [1, 2000].                        */
+olsgd_status olsgd_selftest_wait_timeout(olsgd_ctx* ctx, int32_t limit_ms);
+olsgd_status olsgd_clear_status(olsgd_ctx* ctx);
+
 /* Same iteration for OLSGD_FLAT: the stacked gradients G_k (Eq. 7 without its
  * zero column) come from the caller.
  *   g_device  float32 [m][P], device, row stride P; read on the main stream */

@@ -64,6 +64,8 @@ def load_library():
         "olsgd_local_step_with_grads": (i32, [vp, vp]),
         "olsgd_local_step_host": (i32, [vp, vp, vp, vp]),
         "olsgd_join": (i32, [vp]),
+        "olsgd_selftest_wait_timeout": (i32, [vp, i32]),
+        "olsgd_clear_status": (i32, [vp]),
         "olsgd_period_sync": (i32, [vp]),
         "olsgd_run": (i32, [vp, i64, vp]),
         "olsgd_get_params": (i32, [vp, i32, vp, C.c_size_t]),
@@ -185,6 +187,12 @@ class OverlapLocalSGD:
 
     def join(self):
         _check(self.lib, self.lib.olsgd_join(self.ctx), self.ctx)
+
+    def selftest_wait_timeout(self, limit_ms):
+        _check(self.lib, self.lib.olsgd_selftest_wait_timeout(self.ctx, int(limit_ms)), self.ctx)
+
+    def clear_status(self):
+        _check(self.lib, self.lib.olsgd_clear_status(self.ctx), self.ctx)
 
     def period_sync(self):
         _check(self.lib, self.lib.olsgd_period_sync(self.ctx), self.ctx)

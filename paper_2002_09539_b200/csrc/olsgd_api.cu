@@ -547,6 +547,23 @@ olsgd_status olsgd_local_step_host(olsgd_ctx* c, const float* Xb_host, const voi
   return OLSGD_OK;
 }
 
+olsgd_status olsgd_selftest_wait_timeout(olsgd_ctx* c, int32_t limit_ms) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  if (limit_ms < 1 || limit_ms > 2000) return fail(c, OLSGD_EINVAL, "limit_ms must be in [1, 2000]");
+  Launch l(c, OLSGD_KC_OTHER, c->main);
+  OLSGD_CUDA(c, launch_wait_selftest(c->dev_status, (uint64_t)limit_ms * 1000000ull, c->main));
+  return OLSGD_OK;
+}
+
+olsgd_status olsgd_clear_status(olsgd_ctx* c) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  OLSGD_CUDA(c, cudaStreamSynchronize(c->side));
+  OLSGD_CUDA(c, cudaMemsetAsync(c->dev_status, 0, sizeof(int), c->main));
+  OLSGD_CUDA(c, cudaStreamSynchronize(c->main));
+  c->err.clear();
+  return OLSGD_OK;
+}
+
 olsgd_status olsgd_join(olsgd_ctx* c) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
   if (c->copy) OLSGD_CUDA(c, cudaStreamSynchronize(c->copy));

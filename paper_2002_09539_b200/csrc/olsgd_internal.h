@@ -158,6 +158,8 @@ cudaError_t launch_gemm_simt(const GemmArgs& a, cudaStream_t s);
 // tcgen05 / TMEM / TMA version.  Needs Ma % 128 == 0, K % 64 == 0, Nb % 16 == 0.
 bool gemm_tc_supported(const GemmArgs& a);
 cudaError_t launch_gemm_tc(const GemmArgs& a, cudaStream_t s);
+// One thread waits (bounded by limit_ns) on a barrier nothing arrives on and reports the time-out.
+cudaError_t launch_wait_selftest(int* status, uint64_t limit_ns, cudaStream_t s);
 // Weight-gradient specialisation (short K, fp32 store): needs Ma % 128 == 0, Nb % 128 == 0,
 // K in {64, 128, 192, 256}, epilogue GEMM_EPI_STORE_F32.
 bool wgrad_tc_supported(const GemmArgs& a);

@@ -245,6 +245,21 @@ cudaError_t launch_one(const GemmArgs& a, const CUtensorMap& ma, const CUtensorM
   return cudaGetLastError();
 }
 
+// Self-test of the bounded wait: one thread waits on an mbarrier that nothing ever
+// arrives on, gives up after `limit_ns` and reports OLSGD_ETIMEOUT exactly as the GEMM
+// kernels do.  The context stays usable.
+__global__ void wait_selftest_kernel(int* status, uint64_t limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const bool ok = mbar_wait_ns(smem_u32(&bar), 0, &abort_flag, limit_ns);
+    if (!ok && status) atomicExch(status, (int)OLSGD_ETIMEOUT);
+  }
+}
+
 }  // namespace
 
 bool gemm_tc_supported(const GemmArgs& a) {
@@ -274,6 +289,11 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, cudaStream_t s) {
     case 128: return short_k ? launch_one<128, 2>(a, ma, mb, s) : launch_one<128, 6>(a, ma, mb, s);
     default:  return short_k ? launch_one<64, 2>(a, ma, mb, s) : launch_one<64, 8>(a, ma, mb, s);
   }
+}
+
+cudaError_t launch_wait_selftest(int* status, uint64_t limit_ns, cudaStream_t s) {
+  wait_selftest_kernel<<<1, 32, 0, s>>>(status, limit_ns);
+  return cudaGetLastError();
 }
 
 }  // namespace olsgd

@@ -124,3 +124,32 @@ def test_call_order_is_enforced():
     assert opt.iteration == 2
     opt.local_step_with_grads(g)
     assert opt.iteration == 3 and opt.launch_count >= 4
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    # no fault, no hang: one thread waits 20 ms on a barrier nothing arrives on, gives up,
+    # and the host reads OLSGD_ETIMEOUT at the next join
+    import time
+    from paper_2002_09539_b200 import OverlapLocalSGD, OlsgdError
+    P, m = 1024, 2
+    x0 = si.flat_init(3, P)
+    opt = OverlapLocalSGD("flat", m=m, tau=2, gamma=0.1, alpha=0.5, flat_P=P, x0=x0)
+    g = to_dev(si.flat_grads(3, 0, m, P))
+    opt.local_step_with_grads(g)
+    opt.join()
+    t0 = time.time()
+    opt.selftest_wait_timeout(20)
+    with pytest.raises(OlsgdError) as e:
+        opt.join()
+    assert e.value.status == 5                      # OLSGD_ETIMEOUT
+    assert time.time() - t0 < 5.0
+    with pytest.raises(OlsgdError):
+        opt.get_params(0)                           # still reported until cleared
+    opt.clear_status()
+    opt.join()
+    opt.local_step_with_grads(g)                    # the context works as before
+    opt.period_sync()
+    x = opt.get_params(0)
+    want = x0.astype(np.float64) - 0.1 * 2 * g[0].cpu().numpy().astype(np.float64)
+    want = want - 0.5 * (want - x0)
+    assert max_rel_err([x], [want]) <= 1e-6
