@@ -102,8 +102,6 @@ bool plan_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, ModelPlan
     mp->off_da[l] = take(m * B * w * e);
     mp->off_dat[l] = take(m * B * w * e);
   }
-  for (int l = 1; l < L - 1; ++l)  // layers whose input gradient is a GEMM
-    mp->off_wt[l] = take(m * (size_t)spec.dims[l + 1] * spec.dims[l] * e);
   mp->bytes = off;
   return true;
 }
@@ -142,7 +140,6 @@ bool bind_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, const Mod
     mb->da[l] = bp(mp.off_da[l]);
     mb->dat[l] = bp(mp.off_dat[l]);
   }
-  for (int l = 1; l < L - 1; ++l) mb->wt[l] = bp(mp.off_wt[l]);
   // gemm_bf16 == 1: hidden-layer weight matrices whose shape the weight-gradient kernel
   // takes are updated in its epilogue; everything else goes to the update kernel
   int64_t P = off;
@@ -245,6 +242,30 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
   // hidden layers, backward
   bool waited = false;
   for (int l = L - 1; l >= 1; --l) {
+    if (l >= 2) {
+      // dA_{l-1}^T [d_{l-1}][B] = (W_l^T [d_{l-1}][d_l] * dA_l [B][d_l]^T) .* (H_{l-1}^T > 0).
+      // W_l^T is read in place from the bf16 shadow of W_l [d_l][d_{l-1}] as an MN-major
+      // operand, and BEFORE the weight-gradient GEMM of this layer, whose fused epilogue
+      // overwrites that shadow with W_l of the next iteration.
+      GemmArgs gd{};
+      gd.A = io.shadow + mb.w_off[l - 1];
+      gd.a_mn_major = 1;
+      gd.lda = spec.dims[l - 1];
+      gd.a_batch = io.ld;
+      gd.B = mb.da[l];
+      gd.ldb = spec.dims[l];
+      gd.b_batch = (int64_t)B * spec.dims[l];
+      gd.m = m;
+      gd.Ma = spec.dims[l - 1];
+      gd.Nb = B;
+      gd.K = spec.dims[l];
+      gd.epilogue = GEMM_EPI_RELU_MASK;
+      gd.mask = mb.ht[l - 1];
+      gd.out_t = mb.dat[l - 1];
+      gd.out_n = mb.da[l - 1];
+      Scope sc(hook, OLSGD_KC_BACKWARD, s);
+      OLSGD_TRY(run_gemm(spec, gd, io.status, s));
+    }
     // dW_l [d_l][d_{l-1}] = dA_l^T [d_l][B] * (H_{l-1}^T [d_{l-1}][B])^T
     GemmArgs gw{};
     gw.A = mb.dat[l];
@@ -279,26 +300,6 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
       Scope sc(hook, OLSGD_KC_BACKWARD, s);
       OLSGD_TRY(launch_bias_grad(mb.dat[l], io.g, io.ld, mb.b_off[l - 1], m, spec.dims[l], B, s));
     }
-    if (l >= 2) {
-      // dA_{l-1}^T [d_{l-1}][B] = (W_l^T [d_{l-1}][d_l] * dA_l [B][d_l]^T) .* (H_{l-1}^T > 0)
-      GemmArgs gd{};
-      gd.A = mb.wt[l - 1];
-      gd.lda = spec.dims[l];
-      gd.a_batch = (int64_t)spec.dims[l] * spec.dims[l - 1];
-      gd.B = mb.da[l];
-      gd.ldb = spec.dims[l];
-      gd.b_batch = (int64_t)B * spec.dims[l];
-      gd.m = m;
-      gd.Ma = spec.dims[l - 1];
-      gd.Nb = B;
-      gd.K = spec.dims[l];
-      gd.epilogue = GEMM_EPI_RELU_MASK;
-      gd.mask = mb.ht[l - 1];
-      gd.out_t = mb.dat[l - 1];
-      gd.out_n = mb.da[l - 1];
-      Scope sc(hook, OLSGD_KC_BACKWARD, s);
-      OLSGD_TRY(run_gemm(spec, gd, io.status, s));
-    }
   }
   return cudaSuccess;
 }
@@ -306,16 +307,9 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
 cudaError_t model_post_update(const olsgd_model_spec& spec, const olsgd_hparams& hp,
                               const ModelBuffers& mb, const __nv_bfloat16* shadow, int64_t ld,
                               cudaStream_t s, const ProfHook& hook) {
-  if (!bf16_path(spec)) return cudaSuccess;
-  const int L = n_layers(spec);
-  // layer index l here is 0-based in the parameter layout: weights of the
-  // (l+1)-th layer map dims[l] -> dims[l+1]; its transposed copy feeds dgrad
-  for (int l = 1; l < L - 1; ++l) {
-    Scope sc(hook, OLSGD_KC_OTHER, s);
-    OLSGD_TRY(launch_transpose_bf16(shadow, ld, mb.w_off[l], mb.wt[l],
-                                    (int64_t)spec.dims[l + 1] * spec.dims[l], hp.m,
-                                    spec.dims[l + 1], spec.dims[l], s));
-  }
+  // nothing is derived from the parameters any more: the input-gradient GEMM reads the
+  // bf16 shadow of W_l in place as an MN-major operand
+  (void)spec; (void)hp; (void)mb; (void)shadow; (void)ld; (void)s; (void)hook;
   return cudaSuccess;
 }
 

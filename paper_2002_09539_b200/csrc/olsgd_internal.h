@@ -105,14 +105,10 @@ cudaError_t launch_head_wgrad(const HeadArgs& a, float* g, float* loss, cudaStre
 cudaError_t launch_bias_grad(const __nv_bfloat16* dat, float* g, int64_t ld, int64_t b_off, int m,
                              int R, int batch, cudaStream_t s);
 
-// dst[i][c][r] = src[i][r][c] for a [R][C] bf16 matrix inside every row of a [m][ld] array
-cudaError_t launch_transpose_bf16(const __nv_bfloat16* src, int64_t src_ld, int64_t src_off,
-                                  __nv_bfloat16* dst, int64_t dst_batch, int m, int R, int C,
-                                  cudaStream_t s);
-
 // ---- gemm --------------------------------------------------------------------
 // Worker-batched D[i] = A[i] * B[i]^T with both operands K-major bf16:
-//   A [m][Ma][K] (row pitch lda, batch pitch a_batch, in elements)
+//   A [m][Ma][K] (row pitch lda, batch pitch a_batch, in elements); with a_mn_major the
+//     same operand is stored transposed, [m][K][Ma] (row pitch lda), and read in place
 //   B [m][Nb][K] (row pitch ldb, batch pitch b_batch)
 // D is [Ma][Nb] per worker, fp32 accumulate, consumed by one of three epilogues.
 enum GemmEpilogue {
@@ -142,6 +138,7 @@ struct GemmArgs {
   const __nv_bfloat16* B;
   int64_t lda, a_batch, ldb, b_batch;
   int m, Ma, Nb, K;
+  int a_mn_major;            // A is stored [K][Ma]
   int epilogue;
   const float* bias;         // BIAS_RELU: bias[i * bias_batch + row]
   int64_t bias_batch;
@@ -174,7 +171,6 @@ struct ModelPlan {
          off_loss = 0;
   size_t off_h[OLSGD_MAX_DIMS] = {0}, off_ht[OLSGD_MAX_DIMS] = {0};    // hidden activations
   size_t off_da[OLSGD_MAX_DIMS] = {0}, off_dat[OLSGD_MAX_DIMS] = {0};  // their gradients
-  size_t off_wt[OLSGD_MAX_DIMS] = {0};  // transposed bf16 weights of layer l (for dgrad)
 };
 struct ModelBuffers {
   char error[160] = {0};
@@ -186,7 +182,6 @@ struct ModelBuffers {
   __nv_bfloat16* ht[OLSGD_MAX_DIMS] = {nullptr};
   __nv_bfloat16* da[OLSGD_MAX_DIMS] = {nullptr};
   __nv_bfloat16* dat[OLSGD_MAX_DIMS] = {nullptr};
-  __nv_bfloat16* wt[OLSGD_MAX_DIMS] = {nullptr};
   int64_t w_off[OLSGD_MAX_DIMS] = {0}, b_off[OLSGD_MAX_DIMS] = {0};
   // weights of parameter layer p are updated inside their weight-gradient GEMM
   bool fused_layer[OLSGD_MAX_DIMS] = {false};
@@ -217,7 +212,7 @@ bool bind_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, const Mod
 cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hparams& hp,
                                    const olsgd_data& data, const ModelBuffers& mb,
                                    const StepIO& io, cudaStream_t s, const ProfHook& hook);
-// Work that must follow every parameter update (transposed bf16 weights for dgrad).
+// Work that must follow every parameter update (none at present).
 cudaError_t model_post_update(const olsgd_model_spec& spec, const olsgd_hparams& hp,
                               const ModelBuffers& mb, const __nv_bfloat16* shadow, int64_t ld,
                               cudaStream_t s, const ProfHook& hook);

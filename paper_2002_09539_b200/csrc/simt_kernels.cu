@@ -1,5 +1,5 @@
 // CUDA-core kernels of the forward/backward path: minibatch gather, linear
-// regression, bias gradients, bf16 casts and transposes, and a plain reference GEMM.
+// regression, bias gradients, bf16 casts, and a plain reference GEMM.
 //
 // Every reduction runs in a fixed order (no floating-point atomics), so a step
 // is reproducible bit for bit from run to run.
@@ -178,39 +178,6 @@ __global__ void bias_grad_kernel(const __nv_bfloat16* __restrict__ dat, float* _
   if (lane == 0) g[(int64_t)i * ld + b_off + r] = acc;
 }
 
-// ------------------------------------------------------------------ bf16 transpose
-
-// 64 x 64 tiles, two bf16 per global access (128 bytes per row segment both ways).
-__global__ void __launch_bounds__(256)
-transpose_bf16_kernel(const __nv_bfloat16* __restrict__ src, int64_t src_ld, int64_t src_off,
-                      __nv_bfloat16* __restrict__ dst, int64_t dst_batch, int R, int C) {
-  __shared__ __nv_bfloat16 tile[64][66];
-  const int i = blockIdx.z;
-  const __nv_bfloat16* s = src + (int64_t)i * src_ld + src_off;
-  __nv_bfloat16* d = dst + (int64_t)i * dst_batch;
-  const int c0 = blockIdx.x * 64, r0 = blockIdx.y * 64;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  uint32_t w[8];
-#pragma unroll
-  for (int t = 0; t < 8; ++t) {
-    const int r = r0 + warp + 8 * t, c = c0 + 2 * lane;
-    w[t] = 0;
-    if (r < R && c < C) w[t] = __ldcs(reinterpret_cast<const uint32_t*>(s + (int64_t)r * C + c));
-  }
-#pragma unroll
-  for (int t = 0; t < 8; ++t)
-    *reinterpret_cast<uint32_t*>(&tile[warp + 8 * t][2 * lane]) = w[t];
-  __syncthreads();
-  for (int cc = warp; cc < 64; cc += 8) {
-    const int c = c0 + cc, r = r0 + 2 * lane;
-    if (r < R && c < C) {
-      const uint16_t lo = *reinterpret_cast<const uint16_t*>(&tile[2 * lane][cc]);
-      const uint16_t hi = *reinterpret_cast<const uint16_t*>(&tile[2 * lane + 1][cc]);
-      *reinterpret_cast<uint32_t*>(d + (int64_t)c * R + r) = (uint32_t)lo | ((uint32_t)hi << 16);
-    }
-  }
-}
-
 // ------------------------------------------------------------------ reference GEMM
 
 constexpr int kRefTile = 32;
@@ -226,7 +193,10 @@ gemm_simt_kernel(GemmArgs a) {
   float acc = 0.f;
   for (int k0 = 0; k0 < a.K; k0 += kRefTile) {
     const int k = k0 + tx;
-    As[ty][tx] = (row0 + ty < a.Ma && k < a.K) ? __bfloat162float(A[(int64_t)(row0 + ty) * a.lda + k]) : 0.f;
+    As[ty][tx] = (row0 + ty < a.Ma && k < a.K)
+                     ? __bfloat162float(a.a_mn_major ? A[(int64_t)k * a.lda + row0 + ty]
+                                                     : A[(int64_t)(row0 + ty) * a.lda + k])
+                     : 0.f;
     Bs[ty][tx] = (col0 + ty < a.Nb && k < a.K) ? __bfloat162float(B[(int64_t)(col0 + ty) * a.ldb + k]) : 0.f;
     __syncthreads();
 #pragma unroll
@@ -286,15 +256,6 @@ cudaError_t launch_bias_grad(const __nv_bfloat16* dat, float* g, int64_t ld, int
   const int warps = 8;
   dim3 grid((R + warps - 1) / warps, m), block(warps * 32);
   bias_grad_kernel<<<grid, block, 0, s>>>(dat, g, ld, b_off, R, batch);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_transpose_bf16(const __nv_bfloat16* src, int64_t src_ld, int64_t src_off,
-                                  __nv_bfloat16* dst, int64_t dst_batch, int m, int R, int C,
-                                  cudaStream_t s) {
-  if (R % 2 || C % 2 || src_off % 2 || src_ld % 2 || dst_batch % 2) return cudaErrorInvalidValue;
-  dim3 grid((C + 63) / 64, (R + 63) / 64, m);
-  transpose_bf16_kernel<<<grid, 256, 0, s>>>(src, src_ld, src_off, dst, dst_batch, R, C);
   return cudaGetLastError();
 }
 

@@ -165,7 +165,23 @@ __device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t addr) {
   return d;
 }
 
+// Shared-memory matrix descriptor of an MN-major operand tile: the tile arrives as TMA
+// boxes of 64 MN elements (128 bytes, swizzled) by 64 K rows, one box per 64 MN elements.
+// Inside a box the K rows are 128 B apart, so groups of eight K rows are 1024 B apart
+// (stride byte offset); consecutive 64-element MN blocks are one box = 8192 B apart
+// (leading byte offset).
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(8192 >> 4) << 16;          // leading byte offset: next 64 MN elements
+  d |= (uint64_t)(1024 >> 4) << 32;          // stride byte offset: next eight K rows
+  d |= (uint64_t)1 << 46;                    // descriptor version
+  d |= (uint64_t)2 << 61;                    // SWIZZLE_128B
+  return d;
+}
+
 // Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = bn.
+// Bit 15 set makes A MN-major (its M index is the contiguous one in memory).
 __host__ __device__ constexpr uint32_t instr_desc_bf16(int bn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) |
          ((uint32_t)(kBM >> 4) << 24);

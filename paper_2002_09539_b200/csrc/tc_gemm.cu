@@ -47,7 +47,7 @@ struct SharedCtl {
 template <int BN, int STAGES>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               int num_kb, EpiArgs ea) {
+               int num_kb, int a_mn, EpiArgs ea) {
   constexpr uint32_t kABytes = kBM * kBK * 2;
   constexpr uint32_t kBBytes = BN * kBK * 2;
   constexpr uint32_t kStageBytes = kABytes + kBBytes;
@@ -88,7 +88,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const uint32_t full = smem_u32(&ctl->full[s]);
       mbar_expect_tx(full, kStageBytes);
       const uint32_t a_dst = smem_u32(tiles + s * kStageBytes);
-      tma_load_3d(a_dst, &map_a, full, kb * kBK, m0, worker);
+      if (a_mn) {
+        // A is stored [K][Ma]: two boxes of 64 (Ma) x 64 (K rows)
+        tma_load_3d(a_dst, &map_a, full, m0, kb * kBK, worker);
+        tma_load_3d(a_dst + kABytes / 2, &map_a, full, m0 + 64, kb * kBK, worker);
+      } else {
+        tma_load_3d(a_dst, &map_a, full, kb * kBK, m0, worker);
+      }
       tma_load_3d(a_dst + kABytes, &map_b, full, kb * kBK, n0, worker);
       issued = kb + 1;
     }
@@ -104,7 +110,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
   } else if (warp == 1 && lane == 0) {
     // ---------------- MMA issuer
-    constexpr uint32_t idesc = instr_desc_bf16(BN);
+    const uint32_t idesc = instr_desc_bf16(BN) | (a_mn ? (1u << 15) : 0u);
     bool ok = true;
     for (int kb = 0; kb < num_kb && ok; ++kb) {
       const int s = kb % STAGES;
@@ -113,12 +119,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (!ok) break;
       tc_fence_after();
       const uint32_t a_addr = smem_u32(tiles + s * kStageBytes);
-      const uint64_t a_desc = smem_desc_k_sw128(a_addr);
+      const uint64_t a_desc = a_mn ? smem_desc_mn_sw128(a_addr) : smem_desc_k_sw128(a_addr);
+      // one MMA consumes 16 K elements: 32 bytes along a K-major row, or 16 K rows of
+      // 128 bytes (2048 bytes) of an MN-major tile; in 16-byte descriptor units
+      const uint64_t a_step = a_mn ? 128u : 2u;
       const uint64_t b_desc = smem_desc_k_sw128(a_addr + kABytes);
 #pragma unroll
       for (int k = 0; k < kBK / kUmmaK; ++k) {
         // 16 K elements = 32 bytes = 2 units of the descriptor's start address
-        umma_bf16(tmem_base, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+        umma_bf16(tmem_base, a_desc + a_step * (uint64_t)k, b_desc + (uint64_t)(2 * k), idesc,
                   (kb > 0 || k > 0) ? 1u : 0u);
       }
       umma_commit(smem_u32(&ctl->empty[s]));  // stage reusable once these MMAs retire
@@ -241,7 +250,7 @@ cudaError_t launch_one(const GemmArgs& a, const CUtensorMap& ma, const CUtensorM
   ea.out_batch = a.out_batch;
   ea.status = a.status;
   dim3 grid(a.Nb / BN, a.Ma / kBM, a.m);
-  kern<<<grid, kThreads, smem, s>>>(ma, mb, a.K / kBK, ea);
+  kern<<<grid, kThreads, smem, s>>>(ma, mb, a.K / kBK, a.a_mn_major ? 1 : 0, ea);
   return cudaGetLastError();
 }
 
@@ -280,7 +289,12 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, cudaStream_t s) {
   if (!gemm_tc_supported(a)) return cudaErrorInvalidValue;
   const int bn = pick_bn(a.Nb);
   CUtensorMap ma, mb;
-  if (!make_map(&ma, a.A, a.K, a.Ma, a.m, a.lda, a.a_batch, kBM)) return cudaErrorInvalidValue;
+  if (a.a_mn_major) {
+    // A stored [K][Ma] (Ma contiguous): 64-element boxes along Ma, 64 rows along K
+    if (!make_map(&ma, a.A, a.Ma, a.K, a.m, a.lda, a.a_batch, 64)) return cudaErrorInvalidValue;
+  } else if (!make_map(&ma, a.A, a.K, a.Ma, a.m, a.lda, a.a_batch, kBM)) {
+    return cudaErrorInvalidValue;
+  }
   if (!make_map(&mb, a.B, a.K, a.Nb, a.m, a.ldb, a.b_batch, bn)) return cudaErrorInvalidValue;
   // short K (weight gradients, K = batch): few stages so several CTAs share an SM
   const bool short_k = a.K / kBK <= 2;
