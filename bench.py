@@ -195,6 +195,9 @@ def run_ours(args, rank, world):
     c = dict(si.CONFIGS[name])
     if c["gemm_bf16"] and args.gemm_mode:
         c["gemm_bf16"] = args.gemm_mode
+    local_sgd = args.method != "overlap"
+    if args.method == "sync_sgd":
+        c["tau"] = 1                 # fully synchronous SGD = Eq. 2 with tau = 1
     seed = rank                      # every rank is an independent replica
     table = None
     if c.get("non_iid"):
@@ -204,7 +207,7 @@ def run_ours(args, rank, world):
     Xd, yd = torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda()
     opt = OverlapLocalSGD(c["kind"], m=c["m"], tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"],
                           beta=c["beta"], mu=c["mu"], batch=c["batch"], seed=seed, dims=c["dims"],
-                          gemm_bf16=c["gemm_bf16"], x0=x0, X=Xd, y=yd)
+                          gemm_bf16=c["gemm_bf16"], x0=x0, X=Xd, y=yd, local_sgd=local_sgd)
     m, K, W = c["m"], args.steps, args.warmup
 
     def barrier():
@@ -271,7 +274,7 @@ def run_ours(args, rank, world):
     def e2e_steps(k0, count):
         for t in range(k0, k0 + count):
             opt.local_step_host(Xh[t % pool], yh[t % pool], loss_h[t])
-            if (opt.iteration) % c["tau"] == 0:
+            if (opt.iteration) % c["tau"] == 0 and not local_sgd:
                 opt.period_sync()
 
     e2e_steps(0, W)
@@ -301,7 +304,7 @@ def run_ours(args, rank, world):
             "config": {"workload": workload_name(name, c), "m": m, "tau": c["tau"],
                        "batch": B, "dims": c["dims"], "P": P, "gamma": c["gamma"],
                        "alpha": c["alpha"], "beta": c["beta"], "mu": c["mu"],
-                       "gemm_mode": c["gemm_bf16"],
+                       "gemm_mode": c["gemm_bf16"], "method": args.method,
                        "l2": "no flush: resident inputs+state %.0f MB exceed the %d MB L2"
                              % (resident / 1e6, L2_BYTES >> 20) if resident > L2_BYTES else
                              "state fits in L2 (%.1f MB): steady-state training keeps it there"
@@ -507,6 +510,9 @@ def main():
     ap.add_argument("--gemm-mode", type=int, default=0, choices=[0, 1, 2, 3],
                     help="MLP workloads: 1 tensor cores + update fused into the weight-gradient "
                          "GEMM (default), 3 tensor cores + separate update kernel, 2 CUDA cores")
+    ap.add_argument("--method", default="overlap", choices=["overlap", "local_sgd", "sync_sgd"],
+                    help="overlap: Overlap-Local-SGD (Eq. 3-5, 10-11); local_sgd: blocking periodic "
+                         "averaging (Eq. 2); sync_sgd: Eq. 2 with tau = 1")
     ap.add_argument("--P", type=int, default=0, help="c5 only: one parameter count")
     ap.add_argument("--m", type=int, default=0, help="c5 only: one worker count")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

@@ -70,8 +70,17 @@ typedef struct {
  * momentum factor (Eq. 10).  mu is the factor of the "common Nesterov
  * momentum" of the local step (u <- mu u + g, x <- x - gamma (g + mu u));
  * mu = 0 is plain SGD, beta = 0 is the vanilla anchor refresh of Eq. 5.     */
+typedef enum {
+  OLSGD_MODE_OVERLAP = 0,    /* Overlap-Local-SGD: Eq. 3-5 (and Eq. 10-11)                 */
+  OLSGD_MODE_LOCAL_SGD = 1   /* Local SGD / periodic averaging, Eq. 2: on a sync step every
+                                worker model is replaced by the average of all of them,
+                                on the main stream (blocking); tau = 1 is fully synchronous
+                                SGD.  alpha and beta are ignored, olsgd_period_sync is
+                                never due, and z reports the last average                */
+} olsgd_mode;
+
 typedef struct {
-  int32_t m, tau, batch, reserved;
+  int32_t m, tau, batch, mode /* olsgd_mode */;
   float gamma, alpha, beta, mu;
   uint64_t seed;                /* seeds the minibatch index rule                    */
 } olsgd_hparams;

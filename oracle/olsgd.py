@@ -86,6 +86,48 @@ class OverlapLocalSGD:
         return self.x.mean(axis=0)
 
 
+class LocalSGD:
+    """Local SGD / periodic averaging, the baseline the paper starts from (Eq. 2):
+
+        x_{k+1}^(i) = (1/m) sum_j [x_k^(j) - gamma g_j]   when (k+1) mod tau == 0
+                    = x_k^(i) - gamma g_i                  otherwise.
+
+    tau = 1 is fully synchronous SGD.  A local Nesterov buffer (mu > 0) is fed by local
+    gradients only and is not averaged, as in OverlapLocalSGD.  `z` mirrors the last
+    average so that both classes expose the same fields.
+    """
+
+    def __init__(self, x0, m, tau, gamma, mu=0.0):
+        x0 = np.asarray(x0, dtype=np.float64)
+        self.m, self.tau, self.gamma, self.mu = int(m), int(tau), float(gamma), float(mu)
+        self.x = np.tile(x0, (self.m, 1))
+        self.u = np.zeros_like(self.x)
+        self.z = x0.copy()
+        self.v = np.zeros_like(x0)
+        self.k = 0
+
+    def step(self, g):
+        g = np.asarray(g, dtype=np.float64)
+        for i in range(self.m):
+            if self.mu != 0.0:
+                self.u[i] = self.mu * self.u[i] + g[i]
+                self.x[i] = self.x[i] - self.gamma * (g[i] + self.mu * self.u[i])
+            else:
+                self.x[i] = self.x[i] - self.gamma * g[i]
+        if (self.k + 1) % self.tau == 0:
+            s = np.zeros_like(self.z)
+            for i in range(self.m):
+                s += self.x[i]
+            s /= self.m
+            for i in range(self.m):
+                self.x[i] = s
+            self.z = s.copy()
+        self.k += 1
+
+    def mean_model(self):
+        return self.x.mean(axis=0)
+
+
 def mixing_matrix(m, alpha):
     """The sync-step W of Eq. 9, (m+1) x (m+1), column-stochastic."""
     W = np.zeros((m + 1, m + 1))

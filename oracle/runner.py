@@ -11,14 +11,15 @@ from . import models, olsgd, sampling
 
 
 def run_model(kind, dims, X, y, x0, *, m, tau, batch, gamma, alpha, beta, mu, seed,
-              iters, bf16_operands=False, snapshots=()):
+              iters, bf16_operands=False, snapshots=(), local_sgd=False):
     """Run `iters` iterations; returns (state, losses[iters][m], {k: state copy}).
 
     X [m][n][d_in], y [m][n]; worker i only ever touches X[i], y[i] (Eq. 1).
     `snapshots` lists iteration counts k at which (x, z, v) are copied out.
     """
     n = X.shape[1]
-    st = olsgd.OverlapLocalSGD(x0, m, tau, gamma, alpha, beta, mu)
+    st = (olsgd.LocalSGD(x0, m, tau, gamma, mu) if local_sgd
+          else olsgd.OverlapLocalSGD(x0, m, tau, gamma, alpha, beta, mu))
     losses = np.zeros((iters, m))
     g = np.zeros_like(st.x)
     snaps = {}
@@ -35,9 +36,10 @@ def run_model(kind, dims, X, y, x0, *, m, tau, batch, gamma, alpha, beta, mu, se
     return st, losses, snaps
 
 
-def run_flat(x0, grads, *, m, tau, gamma, alpha, beta, mu):
+def run_flat(x0, grads, *, m, tau, gamma, alpha, beta, mu, local_sgd=False):
     """External-gradient workload: grads is a sequence of [m][P] arrays."""
-    st = olsgd.OverlapLocalSGD(x0, m, tau, gamma, alpha, beta, mu)
+    st = (olsgd.LocalSGD(x0, m, tau, gamma, mu) if local_sgd
+          else olsgd.OverlapLocalSGD(x0, m, tau, gamma, alpha, beta, mu))
     for g in grads:
         st.step(g)
     return st

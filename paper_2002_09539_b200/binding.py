@@ -31,7 +31,7 @@ class _ModelSpec(C.Structure):
 
 
 class _HParams(C.Structure):
-    _fields_ = [("m", C.c_int32), ("tau", C.c_int32), ("batch", C.c_int32), ("reserved", C.c_int32),
+    _fields_ = [("m", C.c_int32), ("tau", C.c_int32), ("batch", C.c_int32), ("mode", C.c_int32),
                 ("gamma", C.c_float), ("alpha", C.c_float), ("beta", C.c_float), ("mu", C.c_float),
                 ("seed", C.c_uint64)]
 
@@ -131,11 +131,11 @@ class OverlapLocalSGD:
 
     def __init__(self, kind, *, m, tau, gamma, alpha, beta=0.0, mu=0.0, batch=1, seed=0,
                  dims=(), gemm_bf16=0, flat_P=0, x0, X=None, y=None, overlap=True,
-                 device="cuda"):
+                 local_sgd=False, device="cuda"):
         self.lib = load_library()
         self.device = torch.device(device)
         self.spec = _spec(kind, dims, gemm_bf16, flat_P)
-        self.hp = _HParams(int(m), int(tau), int(batch), 0, float(gamma), float(alpha),
+        self.hp = _HParams(int(m), int(tau), int(batch), 1 if local_sgd else 0, float(gamma), float(alpha),
                            float(beta), float(mu), int(seed))
         self.m, self.tau, self.batch, self.kind = int(m), int(tau), int(batch), kind
         P = C.c_int64()

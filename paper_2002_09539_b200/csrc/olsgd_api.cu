@@ -203,6 +203,8 @@ olsgd_status check_hp(const olsgd_hparams* hp) {
   if (!(hp->beta >= 0.f && hp->beta < 1.f))
     return fail(nullptr, OLSGD_EINVAL, "beta must be in [0, 1)");
   if (!(hp->mu >= 0.f && hp->mu < 1.f)) return fail(nullptr, OLSGD_EINVAL, "mu must be in [0, 1)");
+  if (hp->mode != OLSGD_MODE_OVERLAP && hp->mode != OLSGD_MODE_LOCAL_SGD)
+    return fail(nullptr, OLSGD_EINVAL, "mode must be OLSGD_MODE_OVERLAP or OLSGD_MODE_LOCAL_SGD");
   return OLSGD_OK;
 }
 
@@ -267,7 +269,9 @@ olsgd_status drain_profile(olsgd_ctx* c) {
 
 // Eq. 3 / Eq. 4 for all workers: reads x[cur], writes x[1-cur], flips.
 olsgd_status apply_update(olsgd_ctx* c, const float* g, int64_t ldg) {
-  const bool sync = (c->k + 1) % c->hp.tau == 0;
+  const bool period_end = (c->k + 1) % c->hp.tau == 0;
+  const bool local_sgd = c->hp.mode == OLSGD_MODE_LOCAL_SGD;
+  const bool sync = period_end && !local_sgd;   // Eq. 4 belongs to the overlap method only
   const int nxt = 1 - c->cur;
   // The anchor refresh of the previous period runs on the side stream.  It must
   // have finished before a pull-back reads z, and before its input buffer is
@@ -300,6 +304,12 @@ olsgd_status apply_update(olsgd_ctx* c, const float* g, int64_t ldg) {
     Launch l(c, OLSGD_KC_UPDATE, c->main);
     OLSGD_CUDA(c, launch_fused_update(a, c->main));
   }
+  if (period_end && local_sgd) {
+    // Eq. 2: blocking average of all worker models, in place, on the main stream
+    Launch l(c, OLSGD_KC_ANCHOR, c->main);
+    OLSGD_CUDA(c, launch_worker_mean_broadcast(c->x[nxt], c->shadow, c->z, c->P, c->ld, c->hp.m,
+                                               c->main));
+  }
   c->cur = nxt;
   c->k += 1;
   if (sync) c->need_sync = true;
@@ -321,7 +331,7 @@ olsgd_status step_body(olsgd_ctx* c, const olsgd_data& data, const int32_t* idx,
   memset(&io.upd, 0, sizeof io.upd);
   io.wait_before_update = nullptr;
   if (c->spec.kind == OLSGD_MLP && c->spec.gemm_bf16 == 1) {
-    const bool sync = (c->k + 1) % c->hp.tau == 0;
+    const bool sync = (c->k + 1) % c->hp.tau == 0 && c->hp.mode == OLSGD_MODE_OVERLAP;
     const int nxt = 1 - c->cur;
     io.upd.enabled = 1;
     io.upd.x_in = c->x[c->cur];

@@ -43,6 +43,11 @@ struct AnchorArgs {
 };
 cudaError_t launch_worker_mean_anchor(const AnchorArgs& a, cudaStream_t s);
 
+// Eq. 2 on a sync step: every worker row of x (and of its bf16 shadow, if any) and z are
+// replaced by the worker mean, summed in worker order.
+cudaError_t launch_worker_mean_broadcast(float* x, __nv_bfloat16* shadow, float* z, int64_t P,
+                                         int64_t ld, int m, cudaStream_t s);
+
 // dst[j] = (1-alpha) * mean_i x_i[j] + alpha * z[j]   (alpha = 0: mean model)
 cudaError_t launch_virtual_sequence(const float* x, const float* z, float* dst, int64_t P,
                                     int64_t ld, int m, float alpha, cudaStream_t s);

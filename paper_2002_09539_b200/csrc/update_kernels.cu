@@ -146,6 +146,41 @@ worker_mean_anchor_kernel(const float* __restrict__ x, float* __restrict__ z,
   }
 }
 
+// Blocking average of Local SGD (Eq. 2): one thread per 16-byte column strip sums the m
+// worker rows in worker order (four loads in flight), then overwrites all of them.
+__global__ void __launch_bounds__(kUpdateThreads)
+worker_mean_broadcast_kernel(float* __restrict__ x, __nv_bfloat16* __restrict__ shadow,
+                             float* __restrict__ z, int64_t n4, int64_t ld, int m, float m_f) {
+  const int64_t col4 = (int64_t)blockIdx.x * kUpdateThreads + threadIdx.x;
+  if (col4 >= n4) return;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int ib = 0; ib < m; ib += kUnroll) {
+    float4 xv[kUnroll];
+#pragma unroll
+    for (int t = 0; t < kUnroll; ++t)
+      if (ib + t < m) xv[t] = reinterpret_cast<const float4*>(x + (int64_t)(ib + t) * ld)[col4];
+#pragma unroll
+    for (int t = 0; t < kUnroll; ++t) {
+      if (ib + t < m) {
+        acc.x += xv[t].x;
+        acc.y += xv[t].y;
+        acc.z += xv[t].z;
+        acc.w += xv[t].w;
+      }
+    }
+  }
+  acc.x /= m_f;
+  acc.y /= m_f;
+  acc.z /= m_f;
+  acc.w /= m_f;
+  reinterpret_cast<float4*>(z)[col4] = acc;
+  const uint2 pk = pack_bf16x4(acc);
+  for (int i = 0; i < m; ++i) {
+    reinterpret_cast<float4*>(x + (int64_t)i * ld)[col4] = acc;
+    if (shadow) reinterpret_cast<uint2*>(shadow + (int64_t)i * ld)[col4] = pk;
+  }
+}
+
 __global__ void virtual_sequence_kernel(const float* __restrict__ x, const float* __restrict__ z,
                                         float* __restrict__ dst, int64_t P, int64_t ld, int m,
                                         float alpha, float m_f) {
@@ -209,6 +244,14 @@ cudaError_t launch_worker_mean_anchor(const AnchorArgs& a, cudaStream_t s) {
   if (a.m >= 16) return launch_mean<4>(a, s);
   if (a.m >= 8) return launch_mean<2>(a, s);
   return launch_mean<1>(a, s);
+}
+
+cudaError_t launch_worker_mean_broadcast(float* x, __nv_bfloat16* shadow, float* z, int64_t P,
+                                         int64_t ld, int m, cudaStream_t s) {
+  const int64_t n4 = (P + 3) / 4;
+  worker_mean_broadcast_kernel<<<(unsigned)((n4 + kUpdateThreads - 1) / kUpdateThreads),
+                                 kUpdateThreads, 0, s>>>(x, shadow, z, n4, ld, m, (float)m);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_virtual_sequence(const float* x, const float* z, float* dst, int64_t P,

@@ -45,14 +45,14 @@ def test_param_count_matches_the_flat_layout(lib):
 def _hp(**kw):
     d = dict(m=4, tau=2, batch=8, gamma=0.1, alpha=0.5, beta=0.0, mu=0.0, seed=0)
     d.update(kw)
-    return binding._HParams(d["m"], d["tau"], d["batch"], 0, d["gamma"], d["alpha"], d["beta"],
+    return binding._HParams(d["m"], d["tau"], d["batch"], d.get("mode", 0), d["gamma"], d["alpha"], d["beta"],
                             d["mu"], d["seed"])
 
 
 @pytest.mark.parametrize("bad", [dict(m=0), dict(tau=0), dict(batch=0), dict(gamma=0.0),
                                  dict(gamma=-1.0), dict(alpha=-0.1), dict(alpha=1.5),
                                  dict(beta=1.0), dict(beta=-0.1), dict(mu=1.0),
-                                 dict(gamma=float("nan"))])
+                                 dict(gamma=float("nan")), dict(mode=2), dict(mode=-1)])
 def test_bad_hyper_parameters_are_rejected(lib, bad):
     s = binding._spec("flat", flat_P=100)
     n = C.c_size_t()

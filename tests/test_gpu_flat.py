@@ -153,3 +153,26 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
     want = x0.astype(np.float64) - 0.1 * 2 * g[0].cpu().numpy().astype(np.float64)
     want = want - 0.5 * (want - x0)
     assert max_rel_err([x], [want]) <= 1e-6
+
+
+@pytest.mark.parametrize("P,m,tau,mu", [(4 * 256 * 3 + 7, 8, 4, 0.0), (70001, 37, 3, 0.9),
+                                        (1000003, 16, 1, 0.9), (5, 3, 2, 0.0)])
+def test_local_sgd_mode_parity(P, m, tau, mu):
+    # Eq. 2: blocking periodic averaging; tau = 1 is fully synchronous SGD
+    from paper_2002_09539_b200 import OverlapLocalSGD, OlsgdError
+    iters = 3 * tau + 1
+    x0 = si.flat_init(4, P)
+    grads = [si.flat_grads(4, k, m, P) for k in range(iters)]
+    st = runner.run_flat(x0, grads, m=m, tau=tau, gamma=0.05, alpha=0.5, beta=0.0, mu=mu,
+                         local_sgd=True)
+    opt = OverlapLocalSGD("flat", m=m, tau=tau, gamma=0.05, alpha=0.5, mu=mu, flat_P=P, x0=x0,
+                          local_sgd=True)
+    for k in range(iters):
+        opt.local_step_with_grads(to_dev(grads[k]))
+        if (k + 1) % tau == 0:
+            x, z, _ = opt.state()
+            assert all(np.array_equal(x[i], x[0]) for i in range(m))    # all workers agree
+            assert np.array_equal(z, x[0])
+            with pytest.raises(OlsgdError):
+                opt.period_sync()                                        # never due in this mode
+    assert state_err(opt, st) <= TOL

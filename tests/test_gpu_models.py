@@ -144,3 +144,26 @@ def test_fused_weight_gradient_update_gives_the_bits_of_the_separate_kernel(dims
     assert np.array_equal(xa, xb) and np.array_equal(za, zb) and np.array_equal(va, vb)
     for i in (0, m - 1):
         assert np.array_equal(a.get_params(-5 - i), b.get_params(-5 - i))
+
+
+@pytest.mark.parametrize("kind,dims,gemm", [("softmax", [100, 7], 0), ("mlp", [128, 256, 128, 10], 1),
+                                            ("mlp", [128, 256, 128, 10], 3)])
+def test_local_sgd_mode_with_models(kind, dims, gemm):
+    # Eq. 2 through the model paths, including the fused weight-gradient/update kernel
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    m, n, batch, tau, iters = 3, 120, 64, 2, 5
+    X, y = si.mixture_data(9, m, n, dims[0])
+    y = (y % dims[-1]).astype(np.int32)
+    rng = np.random.default_rng(9)
+    x0 = (si.model_init(9, "mlp", dims) if kind == "mlp"
+          else (0.1 * rng.standard_normal(models.n_params(kind, dims))).astype(np.float32))
+    kw = dict(m=m, tau=tau, batch=batch, gamma=0.05, alpha=0.5, beta=0.0, mu=0.9, seed=9)
+    st, lo, _ = runner.run_model(kind, dims, X, y, x0, iters=iters, bf16_operands=gemm != 0,
+                                 local_sgd=True, **kw)
+    opt = OverlapLocalSGD(kind, dims=dims, gemm_bf16=gemm, x0=x0, X=to_dev(X), y=to_dev(y),
+                          local_sgd=True, **kw)
+    loss = torch.zeros((iters, m), device="cuda")
+    opt.run(iters, loss)
+    tol = TOL_FP32 if gemm == 0 else TOL_BF16_PARAM
+    assert state_err(opt, st) <= tol
+    assert np.abs(loss.cpu().numpy() - lo).max() <= (2e-5 if gemm == 0 else TOL_BF16_LOSS) * np.abs(lo).max()

@@ -320,3 +320,68 @@ def test_brute_force_tiny_problem_with_real_minibatches():
             z = [sum(xs[i][j] for i in range(m)) / m for j in range(d)]
     assert np.allclose(st.x, np.array(xs), rtol=1e-12, atol=1e-14)
     assert np.allclose(st.z, np.array(z), rtol=1e-12, atol=1e-14)
+
+
+# ------------------------------------------------------------ Eq. 2, Local SGD
+
+def test_local_sgd_tau_one_is_sgd_on_the_averaged_gradient():
+    # fully synchronous SGD: all workers stay equal and move by the mean gradient
+    rng = np.random.default_rng(20)
+    x0 = rng.standard_normal(5)
+    gs = _rand_grads(rng, 7, 4, 5)
+    st = olsgd.LocalSGD(x0, 4, 1, 0.1)
+    x = x0.copy()
+    for g in gs:
+        st.step(g)
+        x = x - 0.1 * g.mean(axis=0)
+        assert np.allclose(st.x, x, rtol=1e-14, atol=1e-15)
+
+
+def test_local_sgd_written_out_by_hand():
+    # m = 2, tau = 2, gamma = 1, gradients (1, 3) then (2, 0):
+    # k=0: x = (-1, -3);  k=1: x = (-3, -3) -> average -3 for both
+    st = olsgd.LocalSGD(np.zeros(1), 2, 2, 1.0)
+    st.step(np.array([[1.0], [3.0]]))
+    assert st.x[:, 0].tolist() == [-1.0, -3.0] and st.z[0] == 0.0
+    st.step(np.array([[2.0], [0.0]]))
+    assert st.x[:, 0].tolist() == [-3.0, -3.0] and st.z[0] == -3.0
+
+
+def test_local_sgd_mean_follows_the_mean_gradient_and_workers_agree_after_sync():
+    rng = np.random.default_rng(21)
+    m, d, tau, gamma = 5, 4, 3, 0.07
+    st = olsgd.LocalSGD(rng.standard_normal(d), m, tau, gamma)
+    for k, g in enumerate(_rand_grads(rng, 10, m, d)):
+        mean_before = st.x.mean(axis=0)
+        st.step(g)
+        assert np.allclose(st.x.mean(axis=0), mean_before - gamma * g.mean(axis=0), atol=1e-14)
+        if (k + 1) % tau == 0:
+            assert all(np.array_equal(st.x[i], st.x[0]) for i in range(m))
+            assert np.array_equal(st.z, st.x[0])
+
+
+def test_local_sgd_equals_the_matrix_form_with_full_averaging():
+    # Eq. 2 as X_{k+1} = (X_k - gamma G_k) W with W = 1 1^T / m on sync steps
+    rng = np.random.default_rng(22)
+    m, d, tau, gamma = 4, 3, 2, 0.1
+    x0 = rng.standard_normal(d)
+    st = olsgd.LocalSGD(x0, m, tau, gamma)
+    X = np.tile(x0[:, None], (1, m))
+    for k, g in enumerate(_rand_grads(rng, 6, m, d)):
+        W = np.full((m, m), 1.0 / m) if (k + 1) % tau == 0 else np.eye(m)
+        X = (X - gamma * g.T) @ W
+        st.step(g)
+        assert np.allclose(st.x.T, X, rtol=1e-13, atol=1e-14)
+
+
+def test_overlap_with_alpha_one_half_differs_from_local_sgd_only_through_the_lag():
+    # one worker: Local SGD is plain SGD; Overlap-Local-SGD with m = 1 pulls toward the
+    # previous period's model, so the two differ after the first period
+    x0 = np.array([4.0])
+    a = olsgd.LocalSGD(x0, 1, 2, 0.25)
+    b = olsgd.OverlapLocalSGD(x0, 1, 2, 0.25, 0.5)
+    for _ in range(2):
+        a.step(a.x.copy())
+        b.step(b.x.copy())
+    assert a.x[0, 0] == 4.0 * 0.75 ** 2
+    assert b.x[0, 0] == 0.5 * 4.0 * 0.75 ** 2 + 0.5 * 4.0
