@@ -420,6 +420,96 @@ def run_flat_sweep(args, rank, world):
     }
 
 
+def run_sharded(args, rank, world):
+    """--shard-workers: ONE m-worker job whose worker dimension is split over the ranks
+    (m / N workers per GPU, same data set and minibatches as the single-GPU job).  The only
+    exchange is the sum of Eq. 5, an NCCL all-reduce of P floats per period issued on the
+    side stream between olsgd_period_sync_begin and olsgd_period_sync_finish, so it overlaps
+    the next period's local steps as in the paper.  Total work is fixed: strong scaling."""
+    import torch
+    import torch.distributed as dist
+    from paper_2002_09539_b200 import OverlapLocalSGD, class_pairs
+    from paper_2002_09539_b200.build import build
+
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if not dist.is_initialized():
+        if "MASTER_ADDR" not in os.environ:
+            os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT="29533")
+        dist.init_process_group("nccl", rank=rank, world_size=world,
+                                device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        build()
+    dist.barrier()
+    name = args.workload
+    c = dict(si.CONFIGS[name])
+    if c["gemm_bf16"] and args.gemm_mode:
+        c["gemm_bf16"] = args.gemm_mode
+    m, K, W = c["m"], args.steps, args.warmup
+    if m % world:
+        raise SystemExit("--shard-workers needs m (%d) divisible by the number of GPUs (%d)" % (m, world))
+    m_loc, off = m // world, rank * (m // world)
+    table = class_pairs(0, m, device="cpu").numpy() if c.get("non_iid") else None
+    X, y, x0 = make_inputs(name, 0, table)          # every rank builds the same data set
+    P = n_params(c)
+    Xd = torch.from_numpy(np.ascontiguousarray(X[off:off + m_loc])).cuda()
+    yd = torch.from_numpy(np.ascontiguousarray(y[off:off + m_loc])).cuda()
+    opt = OverlapLocalSGD(c["kind"], m=m_loc, tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"],
+                          beta=c["beta"], mu=c["mu"], batch=c["batch"], seed=0, dims=c["dims"],
+                          gemm_bf16=c["gemm_bf16"], x0=x0, X=Xd, y=yd, worker_offset=off, m_total=m)
+    buf = torch.zeros(opt.lib.olsgd_row_floats(opt.ctx), device="cuda")
+
+    def steps(count):
+        for _ in range(count):
+            opt.local_step()
+            if opt.iteration % c["tau"] == 0:
+                opt.period_sync_sharded(buf)
+
+    steps(W)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    dist.barrier()
+    torch.cuda.synchronize()
+    n0 = opt.launch_count
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    steps(K)
+    opt.main.wait_stream(opt.side)
+    e1.record()
+    dist.barrier()
+    torch.cuda.synchronize()
+    ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
+    launches = opt.launch_count - n0
+    clocks = sampler.stop() if rank == 0 else None
+    opt.profile_enable(True)
+    steps(K)
+    prof = opt.profile_read()
+    opt.profile_enable(False)
+    zsum = float(np.abs(opt.get_params(-1)).sum())
+    opt.close()
+    out = None
+    if rank == 0:
+        busy = {k: v for k, v in prof.items() if v[0] > 0}
+        out = {
+            "metric": METRIC, "value": round(m * K / (ms * 1e-3), 1), "unit": UNIT, "n_gpus": world,
+            "steps": K, "warmup": W, "ms_per_step": round(ms / K, 4), "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None,
+            "dtype": "bf16" if c["gemm_bf16"] else "f32", "data": "synthetic",
+            "config": {"workload": workload_name(name, c), "m": m, "workers_per_gpu": m_loc,
+                       "tau": c["tau"], "batch": c["batch"], "dims": c["dims"], "P": P,
+                       "parallelism": "workers sharded over %d GPU(s), all-reduce of the anchor sum" % world,
+                       "allreduce_bytes_per_period": int(P * 4), "anchor_abs_sum": zsum},
+            "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
+            "roofline": dict(bound="hbm", kernel=None, traffic=None,
+                             class_us_per_step={k: round(v[1] * 1e3 / K, 2) for k, v in busy.items()}),
+            "cpu_baseline": None,
+        }
+    dist.barrier()
+    dist.destroy_process_group()
+    return out
+
+
 def max_over_ranks(value, world, device):
     """The slowest rank's value (timings are reported as the max over ranks)."""
     if world <= 1:
@@ -513,6 +603,9 @@ def main():
     ap.add_argument("--method", default="overlap", choices=["overlap", "local_sgd", "sync_sgd"],
                     help="overlap: Overlap-Local-SGD (Eq. 3-5, 10-11); local_sgd: blocking periodic "
                          "averaging (Eq. 2); sync_sgd: Eq. 2 with tau = 1")
+    ap.add_argument("--shard-workers", action="store_true",
+                    help="split the m workers of ONE job over the GPUs (strong scaling) instead of "
+                         "running one replica of the job per GPU")
     ap.add_argument("--P", type=int, default=0, help="c5 only: one parameter count")
     ap.add_argument("--m", type=int, default=0, help="c5 only: one worker count")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -523,6 +616,8 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":
         out = run_reference(args, rank, world)
+    elif args.shard_workers:
+        out = run_sharded(args, rank, world)
     elif args.workload == "c5":
         out = run_flat_sweep(args, rank, world) if rank == 0 else None
     else:

@@ -83,6 +83,12 @@ typedef struct {
   int32_t m, tau, batch, mode /* olsgd_mode */;
   float gamma, alpha, beta, mu;
   uint64_t seed;                /* seeds the minibatch index rule                    */
+  /* Sharding of the worker dimension over several contexts (one per GPU).  This context
+   * holds the workers worker_offset .. worker_offset + m - 1 of m_total; the minibatch rule
+   * uses the global worker id and the anchor is the mean over all m_total workers, formed
+   * with olsgd_period_sync_begin / _finish around the caller's all-reduce.  m_total = 0
+   * means "not sharded" (m_total = m, worker_offset = 0).                              */
+  int32_t worker_offset, m_total;
 } olsgd_hparams;
 
 /* Worker i's data set D_i (Eq. 1).  Device pointers, borrowed for the life of
@@ -169,6 +175,24 @@ olsgd_status olsgd_local_step_with_grads(olsgd_ctx* ctx, const float* g_device);
  * Legal exactly once per period, when k > 0 and k mod tau == 0; otherwise
  * OLSGD_ESTATE.                                                             */
 olsgd_status olsgd_period_sync(olsgd_ctx* ctx);
+
+/* The anchor refresh split in two for a worker dimension that is sharded over several
+ * contexts: the only exchange of the method is the sum in Eq. 5.
+ *   olsgd_period_sync_begin   legal exactly when olsgd_period_sync would be; on the side
+ *                             stream, after the pull-back that closed the period, writes
+ *                             the undivided sum of THIS context's worker models into
+ *                             partial_sum_device (P floats rounded up to a multiple of 64,
+ *                             device, 16-byte aligned; olsgd_row_floats gives the count)
+ *   (caller)                  sums that buffer over all contexts, in place, ordered after the
+ *                             side stream's work and before the next call: ncclAllReduce on
+ *                             the side stream, or any other means
+ *   olsgd_period_sync_finish  on the side stream: s = total / m_total, then Eq. 5 or Eq. 10-11
+ * Both return at once; the next period's local steps overlap with all three stages, exactly
+ * as with olsgd_period_sync.  OLSGD_MODE_OVERLAP only.                                   */
+olsgd_status olsgd_period_sync_begin(olsgd_ctx* ctx, float* partial_sum_device);
+olsgd_status olsgd_period_sync_finish(olsgd_ctx* ctx, const float* total_sum_device);
+/* Floats in one padded state row (P rounded up to a multiple of 64).                    */
+int64_t olsgd_row_floats(const olsgd_ctx* ctx);
 
 /* n_iters iterations in one call: olsgd_local_step, followed by
  * olsgd_period_sync whenever a period ends.  Not for OLSGD_FLAT.

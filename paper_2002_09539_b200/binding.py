@@ -33,7 +33,7 @@ class _ModelSpec(C.Structure):
 class _HParams(C.Structure):
     _fields_ = [("m", C.c_int32), ("tau", C.c_int32), ("batch", C.c_int32), ("mode", C.c_int32),
                 ("gamma", C.c_float), ("alpha", C.c_float), ("beta", C.c_float), ("mu", C.c_float),
-                ("seed", C.c_uint64)]
+                ("seed", C.c_uint64), ("worker_offset", C.c_int32), ("m_total", C.c_int32)]
 
 
 class _Data(C.Structure):
@@ -67,6 +67,9 @@ def load_library():
         "olsgd_selftest_wait_timeout": (i32, [vp, i32]),
         "olsgd_clear_status": (i32, [vp]),
         "olsgd_period_sync": (i32, [vp]),
+        "olsgd_period_sync_begin": (i32, [vp, vp]),
+        "olsgd_period_sync_finish": (i32, [vp, vp]),
+        "olsgd_row_floats": (i64, [vp]),
         "olsgd_run": (i32, [vp, i64, vp]),
         "olsgd_get_params": (i32, [vp, i32, vp, C.c_size_t]),
         "olsgd_get_indices": (i32, [vp, i64, vp]),
@@ -131,12 +134,12 @@ class OverlapLocalSGD:
 
     def __init__(self, kind, *, m, tau, gamma, alpha, beta=0.0, mu=0.0, batch=1, seed=0,
                  dims=(), gemm_bf16=0, flat_P=0, x0, X=None, y=None, overlap=True,
-                 local_sgd=False, device="cuda"):
+                 local_sgd=False, worker_offset=0, m_total=0, device="cuda"):
         self.lib = load_library()
         self.device = torch.device(device)
         self.spec = _spec(kind, dims, gemm_bf16, flat_P)
         self.hp = _HParams(int(m), int(tau), int(batch), 1 if local_sgd else 0, float(gamma), float(alpha),
-                           float(beta), float(mu), int(seed))
+                           float(beta), float(mu), int(seed), int(worker_offset), int(m_total))
         self.m, self.tau, self.batch, self.kind = int(m), int(tau), int(batch), kind
         P = C.c_int64()
         _check(self.lib, self.lib.olsgd_param_count(C.byref(self.spec), C.byref(P)))
@@ -196,6 +199,24 @@ class OverlapLocalSGD:
 
     def period_sync(self):
         _check(self.lib, self.lib.olsgd_period_sync(self.ctx), self.ctx)
+
+    def period_sync_begin(self, partial_sum):
+        assert partial_sum.is_cuda and partial_sum.dtype == torch.float32
+        assert partial_sum.numel() >= self.lib.olsgd_row_floats(self.ctx)
+        _check(self.lib, self.lib.olsgd_period_sync_begin(self.ctx, partial_sum.data_ptr()), self.ctx)
+
+    def period_sync_finish(self, total_sum):
+        assert total_sum.is_cuda and total_sum.dtype == torch.float32
+        _check(self.lib, self.lib.olsgd_period_sync_finish(self.ctx, total_sum.data_ptr()), self.ctx)
+
+    def period_sync_sharded(self, buf, group=None):
+        """Anchor refresh of a context that holds a shard of the workers: partial sum, all-reduce
+        over `group` (torch.distributed, issued on the side stream), anchor update."""
+        import torch.distributed as dist
+        self.period_sync_begin(buf)
+        with torch.cuda.stream(self.side):
+            dist.all_reduce(buf, op=dist.ReduceOp.SUM, group=group)
+        self.period_sync_finish(buf)
 
     def run(self, n_iters, loss=None):
         if loss is not None:

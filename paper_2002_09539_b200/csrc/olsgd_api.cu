@@ -56,6 +56,7 @@ struct olsgd_ctx {
   bool reduce_pending = false;  // an anchor refresh was launched and not yet waited for
   int reduce_reads = -1;        // which x buffer that refresh reads
   bool need_sync = false;       // a period ended; olsgd_period_sync is due
+  bool sync_begun = false;      // olsgd_period_sync_begin ran; _finish is due
 
   int64_t k = 0;
   int64_t launches = 0;
@@ -203,6 +204,12 @@ olsgd_status check_hp(const olsgd_hparams* hp) {
   if (!(hp->beta >= 0.f && hp->beta < 1.f))
     return fail(nullptr, OLSGD_EINVAL, "beta must be in [0, 1)");
   if (!(hp->mu >= 0.f && hp->mu < 1.f)) return fail(nullptr, OLSGD_EINVAL, "mu must be in [0, 1)");
+  if (hp->m_total != 0 && (hp->worker_offset < 0 || hp->worker_offset + hp->m > hp->m_total))
+    return fail(nullptr, OLSGD_EINVAL, "worker_offset + m must not exceed m_total");
+  if (hp->m_total == 0 && hp->worker_offset != 0)
+    return fail(nullptr, OLSGD_EINVAL, "worker_offset needs m_total");
+  if (hp->m_total != 0 && hp->mode != OLSGD_MODE_OVERLAP)
+    return fail(nullptr, OLSGD_EINVAL, "sharded contexts support OLSGD_MODE_OVERLAP only");
   if (hp->mode != OLSGD_MODE_OVERLAP && hp->mode != OLSGD_MODE_LOCAL_SGD)
     return fail(nullptr, OLSGD_EINVAL, "mode must be OLSGD_MODE_OVERLAP or OLSGD_MODE_LOCAL_SGD");
   return OLSGD_OK;
@@ -523,7 +530,7 @@ olsgd_status olsgd_local_step(olsgd_ctx* c, float* loss_device) {
   {
     Launch l(c, OLSGD_KC_INDEX, c->main);
     OLSGD_CUDA(c, launch_minibatch_indices(c->idx, c->hp.seed, c->hp.m, c->k, c->hp.batch,
-                                           c->data.n_per_worker, c->main));
+                                           c->data.n_per_worker, c->hp.worker_offset, c->main));
   }
   return step_body(c, c->data, c->idx, loss_device, -1);
 }
@@ -585,7 +592,7 @@ olsgd_status olsgd_join(olsgd_ctx* c) {
 
 olsgd_status olsgd_period_sync(olsgd_ctx* c) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
-  if (!c->need_sync)
+  if (!c->need_sync || c->sync_begun)
     return fail(c, OLSGD_ESTATE, "olsgd_period_sync is legal once, right after a period ends (k=%lld, tau=%d)",
                 (long long)c->k, c->hp.tau);
   // S7 on the side stream, ordered after the pull-back that closed the period
@@ -599,6 +606,10 @@ olsgd_status olsgd_period_sync(olsgd_ctx* c) {
   a.ld = c->ld;
   a.m = c->hp.m;
   a.beta = c->hp.beta;
+  a.partial = nullptr;
+  if (c->hp.m_total != 0 && c->hp.m_total != c->hp.m)
+    return fail(c, OLSGD_ESTATE, "this context holds a shard of the workers: use "
+                                 "olsgd_period_sync_begin / olsgd_period_sync_finish");
   {
     Launch l(c, OLSGD_KC_ANCHOR, c->side);
     OLSGD_CUDA(c, launch_worker_mean_anchor(a, c->side));
@@ -609,6 +620,55 @@ olsgd_status olsgd_period_sync(olsgd_ctx* c) {
   c->need_sync = false;
   return OLSGD_OK;
 }
+
+olsgd_status olsgd_period_sync_begin(olsgd_ctx* c, float* partial_sum_device) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  if (!partial_sum_device || (reinterpret_cast<uintptr_t>(partial_sum_device) & 15))
+    return fail(c, OLSGD_EINVAL, "partial_sum_device must be non-null and 16-byte aligned");
+  if (!c->need_sync || c->sync_begun)
+    return fail(c, OLSGD_ESTATE, "olsgd_period_sync_begin is legal once, right after a period ends");
+  OLSGD_CUDA(c, cudaEventRecord(c->pullback_done, c->main));
+  OLSGD_CUDA(c, cudaStreamWaitEvent(c->side, c->pullback_done, 0));
+  AnchorArgs a;
+  a.x = c->x[c->cur];
+  a.z = c->z;
+  a.v = c->v;
+  a.P = c->P;
+  a.ld = c->ld;
+  a.m = c->hp.m;
+  a.beta = c->hp.beta;
+  a.partial = partial_sum_device;
+  {
+    Launch l(c, OLSGD_KC_ANCHOR, c->side);
+    OLSGD_CUDA(c, launch_worker_mean_anchor(a, c->side));
+  }
+  // from here on the worker models are no longer read by the refresh, but z is not ready:
+  // the main stream must still wait for reduce_done (recorded by _finish) before it reads z
+  c->sync_begun = true;
+  return OLSGD_OK;
+}
+
+olsgd_status olsgd_period_sync_finish(olsgd_ctx* c, const float* total_sum_device) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  if (!total_sum_device || (reinterpret_cast<uintptr_t>(total_sum_device) & 15))
+    return fail(c, OLSGD_EINVAL, "total_sum_device must be non-null and 16-byte aligned");
+  if (!c->sync_begun)
+    return fail(c, OLSGD_ESTATE, "olsgd_period_sync_finish needs olsgd_period_sync_begin first");
+  const int m_total = c->hp.m_total ? c->hp.m_total : c->hp.m;
+  {
+    Launch l(c, OLSGD_KC_ANCHOR, c->side);
+    OLSGD_CUDA(c, launch_anchor_from_sum(total_sum_device, c->z, c->v, c->P, c->hp.beta, m_total,
+                                         c->side));
+  }
+  OLSGD_CUDA(c, cudaEventRecord(c->reduce_done, c->side));
+  c->reduce_pending = true;
+  c->reduce_reads = c->cur;
+  c->need_sync = false;
+  c->sync_begun = false;
+  return OLSGD_OK;
+}
+
+int64_t olsgd_row_floats(const olsgd_ctx* c) { return c ? c->ld : -1; }
 
 olsgd_status olsgd_run(olsgd_ctx* c, int64_t n_iters, float* loss_device) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
@@ -663,7 +723,7 @@ olsgd_status olsgd_get_indices(olsgd_ctx* c, int64_t k, int32_t* dst) {
   {
     Launch l(c, OLSGD_KC_INDEX, c->main);
     OLSGD_CUDA(c, launch_minibatch_indices(c->idx, c->hp.seed, c->hp.m, k, c->hp.batch,
-                                           c->data.n_per_worker, c->main));
+                                           c->data.n_per_worker, c->hp.worker_offset, c->main));
   }
   return copy_out(c, dst, c->idx, (size_t)c->hp.m * c->hp.batch * sizeof(int32_t));
 }

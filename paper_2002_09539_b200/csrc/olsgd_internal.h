@@ -40,8 +40,12 @@ struct AnchorArgs {
   int64_t P, ld;
   int m;
   float beta;
+  float* partial;   // non-null: only write the undivided column sums there (sharded sync)
 };
 cudaError_t launch_worker_mean_anchor(const AnchorArgs& a, cudaStream_t s);
+// Eq. 5 / Eq. 10-11 from column sums over all m_total workers (sum is padded like a state row).
+cudaError_t launch_anchor_from_sum(const float* sum, float* z, float* v, int64_t P, float beta,
+                                   int m_total, cudaStream_t s);
 
 // Eq. 2 on a sync step: every worker row of x (and of its bf16 shadow, if any) and z are
 // replaced by the worker mean, summed in worker order.
@@ -53,8 +57,10 @@ cudaError_t launch_virtual_sequence(const float* x, const float* z, float* dst, 
                                     int64_t ld, int m, float alpha, cudaStream_t s);
 
 // ---- sampling_kernels.cu ----------------------------------------------------
+// worker_offset: global id of this context's first worker (the rule is a function of the
+// global worker id, so a sharded run draws the same minibatches as an unsharded one)
 cudaError_t launch_minibatch_indices(int32_t* idx, uint64_t seed, int m, int64_t k, int batch,
-                                     int64_t n, cudaStream_t s);
+                                     int64_t n, int worker_offset, cudaStream_t s);
 cudaError_t launch_class_pairs(int32_t* dst, uint64_t seed, int m, cudaStream_t s);
 // idx[i][j] = j: the "indices" of a minibatch that is already contiguous
 cudaError_t launch_identity_indices(int32_t* idx, int m, int batch, cudaStream_t s);

@@ -36,12 +36,13 @@ constexpr uint32_t kStreamPartition = 2;
 
 // One thread per Philox block: four consecutive slots of one worker.
 __global__ void minibatch_indices_kernel(int32_t* __restrict__ idx, uint32_t k0, uint32_t k1,
-                                         int m, uint32_t k, int batch, uint32_t n) {
+                                         int m, uint32_t k, int batch, uint32_t n,
+                                         uint32_t worker_offset) {
   const int blocks_per_worker = (batch + 3) / 4;
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= m * blocks_per_worker) return;
   const int i = t / blocks_per_worker, q = t % blocks_per_worker;
-  const U4 r = philox4x32_10((uint32_t)q, k, (uint32_t)i, kStreamMinibatch, k0, k1);
+  const U4 r = philox4x32_10((uint32_t)q, k, (uint32_t)i + worker_offset, kStreamMinibatch, k0, k1);
 #pragma unroll
   for (int lane = 0; lane < 4; ++lane) {
     const int j = q * 4 + lane;
@@ -84,12 +85,12 @@ cudaError_t launch_identity_indices(int32_t* idx, int m, int batch, cudaStream_t
 }
 
 cudaError_t launch_minibatch_indices(int32_t* idx, uint64_t seed, int m, int64_t k, int batch,
-                                     int64_t n, cudaStream_t s) {
+                                     int64_t n, int worker_offset, cudaStream_t s) {
   const int total = m * ((batch + 3) / 4);
   const int threads = 128;
   minibatch_indices_kernel<<<(total + threads - 1) / threads, threads, 0, s>>>(
       idx, (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), m, (uint32_t)k, batch,
-      (uint32_t)n);
+      (uint32_t)n, (uint32_t)worker_offset);
   return cudaGetLastError();
 }
 

@@ -79,11 +79,14 @@ constexpr int kMeanThreads = 256;
 // sequentially (four loads in flight), the partial sums are staged in shared
 // memory and slice 0 adds them in slice order.  SLICES depends on m only, so the
 // result does not depend on P, on the launch shape or on timing.
+// With `partial` non-null the kernel stops after the sum: it writes the undivided column
+// sums of this GPU's workers there (the input of the cross-GPU all-reduce) and leaves z, v
+// alone.
 template <bool MOM, int SLICES>
 __global__ void __launch_bounds__(kMeanThreads)
 worker_mean_anchor_kernel(const float* __restrict__ x, float* __restrict__ z,
-                          float* __restrict__ v, int64_t n4, int64_t ld, int m, float beta,
-                          float m_f) {
+                          float* __restrict__ v, float* __restrict__ partial, int64_t n4,
+                          int64_t ld, int m, float beta, float m_f) {
   constexpr int kMeanCols = kMeanThreads / SLICES;
   constexpr int kMeanSlices = SLICES;
   __shared__ float4 part[kMeanSlices][kMeanCols];
@@ -121,6 +124,10 @@ worker_mean_anchor_kernel(const float* __restrict__ x, float* __restrict__ z,
     s.y += p.y;
     s.z += p.z;
     s.w += p.w;
+  }
+  if (partial) {
+    reinterpret_cast<float4*>(partial)[col4] = s;
+    return;
   }
   s.x /= m_f;
   s.y /= m_f;
@@ -181,6 +188,38 @@ worker_mean_broadcast_kernel(float* __restrict__ x, __nv_bfloat16* __restrict__ 
   }
 }
 
+// Second half of a sharded anchor refresh: `sum` holds the column sums over ALL workers
+// (after the all-reduce); Eq. 5 or Eq. 10-11 with s = sum / m_total.
+template <bool MOM>
+__global__ void __launch_bounds__(kUpdateThreads)
+anchor_from_sum_kernel(const float* __restrict__ sum, float* __restrict__ z, float* __restrict__ v,
+                       int64_t n4, float beta, float m_f) {
+  const int64_t col4 = (int64_t)blockIdx.x * kUpdateThreads + threadIdx.x;
+  if (col4 >= n4) return;
+  float4 s = reinterpret_cast<const float4*>(sum)[col4];
+  s.x /= m_f;
+  s.y /= m_f;
+  s.z /= m_f;
+  s.w /= m_f;
+  float4* z4 = reinterpret_cast<float4*>(z) + col4;
+  if (MOM) {
+    float4* v4 = reinterpret_cast<float4*>(v) + col4;
+    float4 zz = *z4, vv = *v4;
+    vv.x = fmaf(beta, vv.x, s.x - zz.x);
+    vv.y = fmaf(beta, vv.y, s.y - zz.y);
+    vv.z = fmaf(beta, vv.z, s.z - zz.z);
+    vv.w = fmaf(beta, vv.w, s.w - zz.w);
+    zz.x += vv.x;
+    zz.y += vv.y;
+    zz.z += vv.z;
+    zz.w += vv.w;
+    *v4 = vv;
+    *z4 = zz;
+  } else {
+    *z4 = s;
+  }
+}
+
 __global__ void virtual_sequence_kernel(const float* __restrict__ x, const float* __restrict__ z,
                                         float* __restrict__ dst, int64_t P, int64_t ld, int m,
                                         float alpha, float m_f) {
@@ -232,9 +271,9 @@ cudaError_t launch_mean(const AnchorArgs& a, cudaStream_t s) {
   dim3 grid((unsigned)((n4 + cols - 1) / cols)), block(cols, SLICES);
   const float m_f = (float)a.m;
   if (a.beta != 0.f)
-    worker_mean_anchor_kernel<true, SLICES><<<grid, block, 0, s>>>(a.x, a.z, a.v, n4, a.ld, a.m, a.beta, m_f);
+    worker_mean_anchor_kernel<true, SLICES><<<grid, block, 0, s>>>(a.x, a.z, a.v, a.partial, n4, a.ld, a.m, a.beta, m_f);
   else
-    worker_mean_anchor_kernel<false, SLICES><<<grid, block, 0, s>>>(a.x, a.z, a.v, n4, a.ld, a.m, a.beta, m_f);
+    worker_mean_anchor_kernel<false, SLICES><<<grid, block, 0, s>>>(a.x, a.z, a.v, a.partial, n4, a.ld, a.m, a.beta, m_f);
   return cudaGetLastError();
 }
 
@@ -251,6 +290,17 @@ cudaError_t launch_worker_mean_broadcast(float* x, __nv_bfloat16* shadow, float*
   const int64_t n4 = (P + 3) / 4;
   worker_mean_broadcast_kernel<<<(unsigned)((n4 + kUpdateThreads - 1) / kUpdateThreads),
                                  kUpdateThreads, 0, s>>>(x, shadow, z, n4, ld, m, (float)m);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_anchor_from_sum(const float* sum, float* z, float* v, int64_t P, float beta,
+                                   int m_total, cudaStream_t s) {
+  const int64_t n4 = (P + 3) / 4;
+  const unsigned grid = (unsigned)((n4 + kUpdateThreads - 1) / kUpdateThreads);
+  if (beta != 0.f)
+    anchor_from_sum_kernel<true><<<grid, kUpdateThreads, 0, s>>>(sum, z, v, n4, beta, (float)m_total);
+  else
+    anchor_from_sum_kernel<false><<<grid, kUpdateThreads, 0, s>>>(sum, z, v, n4, beta, (float)m_total);
   return cudaGetLastError();
 }
 
