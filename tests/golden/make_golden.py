@@ -50,6 +50,10 @@ def main(names):
             "F_mean_model": models.full_objective(c["kind"], c["dims"], xbar, X, y),
             "F_anchor": models.full_objective(c["kind"], c["dims"], st.z, X, y),
             "minibatch_loss_mean_every_50": [float(v) for v in losses.mean(axis=1)[49::50]],
+            # mean over workers AND over each block of 50 iterations: a far less noisy
+            # statistic of the trajectory than one iteration's loss
+            "minibatch_loss_block_mean_50": [float(losses[b:b + 50].mean())
+                                             for b in range(0, losses.shape[0] - 49, 50)],
             "minibatch_loss_last10_mean": float(losses[-10:].mean()),
             "norm2_mean_model": float(np.linalg.norm(xbar)),
             "norm2_anchor": float(np.linalg.norm(st.z)),

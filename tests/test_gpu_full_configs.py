@@ -83,14 +83,17 @@ def test_mlp_configs_first_iterations_against_exact_oracle(name, iters, tol_para
 
 # How long the stored trajectory can be followed.  The momentum configurations are
 # chaotic once the loss is small: the SAME kernels started from x0 with 1e-7 added to
-# one entry end config 3 with a 40 % different objective, and two fp64 oracle runs
-# that differ by that perturbation drift apart likewise (tests/golden/c3_perturbed.json).
+# one entry end config 3 with a 40 % different objective, and two fp64 ORACLE runs
+# that differ by that perturbation agree to 6 digits up to iteration 250, by 1 % at 400,
+# 3 % at 450, 45 % at 700 and end 22 % apart (tests/golden/c3_final.json vs
+# c3_perturbed.json).  A perturbation of bf16 size (2^-8 per operand) gets there sooner.
 # No implementation can meet a 2e-2 bound on the loss after the full 1000 iterations,
 # so the bound is enforced on the stored checkpoints up to STRICT_UNTIL and the end of
 # the run is checked for having trained to the same level.
 # Config 4 (tau = 8, alpha = 0.5) stays reproducible to the end, so there the 2e-2 bound is
 # enforced on every checkpoint and on the final objective.
-STRICT_UNTIL = {"c3": 250, "c4": 800}
+STRICT_UNTIL = {"c3": 150, "c4": 800}          # one iteration's worker-mean loss
+STRICT_BLOCKS_UNTIL = {"c3": 250, "c4": 800}   # mean over blocks of 50 iterations
 FINAL_STRICT = {"c3": False, "c4": True}
 
 
@@ -108,6 +111,11 @@ def test_mlp_configs_full_length(name):
         k = 50 * (t + 1)
         if k <= STRICT_UNTIL[name]:
             assert abs(every50[t] - want) <= TOL_BF16_LOSS * want, (k, every50[t], want)
+    blocks = gold.get("minibatch_loss_block_mean_50", [])
+    for t, want in enumerate(blocks):
+        if 50 * (t + 1) <= STRICT_BLOCKS_UNTIL[name]:
+            got = float(lg[50 * t:50 * t + 50].mean())
+            assert abs(got - want) <= TOL_BF16_LOSS * want, (50 * (t + 1), got, want)
     xbar, z = opt.get_params(-4).copy(), opt.get_params(-1).copy()
     F_mean = models.full_objective("mlp", c["dims"], xbar, X, y)
     F_anchor = models.full_objective("mlp", c["dims"], z, X, y)
