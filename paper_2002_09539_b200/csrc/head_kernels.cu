@@ -27,6 +27,21 @@ __device__ __forceinline__ float load_in<__nv_bfloat16>(const __nv_bfloat16* p) 
   return __bfloat162float(*p);
 }
 
+// Row b of worker i of the layer's input, and its label, with or without the fused gather.
+template <typename InT>
+__device__ __forceinline__ const InT* head_row(const HeadArgs& a, int i, int b) {
+  if (sizeof(InT) == 4) {
+    const int64_t row = a.row_idx ? (int64_t)i * a.n_rows + a.row_idx[(int64_t)i * a.batch + b]
+                                  : (int64_t)i * a.batch + b;
+    return reinterpret_cast<const InT*>(a.in32) + row * a.K;
+  }
+  return reinterpret_cast<const InT*>(a.in16) + ((int64_t)i * a.batch + b) * a.K;
+}
+__device__ __forceinline__ int head_label(const HeadArgs& a, int i, int b) {
+  if (a.row_idx) return a.y_all[(int64_t)i * a.n_rows + a.row_idx[(int64_t)i * a.batch + b]];
+  return a.yb[(int64_t)i * a.batch + b];
+}
+
 constexpr int kHeadThreads = 128;
 
 // Forward, loss and input gradient of the output layer for R batch rows of one worker.
@@ -48,12 +63,12 @@ head_forward_kernel(HeadArgs a) {
   const int i = blockIdx.y, b0 = blockIdx.x * R;
   const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
   const int K = a.K, C = a.C, B = a.batch;
-  const InT* in = (sizeof(InT) == 4 ? reinterpret_cast<const InT*>(a.in32)
-                                    : reinterpret_cast<const InT*>(a.in16)) +
-                  ((int64_t)i * B + b0) * K;
   const float* W = a.x + (int64_t)i * a.ld + a.w_off;
   const float* bias = a.x + (int64_t)i * a.ld + a.b_off;
   const int rows = min(R, B - b0);
+  const InT* rowp[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r) rowp[r] = head_row<InT>(a, i, b0 + (r < rows ? r : 0));
 
   float acc[R][CMAX];
 #pragma unroll
@@ -67,7 +82,7 @@ head_forward_kernel(HeadArgs a) {
 #pragma unroll
     for (int c = 0; c < CMAX; ++c) w[c] = (c < C) ? W[(int64_t)c * K + k] : 0.f;
 #pragma unroll
-    for (int r = 0; r < R; ++r) xv[r] = (r < rows) ? load_in<InT>(in + (int64_t)r * K + k) : 0.f;
+    for (int r = 0; r < R; ++r) xv[r] = (r < rows) ? load_in<InT>(rowp[r] + k) : 0.f;
     if (a.round_w_bf16) {
 #pragma unroll
       for (int c = 0; c < CMAX; ++c) w[c] = bf16_round(w[c]);
@@ -103,7 +118,7 @@ head_forward_kernel(HeadArgs a) {
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     const float e = (lane < C) ? expf(logit - mx) : 0.f;
     const float lse = mx + logf(warp_sum(e));
-    const int label = live ? a.yb[(int64_t)i * B + b] : 0;
+    const int label = live ? head_label(a, i, b) : 0;
     const float picked = __shfl_sync(0xffffffffu, logit, label);
     float dl = 0.f;
     if (lane < C) dl = (expf(logit - lse) - (lane == label ? 1.f : 0.f)) / (float)B;
@@ -127,7 +142,7 @@ head_forward_kernel(HeadArgs a) {
 #pragma unroll
     for (int c = 0; c < CMAX; ++c) w[c] = (c < C) ? W[(int64_t)c * K + k] : 0.f;
 #pragma unroll
-    for (int r = 0; r < R; ++r) xv[r] = (r < rows) ? load_in<InT>(in + (int64_t)r * K + k) : 0.f;
+    for (int r = 0; r < R; ++r) xv[r] = (r < rows) ? load_in<InT>(rowp[r] + k) : 0.f;
     if (a.round_w_bf16) {
 #pragma unroll
       for (int c = 0; c < CMAX; ++c) w[c] = bf16_round(w[c]);
@@ -181,9 +196,6 @@ head_wgrad_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ loss) {
   const int tx = threadIdx.x, ty = threadIdx.y, tid = ty * kWgCols + tx;
   const int j = blockIdx.x * kWgCols + tx;
   const int K = a.K, C = a.C, B = a.batch;
-  const InT* in = (sizeof(InT) == 4 ? reinterpret_cast<const InT*>(a.in32)
-                                    : reinterpret_cast<const InT*>(a.in16)) +
-                  (int64_t)i * B * K;
   const float* dl = a.dlogits + (int64_t)i * B * C;
   float acc[CMAX];
 #pragma unroll
@@ -204,7 +216,7 @@ head_wgrad_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ loss) {
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
           const int r = rb + u * kWgSlices;
-          xs[u] = (r < rc) ? load_in<InT>(in + (int64_t)(r0 + r) * K + j) : 0.f;
+          xs[u] = (r < rc) ? load_in<InT>(head_row<InT>(a, i, r0 + r) + j) : 0.f;
         }
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
@@ -246,6 +258,107 @@ head_wgrad_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ loss) {
   }
 }
 
+// The same product for K % 4 == 0 and at most 16 classes: a thread owns FOUR adjacent input
+// columns (one 16-byte fp32 or 8-byte bf16 load per row, eight in flight) and a block of
+// 32 x 4 threads covers 128 columns with four batch slices.  Fixed order as above.
+constexpr int kWvCols = 32, kWvSlices = 4, kWvRows = 128, kWvFlight = 8;
+
+__device__ __forceinline__ float4 load4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
+  const uint2 w = *reinterpret_cast<const uint2*>(p);
+  const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&w.x);
+  const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&w.y);
+  return make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
+}
+
+template <typename InT, int CMAX>
+__global__ void __launch_bounds__(kWvCols* kWvSlices)
+head_wgrad_vec_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ loss) {
+  __shared__ float dsm[kWvRows][CMAX + 1];
+  __shared__ __align__(16) float part[kWvSlices][CMAX][kWvCols * 4];
+  const int i = blockIdx.y;
+  const int tx = threadIdx.x, ty = threadIdx.y, tid = ty * kWvCols + tx;
+  const int j = (blockIdx.x * kWvCols + tx) * 4;
+  const int K = a.K, C = a.C, B = a.batch;
+  const float* dl = a.dlogits + (int64_t)i * B * C;
+  float acc[4][CMAX];
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+#pragma unroll
+    for (int c = 0; c < CMAX; ++c) acc[q][c] = 0.f;
+  float bsum = 0.f;
+  for (int r0 = 0; r0 < B; r0 += kWvRows) {
+    const int rc = min(kWvRows, B - r0);
+    __syncthreads();
+    for (int e = tid; e < rc * C; e += kWvCols * kWvSlices) {
+      float d = dl[(int64_t)r0 * C + e];
+      if (a.round_w_bf16) d = bf16_round(d);
+      dsm[e / C][e % C] = d;
+    }
+    __syncthreads();
+    if (j < K) {
+      for (int rb = ty; rb < rc; rb += kWvSlices * kWvFlight) {
+        float4 xs[kWvFlight];
+#pragma unroll
+        for (int u = 0; u < kWvFlight; ++u) {
+          const int r = rb + u * kWvSlices;
+          xs[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (r < rc) xs[u] = load4(head_row<InT>(a, i, r0 + r) + j);
+        }
+#pragma unroll
+        for (int u = 0; u < kWvFlight; ++u) {
+          const int r = rb + u * kWvSlices;
+          if (r < rc) {
+#pragma unroll
+            for (int c = 0; c < CMAX; ++c) {
+              if (c < C) {
+                const float d = dsm[r][c];
+                acc[0][c] = fmaf(d, xs[u].x, acc[0][c]);
+                acc[1][c] = fmaf(d, xs[u].y, acc[1][c]);
+                acc[2][c] = fmaf(d, xs[u].z, acc[2][c]);
+                acc[3][c] = fmaf(d, xs[u].w, acc[3][c]);
+              }
+            }
+          }
+        }
+      }
+    }
+    if (blockIdx.x == 0 && tid < C)
+      for (int r = 0; r < rc; ++r) bsum += dl[(int64_t)(r0 + r) * C + tid];
+  }
+#pragma unroll
+  for (int c = 0; c < CMAX; ++c)
+    if (c < C)
+      *reinterpret_cast<float4*>(&part[ty][c][tx * 4]) =
+          make_float4(acc[0][c], acc[1][c], acc[2][c], acc[3][c]);
+  __syncthreads();
+  float* gi = g + (int64_t)i * a.ld;
+  for (int e = tid; e < C * kWvCols; e += kWvCols * kWvSlices) {
+    const int c = e / kWvCols, col4 = e % kWvCols;
+    const int jj = (blockIdx.x * kWvCols + col4) * 4;
+    if (jj < K) {
+      float4 s = *reinterpret_cast<const float4*>(&part[0][c][col4 * 4]);
+#pragma unroll
+      for (int t = 1; t < kWvSlices; ++t) {
+        const float4 p = *reinterpret_cast<const float4*>(&part[t][c][col4 * 4]);
+        s.x += p.x;
+        s.y += p.y;
+        s.z += p.z;
+        s.w += p.w;
+      }
+      *reinterpret_cast<float4*>(gi + a.w_off + (int64_t)c * K + jj) = s;
+    }
+  }
+  if (blockIdx.x == 0) {
+    if (tid < C) gi[a.b_off + tid] = bsum;
+    if (loss && tid == kWvCols * kWvSlices - 1) {
+      float s = 0.f;
+      for (int r = 0; r < B; ++r) s += a.rowloss[(int64_t)i * B + r];
+      loss[i] = s / (float)B;
+    }
+  }
+}
+
 template <typename InT, int CMAX, int R>
 cudaError_t launch_fwd(const HeadArgs& a, cudaStream_t s) {
   const size_t smem = ((size_t)R * CMAX * (kHeadThreads + 1) + (size_t)R * CMAX) * sizeof(float);
@@ -275,8 +388,19 @@ cudaError_t launch_head_forward(const HeadArgs& a, cudaStream_t s) {
 }
 
 cudaError_t launch_head_wgrad(const HeadArgs& a, float* g, float* loss, cudaStream_t s) {
-  dim3 grid((a.K + kWgCols - 1) / kWgCols, a.m), block(kWgCols, kWgSlices);
   const bool f32 = a.in32 != nullptr;
+  if (a.K % 4 == 0 && a.C <= 16 && a.w_off % 4 == 0 && a.ld % 4 == 0) {
+    dim3 vgrid((a.K / 4 + kWvCols - 1) / kWvCols, a.m), vblock(kWvCols, kWvSlices);
+    if (a.C <= 10) {
+      if (f32) head_wgrad_vec_kernel<float, 10><<<vgrid, vblock, 0, s>>>(a, g, loss);
+      else head_wgrad_vec_kernel<__nv_bfloat16, 10><<<vgrid, vblock, 0, s>>>(a, g, loss);
+    } else {
+      if (f32) head_wgrad_vec_kernel<float, 16><<<vgrid, vblock, 0, s>>>(a, g, loss);
+      else head_wgrad_vec_kernel<__nv_bfloat16, 16><<<vgrid, vblock, 0, s>>>(a, g, loss);
+    }
+    return cudaGetLastError();
+  }
+  dim3 grid((a.K + kWgCols - 1) / kWgCols, a.m), block(kWgCols, kWgSlices);
   if (a.C <= 16) {
     if (f32) head_wgrad_kernel<float, 16><<<grid, block, 0, s>>>(a, g, loss);
     else head_wgrad_kernel<__nv_bfloat16, 16><<<grid, block, 0, s>>>(a, g, loss);

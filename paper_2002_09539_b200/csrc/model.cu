@@ -182,7 +182,10 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
   const int L = n_layers(spec);
   const int d0 = spec.dims[0], C = spec.dims[L];
   const bool bf = bf16_path(spec);
-  {
+  // softmax regression in fp32 reads its rows straight from the data set (gather fused into
+  // the two output-layer kernels); every other model stages the minibatch
+  const bool fused_gather = !bf && L == 1;
+  if (!fused_gather) {
     Scope sc(hook, OLSGD_KC_GATHER, s);
     OLSGD_TRY(launch_gather(X, static_cast<const int32_t*>(data.y), io.idx, bf ? nullptr : mb.xb32,
                             bf ? mb.xb16 : nullptr, bf ? mb.xb16t : nullptr, mb.yb, m, B, n, d0,
@@ -213,7 +216,10 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
 
   // output layer: forward, loss, and backward to its input
   HeadArgs ha{};
-  ha.in32 = bf ? nullptr : mb.xb32;
+  ha.in32 = bf ? nullptr : (fused_gather ? X : mb.xb32);
+  ha.row_idx = fused_gather ? io.idx : nullptr;
+  ha.n_rows = n;
+  ha.y_all = static_cast<const int32_t*>(data.y);
   ha.in16 = bf ? mb.h[L - 1] : nullptr;
   ha.x = io.x;
   ha.ld = io.ld;

@@ -104,6 +104,12 @@ struct HeadArgs {
   __nv_bfloat16* din16t;
   int m, batch, K, C;
   bool round_w_bf16;     // round W to bf16 before use (tensor-core path's operand rule)
+  // Gather fused in (fp32 input only): when row_idx is non-null, in32 is the whole data set
+  // [m][n_rows][K], batch row b of worker i is its row row_idx[i * batch + b], and the label
+  // comes from y_all [m][n_rows] instead of yb.
+  const int32_t* row_idx;
+  int64_t n_rows;
+  const int32_t* y_all;
 };
 cudaError_t launch_head_forward(const HeadArgs& a, cudaStream_t s);
 
