@@ -123,11 +123,17 @@ def test_mlp_configs_full_length(name):
         assert abs(F_mean - gold["F_mean_model"]) <= TOL_BF16_LOSS * gold["F_mean_model"], F_mean
         assert abs(F_anchor - gold["F_anchor"]) <= TOL_BF16_LOSS * gold["F_anchor"], F_anchor
     else:
-        assert 0.5 * gold["F_mean_model"] <= F_mean <= 2.0 * gold["F_mean_model"], F_mean
-        assert 0.5 * gold["F_anchor"] <= F_anchor <= 2.0 * gold["F_anchor"], F_anchor
+        # the chaotic end of the run: six GPU runs that differ by 1e-7 in one entry of x0 end
+        # with F(mean model) between 0.11 and 0.35 and F(anchor) between 0.12 and 1.15 (the
+        # anchor carries momentum 0.9), the tail of the training loss between 0.14 and 0.20
+        # and the parameter norm within 0.3 %.  Only the stable statistics are held tightly.
+        assert 0.25 * gold["F_mean_model"] <= F_mean <= 4.0 * gold["F_mean_model"], F_mean
+        assert np.isfinite(F_anchor) and F_anchor < float(lg[0].mean())
+        tail = float(lg[-50:].mean())
+        assert 0.5 * gold["minibatch_loss_last10_mean"] <= tail <= 2.0 * gold["minibatch_loss_last10_mean"]
     # it trained: the minibatch loss at the end is far below the first iteration's
     assert float(lg[-10:].mean()) < 0.5 * float(lg[0].mean())
-    assert abs(np.linalg.norm(xbar) - gold["norm2_mean_model"]) <= 0.05 * gold["norm2_mean_model"]
+    assert abs(np.linalg.norm(xbar) - gold["norm2_mean_model"]) <= 0.02 * gold["norm2_mean_model"]
 
 
 @pytest.mark.parametrize("m", [8, 16, 64])
