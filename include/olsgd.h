@@ -207,6 +207,23 @@ olsgd_status olsgd_run(olsgd_ctx* ctx, int64_t n_iters, float* loss_device);
  *   n_floats  must equal P                                                   */
 olsgd_status olsgd_get_params(olsgd_ctx* ctx, int32_t which, float* dst, size_t n_floats);
 
+/* Overwrite one vector of the state (checkpoint / resume together with
+ * olsgd_get_params and olsgd_set_iteration).  Joins both streams.  which: 0..m-1 worker
+ * model (its bf16 copy for the tensor cores is refreshed too); -1 anchor z; -2 anchor
+ * momentum v; -5 - i local momentum u_i.
+ *   src       host or device memory, n_floats == P                                  */
+olsgd_status olsgd_set_params(olsgd_ctx* ctx, int32_t which, const float* src, size_t n_floats);
+
+/* Set the iteration counter k (k >= 0, k mod tau == 0: a period boundary, no anchor
+ * refresh pending).  With the state vectors restored this resumes a run exactly: the
+ * minibatch rule is a function of k.                                                 */
+olsgd_status olsgd_set_iteration(olsgd_ctx* ctx, int64_t k);
+
+/* Consensus distance sum_i ||x^(i) - z||^2 of the current state (the quantity the
+ * convergence proof bounds, Appendix A), summed in double precision in a fixed order on
+ * the device.  Joins both streams.  out_host: one double on the host.                */
+olsgd_status olsgd_consensus_distance(olsgd_ctx* ctx, double* out_host);
+
 /* The minibatch indices xi_k^(i) that iteration k uses (or used): slot j of
  * worker i is floor(w * n / 2^32) with w word (j mod 4) of the Philox4x32-10
  * block (Salmon et al., SC'11) of counter (j div 4, k, i, 1) and key

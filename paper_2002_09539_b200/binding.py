@@ -73,6 +73,9 @@ def load_library():
         "olsgd_run": (i32, [vp, i64, vp]),
         "olsgd_get_params": (i32, [vp, i32, vp, C.c_size_t]),
         "olsgd_get_indices": (i32, [vp, i64, vp]),
+        "olsgd_set_params": (i32, [vp, i32, vp, C.c_size_t]),
+        "olsgd_set_iteration": (i32, [vp, i64]),
+        "olsgd_consensus_distance": (i32, [vp, C.POINTER(C.c_double)]),
         "olsgd_class_pairs": (i32, [u64, i32, vp, vp]),
         "olsgd_class_pairs_noalloc": (i32, [u64, i32, vp, vp]),
         "olsgd_iteration": (i64, [vp]),
@@ -233,6 +236,20 @@ class OverlapLocalSGD:
         _check(self.lib, self.lib.olsgd_get_params(self.ctx, int(which), out.data_ptr(), self.P),
                self.ctx)
         return out.numpy() if not out.is_cuda else out
+
+    def set_params(self, which, src):
+        src = torch.as_tensor(src, dtype=torch.float32).contiguous()
+        assert src.numel() == self.P
+        _check(self.lib, self.lib.olsgd_set_params(self.ctx, int(which), src.data_ptr(), self.P),
+               self.ctx)
+
+    def set_iteration(self, k):
+        _check(self.lib, self.lib.olsgd_set_iteration(self.ctx, int(k)), self.ctx)
+
+    def consensus_distance(self):
+        out = C.c_double()
+        _check(self.lib, self.lib.olsgd_consensus_distance(self.ctx, C.byref(out)), self.ctx)
+        return out.value
 
     def get_indices(self, k):
         out = torch.empty((self.m, self.batch), dtype=torch.int32)

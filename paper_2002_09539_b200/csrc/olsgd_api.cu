@@ -714,6 +714,59 @@ olsgd_status olsgd_get_params(olsgd_ctx* c, int32_t which, float* dst, size_t n_
   return copy_out(c, dst, c->tmp, bytes);
 }
 
+olsgd_status olsgd_set_params(olsgd_ctx* c, int32_t which, const float* src, size_t n_floats) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  if (!src) return fail(c, OLSGD_EINVAL, "src is NULL");
+  if (n_floats != (size_t)c->P)
+    return fail(c, OLSGD_EINVAL, "n_floats is %zu but P is %lld", n_floats, (long long)c->P);
+  const int m = c->hp.m;
+  if (which >= m || which < -5 - (m - 1) || which == -3 || which == -4)
+    return fail(c, OLSGD_EINVAL, "which = %d cannot be set", which);
+  if (which <= -5 && !c->u) return fail(c, OLSGD_EINVAL, "no local momentum buffer (mu = 0)");
+  OLSGD_CUDA(c, cudaStreamSynchronize(c->side));
+  c->reduce_pending = false;
+  OLSGD_CUDA(c, cudaStreamSynchronize(c->main));
+  float* dst = which >= 0   ? c->x[c->cur] + (int64_t)which * c->ld
+               : which == -1 ? c->z
+               : which == -2 ? c->v
+                             : c->u + (int64_t)(-5 - which) * c->ld;
+  OLSGD_CUDA(c, cudaMemcpyAsync(dst, src, (size_t)c->P * sizeof(float), cudaMemcpyDefault, c->main));
+  if (which >= 0 && c->shadow) {
+    Launch l(c, OLSGD_KC_OTHER, c->main);
+    OLSGD_CUDA(c, launch_cast_bf16(dst, c->shadow + (int64_t)which * c->ld, c->ld, c->main));
+  }
+  OLSGD_CUDA(c, cudaStreamSynchronize(c->main));
+  return OLSGD_OK;
+}
+
+olsgd_status olsgd_set_iteration(olsgd_ctx* c, int64_t k) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  if (k < 0 || k % c->hp.tau != 0)
+    return fail(c, OLSGD_EINVAL, "k must be a non-negative multiple of tau");
+  if (c->need_sync) return fail(c, OLSGD_ESTATE, "a period ended: call olsgd_period_sync first");
+  c->k = k;
+  return OLSGD_OK;
+}
+
+olsgd_status olsgd_consensus_distance(olsgd_ctx* c, double* out_host) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  if (!out_host) return fail(c, OLSGD_EINVAL, "out_host is NULL");
+  OLSGD_CUDA(c, cudaStreamSynchronize(c->side));
+  c->reduce_pending = false;
+  OLSGD_CUDA(c, cudaStreamSynchronize(c->main));
+  // the scratch row holds ld floats = ld / 2 doubles: slot 0 the result, then the partials
+  int n_partials = (int)(c->ld / 2 - 1);
+  if (n_partials > 592) n_partials = 592;
+  double* scratch = reinterpret_cast<double*>(c->tmp);
+  {
+    Launch l(c, OLSGD_KC_OTHER, c->main);
+    OLSGD_CUDA(c, launch_consensus_distance(c->x[c->cur], c->z, scratch, n_partials, c->P, c->ld,
+                                            c->hp.m, c->main));
+    c->launches++;
+  }
+  return copy_out(c, out_host, scratch, sizeof(double));
+}
+
 olsgd_status olsgd_get_indices(olsgd_ctx* c, int64_t k, int32_t* dst) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
   if (!dst) return fail(c, OLSGD_EINVAL, "dst is NULL");

@@ -52,6 +52,11 @@ cudaError_t launch_anchor_from_sum(const float* sum, float* z, float* v, int64_t
 cudaError_t launch_worker_mean_broadcast(float* x, __nv_bfloat16* shadow, float* z, int64_t P,
                                          int64_t ld, int m, cudaStream_t s);
 
+// *out = sum_i ||x_i - z||^2 in double; scratch holds at least 2 * n_partials floats.
+cudaError_t launch_consensus_distance(const float* x, const float* z, double* scratch,
+                                      int n_partials, int64_t P, int64_t ld, int m,
+                                      cudaStream_t s);
+
 // dst[j] = (1-alpha) * mean_i x_i[j] + alpha * z[j]   (alpha = 0: mean model)
 cudaError_t launch_virtual_sequence(const float* x, const float* z, float* dst, int64_t P,
                                     int64_t ld, int m, float alpha, cudaStream_t s);

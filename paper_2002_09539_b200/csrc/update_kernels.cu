@@ -220,6 +220,33 @@ anchor_from_sum_kernel(const float* __restrict__ sum, float* __restrict__ z, flo
   }
 }
 
+// Stage 1: block b adds (x_i[j] - z[j])^2 over its strided share of the m * P entries, each
+// thread sequentially, then the threads in a fixed tree.  Stage 2: one thread adds the block
+// partials in order.  Double precision throughout.
+__global__ void __launch_bounds__(256)
+consensus_partial_kernel(const float* __restrict__ x, const float* __restrict__ z,
+                         double* __restrict__ partial, int64_t P, int64_t ld, int m) {
+  __shared__ double sm[256];
+  double acc = 0.0;
+  for (int i = 0; i < m; ++i)
+    for (int64_t j = (int64_t)blockIdx.x * 256 + threadIdx.x; j < P; j += (int64_t)gridDim.x * 256) {
+      const double d = (double)x[(int64_t)i * ld + j] - (double)z[j];
+      acc += d * d;
+    }
+  sm[threadIdx.x] = acc;
+  __syncthreads();
+  for (int s = 128; s > 0; s >>= 1) {
+    if ((int)threadIdx.x < s) sm[threadIdx.x] += sm[threadIdx.x + s];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) partial[blockIdx.x + 1] = sm[0];
+}
+__global__ void consensus_final_kernel(double* partial, int n) {
+  double s = 0.0;
+  for (int b = 0; b < n; ++b) s += partial[b + 1];
+  partial[0] = s;
+}
+
 __global__ void virtual_sequence_kernel(const float* __restrict__ x, const float* __restrict__ z,
                                         float* __restrict__ dst, int64_t P, int64_t ld, int m,
                                         float alpha, float m_f) {
@@ -301,6 +328,14 @@ cudaError_t launch_anchor_from_sum(const float* sum, float* z, float* v, int64_t
     anchor_from_sum_kernel<true><<<grid, kUpdateThreads, 0, s>>>(sum, z, v, n4, beta, (float)m_total);
   else
     anchor_from_sum_kernel<false><<<grid, kUpdateThreads, 0, s>>>(sum, z, v, n4, beta, (float)m_total);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_consensus_distance(const float* x, const float* z, double* scratch,
+                                      int n_partials, int64_t P, int64_t ld, int m,
+                                      cudaStream_t s) {
+  consensus_partial_kernel<<<n_partials, 256, 0, s>>>(x, z, scratch, P, ld, m);
+  consensus_final_kernel<<<1, 1, 0, s>>>(scratch, n_partials);
   return cudaGetLastError();
 }
 

@@ -167,3 +167,42 @@ def test_local_sgd_mode_with_models(kind, dims, gemm):
     tol = TOL_FP32 if gemm == 0 else TOL_BF16_PARAM
     assert state_err(opt, st) <= tol
     assert np.abs(loss.cpu().numpy() - lo).max() <= (2e-5 if gemm == 0 else TOL_BF16_LOSS) * np.abs(lo).max()
+
+
+def test_checkpoint_and_resume_reproduce_the_run_bit_for_bit():
+    # export (x, u, z, v) at a period boundary, restore into a fresh context, continue
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    dims, m, n, batch, tau = [128, 128, 10], 3, 90, 64, 2
+    X, y = si.mixture_data(11, m, n, dims[0])
+    x0 = si.model_init(11, "mlp", dims)
+    kw = dict(dims=dims, gemm_bf16=1, m=m, tau=tau, batch=batch, gamma=0.05, alpha=0.6, beta=0.9,
+              mu=0.9, seed=11, X=to_dev(X), y=to_dev(y))
+    a = OverlapLocalSGD("mlp", x0=x0, **kw)
+    a.run(10)
+    b = OverlapLocalSGD("mlp", x0=x0, **kw)
+    b.run(6)
+    saved = {w: b.get_params(w).copy() for w in list(range(m)) + [-1, -2] + [-5 - i for i in range(m)]}
+    c = OverlapLocalSGD("mlp", x0=np.zeros_like(x0), **kw)
+    for w, vec in saved.items():
+        c.set_params(w, vec)
+    c.set_iteration(6)
+    c.run(4)
+    xa, za, va = a.state()
+    xc, zc, vc = c.state()
+    assert np.array_equal(xa, xc) and np.array_equal(za, zc) and np.array_equal(va, vc)
+    assert c.iteration == 10
+
+
+def test_consensus_distance_matches_the_state():
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    P, m = 70001, 5
+    x0 = si.flat_init(12, P)
+    opt = OverlapLocalSGD("flat", m=m, tau=3, gamma=0.1, alpha=0.5, beta=0.5, mu=0.9, flat_P=P, x0=x0)
+    assert opt.consensus_distance() == 0.0          # all models start at the anchor
+    for k in range(4):
+        opt.local_step_with_grads(to_dev(si.flat_grads(12, k, m, P)))
+        if (k + 1) % 3 == 0:
+            opt.period_sync()
+    x, z, _ = opt.state()
+    want = float(((x.astype(np.float64) - z.astype(np.float64)) ** 2).sum())
+    assert abs(opt.consensus_distance() - want) <= 1e-12 * want
