@@ -301,7 +301,13 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, cudaStream_t s) {
   switch (bn) {
     case 256: return short_k ? launch_one<256, 2>(a, ma, mb, s) : launch_one<256, 4>(a, ma, mb, s);
     case 128: return short_k ? launch_one<128, 2>(a, ma, mb, s) : launch_one<128, 6>(a, ma, mb, s);
-    default:  return short_k ? launch_one<64, 2>(a, ma, mb, s) : launch_one<64, 8>(a, ma, mb, s);
+    default: {
+      // more tiles than SMs: four stages (96 KB) so that two CTAs share an SM and the
+      // whole grid is resident in one wave
+      const int64_t ctas = (int64_t)(a.Nb / 64) * (a.Ma / kBM) * a.m;
+      if (short_k) return launch_one<64, 2>(a, ma, mb, s);
+      return ctas > 148 ? launch_one<64, 4>(a, ma, mb, s) : launch_one<64, 8>(a, ma, mb, s);
+    }
   }
 }
 
