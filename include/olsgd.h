@@ -6,9 +6,10 @@
  * One context holds the m worker models x^(1..m), their local momentum
  * buffers, the anchor z and the anchor momentum buffer v, all resident in
  * device memory that the CALLER allocates and hands over as one workspace.
- * The library owns host memory and CUDA events only.  It never allocates
- * device memory, never throws, never aborts: every call returns a status and
- * `olsgd_last_error` gives the reason as text.
+ * A context owns host memory, CUDA events and one stream for host-to-device
+ * staging copies.  The library never allocates device memory, never throws,
+ * never aborts: every call returns a status and `olsgd_last_error` gives the
+ * reason as text.
  *
  * Conventions
  *   - "device pointer": memory on the current CUDA device, 16-byte aligned.
