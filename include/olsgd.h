@@ -90,6 +90,14 @@ typedef struct {
    * with olsgd_period_sync_begin / _finish around the caller's all-reduce.  m_total = 0
    * means "not sharded" (m_total = m, worker_offset = 0).                              */
   int32_t worker_offset, m_total;
+  /* Minibatch rule.  0: independent uniform draws with replacement (see olsgd_get_indices).
+   * 1: one pass over D_i per epoch without replacement: draw t = k * batch + j of worker i
+   * takes sample pi(t mod n) of epoch e = t div n, where pi is a four-round balanced Feistel
+   * permutation of 0..n-1 with cycle walking (Black and Rogaway, CT-RSA 2002) on two halves
+   * of h = ceil(ceil(log2 n) / 2) bits; round r maps (L, R) to (R, L xor F) with F the low h
+   * bits of word 0 of the Philox4x32-10 block of counter (R, 4 e + r, i, 3) and the same
+   * key; the network is applied again while the value is >= n.                          */
+  int32_t sampling, reserved2;
 } olsgd_hparams;
 
 /* Worker i's data set D_i (Eq. 1).  Device pointers, borrowed for the life of

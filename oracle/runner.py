@@ -11,7 +11,8 @@ from . import models, olsgd, sampling
 
 
 def run_model(kind, dims, X, y, x0, *, m, tau, batch, gamma, alpha, beta, mu, seed,
-              iters, bf16_operands=False, snapshots=(), local_sgd=False):
+              iters, bf16_operands=False, snapshots=(), local_sgd=False,
+              epoch_sampling=False):
     """Run `iters` iterations; returns (state, losses[iters][m], {k: state copy}).
 
     X [m][n][d_in], y [m][n]; worker i only ever touches X[i], y[i] (Eq. 1).
@@ -24,7 +25,8 @@ def run_model(kind, dims, X, y, x0, *, m, tau, batch, gamma, alpha, beta, mu, se
     g = np.zeros_like(st.x)
     snaps = {}
     for k in range(iters):
-        idx = sampling.minibatch_indices(seed, m, k, batch, n)
+        idx = (sampling.minibatch_indices_epoch(seed, m, k, batch, n) if epoch_sampling
+               else sampling.minibatch_indices(seed, m, k, batch, n))
         for i in range(m):
             Xb = X[i][idx[i]]
             yb = y[i][idx[i]]

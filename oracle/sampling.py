@@ -28,6 +28,7 @@ from .philox import philox4x32_10
 
 STREAM_MINIBATCH = 1
 STREAM_PARTITION = 2
+STREAM_EPOCH = 3
 N_CLASSES = 10
 
 
@@ -62,3 +63,51 @@ def class_pairs(seed, m):
             perm[p], perm[q] = perm[q], perm[p]
         slots.extend(perm)
     return np.asarray(slots[:2 * m], dtype=np.int32).reshape(m, 2)
+
+
+# ---------------------------------------------------------------------------
+# Second sampling rule: one pass over D_i per epoch, without replacement.
+#
+# The paper's runs go through each node's partition epoch by epoch (Section 4: the data
+# "is evenly partitioned across all nodes and not shuffled" between nodes).  Reading: worker
+# i's draws are numbered t = k * B + j; draw t belongs to epoch e = t // n and takes sample
+# pi_{i,e}(t mod n), where pi_{i,e} is a permutation of 0..n-1 that is a pure function of
+# (seed, i, e), so no state is carried from step to step.
+#
+# pi is a balanced Feistel network with cycle walking (Black and Rogaway, "Ciphers with
+# arbitrary finite domains", CT-RSA 2002): with h = ceil(ceil(log2 n) / 2) the value is split
+# into two h-bit halves (L, R); four rounds (L, R) <- (R, L xor F_r(R)) permute 0..2^(2h)-1;
+# the network is applied again until the result is below n.  F_r(R) is the low h bits of word
+# 0 of the Philox4x32-10 block with counter (R, 4 * e + r, i, 3) and key (seed lo, seed hi).
+
+
+def _half_bits(n):
+    bits = max(1, int(n - 1).bit_length())
+    return (bits + 1) // 2
+
+
+def epoch_permutation(seed, i, e, o, n):
+    """pi_{i,e}(o) for 0 <= o < n, as a Python int."""
+    k0, k1 = _key(seed)
+    h = _half_bits(n)
+    mask = (1 << h) - 1
+    v = int(o)
+    while True:
+        left, right = v >> h, v & mask
+        for r in range(4):
+            f = int(philox4x32_10(right, (4 * int(e) + r) & 0xFFFFFFFF, i, STREAM_EPOCH,
+                                  k0, k1)[0]) & mask
+            left, right = right, left ^ f
+        v = (left << h) | right
+        if v < n:
+            return v
+
+
+def minibatch_indices_epoch(seed, m, k, batch, n, worker_offset=0):
+    """int32 [m][batch]: the epoch rule's indices of every worker at iteration k."""
+    out = np.empty((m, batch), dtype=np.int32)
+    for i in range(m):
+        for j in range(batch):
+            t = int(k) * batch + j
+            out[i, j] = epoch_permutation(seed, i + worker_offset, t // n, t % n, n)
+    return out

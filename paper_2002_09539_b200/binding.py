@@ -33,7 +33,8 @@ class _ModelSpec(C.Structure):
 class _HParams(C.Structure):
     _fields_ = [("m", C.c_int32), ("tau", C.c_int32), ("batch", C.c_int32), ("mode", C.c_int32),
                 ("gamma", C.c_float), ("alpha", C.c_float), ("beta", C.c_float), ("mu", C.c_float),
-                ("seed", C.c_uint64), ("worker_offset", C.c_int32), ("m_total", C.c_int32)]
+                ("seed", C.c_uint64), ("worker_offset", C.c_int32), ("m_total", C.c_int32),
+                ("sampling", C.c_int32), ("reserved2", C.c_int32)]
 
 
 class _Data(C.Structure):
@@ -137,12 +138,14 @@ class OverlapLocalSGD:
 
     def __init__(self, kind, *, m, tau, gamma, alpha, beta=0.0, mu=0.0, batch=1, seed=0,
                  dims=(), gemm_bf16=0, flat_P=0, x0, X=None, y=None, overlap=True,
-                 local_sgd=False, worker_offset=0, m_total=0, device="cuda"):
+                 local_sgd=False, worker_offset=0, m_total=0, epoch_sampling=False,
+                 device="cuda"):
         self.lib = load_library()
         self.device = torch.device(device)
         self.spec = _spec(kind, dims, gemm_bf16, flat_P)
         self.hp = _HParams(int(m), int(tau), int(batch), 1 if local_sgd else 0, float(gamma), float(alpha),
-                           float(beta), float(mu), int(seed), int(worker_offset), int(m_total))
+                           float(beta), float(mu), int(seed), int(worker_offset), int(m_total),
+                           1 if epoch_sampling else 0, 0)
         self.m, self.tau, self.batch, self.kind = int(m), int(tau), int(batch), kind
         P = C.c_int64()
         _check(self.lib, self.lib.olsgd_param_count(C.byref(self.spec), C.byref(P)))

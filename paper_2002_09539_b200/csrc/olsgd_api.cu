@@ -210,6 +210,8 @@ olsgd_status check_hp(const olsgd_hparams* hp) {
     return fail(nullptr, OLSGD_EINVAL, "worker_offset needs m_total");
   if (hp->m_total != 0 && hp->mode != OLSGD_MODE_OVERLAP)
     return fail(nullptr, OLSGD_EINVAL, "sharded contexts support OLSGD_MODE_OVERLAP only");
+  if (hp->sampling != 0 && hp->sampling != 1)
+    return fail(nullptr, OLSGD_EINVAL, "sampling must be 0 (with replacement) or 1 (epoch rule)");
   if (hp->mode != OLSGD_MODE_OVERLAP && hp->mode != OLSGD_MODE_LOCAL_SGD)
     return fail(nullptr, OLSGD_EINVAL, "mode must be OLSGD_MODE_OVERLAP or OLSGD_MODE_LOCAL_SGD");
   return OLSGD_OK;
@@ -321,6 +323,15 @@ olsgd_status apply_update(olsgd_ctx* c, const float* g, int64_t ldg) {
   c->k += 1;
   if (sync) c->need_sync = true;
   return OLSGD_OK;
+}
+
+// S1: the minibatch indices of iteration k into c->idx, by the context's sampling rule.
+cudaError_t draw_indices(olsgd_ctx* c, int64_t k) {
+  if (c->hp.sampling == 1)
+    return launch_minibatch_indices_epoch(c->idx, c->hp.seed, c->hp.m, k, c->hp.batch,
+                                          c->data.n_per_worker, c->hp.worker_offset, c->main);
+  return launch_minibatch_indices(c->idx, c->hp.seed, c->hp.m, k, c->hp.batch,
+                                  c->data.n_per_worker, c->hp.worker_offset, c->main);
 }
 
 // S2-S6 of one iteration on the main stream, reading the minibatch rows
@@ -529,8 +540,7 @@ olsgd_status olsgd_local_step(olsgd_ctx* c, float* loss_device) {
   // S1: minibatch indices xi_k^(i)
   {
     Launch l(c, OLSGD_KC_INDEX, c->main);
-    OLSGD_CUDA(c, launch_minibatch_indices(c->idx, c->hp.seed, c->hp.m, c->k, c->hp.batch,
-                                           c->data.n_per_worker, c->hp.worker_offset, c->main));
+    OLSGD_CUDA(c, draw_indices(c, c->k));
   }
   return step_body(c, c->data, c->idx, loss_device, -1);
 }
@@ -775,8 +785,7 @@ olsgd_status olsgd_get_indices(olsgd_ctx* c, int64_t k, int32_t* dst) {
   OLSGD_CUDA(c, cudaStreamSynchronize(c->main));
   {
     Launch l(c, OLSGD_KC_INDEX, c->main);
-    OLSGD_CUDA(c, launch_minibatch_indices(c->idx, c->hp.seed, c->hp.m, k, c->hp.batch,
-                                           c->data.n_per_worker, c->hp.worker_offset, c->main));
+    OLSGD_CUDA(c, draw_indices(c, k));
   }
   return copy_out(c, dst, c->idx, (size_t)c->hp.m * c->hp.batch * sizeof(int32_t));
 }

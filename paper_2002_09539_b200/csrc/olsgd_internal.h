@@ -66,6 +66,9 @@ cudaError_t launch_virtual_sequence(const float* x, const float* z, float* dst, 
 // global worker id, so a sharded run draws the same minibatches as an unsharded one)
 cudaError_t launch_minibatch_indices(int32_t* idx, uint64_t seed, int m, int64_t k, int batch,
                                      int64_t n, int worker_offset, cudaStream_t s);
+// The epoch rule (one pass over the worker's samples per epoch, Feistel permutation).
+cudaError_t launch_minibatch_indices_epoch(int32_t* idx, uint64_t seed, int m, int64_t k, int batch,
+                                           int64_t n, int worker_offset, cudaStream_t s);
 cudaError_t launch_class_pairs(int32_t* dst, uint64_t seed, int m, cudaStream_t s);
 // idx[i][j] = j: the "indices" of a minibatch that is already contiguous
 cudaError_t launch_identity_indices(int32_t* idx, int m, int batch, cudaStream_t s);

@@ -33,6 +33,7 @@ __device__ __forceinline__ U4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c
 
 constexpr uint32_t kStreamMinibatch = 1;
 constexpr uint32_t kStreamPartition = 2;
+constexpr uint32_t kStreamEpoch = 3;
 
 // One thread per Philox block: four consecutive slots of one worker.
 __global__ void minibatch_indices_kernel(int32_t* __restrict__ idx, uint32_t k0, uint32_t k1,
@@ -71,6 +72,36 @@ __global__ void class_pairs_kernel(int32_t* __restrict__ dst, uint32_t k0, uint3
   }
 }
 
+// Epoch rule, one thread per slot: draw t = k * batch + j belongs to epoch e = t / n and takes
+// sample pi(t % n); pi is a four-round balanced Feistel network on two h-bit halves whose
+// round function is a Philox word, applied again while the result is >= n (cycle walking;
+// at most a handful of passes since 2^(2h) < 4 n).
+__global__ void minibatch_indices_epoch_kernel(int32_t* __restrict__ idx, uint32_t k0, uint32_t k1,
+                                               int m, uint64_t k, int batch, uint32_t n, int h,
+                                               uint32_t worker_offset) {
+  const int t_id = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t_id >= m * batch) return;
+  const int i = t_id / batch, j = t_id % batch;
+  const uint64_t t = k * (uint64_t)batch + (uint64_t)j;
+  const uint32_t e = (uint32_t)(t / n);
+  uint32_t v = (uint32_t)(t % n);
+  const uint32_t mask = (1u << h) - 1u;
+  for (int walk = 0; walk < 64; ++walk) {       // bounded; a valid value appears long before
+    uint32_t left = v >> h, right = v & mask;
+#pragma unroll
+    for (uint32_t r = 0; r < 4; ++r) {
+      const U4 w = philox4x32_10(right, 4u * e + r, (uint32_t)i + worker_offset, kStreamEpoch, k0, k1);
+      const uint32_t f = w.w[0] & mask;
+      const uint32_t nl = right;
+      right = left ^ f;
+      left = nl;
+    }
+    v = (left << h) | right;
+    if (v < n) break;
+  }
+  idx[t_id] = (int32_t)v;
+}
+
 __global__ void identity_indices_kernel(int32_t* __restrict__ idx, int total, int batch) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t < total) idx[t] = t % batch;
@@ -91,6 +122,18 @@ cudaError_t launch_minibatch_indices(int32_t* idx, uint64_t seed, int m, int64_t
   minibatch_indices_kernel<<<(total + threads - 1) / threads, threads, 0, s>>>(
       idx, (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), m, (uint32_t)k, batch,
       (uint32_t)n, (uint32_t)worker_offset);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_minibatch_indices_epoch(int32_t* idx, uint64_t seed, int m, int64_t k, int batch,
+                                           int64_t n, int worker_offset, cudaStream_t s) {
+  int bits = 1;
+  while (((int64_t)1 << bits) < n) ++bits;       // ceil(log2 n), at least 1
+  const int h = (bits + 1) / 2;
+  const int total = m * batch, threads = 128;
+  minibatch_indices_epoch_kernel<<<(total + threads - 1) / threads, threads, 0, s>>>(
+      idx, (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), m, (uint64_t)k, batch,
+      (uint32_t)n, h, (uint32_t)worker_offset);
   return cudaGetLastError();
 }
 

@@ -206,3 +206,21 @@ def test_consensus_distance_matches_the_state():
     x, z, _ = opt.state()
     want = float(((x.astype(np.float64) - z.astype(np.float64)) ** 2).sum())
     assert abs(opt.consensus_distance() - want) <= 1e-12 * want
+
+
+def test_epoch_sampling_rule_end_to_end():
+    # the second minibatch rule (one pass per epoch, no replacement) through a whole run
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    m, n, d, C, batch, tau, iters = 3, 40, 36, 5, 16, 2, 7      # 2.5 iterations per epoch
+    rng = np.random.default_rng(13)
+    X = rng.standard_normal((m, n, d)).astype(np.float32)
+    y = rng.integers(0, C, size=(m, n)).astype(np.int32)
+    x0 = (0.1 * rng.standard_normal(d * C + C)).astype(np.float32)
+    kw = dict(m=m, tau=tau, batch=batch, gamma=0.05, alpha=0.5, beta=0.7, mu=0.9, seed=13)
+    st, lo, _ = runner.run_model("softmax", [d, C], X, y, x0, iters=iters, epoch_sampling=True, **kw)
+    opt = OverlapLocalSGD("softmax", dims=[d, C], x0=x0, X=to_dev(X), y=to_dev(y),
+                          epoch_sampling=True, **kw)
+    loss = torch.zeros((iters, m), device="cuda")
+    opt.run(iters, loss)
+    assert state_err(opt, st) <= TOL_FP32
+    assert np.abs(loss.cpu().numpy() - lo).max() <= 2e-5 * np.abs(lo).max()

@@ -49,3 +49,19 @@ def test_class_pairs_bit_exact(seed, m):
     got_host = class_pairs(seed, m, device="cpu").numpy()
     assert np.array_equal(got_dev, want)
     assert np.array_equal(got_host, want)
+
+
+@pytest.mark.parametrize("seed,m,batch,n,offset", [(0, 4, 32, 1000, 0), (7, 3, 13, 17, 0),
+                                                   (2**40 + 3, 2, 64, 5000, 6), (1, 2, 8, 1, 0),
+                                                   (5, 2, 16, 1024, 0)])
+def test_epoch_rule_indices_bit_exact(seed, m, batch, n, offset):
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    d = 8
+    X = torch.zeros((m, n, d), device="cuda")
+    y = torch.zeros((m, n), device="cuda")
+    opt = OverlapLocalSGD("linreg", m=m, tau=2, gamma=0.1, alpha=0.5, batch=batch, seed=seed,
+                          dims=[d], x0=np.zeros(d, np.float32), X=X, y=y, epoch_sampling=True,
+                          worker_offset=offset, m_total=offset + m)
+    for k in (0, 1, 2, n // batch, 3 * n + 1, 12345):
+        want = sampling.minibatch_indices_epoch(seed, m, k, batch, n, worker_offset=offset)
+        assert np.array_equal(opt.get_indices(k), want), k

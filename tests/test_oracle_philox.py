@@ -109,3 +109,64 @@ def test_class_pairs_shuffle_is_uniform():
     chi2 = ((counts - 300.0) ** 2 / 300.0).sum()
     # 81 degrees of freedom, sd ~12.7
     assert chi2 < 160, chi2
+
+
+# ------------------------------------------------------------ epoch rule
+
+def test_epoch_permutation_is_a_bijection_for_awkward_sizes():
+    for n in (1, 2, 3, 5, 16, 17, 100, 1000, 1024, 1025):
+        for seed, i, e in ((0, 0, 0), (9, 3, 7)):
+            vals = [sampling.epoch_permutation(seed, i, e, o, n) for o in range(n)]
+            assert sorted(vals) == list(range(n)), (n, seed, i, e)
+
+
+def test_epoch_permutation_inverts_round_by_round():
+    # structural pin: undo the four Feistel rounds (and the cycle walk) with the inverse
+    # network written here; a wrong half swap or round index would not invert
+    n, seed, i, e = 777, 5, 2, 3
+    k0, k1 = seed & 0xFFFFFFFF, seed >> 32
+    h = ((n - 1).bit_length() + 1) // 2
+    mask = (1 << h) - 1
+
+    def inverse(v):
+        while True:
+            left, right = v >> h, v & mask
+            for r in (3, 2, 1, 0):
+                f = int(philox.philox4x32_10(left, 4 * e + r, i, 3, k0, k1)[0]) & mask
+                left, right = right ^ f, left
+            v = (left << h) | right
+            if v < n:
+                return v
+
+    for o in range(0, n, 7):
+        assert inverse(sampling.epoch_permutation(seed, i, e, o, n)) == o
+
+
+def test_epoch_rule_visits_every_sample_once_per_epoch():
+    seed, m, B, n = 4, 3, 8, 40               # 5 iterations per epoch
+    seen = np.concatenate([sampling.minibatch_indices_epoch(seed, m, k, B, n) for k in range(5)], axis=1)
+    for i in range(m):
+        assert sorted(seen[i]) == list(range(n))
+    nxt = np.concatenate([sampling.minibatch_indices_epoch(seed, m, k, B, n) for k in range(5, 10)], axis=1)
+    for i in range(m):
+        assert sorted(nxt[i]) == list(range(n)) and not np.array_equal(nxt[i], seen[i])
+    assert not np.array_equal(seen[0], seen[1])
+
+
+def test_epoch_rule_straddles_epochs_and_respects_worker_offset():
+    seed, B, n = 6, 16, 40                    # iteration 2 takes draws 32..47: epochs 0 and 1
+    a = sampling.minibatch_indices_epoch(seed, 4, 2, B, n)
+    for j in range(B):
+        t = 2 * B + j
+        assert a[1, j] == sampling.epoch_permutation(seed, 1, t // n, t % n, n)
+    b = sampling.minibatch_indices_epoch(seed, 2, 2, B, n, worker_offset=2)
+    assert np.array_equal(b, a[2:])
+
+
+def test_epoch_permutation_first_position_is_uniform():
+    n = 20
+    counts = np.zeros(n)
+    for seed in range(2000):
+        counts[sampling.epoch_permutation(seed, 0, 0, 0, n)] += 1
+    chi2 = ((counts - 100.0) ** 2 / 100.0).sum()
+    assert chi2 < 60, chi2                      # 19 degrees of freedom
