@@ -190,6 +190,9 @@ def run_ours(args, rank, world):
         build()
     if world > 1:
         dist.barrier()
+    # everything below runs on one real stream (the library's main stream, the timing events,
+    # torch's copies): olsgd_run can only capture its CUDA graph on a non-default stream
+    torch.cuda.set_stream(torch.cuda.Stream())
 
     name = args.workload
     c = dict(si.CONFIGS[name])
@@ -233,6 +236,7 @@ def run_ours(args, rank, world):
     launches0 = opt.launch_count
     ms = timed(lambda: opt.run(K))
     launches = opt.launch_count - launches0
+    replays = opt.graph_replays
     clocks = sampler.stop() if rank == 0 else None
     value = world * m * K / (ms * 1e-3)
 
@@ -311,6 +315,7 @@ def run_ours(args, rank, world):
                              % (resident / 1e6),
                        "replicas": world},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+            "graph_replays": int(replays),
             "roofline": roofline, "cpu_baseline": cpu,
         }
     opt.close()

@@ -208,6 +208,14 @@ int64_t olsgd_row_floats(const olsgd_ctx* ctx);
  *   loss_device  n_iters * m floats ([iteration][worker]), device; or NULL  */
 olsgd_status olsgd_run(olsgd_ctx* ctx, int64_t n_iters, float* loss_device);
 
+/* How often olsgd_run has replayed its captured CUDA graph on this context so far.  Long
+ * runs (at least three blocks of max(8, 2 tau)-odd iterations) are executed as replays of
+ * one captured block; the iteration number the minibatch rule needs is then read from
+ * device memory.  Capturing needs main_stream to be a real stream: with the legacy default
+ * stream (NULL) olsgd_run keeps launching kernel by kernel and this stays 0.  The results
+ * are the same bits either way.                                                        */
+int64_t olsgd_graph_replays(const olsgd_ctx* ctx);
+
 /* Copy one vector of the state to the caller.  Joins both streams (blocks
  * the host).  which: 0..m-1 worker model x^(i); -1 anchor z; -2 anchor
  * momentum v; -3 virtual sequence y = (1-alpha) mean_i x^(i) + alpha z

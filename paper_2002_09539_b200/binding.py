@@ -81,6 +81,7 @@ def load_library():
         "olsgd_class_pairs_noalloc": (i32, [u64, i32, vp, vp]),
         "olsgd_iteration": (i64, [vp]),
         "olsgd_launch_count": (i64, [vp]),
+        "olsgd_graph_replays": (i64, [vp]),
         "olsgd_profile_enable": (i32, [vp, i32]),
         "olsgd_profile_read": (i32, [vp, C.POINTER(i64), C.POINTER(C.c_double), i32]),
         "olsgd_last_error": (C.c_char_p, [vp]),
@@ -266,6 +267,10 @@ class OverlapLocalSGD:
     @property
     def launch_count(self):
         return self.lib.olsgd_launch_count(self.ctx)
+
+    @property
+    def graph_replays(self):
+        return self.lib.olsgd_graph_replays(self.ctx)
 
     def profile_enable(self, on=True):
         _check(self.lib, self.lib.olsgd_profile_enable(self.ctx, 1 if on else 0), self.ctx)

@@ -44,6 +44,8 @@ struct olsgd_ctx {
   int32_t* idx = nullptr;            // [m][batch]
   int32_t* ident = nullptr;          // [m][batch], ident[i][j] = j
   int* dev_status = nullptr;         // one word: a kernel's bounded wait gave up
+  int64_t* dev_k = nullptr;          // iteration number read by the index kernel inside a graph
+  float* loss_ring = nullptr;        // [graph_block][m] losses of one replayed block
   float* stage_x[2] = {nullptr, nullptr};  // host-fed minibatches [m][batch][d_in]
   void* stage_y[2] = {nullptr, nullptr};   // [m][batch] targets / labels
   ModelBuffers mb;
@@ -57,6 +59,17 @@ struct olsgd_ctx {
   int reduce_reads = -1;        // which x buffer that refresh reads
   bool need_sync = false;       // a period ended; olsgd_period_sync is due
   bool sync_begun = false;      // olsgd_period_sync_begin ran; _finish is due
+
+  // olsgd_run replays a captured CUDA graph of `graph_block` iterations (a whole number of
+  // periods, an even number of steps so that the ping-pong buffers return to their places)
+  int graph_block = 0;
+  cudaGraphExec_t graph_exec = nullptr;
+  int graph_cur = -1;            // c->cur at capture time
+  bool graph_off = false;        // capture failed once: stay on the plain path
+  bool capturing = false;        // the index kernel reads k from dev_k
+  int64_t capture_k0 = 0;        // k at the start of the block being captured
+  int64_t graph_launches = 0;    // kernel launches of one block
+  int64_t graph_replays = 0;
 
   int64_t k = 0;
   int64_t launches = 0;
@@ -138,6 +151,7 @@ void free_host_side(olsgd_ctx* c) {
     if (c->stage_free[b]) cudaEventDestroy(c->stage_free[b]);
   }
   if (c->copy) cudaStreamDestroy(c->copy);
+  if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
   delete c;
 }
 
@@ -151,10 +165,18 @@ ProfHook make_hook(olsgd_ctx* c) {
   return hook;
 }
 
+// Iterations in one captured block: whole periods, an even count, at least eight steps.
+int graph_block_len(int tau) {
+  int periods = (8 + tau - 1) / tau;
+  if ((periods * tau) % 2) periods *= 2;
+  return periods * tau;
+}
+
 struct Plan {
   int64_t P = 0, ld = 0;
   size_t off_x0 = 0, off_x1 = 0, off_u = 0, off_g = 0, off_z = 0, off_v = 0, off_tmp = 0,
-         off_shadow = 0, off_idx = 0, off_ident = 0, off_status = 0, off_stage_x[2] = {0, 0},
+         off_shadow = 0, off_idx = 0, off_ident = 0, off_status = 0, off_dev_k = 0,
+         off_loss_ring = 0, off_stage_x[2] = {0, 0},
          off_stage_y[2] = {0, 0}, off_model = 0, total = 0;
   bool has_u = false, has_g = false, has_shadow = false;
   ModelPlan mp;
@@ -242,6 +264,8 @@ olsgd_status make_plan(const olsgd_model_spec* spec, const olsgd_hparams* hp, Pl
   pl->off_v = take(row);
   pl->off_tmp = take(row);
   pl->off_status = take(sizeof(int));
+  pl->off_dev_k = take(sizeof(int64_t));
+  pl->off_loss_ring = take((size_t)graph_block_len(hp->tau) * m * sizeof(float));
   pl->off_shadow = pl->has_shadow ? take((size_t)pl->ld * m * sizeof(__nv_bfloat16)) : 0;
   pl->off_idx = pl->has_g ? take((size_t)m * hp->batch * sizeof(int32_t)) : 0;
   if (pl->has_g) {
@@ -327,11 +351,16 @@ olsgd_status apply_update(olsgd_ctx* c, const float* g, int64_t ldg) {
 
 // S1: the minibatch indices of iteration k into c->idx, by the context's sampling rule.
 cudaError_t draw_indices(olsgd_ctx* c, int64_t k) {
+  // while a graph is being captured the kernel gets the offset inside the block and adds
+  // the block's first iteration from device memory, so that every replay draws new batches
+  const int64_t* k_ptr = c->capturing ? c->dev_k : nullptr;
+  if (c->capturing) k -= c->capture_k0;
   if (c->hp.sampling == 1)
     return launch_minibatch_indices_epoch(c->idx, c->hp.seed, c->hp.m, k, c->hp.batch,
-                                          c->data.n_per_worker, c->hp.worker_offset, c->main);
+                                          c->data.n_per_worker, c->hp.worker_offset, k_ptr,
+                                          c->main);
   return launch_minibatch_indices(c->idx, c->hp.seed, c->hp.m, k, c->hp.batch,
-                                  c->data.n_per_worker, c->hp.worker_offset, c->main);
+                                  c->data.n_per_worker, c->hp.worker_offset, k_ptr, c->main);
 }
 
 // S2-S6 of one iteration on the main stream, reading the minibatch rows
@@ -460,6 +489,9 @@ olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const ols
   c->v = reinterpret_cast<float*>(ws + pl.off_v);
   c->tmp = reinterpret_cast<float*>(ws + pl.off_tmp);
   c->dev_status = reinterpret_cast<int*>(ws + pl.off_status);
+  c->dev_k = reinterpret_cast<int64_t*>(ws + pl.off_dev_k);
+  c->loss_ring = reinterpret_cast<float*>(ws + pl.off_loss_ring);
+  c->graph_block = graph_block_len(hp->tau);
   c->shadow = pl.has_shadow ? reinterpret_cast<__nv_bfloat16*>(ws + pl.off_shadow) : nullptr;
   c->idx = pl.has_g ? reinterpret_cast<int32_t*>(ws + pl.off_idx) : nullptr;
   if (pl.has_g) {
@@ -680,18 +712,116 @@ olsgd_status olsgd_period_sync_finish(olsgd_ctx* c, const float* total_sum_devic
 
 int64_t olsgd_row_floats(const olsgd_ctx* c) { return c ? c->ld : -1; }
 
+// One iteration of olsgd_run: a local step and, when a period ends, the anchor refresh.
+static olsgd_status run_one(olsgd_ctx* c, float* loss) {
+  olsgd_status st = olsgd_local_step(c, loss);
+  if (st != OLSGD_OK) return st;
+  if (c->need_sync) st = olsgd_period_sync(c);
+  return st;
+}
+
+// Captures one block of iterations (starting at the current, period-aligned state) into a
+// graph.  The block ends with the side stream joined and with the device counter advanced,
+// so that replaying it continues the run.  On any failure the context falls back to plain
+// launches for good; the run itself is never affected because a capture executes nothing.
+static bool capture_block(olsgd_ctx* c) {
+  if (c->graph_exec) {
+    cudaGraphExecDestroy(c->graph_exec);
+    c->graph_exec = nullptr;
+  }
+  const int64_t k0 = c->k, launches0 = c->launches;
+  const int cur0 = c->cur;
+  cudaGraph_t graph = nullptr;
+  if (cudaStreamBeginCapture(c->main, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    cudaGetLastError();
+    c->graph_off = true;
+    return false;
+  }
+  c->capturing = true;
+  c->capture_k0 = k0;
+  bool ok = true;
+  for (int j = 0; j < c->graph_block && ok; ++j)
+    ok = run_one(c, c->loss_ring + (int64_t)j * c->hp.m) == OLSGD_OK;
+  if (ok && c->reduce_pending) {
+    ok = cudaStreamWaitEvent(c->main, c->reduce_done, 0) == cudaSuccess;
+    c->reduce_pending = false;
+  }
+  if (ok) ok = launch_counter(c->dev_k, 0, c->graph_block, false, c->main) == cudaSuccess;
+  c->capturing = false;
+  const cudaError_t e = cudaStreamEndCapture(c->main, &graph);
+  // nothing ran: put the host-side state back to the start of the block
+  c->graph_launches = c->launches - launches0 + 1;
+  c->launches = launches0;
+  c->k = k0;
+  c->cur = cur0;
+  c->need_sync = false;
+  c->reduce_pending = false;
+  if (!ok || e != cudaSuccess || !graph) {
+    if (graph) cudaGraphDestroy(graph);
+    cudaGetLastError();
+    c->graph_off = true;
+    return false;
+  }
+  const cudaError_t ie = cudaGraphInstantiate(&c->graph_exec, graph, 0);
+  cudaGraphDestroy(graph);
+  if (ie != cudaSuccess) {
+    cudaGetLastError();
+    c->graph_exec = nullptr;
+    c->graph_off = true;
+    return false;
+  }
+  c->graph_cur = cur0;
+  return true;
+}
+
 olsgd_status olsgd_run(olsgd_ctx* c, int64_t n_iters, float* loss_device) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
   if (n_iters < 0) return fail(c, OLSGD_EINVAL, "n_iters must be >= 0");
-  for (int64_t t = 0; t < n_iters; ++t) {
-    olsgd_status st = olsgd_local_step(c, loss_device ? loss_device + t * c->hp.m : nullptr);
-    if (st != OLSGD_OK) return st;
-    if (c->need_sync) {
-      st = olsgd_period_sync(c);
+  if (c->spec.kind == OLSGD_FLAT)
+    return fail(c, OLSGD_ESTATE, "OLSGD_FLAT contexts take olsgd_local_step_with_grads");
+  int64_t t = 0;
+  auto plain = [&](int64_t count) -> olsgd_status {
+    for (int64_t j = 0; j < count; ++j, ++t) {
+      olsgd_status st = run_one(c, loss_device ? loss_device + t * c->hp.m : nullptr);
       if (st != OLSGD_OK) return st;
     }
+    return OLSGD_OK;
+  };
+  const int block = c->graph_block;
+  // the legacy default stream cannot be captured
+  const bool real_stream = c->main != nullptr && c->main != cudaStreamLegacy &&
+                           c->main != cudaStreamPerThread;
+  const bool want_graph = real_stream && !c->graph_off && !c->prof && block > 0 &&
+                          n_iters >= 3 * (int64_t)block;
+  if (!want_graph) return plain(n_iters);
+  // reach a period boundary, then run one block with plain launches (this also performs every
+  // one-time kernel attribute set-up, which must not happen inside a capture)
+  olsgd_status st = OLSGD_OK;
+  while (c->k % c->hp.tau != 0 && t < n_iters)
+    if ((st = plain(1)) != OLSGD_OK) return st;
+  if (n_iters - t < 2 * (int64_t)block) return plain(n_iters - t);
+  if ((st = plain(block)) != OLSGD_OK) return st;
+  if (c->reduce_pending) {
+    OLSGD_CUDA(c, cudaStreamWaitEvent(c->main, c->reduce_done, 0));
+    c->reduce_pending = false;
   }
-  return OLSGD_OK;
+  if ((!c->graph_exec || c->graph_cur != c->cur) && !capture_block(c)) return plain(n_iters - t);
+  {
+    Launch l(c, OLSGD_KC_INDEX, c->main);
+    OLSGD_CUDA(c, launch_counter(c->dev_k, c->k, 0, true, c->main));
+  }
+  while (n_iters - t >= block) {
+    OLSGD_CUDA(c, cudaGraphLaunch(c->graph_exec, c->main));
+    if (loss_device)
+      OLSGD_CUDA(c, cudaMemcpyAsync(loss_device + t * c->hp.m, c->loss_ring,
+                                    (size_t)block * c->hp.m * sizeof(float),
+                                    cudaMemcpyDeviceToDevice, c->main));
+    c->k += block;
+    c->graph_replays += 1;
+    c->launches += c->graph_launches;
+    t += block;
+  }
+  return plain(n_iters - t);
 }
 
 olsgd_status olsgd_get_params(olsgd_ctx* c, int32_t which, float* dst, size_t n_floats) {
@@ -819,6 +949,7 @@ olsgd_status olsgd_class_pairs(uint64_t seed, int32_t m, int32_t* dst, void* str
 
 int64_t olsgd_iteration(const olsgd_ctx* c) { return c ? c->k : -1; }
 int64_t olsgd_launch_count(const olsgd_ctx* c) { return c ? c->launches : -1; }
+int64_t olsgd_graph_replays(const olsgd_ctx* c) { return c ? c->graph_replays : -1; }
 
 olsgd_status olsgd_profile_enable(olsgd_ctx* c, int32_t on) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");

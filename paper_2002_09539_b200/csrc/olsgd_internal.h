@@ -64,11 +64,16 @@ cudaError_t launch_virtual_sequence(const float* x, const float* z, float* dst, 
 // ---- sampling_kernels.cu ----------------------------------------------------
 // worker_offset: global id of this context's first worker (the rule is a function of the
 // global worker id, so a sharded run draws the same minibatches as an unsharded one)
+// k_ptr: if non-null the iteration number is k + *k_ptr, read on the device (captured graphs)
 cudaError_t launch_minibatch_indices(int32_t* idx, uint64_t seed, int m, int64_t k, int batch,
-                                     int64_t n, int worker_offset, cudaStream_t s);
+                                     int64_t n, int worker_offset, const int64_t* k_ptr,
+                                     cudaStream_t s);
+// *p = value (set) or *p += by
+cudaError_t launch_counter(int64_t* p, int64_t value, int64_t by, bool set, cudaStream_t s);
 // The epoch rule (one pass over the worker's samples per epoch, Feistel permutation).
 cudaError_t launch_minibatch_indices_epoch(int32_t* idx, uint64_t seed, int m, int64_t k, int batch,
-                                           int64_t n, int worker_offset, cudaStream_t s);
+                                           int64_t n, int worker_offset, const int64_t* k_ptr,
+                                           cudaStream_t s);
 cudaError_t launch_class_pairs(int32_t* dst, uint64_t seed, int m, cudaStream_t s);
 // idx[i][j] = j: the "indices" of a minibatch that is already contiguous
 cudaError_t launch_identity_indices(int32_t* idx, int m, int batch, cudaStream_t s);

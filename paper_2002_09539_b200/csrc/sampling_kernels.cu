@@ -37,8 +37,10 @@ constexpr uint32_t kStreamEpoch = 3;
 
 // One thread per Philox block: four consecutive slots of one worker.
 __global__ void minibatch_indices_kernel(int32_t* __restrict__ idx, uint32_t k0, uint32_t k1,
-                                         int m, uint32_t k, int batch, uint32_t n,
-                                         uint32_t worker_offset) {
+                                         int m, uint64_t k_base, const long long* k_ptr,
+                                         int batch, uint32_t n, uint32_t worker_offset) {
+  // inside a captured graph the iteration number lives in device memory
+  const uint32_t k = (uint32_t)(k_base + (k_ptr ? (uint64_t)*k_ptr : 0ull));
   const int blocks_per_worker = (batch + 3) / 4;
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= m * blocks_per_worker) return;
@@ -77,8 +79,10 @@ __global__ void class_pairs_kernel(int32_t* __restrict__ dst, uint32_t k0, uint3
 // round function is a Philox word, applied again while the result is >= n (cycle walking;
 // at most a handful of passes since 2^(2h) < 4 n).
 __global__ void minibatch_indices_epoch_kernel(int32_t* __restrict__ idx, uint32_t k0, uint32_t k1,
-                                               int m, uint64_t k, int batch, uint32_t n, int h,
+                                               int m, uint64_t k_base, const long long* k_ptr,
+                                               int batch, uint32_t n, int h,
                                                uint32_t worker_offset) {
+  const uint64_t k = k_base + (k_ptr ? (uint64_t)*k_ptr : 0ull);
   const int t_id = blockIdx.x * blockDim.x + threadIdx.x;
   if (t_id >= m * batch) return;
   const int i = t_id / batch, j = t_id % batch;
@@ -102,6 +106,11 @@ __global__ void minibatch_indices_epoch_kernel(int32_t* __restrict__ idx, uint32
   idx[t_id] = (int32_t)v;
 }
 
+// The device-resident iteration counter of a captured graph: *p = value, or *p += by.
+__global__ void counter_kernel(long long* p, long long value, long long by, int set) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) *p = set ? value : *p + by;
+}
+
 __global__ void identity_indices_kernel(int32_t* __restrict__ idx, int total, int batch) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t < total) idx[t] = t % batch;
@@ -116,24 +125,32 @@ cudaError_t launch_identity_indices(int32_t* idx, int m, int batch, cudaStream_t
 }
 
 cudaError_t launch_minibatch_indices(int32_t* idx, uint64_t seed, int m, int64_t k, int batch,
-                                     int64_t n, int worker_offset, cudaStream_t s) {
+                                     int64_t n, int worker_offset, const int64_t* k_ptr,
+                                     cudaStream_t s) {
   const int total = m * ((batch + 3) / 4);
   const int threads = 128;
   minibatch_indices_kernel<<<(total + threads - 1) / threads, threads, 0, s>>>(
-      idx, (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), m, (uint32_t)k, batch,
-      (uint32_t)n, (uint32_t)worker_offset);
+      idx, (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), m, (uint64_t)k,
+      reinterpret_cast<const long long*>(k_ptr), batch, (uint32_t)n, (uint32_t)worker_offset);
   return cudaGetLastError();
 }
 
 cudaError_t launch_minibatch_indices_epoch(int32_t* idx, uint64_t seed, int m, int64_t k, int batch,
-                                           int64_t n, int worker_offset, cudaStream_t s) {
+                                           int64_t n, int worker_offset, const int64_t* k_ptr,
+                                           cudaStream_t s) {
   int bits = 1;
   while (((int64_t)1 << bits) < n) ++bits;       // ceil(log2 n), at least 1
   const int h = (bits + 1) / 2;
   const int total = m * batch, threads = 128;
   minibatch_indices_epoch_kernel<<<(total + threads - 1) / threads, threads, 0, s>>>(
-      idx, (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), m, (uint64_t)k, batch,
-      (uint32_t)n, h, (uint32_t)worker_offset);
+      idx, (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), m, (uint64_t)k,
+      reinterpret_cast<const long long*>(k_ptr), batch, (uint32_t)n, h, (uint32_t)worker_offset);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_counter(int64_t* p, int64_t value, int64_t by, bool set, cudaStream_t s) {
+  counter_kernel<<<1, 32, 0, s>>>(reinterpret_cast<long long*>(p), (long long)value, (long long)by,
+                                  set ? 1 : 0);
   return cudaGetLastError();
 }
 

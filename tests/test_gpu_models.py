@@ -224,3 +224,50 @@ def test_epoch_sampling_rule_end_to_end():
     opt.run(iters, loss)
     assert state_err(opt, st) <= TOL_FP32
     assert np.abs(loss.cpu().numpy() - lo).max() <= 2e-5 * np.abs(lo).max()
+
+
+@pytest.mark.parametrize("kind,dims,gemm,tau,epoch", [("softmax", [100, 7], 0, 2, False),
+                                                      ("mlp", [128, 256, 128, 10], 1, 3, False),
+                                                      ("linreg", [24], 0, 8, True)])
+def test_run_with_replayed_graph_equals_single_steps(kind, dims, gemm, tau, epoch):
+    # olsgd_run replays a captured block of iterations once the run is long enough; the
+    # result must be the bits of the call-by-call loop, losses included
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    m, n, batch = 3, 96, 64
+    if kind == "linreg":
+        X, y, _ = si.linreg_data(14, m, n, dims[0])
+        x0 = np.zeros(dims[0], np.float32)
+    else:
+        X, y = si.mixture_data(14, m, n, dims[0])
+        y = (y % dims[-1]).astype(np.int32)
+        x0 = (si.model_init(14, "mlp", dims) if kind == "mlp" else
+              (0.1 * np.random.default_rng(14).standard_normal(models.n_params(kind, dims))).astype(np.float32))
+    kw = dict(dims=dims, gemm_bf16=gemm, m=m, tau=tau, batch=batch, gamma=0.02, alpha=0.5, beta=0.7,
+              mu=0.9, seed=14, x0=x0, X=to_dev(X), y=to_dev(y), epoch_sampling=epoch)
+    block = -(-8 // tau) * tau
+    if block % 2:
+        block *= 2
+    iters = 4 * block + tau + 1
+    # a graph can only be captured on a real stream, not on the legacy default stream
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(stream):
+        a = OverlapLocalSGD(kind, **kw)
+        la = torch.zeros((iters, m), device="cuda")
+        a.run(1)                               # start off a period boundary on purpose
+        a.run(iters - 1, la[1:])
+        assert a.graph_replays >= 2
+        a.join()
+    torch.cuda.synchronize()
+    b = OverlapLocalSGD(kind, **kw)
+    lb = torch.zeros((iters, m), device="cuda")
+    for k in range(iters):
+        b.local_step(lb[k])
+        if (k + 1) % tau == 0:
+            b.period_sync()
+    xa, za, va = a.state()
+    xb, zb, vb = b.state()
+    assert a.iteration == b.iteration == iters
+    assert np.array_equal(xa, xb) and np.array_equal(za, zb) and np.array_equal(va, vb)
+    assert np.array_equal(la[1:].cpu().numpy(), lb[1:].cpu().numpy())
+    assert a.launch_count >= b.launch_count      # the replayed launches are counted too
