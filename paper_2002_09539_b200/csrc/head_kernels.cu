@@ -42,6 +42,15 @@ __device__ __forceinline__ int head_label(const HeadArgs& a, int i, int b) {
   return a.yb[(int64_t)i * a.batch + b];
 }
 
+// four adjacent inputs of a row (16-byte fp32 or 8-byte bf16 load)
+__device__ __forceinline__ float4 load4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
+  const uint2 w = *reinterpret_cast<const uint2*>(p);
+  const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&w.x);
+  const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&w.y);
+  return make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
+}
+
 constexpr int kHeadThreads = 128;
 
 // Forward, loss and input gradient of the output layer for R batch rows of one worker.
@@ -181,6 +190,165 @@ head_forward_kernel(HeadArgs a) {
   }
 }
 
+// The same kernel for K % 4 == 0: a thread owns FOUR adjacent input columns at a time
+// (k = 4 tid, 4 tid + 512, ...), so every load is 8 or 16 bytes and one sweep needs a quarter
+// of the load instructions.  Same reduction order over threads as above.
+template <typename InT, int CMAX, int R>
+__global__ void __launch_bounds__(kHeadThreads)
+head_forward_vec_kernel(HeadArgs a) {
+  extern __shared__ __align__(16) float head_smem[];
+  float* red = head_smem;                                  // [R * CMAX][kHeadThreads + 1]
+  float* lg = red + R * CMAX * (kHeadThreads + 1);         // [R][CMAX] logits, then dl
+  const int i = blockIdx.y, b0 = blockIdx.x * R;
+  const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
+  const int K = a.K, C = a.C, B = a.batch;
+  const float* W = a.x + (int64_t)i * a.ld + a.w_off;
+  const float* bias = a.x + (int64_t)i * a.ld + a.b_off;
+  const int rows = min(R, B - b0);
+  const InT* rowp[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r) rowp[r] = head_row<InT>(a, i, b0 + (r < rows ? r : 0));
+
+  float acc[R][CMAX];
+#pragma unroll
+  for (int r = 0; r < R; ++r)
+#pragma unroll
+    for (int c = 0; c < CMAX; ++c) acc[r][c] = 0.f;
+
+  for (int k = 4 * tid; k < K; k += 4 * kHeadThreads) {
+    float4 w[CMAX], xv[R];
+#pragma unroll
+    for (int c = 0; c < CMAX; ++c)
+      w[c] = (c < C) ? load4(W + (int64_t)c * K + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+      xv[r] = (r < rows) ? load4(rowp[r] + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+    if (a.round_w_bf16) {
+#pragma unroll
+      for (int c = 0; c < CMAX; ++c) {
+        w[c].x = bf16_round(w[c].x);
+        w[c].y = bf16_round(w[c].y);
+        w[c].z = bf16_round(w[c].z);
+        w[c].w = bf16_round(w[c].w);
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+      for (int c = 0; c < CMAX; ++c) {
+        acc[r][c] = fmaf(xv[r].x, w[c].x, acc[r][c]);
+        acc[r][c] = fmaf(xv[r].y, w[c].y, acc[r][c]);
+        acc[r][c] = fmaf(xv[r].z, w[c].z, acc[r][c]);
+        acc[r][c] = fmaf(xv[r].w, w[c].w, acc[r][c]);
+      }
+  }
+#pragma unroll
+  for (int r = 0; r < R; ++r)
+#pragma unroll
+    for (int c = 0; c < CMAX; ++c) red[(r * CMAX + c) * (kHeadThreads + 1) + tid] = acc[r][c];
+  __syncthreads();
+  for (int o = warp; o < R * CMAX; o += kHeadThreads / 32) {
+    const float* src = red + o * (kHeadThreads + 1);
+    float sum = 0.f;
+#pragma unroll
+    for (int t = 0; t < kHeadThreads / 32; ++t) sum += src[lane + 32 * t];
+    sum = warp_sum(sum);
+    if (lane == 0) lg[o] = sum;
+  }
+  __syncthreads();
+  for (int r = warp; r < R; r += kHeadThreads / 32) {
+    const int b = b0 + r;
+    const bool live = r < rows;
+    const float logit = (lane < C) ? lg[r * CMAX + lane] + bias[lane] : -INFINITY;
+    float mx = logit;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    const float e = (lane < C) ? expf(logit - mx) : 0.f;
+    const float lse = mx + logf(warp_sum(e));
+    const int label = live ? head_label(a, i, b) : 0;
+    const float picked = __shfl_sync(0xffffffffu, logit, label);
+    float dl = 0.f;
+    if (lane < C) dl = (expf(logit - lse) - (lane == label ? 1.f : 0.f)) / (float)B;
+    if (live && lane < C) a.dlogits[((int64_t)i * B + b) * C + lane] = dl;
+    if (live && lane == 0) a.rowloss[(int64_t)i * B + b] = lse - picked;
+    if (lane < CMAX) lg[r * CMAX + lane] = (live && lane < C) ? (a.round_w_bf16 ? bf16_round(dl) : dl) : 0.f;
+  }
+  if (!a.din32 && !a.din16 && !a.din16t) return;
+  __syncthreads();
+
+  // second sweep: dl is read from shared memory (a broadcast), four columns per read
+  const bool vec_t = (R == 8) && (B % 8 == 0) && rows == R;
+  for (int k = 4 * tid; k < K; k += 4 * kHeadThreads) {
+    float4 w[CMAX], xv[R], d[R];
+#pragma unroll
+    for (int c = 0; c < CMAX; ++c)
+      w[c] = (c < C) ? load4(W + (int64_t)c * K + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+      xv[r] = (r < rows) ? load4(rowp[r] + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+    if (a.round_w_bf16) {
+#pragma unroll
+      for (int c = 0; c < CMAX; ++c) {
+        w[c].x = bf16_round(w[c].x);
+        w[c].y = bf16_round(w[c].y);
+        w[c].z = bf16_round(w[c].z);
+        w[c].w = bf16_round(w[c].w);
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int c = 0; c < CMAX; ++c) {
+        const float dl = lg[r * CMAX + c];
+        v.x = fmaf(dl, w[c].x, v.x);
+        v.y = fmaf(dl, w[c].y, v.y);
+        v.z = fmaf(dl, w[c].z, v.z);
+        v.w = fmaf(dl, w[c].w, v.w);
+      }
+      d[r].x = (xv[r].x > 0.f) ? v.x : 0.f;
+      d[r].y = (xv[r].y > 0.f) ? v.y : 0.f;
+      d[r].z = (xv[r].z > 0.f) ? v.z : 0.f;
+      d[r].w = (xv[r].w > 0.f) ? v.w : 0.f;
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      if (r < rows) {
+        const int64_t o = ((int64_t)i * B + b0 + r) * K + k;
+        if (a.din32) *reinterpret_cast<float4*>(a.din32 + o) = d[r];
+        if (a.din16) {
+          const __nv_bfloat162 lo = __floats2bfloat162_rn(d[r].x, d[r].y);
+          const __nv_bfloat162 hi = __floats2bfloat162_rn(d[r].z, d[r].w);
+          *reinterpret_cast<uint2*>(a.din16 + o) = make_uint2(*reinterpret_cast<const uint32_t*>(&lo),
+                                                              *reinterpret_cast<const uint32_t*>(&hi));
+        }
+      }
+    }
+    if (a.din16t) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        __nv_bfloat16* dst = a.din16t + ((int64_t)i * K + k + q) * B + b0;
+        float dq[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) dq[r] = q == 0 ? d[r].x : q == 1 ? d[r].y : q == 2 ? d[r].z : d[r].w;
+        if (vec_t) {
+          uint32_t pk[4];
+#pragma unroll
+          for (int r = 0; r < 4; ++r) {
+            const __nv_bfloat162 p2 = __floats2bfloat162_rn(dq[(2 * r) % R], dq[(2 * r + 1) % R]);
+            pk[r] = *reinterpret_cast<const uint32_t*>(&p2);
+          }
+          *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        } else {
+#pragma unroll
+          for (int r = 0; r < R; ++r)
+            if (r < rows) dst[r] = __float2bfloat16_rn(dq[r]);
+        }
+      }
+    }
+  }
+}
+
 constexpr int kWgCols = 64;    // input columns per block
 constexpr int kWgSlices = 4;   // batch slices per block, combined in slice order
 constexpr int kWgRows = 64;    // dlogits rows staged at a time
@@ -263,13 +431,6 @@ head_wgrad_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ loss) {
 // 32 x 4 threads covers 128 columns with four batch slices.  Fixed order as above.
 constexpr int kWvCols = 32, kWvSlices = 4, kWvRows = 128, kWvFlight = 8;
 
-__device__ __forceinline__ float4 load4(const float* p) { return *reinterpret_cast<const float4*>(p); }
-__device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
-  const uint2 w = *reinterpret_cast<const uint2*>(p);
-  const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&w.x);
-  const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&w.y);
-  return make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
-}
 
 template <typename InT, int CMAX>
 __global__ void __launch_bounds__(kWvCols* kWvSlices)
@@ -362,12 +523,16 @@ head_wgrad_vec_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ los
 template <typename InT, int CMAX, int R>
 cudaError_t launch_fwd(const HeadArgs& a, cudaStream_t s) {
   const size_t smem = ((size_t)R * CMAX * (kHeadThreads + 1) + (size_t)R * CMAX) * sizeof(float);
-  auto kern = head_forward_kernel<InT, CMAX, R>;
-  static bool configured = false;
-  if (!configured) {
+  // four columns per thread where the rows are 16-byte aligned; with 32 classes the
+  // float4 weights would not fit the register file, so that case keeps one column per thread
+  constexpr int VC = CMAX <= 16 ? CMAX : 1;
+  const bool vec = CMAX <= 16 && a.K % 4 == 0 && a.w_off % 4 == 0 && a.ld % 4 == 0;
+  auto kern = vec ? head_forward_vec_kernel<InT, VC, R> : head_forward_kernel<InT, CMAX, R>;
+  static bool configured[2] = {false, false};
+  if (!configured[vec]) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    configured = true;
+    configured[vec] = true;
   }
   dim3 grid((a.batch + R - 1) / R, a.m), block(kHeadThreads);
   kern<<<grid, block, smem, s>>>(a);
