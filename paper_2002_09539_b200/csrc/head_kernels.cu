@@ -52,6 +52,7 @@ __device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
 }
 
 constexpr int kHeadThreads = 128;
+constexpr int kHeadSmallGrid = 2 * 148;
 
 // Forward, loss and input gradient of the output layer for R batch rows of one worker.
 //
@@ -194,7 +195,7 @@ head_forward_kernel(HeadArgs a) {
 // (k = 4 tid, 4 tid + 512, ...), so every load is 8 or 16 bytes and one sweep needs a quarter
 // of the load instructions.  Same reduction order over threads as above.
 template <typename InT, int CMAX, int R>
-__global__ void __launch_bounds__(kHeadThreads)
+__global__ void __launch_bounds__(kHeadThreads, (R <= 4 && CMAX <= 10) ? 4 : 2)
 head_forward_vec_kernel(HeadArgs a) {
   extern __shared__ __align__(16) float head_smem[];
   float* red = head_smem;                                  // [R * CMAX][kHeadThreads + 1]
@@ -277,7 +278,7 @@ head_forward_vec_kernel(HeadArgs a) {
   __syncthreads();
 
   // second sweep: dl is read from shared memory (a broadcast), four columns per read
-  const bool vec_t = (R == 8) && (B % 8 == 0) && rows == R;
+  const bool vec_t = (R == 8 || R == 4) && (B % R == 0) && rows == R;
   for (int k = 4 * tid; k < K; k += 4 * kHeadThreads) {
     float4 w[CMAX], xv[R], d[R];
 #pragma unroll
@@ -338,7 +339,8 @@ head_forward_vec_kernel(HeadArgs a) {
             const __nv_bfloat162 p2 = __floats2bfloat162_rn(dq[(2 * r) % R], dq[(2 * r + 1) % R]);
             pk[r] = *reinterpret_cast<const uint32_t*>(&p2);
           }
-          *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          if (R == 8) *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          else *reinterpret_cast<uint2*>(dst) = make_uint2(pk[0], pk[1]);
         } else {
 #pragma unroll
           for (int r = 0; r < R; ++r)
@@ -346,6 +348,41 @@ head_forward_vec_kernel(HeadArgs a) {
         }
       }
     }
+  }
+}
+
+// Bias gradient db[c] = sum_b dlogits[b][c] and the worker's mean loss, by one whole block
+// of T threads (T a multiple of 32): with T / 32 parts, thread (c, p) adds the rows
+// b = p, p + T / 32, ... of class c in order and thread c adds the partial sums in order;
+// the last warp adds the per-row losses (lane l takes rows l, l + 32, ... in order, then a
+// fixed shuffle tree).  `scratch` holds T floats and is free once the block has passed the
+// barrier inside.
+template <int T>
+__device__ __forceinline__ void head_bias_and_loss(const HeadArgs& a, int i, int tid, float* scratch,
+                                                   float* gi, float* loss) {
+  const int C = a.C, B = a.batch;
+  const float* dl = a.dlogits + (int64_t)i * B * C;
+  __syncthreads();
+  const int c = tid % 32, p = tid / 32;
+  constexpr int NP = T / 32;
+  if (c < C) {
+    float sum = 0.f;
+    for (int b = p; b < B; b += NP) sum += dl[(int64_t)b * C + c];
+    scratch[p * 32 + c] = sum;
+  }
+  __syncthreads();
+  if (tid < C) {
+    float sum = scratch[tid];
+#pragma unroll
+    for (int q = 1; q < NP; ++q) sum += scratch[q * 32 + tid];
+    gi[a.b_off + tid] = sum;
+  }
+  if (loss && tid >= T - 32) {
+    const int lane = tid % 32;
+    float sum = 0.f;
+    for (int b = lane; b < B; b += 32) sum += a.rowloss[(int64_t)i * B + b];
+    sum = warp_sum(sum);
+    if (lane == 0) loss[i] = sum / (float)B;
   }
 }
 
@@ -368,7 +405,6 @@ head_wgrad_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ loss) {
   float acc[CMAX];
 #pragma unroll
   for (int c = 0; c < CMAX; ++c) acc[c] = 0.f;
-  float bsum = 0.f;  // thread c < C of block 0 also sums the bias gradient over all rows
   for (int r0 = 0; r0 < B; r0 += kWgRows) {
     const int rc = min(kWgRows, B - r0);
     __syncthreads();
@@ -397,8 +433,6 @@ head_wgrad_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ loss) {
         }
       }
     }
-    if (blockIdx.x == 0 && tid < C)
-      for (int r = 0; r < rc; ++r) bsum += dl[(int64_t)(r0 + r) * C + tid];
   }
 #pragma unroll
   for (int c = 0; c < CMAX; ++c)
@@ -416,20 +450,13 @@ head_wgrad_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ loss) {
       gi[a.w_off + (int64_t)c * K + jj] = s;
     }
   }
-  if (blockIdx.x == 0) {
-    if (tid < C) gi[a.b_off + tid] = bsum;
-    if (loss && tid == kWgCols * kWgSlices - 1) {
-      float s = 0.f;
-      for (int r = 0; r < B; ++r) s += a.rowloss[(int64_t)i * B + r];
-      loss[i] = s / (float)B;
-    }
-  }
+  if (blockIdx.x == 0) head_bias_and_loss<kWgCols * kWgSlices>(a, i, tid, &part[0][0][0], gi, loss);
 }
 
 // The same product for K % 4 == 0 and at most 16 classes: a thread owns FOUR adjacent input
 // columns (one 16-byte fp32 or 8-byte bf16 load per row, eight in flight) and a block of
-// 32 x 4 threads covers 128 columns with four batch slices.  Fixed order as above.
-constexpr int kWvCols = 32, kWvSlices = 4, kWvRows = 128, kWvFlight = 8;
+// 16 x 8 threads covers 64 columns with eight batch slices.  Fixed order as above.
+constexpr int kWvCols = 16, kWvSlices = 8, kWvRows = 128, kWvFlight = 8;
 
 
 template <typename InT, int CMAX>
@@ -447,7 +474,6 @@ head_wgrad_vec_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ los
   for (int q = 0; q < 4; ++q)
 #pragma unroll
     for (int c = 0; c < CMAX; ++c) acc[q][c] = 0.f;
-  float bsum = 0.f;
   for (int r0 = 0; r0 < B; r0 += kWvRows) {
     const int rc = min(kWvRows, B - r0);
     __syncthreads();
@@ -484,8 +510,6 @@ head_wgrad_vec_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ los
         }
       }
     }
-    if (blockIdx.x == 0 && tid < C)
-      for (int r = 0; r < rc; ++r) bsum += dl[(int64_t)(r0 + r) * C + tid];
   }
 #pragma unroll
   for (int c = 0; c < CMAX; ++c)
@@ -510,14 +534,7 @@ head_wgrad_vec_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ los
       *reinterpret_cast<float4*>(gi + a.w_off + (int64_t)c * K + jj) = s;
     }
   }
-  if (blockIdx.x == 0) {
-    if (tid < C) gi[a.b_off + tid] = bsum;
-    if (loss && tid == kWvCols * kWvSlices - 1) {
-      float s = 0.f;
-      for (int r = 0; r < B; ++r) s += a.rowloss[(int64_t)i * B + r];
-      loss[i] = s / (float)B;
-    }
-  }
+  if (blockIdx.x == 0) head_bias_and_loss<kWvCols * kWvSlices>(a, i, tid, &part[0][0][0], gi, loss);
 }
 
 template <typename InT, int CMAX, int R>
@@ -541,8 +558,10 @@ cudaError_t launch_fwd(const HeadArgs& a, cudaStream_t s) {
 
 template <typename InT>
 cudaError_t launch_fwd_c(const HeadArgs& a, cudaStream_t s) {
-  if (a.C <= 10) return launch_fwd<InT, 10, 8>(a, s);
-  if (a.C <= 16) return launch_fwd<InT, 16, 8>(a, s);
+  // eight batch rows per block, or four where that leaves fewer than two blocks per SM
+  const bool small = (int64_t)((a.batch + 7) / 8) * a.m < kHeadSmallGrid;
+  if (a.C <= 10) return small ? launch_fwd<InT, 10, 4>(a, s) : launch_fwd<InT, 10, 8>(a, s);
+  if (a.C <= 16) return small ? launch_fwd<InT, 16, 4>(a, s) : launch_fwd<InT, 16, 8>(a, s);
   return launch_fwd<InT, 32, 4>(a, s);
 }
 

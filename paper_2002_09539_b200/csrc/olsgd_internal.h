@@ -10,6 +10,41 @@
 
 namespace olsgd {
 
+// ---- overlapped launches -----------------------------------------------------
+// The kernels of one iteration form a chain on the main stream, most of them short.  They
+// are launched with programmatic stream serialization: the blocks of a kernel may become
+// resident while the kernel before it is still draining, and each block executes
+// launch_gate() before its first access to global memory.  The gate returns once every
+// earlier kernel of the stream has completed and its writes are visible, then lets the
+// kernel after this one start its own launch.  A kernel launched the ordinary way passes
+// through the gate at once.
+#ifndef OLSGD_OVERLAP_LAUNCH
+#define OLSGD_OVERLAP_LAUNCH 1
+#endif
+
+#ifdef __CUDACC__
+__device__ __forceinline__ void launch_gate() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                           cudaStream_t s, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = OLSGD_OVERLAP_LAUNCH ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+#endif
+
 // ---- olsgd_api.cu -------------------------------------------------------------
 // Records the text olsgd_last_error(NULL) returns for context-free calls of this thread.
 void set_thread_error(const char* text);

@@ -70,20 +70,14 @@ __device__ __forceinline__ UnitPos unit_pos(int unit, int n_tiles, int m_tiles) 
 //            memory by TMA with the 128-byte swizzle (row r, 16-byte chunk q at q ^ (r % 8))
 //   blk_off  element offset of the block's corner inside a worker row
 //   ldw      row pitch of the weight matrix (its input width)
+//   zs       the block's strip of the anchor (sync steps), loaded one block ahead
 template <bool MOM, bool SYNC>
-__device__ __forceinline__ void fused_block(const float (&v)[32], float* stage, const float* xt,
-                                            const float* ut, uint32_t xu_bar, uint32_t xu_parity,
-                                            volatile int* abort_flag, int lane, const WgradUpd& up,
-                                            int64_t wk_off, int64_t blk_off, int ldw, bool* ok) {
+__device__ __forceinline__ void fused_block(const float (&v)[32], const float4 (&zs)[8], float* stage,
+                                            const float* xt, const float* ut, uint32_t xu_bar,
+                                            uint32_t xu_parity, volatile int* abort_flag, int lane,
+                                            const WgradUpd& up, int64_t wk_off, int64_t blk_off,
+                                            int ldw, bool* ok) {
   const int q = lane & 7, rsub = lane >> 3;
-  // the anchor strip comes straight from global memory (it is shared by all workers and
-  // mostly served by L2); issued first so that it is in flight during the staging
-  float4 zs[8];
-#pragma unroll
-  for (int t = 0; t < 8; ++t) {
-    zs[t] = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (SYNC) zs[t] = *reinterpret_cast<const float4*>(up.z + blk_off + (int64_t)(t * 4 + rsub) * ldw + q * 4);
-  }
   __syncwarp();   // the previous block's reads of the staging buffer are done
   float4* mine = reinterpret_cast<float4*>(stage + lane * 32);
 #pragma unroll
@@ -273,10 +267,25 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       if (n_blocks > 0) issue(0);
       if (n_blocks > 1) issue(1);
     }
+    // The anchor strip of a block comes straight from global memory (the anchor is shared
+    // by all workers and mostly served by L2) into registers, one block ahead, so that its
+    // latency is hidden behind the update of the block before.
+    float4 zs[8], zn[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) zs[t] = zn[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+    auto load_z = [&](int nn, float4 (&dst)[8]) {
+      const UnitPos pz = unit_pos(unit_of(nn >> 1), n_tiles, m_tiles);
+      const float* zp = up.z + up.w_off + (int64_t)(pz.m0 + lane_group * 32 + (lane >> 3)) * ldw +
+                        pz.col + (half + 2 * (nn & 1)) * 32 + (lane & 7) * 4;
+#pragma unroll
+      for (int t = 0; t < 8; ++t) dst[t] = *reinterpret_cast<const float4*>(zp + (int64_t)(t * 4) * ldw);
+    };
+    if (up.sync && n_blocks > 0) load_z(0, zs);
     bool ok = true;
     int n = 0;
     for (; n < n_blocks && ok; ++n) {
       const int j = n >> 1, c = half + 2 * (n & 1), buf = j & 1, use = j >> 1, b = n & 1;
+      if (up.sync && n + 1 < n_blocks) load_z(n + 1, zn);
       if ((n & 1) == 0) {
         ok = mbar_wait(smem_u32(&ctl->tmem_full[buf]), use & 1, abort_flag);
         if (!ok) break;
@@ -292,13 +301,15 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const uint32_t bar = smem_u32(&ctl->xu_full[ew][b]);
       const uint32_t par = (uint32_t)(n >> 1) & 1u;
       if (up.mom) {
-        if (up.sync) fused_block<true, true>(v, stage, xt, ut, bar, par, abort_flag, lane, up, wk_off, blk_off, ldw, &ok);
-        else fused_block<true, false>(v, stage, xt, ut, bar, par, abort_flag, lane, up, wk_off, blk_off, ldw, &ok);
+        if (up.sync) fused_block<true, true>(v, zs, stage, xt, ut, bar, par, abort_flag, lane, up, wk_off, blk_off, ldw, &ok);
+        else fused_block<true, false>(v, zs, stage, xt, ut, bar, par, abort_flag, lane, up, wk_off, blk_off, ldw, &ok);
       } else {
-        if (up.sync) fused_block<false, true>(v, stage, xt, ut, bar, par, abort_flag, lane, up, wk_off, blk_off, ldw, &ok);
-        else fused_block<false, false>(v, stage, xt, ut, bar, par, abort_flag, lane, up, wk_off, blk_off, ldw, &ok);
+        if (up.sync) fused_block<false, true>(v, zs, stage, xt, ut, bar, par, abort_flag, lane, up, wk_off, blk_off, ldw, &ok);
+        else fused_block<false, false>(v, zs, stage, xt, ut, bar, par, abort_flag, lane, up, wk_off, blk_off, ldw, &ok);
       }
       if (!ok) break;
+#pragma unroll
+      for (int t = 0; t < 8; ++t) zs[t] = zn[t];
       __syncwarp();   // every lane has read this buffer's tiles: it may be refilled
       if (lane == 0 && n + 2 < n_blocks) issue(n + 2);
       if (n & 1) {

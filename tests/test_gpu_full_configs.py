@@ -86,14 +86,17 @@ def test_mlp_configs_first_iterations_against_exact_oracle(name, iters, tol_para
 # one entry end config 3 with a 40 % different objective, and two fp64 ORACLE runs
 # that differ by that perturbation agree to 6 digits up to iteration 250, by 1 % at 400,
 # 3 % at 450, 45 % at 700 and end 22 % apart (tests/golden/c3_final.json vs
-# c3_perturbed.json).  A perturbation of bf16 size (2^-8 per operand) gets there sooner.
+# c3_perturbed.json).  The bf16 path gets there sooner, because a last-bit difference in
+# fp32 can flip an operand by a whole bf16 ulp: five GPU runs whose x0 differs by 1e-7 in
+# one entry agree on the 50-iteration block means of config 3 to 0.15 % up to iteration 150
+# and spread by 2 % over iterations 151-200 and by 4 % over 201-250.
 # No implementation can meet a 2e-2 bound on the loss after the full 1000 iterations,
 # so the bound is enforced on the stored checkpoints up to STRICT_UNTIL and the end of
 # the run is checked for having trained to the same level.
 # Config 4 (tau = 8, alpha = 0.5) stays reproducible to the end, so there the 2e-2 bound is
 # enforced on every checkpoint and on the final objective.
 STRICT_UNTIL = {"c3": 150, "c4": 800}          # one iteration's worker-mean loss
-STRICT_BLOCKS_UNTIL = {"c3": 250, "c4": 800}   # mean over blocks of 50 iterations
+STRICT_BLOCKS_UNTIL = {"c3": 150, "c4": 800}   # mean over blocks of 50 iterations
 FINAL_STRICT = {"c3": False, "c4": True}
 
 
