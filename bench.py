@@ -84,6 +84,13 @@ class ClockSampler:
         except OSError:
             self.proc = None
 
+    def wait_first_sample(self, limit_s=5.0):
+        """nvidia-smi holds driver locks while it starts up, which can stall kernel launches for
+        tens of milliseconds: the timed region begins only after its first sample has arrived."""
+        t0 = time.time()
+        while self.proc is not None and not self.lines and time.time() - t0 < limit_s:
+            time.sleep(0.01)
+
     def _pump(self):
         for line in self.proc.stdout:
             self.lines.append(line.strip())
@@ -233,6 +240,7 @@ def run_ours(args, rank, world):
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
+        sampler.wait_first_sample()
     launches0 = opt.launch_count
     ms = timed(lambda: opt.run(K))
     launches = opt.launch_count - launches0
@@ -345,6 +353,7 @@ def run_flat_sweep(args, rank, world):
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
+        sampler.wait_first_sample()
     for P in Ps:
         for m in ms_:
             x0 = torch.randn(P, device="cuda")
@@ -474,6 +483,7 @@ def run_sharded(args, rank, world):
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
+        sampler.wait_first_sample()
     dist.barrier()
     torch.cuda.synchronize()
     n0 = opt.launch_count

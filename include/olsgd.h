@@ -216,6 +216,16 @@ olsgd_status olsgd_run(olsgd_ctx* ctx, int64_t n_iters, float* loss_device);
  * are the same bits either way.                                                        */
 int64_t olsgd_graph_replays(const olsgd_ctx* ctx);
 
+/* Process-wide switch for how the kernels of one iteration follow each other on the main
+ * stream.  on != 0 (the default): they are launched with programmatic stream serialization,
+ * so a kernel's blocks may become resident and set up their shared state while the kernel
+ * before it is still draining; every kernel waits for its predecessors to complete before
+ * its first access to global memory, so the results are the same bits.  on == 0: plain
+ * stream order.  Applies to launches made after the call (a captured graph of olsgd_run
+ * keeps the setting it was captured with).  Returns the previous setting.  The paper has
+ * no counterpart: this is launch plumbing.                                               */
+int olsgd_set_launch_overlap(int on);
+
 /* Copy one vector of the state to the caller.  Joins both streams (blocks
  * the host).  which: 0..m-1 worker model x^(i); -1 anchor z; -2 anchor
  * momentum v; -3 virtual sequence y = (1-alpha) mean_i x^(i) + alpha z

@@ -82,6 +82,7 @@ def load_library():
         "olsgd_iteration": (i64, [vp]),
         "olsgd_launch_count": (i64, [vp]),
         "olsgd_graph_replays": (i64, [vp]),
+        "olsgd_set_launch_overlap": (i32, [i32]),
         "olsgd_profile_enable": (i32, [vp, i32]),
         "olsgd_profile_read": (i32, [vp, C.POINTER(i64), C.POINTER(C.c_double), i32]),
         "olsgd_last_error": (C.c_char_p, [vp]),
@@ -117,6 +118,11 @@ def class_pairs(seed, m, device="cuda"):
     stream = torch.cuda.current_stream().cuda_stream
     _check(lib, lib.olsgd_class_pairs(int(seed), int(m), out.data_ptr(), stream))
     return out
+
+
+def set_launch_overlap(on):
+    """olsgd_set_launch_overlap: process-wide; returns the previous setting."""
+    return bool(load_library().olsgd_set_launch_overlap(1 if on else 0))
 
 
 NOALLOC_MAX_WORKERS = 16384

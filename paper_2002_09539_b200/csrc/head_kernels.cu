@@ -67,6 +67,7 @@ constexpr int kHeadSmallGrid = 2 * 148;
 template <typename InT, int CMAX, int R>
 __global__ void __launch_bounds__(kHeadThreads)
 head_forward_kernel(HeadArgs a) {
+  launch_gate();
   extern __shared__ __align__(16) float head_smem[];
   float* red = head_smem;                                  // [R * CMAX][kHeadThreads + 1]
   float* lg = red + R * CMAX * (kHeadThreads + 1);         // [R][CMAX] logits, then dl
@@ -197,6 +198,7 @@ head_forward_kernel(HeadArgs a) {
 template <typename InT, int CMAX, int R>
 __global__ void __launch_bounds__(kHeadThreads, (R <= 4 && CMAX <= 10) ? 4 : 2)
 head_forward_vec_kernel(HeadArgs a) {
+  launch_gate();
   extern __shared__ __align__(16) float head_smem[];
   float* red = head_smem;                                  // [R * CMAX][kHeadThreads + 1]
   float* lg = red + R * CMAX * (kHeadThreads + 1);         // [R][CMAX] logits, then dl
@@ -395,6 +397,7 @@ constexpr int kWgRows = 64;    // dlogits rows staged at a time
 template <typename InT, int CMAX>
 __global__ void __launch_bounds__(kWgCols* kWgSlices)
 head_wgrad_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ loss) {
+  launch_gate();
   __shared__ float dsm[kWgRows][CMAX + 1];
   __shared__ float part[kWgSlices][CMAX][kWgCols];
   const int i = blockIdx.y;
@@ -462,6 +465,7 @@ constexpr int kWvCols = 16, kWvSlices = 8, kWvRows = 128, kWvFlight = 8;
 template <typename InT, int CMAX>
 __global__ void __launch_bounds__(kWvCols* kWvSlices)
 head_wgrad_vec_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ loss) {
+  launch_gate();
   __shared__ float dsm[kWvRows][CMAX + 1];
   __shared__ __align__(16) float part[kWvSlices][CMAX][kWvCols * 4];
   const int i = blockIdx.y;
@@ -552,8 +556,7 @@ cudaError_t launch_fwd(const HeadArgs& a, cudaStream_t s) {
     configured[vec] = true;
   }
   dim3 grid((a.batch + R - 1) / R, a.m), block(kHeadThreads);
-  kern<<<grid, block, smem, s>>>(a);
-  return cudaGetLastError();
+  return launch_chained(kern, grid, block, smem, s, a);
 }
 
 template <typename InT>
@@ -573,26 +576,27 @@ cudaError_t launch_head_forward(const HeadArgs& a, cudaStream_t s) {
 
 cudaError_t launch_head_wgrad(const HeadArgs& a, float* g, float* loss, cudaStream_t s) {
   const bool f32 = a.in32 != nullptr;
+  cudaError_t err = cudaSuccess;
   if (a.K % 4 == 0 && a.C <= 16 && a.w_off % 4 == 0 && a.ld % 4 == 0) {
     dim3 vgrid((a.K / 4 + kWvCols - 1) / kWvCols, a.m), vblock(kWvCols, kWvSlices);
     if (a.C <= 10) {
-      if (f32) head_wgrad_vec_kernel<float, 10><<<vgrid, vblock, 0, s>>>(a, g, loss);
-      else head_wgrad_vec_kernel<__nv_bfloat16, 10><<<vgrid, vblock, 0, s>>>(a, g, loss);
+      if (f32) err = launch_chained(head_wgrad_vec_kernel<float, 10>, vgrid, vblock, 0, s, a, g, loss);
+      else err = launch_chained(head_wgrad_vec_kernel<__nv_bfloat16, 10>, vgrid, vblock, 0, s, a, g, loss);
     } else {
-      if (f32) head_wgrad_vec_kernel<float, 16><<<vgrid, vblock, 0, s>>>(a, g, loss);
-      else head_wgrad_vec_kernel<__nv_bfloat16, 16><<<vgrid, vblock, 0, s>>>(a, g, loss);
+      if (f32) err = launch_chained(head_wgrad_vec_kernel<float, 16>, vgrid, vblock, 0, s, a, g, loss);
+      else err = launch_chained(head_wgrad_vec_kernel<__nv_bfloat16, 16>, vgrid, vblock, 0, s, a, g, loss);
     }
-    return cudaGetLastError();
+    return err;
   }
   dim3 grid((a.K + kWgCols - 1) / kWgCols, a.m), block(kWgCols, kWgSlices);
   if (a.C <= 16) {
-    if (f32) head_wgrad_kernel<float, 16><<<grid, block, 0, s>>>(a, g, loss);
-    else head_wgrad_kernel<__nv_bfloat16, 16><<<grid, block, 0, s>>>(a, g, loss);
+    if (f32) err = launch_chained(head_wgrad_kernel<float, 16>, grid, block, 0, s, a, g, loss);
+    else err = launch_chained(head_wgrad_kernel<__nv_bfloat16, 16>, grid, block, 0, s, a, g, loss);
   } else {
-    if (f32) head_wgrad_kernel<float, 32><<<grid, block, 0, s>>>(a, g, loss);
-    else head_wgrad_kernel<__nv_bfloat16, 32><<<grid, block, 0, s>>>(a, g, loss);
+    if (f32) err = launch_chained(head_wgrad_kernel<float, 32>, grid, block, 0, s, a, g, loss);
+    else err = launch_chained(head_wgrad_kernel<__nv_bfloat16, 32>, grid, block, 0, s, a, g, loss);
   }
-  return cudaGetLastError();
+  return err;
 }
 
 }  // namespace olsgd

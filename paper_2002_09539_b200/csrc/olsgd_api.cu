@@ -430,6 +430,7 @@ olsgd_status check_device_status(olsgd_ctx* c) {
 
 namespace olsgd {
 void set_thread_error(const char* text) { g_last_error = text ? text : ""; }
+int g_launch_overlap = 1;
 }  // namespace olsgd
 
 extern "C" {
@@ -950,6 +951,12 @@ olsgd_status olsgd_class_pairs(uint64_t seed, int32_t m, int32_t* dst, void* str
 int64_t olsgd_iteration(const olsgd_ctx* c) { return c ? c->k : -1; }
 int64_t olsgd_launch_count(const olsgd_ctx* c) { return c ? c->launches : -1; }
 int64_t olsgd_graph_replays(const olsgd_ctx* c) { return c ? c->graph_replays : -1; }
+
+int olsgd_set_launch_overlap(int on) {
+  const int before = olsgd::g_launch_overlap;
+  olsgd::g_launch_overlap = on ? 1 : 0;
+  return before;
+}
 
 olsgd_status olsgd_profile_enable(olsgd_ctx* c, int32_t on) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");

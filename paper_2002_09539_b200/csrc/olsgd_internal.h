@@ -18,9 +18,7 @@ namespace olsgd {
 // earlier kernel of the stream has completed and its writes are visible, then lets the
 // kernel after this one start its own launch.  A kernel launched the ordinary way passes
 // through the gate at once.
-#ifndef OLSGD_OVERLAP_LAUNCH
-#define OLSGD_OVERLAP_LAUNCH 1
-#endif
+extern int g_launch_overlap;   // olsgd_set_launch_overlap
 
 #ifdef __CUDACC__
 __device__ __forceinline__ void launch_gate() {
@@ -40,7 +38,7 @@ cudaError_t launch_chained(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = OLSGD_OVERLAP_LAUNCH ? 1 : 0;
+  cfg.numAttrs = g_launch_overlap ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 #endif

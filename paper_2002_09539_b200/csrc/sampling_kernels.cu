@@ -39,6 +39,7 @@ constexpr uint32_t kStreamEpoch = 3;
 __global__ void minibatch_indices_kernel(int32_t* __restrict__ idx, uint32_t k0, uint32_t k1,
                                          int m, uint64_t k_base, const long long* k_ptr,
                                          int batch, uint32_t n, uint32_t worker_offset) {
+  launch_gate();
   // inside a captured graph the iteration number lives in device memory
   const uint32_t k = (uint32_t)(k_base + (k_ptr ? (uint64_t)*k_ptr : 0ull));
   const int blocks_per_worker = (batch + 3) / 4;
@@ -82,6 +83,7 @@ __global__ void minibatch_indices_epoch_kernel(int32_t* __restrict__ idx, uint32
                                                int m, uint64_t k_base, const long long* k_ptr,
                                                int batch, uint32_t n, int h,
                                                uint32_t worker_offset) {
+  launch_gate();
   const uint64_t k = k_base + (k_ptr ? (uint64_t)*k_ptr : 0ull);
   const int t_id = blockIdx.x * blockDim.x + threadIdx.x;
   if (t_id >= m * batch) return;
@@ -108,6 +110,7 @@ __global__ void minibatch_indices_epoch_kernel(int32_t* __restrict__ idx, uint32
 
 // The device-resident iteration counter of a captured graph: *p = value, or *p += by.
 __global__ void counter_kernel(long long* p, long long value, long long by, int set) {
+  launch_gate();
   if (threadIdx.x == 0 && blockIdx.x == 0) *p = set ? value : *p + by;
 }
 
@@ -129,10 +132,10 @@ cudaError_t launch_minibatch_indices(int32_t* idx, uint64_t seed, int m, int64_t
                                      cudaStream_t s) {
   const int total = m * ((batch + 3) / 4);
   const int threads = 128;
-  minibatch_indices_kernel<<<(total + threads - 1) / threads, threads, 0, s>>>(
-      idx, (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), m, (uint64_t)k,
-      reinterpret_cast<const long long*>(k_ptr), batch, (uint32_t)n, (uint32_t)worker_offset);
-  return cudaGetLastError();
+  return launch_chained(minibatch_indices_kernel, dim3((total + threads - 1) / threads), dim3(threads),
+                        0, s, idx, (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), m,
+                        (uint64_t)k, reinterpret_cast<const long long*>(k_ptr), batch, (uint32_t)n,
+                        (uint32_t)worker_offset);
 }
 
 cudaError_t launch_minibatch_indices_epoch(int32_t* idx, uint64_t seed, int m, int64_t k, int batch,
@@ -142,16 +145,16 @@ cudaError_t launch_minibatch_indices_epoch(int32_t* idx, uint64_t seed, int m, i
   while (((int64_t)1 << bits) < n) ++bits;       // ceil(log2 n), at least 1
   const int h = (bits + 1) / 2;
   const int total = m * batch, threads = 128;
-  minibatch_indices_epoch_kernel<<<(total + threads - 1) / threads, threads, 0, s>>>(
-      idx, (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), m, (uint64_t)k,
-      reinterpret_cast<const long long*>(k_ptr), batch, (uint32_t)n, h, (uint32_t)worker_offset);
-  return cudaGetLastError();
+  return launch_chained(minibatch_indices_epoch_kernel, dim3((total + threads - 1) / threads),
+                        dim3(threads), 0, s, idx, (uint32_t)(seed & 0xFFFFFFFFu),
+                        (uint32_t)(seed >> 32), m, (uint64_t)k,
+                        reinterpret_cast<const long long*>(k_ptr), batch, (uint32_t)n, h,
+                        (uint32_t)worker_offset);
 }
 
 cudaError_t launch_counter(int64_t* p, int64_t value, int64_t by, bool set, cudaStream_t s) {
-  counter_kernel<<<1, 32, 0, s>>>(reinterpret_cast<long long*>(p), (long long)value, (long long)by,
-                                  set ? 1 : 0);
-  return cudaGetLastError();
+  return launch_chained(counter_kernel, dim3(1), dim3(32), 0, s, reinterpret_cast<long long*>(p),
+                        (long long)value, (long long)by, set ? 1 : 0);
 }
 
 cudaError_t launch_class_pairs(int32_t* dst, uint64_t seed, int m, cudaStream_t s) {

@@ -41,6 +41,7 @@ gather_kernel(const float* __restrict__ X, const int32_t* __restrict__ y,
               const int32_t* __restrict__ idx, float* __restrict__ xb32,
               __nv_bfloat16* __restrict__ xb16, __nv_bfloat16* __restrict__ xb16t,
               int32_t* __restrict__ yb, int batch, int64_t n, int d) {
+  launch_gate();
   __shared__ __nv_bfloat16 tile[kGatherRows][kGatherCols + 2];
   __shared__ int32_t rows[kGatherRows];
   const int i = blockIdx.z;
@@ -84,6 +85,7 @@ gather_vec_kernel(const float* __restrict__ X, const int32_t* __restrict__ y,
                   const int32_t* __restrict__ idx, float* __restrict__ xb32,
                   __nv_bfloat16* __restrict__ xb16, __nv_bfloat16* __restrict__ xb16t,
                   int32_t* __restrict__ yb, int batch, int64_t n, int d) {
+  launch_gate();
   __shared__ __align__(16) __nv_bfloat16 tile[kGvRows][kGvCols + 8];
   __shared__ int32_t rows[kGvRows];
   const int i = blockIdx.z;
@@ -133,6 +135,7 @@ __global__ void __launch_bounds__(128)
 linreg_kernel(const float* __restrict__ X, const float* __restrict__ y,
               const int32_t* __restrict__ idx, const float* __restrict__ x, float* __restrict__ g,
               float* __restrict__ loss, int batch, int64_t n, int d, int64_t ld) {
+  launch_gate();
   extern __shared__ float sm[];  // residuals [batch]
   const int i = blockIdx.x;
   const float* w = x + (int64_t)i * ld;
@@ -167,6 +170,7 @@ linreg_kernel(const float* __restrict__ X, const float* __restrict__ y,
 
 __global__ void bias_grad_kernel(const __nv_bfloat16* __restrict__ dat, float* __restrict__ g,
                                  int64_t ld, int64_t b_off, int R, int batch) {
+  launch_gate();
   const int i = blockIdx.y;
   const int r = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
   const int lane = threadIdx.x % 32;
@@ -235,28 +239,26 @@ cudaError_t launch_gather(const float* X, const int32_t* y, const int32_t* idx, 
                           int64_t n, int d, cudaStream_t s) {
   if (d % kGvCols == 0 && batch % kGvRows == 0) {
     dim3 grid(d / kGvCols, batch / kGvRows, m);
-    gather_vec_kernel<<<grid, 256, 0, s>>>(X, y, idx, xb32, xb16, xb16t, yb, batch, n, d);
-    return cudaGetLastError();
+    return launch_chained(gather_vec_kernel, grid, dim3(256), 0, s, X, y, idx, xb32, xb16, xb16t, yb,
+                          batch, n, d);
   }
   dim3 grid((d + kGatherCols - 1) / kGatherCols, (batch + kGatherRows - 1) / kGatherRows, m);
   dim3 block(kGatherCols, 4);
-  gather_kernel<<<grid, block, 0, s>>>(X, y, idx, xb32, xb16, xb16t, yb, batch, n, d);
-  return cudaGetLastError();
+  return launch_chained(gather_kernel, grid, block, 0, s, X, y, idx, xb32, xb16, xb16t, yb, batch, n, d);
 }
 
 cudaError_t launch_linreg(const float* X, const float* y, const int32_t* idx, const float* x,
                           float* g, float* loss, int m, int batch, int64_t n, int d, int64_t ld,
                           cudaStream_t s) {
-  linreg_kernel<<<m, 128, (size_t)batch * sizeof(float), s>>>(X, y, idx, x, g, loss, batch, n, d, ld);
-  return cudaGetLastError();
+  return launch_chained(linreg_kernel, dim3(m), dim3(128), (size_t)batch * sizeof(float), s, X, y, idx,
+                        x, g, loss, batch, n, d, ld);
 }
 
 cudaError_t launch_bias_grad(const __nv_bfloat16* dat, float* g, int64_t ld, int64_t b_off, int m,
                              int R, int batch, cudaStream_t s) {
   const int warps = 8;
   dim3 grid((R + warps - 1) / warps, m), block(warps * 32);
-  bias_grad_kernel<<<grid, block, 0, s>>>(dat, g, ld, b_off, R, batch);
-  return cudaGetLastError();
+  return launch_chained(bias_grad_kernel, grid, block, 0, s, dat, g, ld, b_off, R, batch);
 }
 
 cudaError_t launch_gemm_simt(const GemmArgs& a, cudaStream_t s) {

@@ -77,6 +77,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
+  // everything above touched only shared and tensor memory: it may run under the tail of
+  // the kernel before this one
+  launch_gate();
 
   if (warp == 0 && lane == 0) {
     // ---------------- TMA producer
@@ -250,8 +253,7 @@ cudaError_t launch_one(const GemmArgs& a, const CUtensorMap& ma, const CUtensorM
   ea.out_batch = a.out_batch;
   ea.status = a.status;
   dim3 grid(a.Nb / BN, a.Ma / kBM, a.m);
-  kern<<<grid, kThreads, smem, s>>>(ma, mb, a.K / kBK, a.a_mn_major ? 1 : 0, ea);
-  return cudaGetLastError();
+  return launch_chained(kern, grid, dim3(kThreads), smem, s, ma, mb, a.K / kBK, a.a_mn_major ? 1 : 0, ea);
 }
 
 // Self-test of the bounded wait: one thread waits on an mbarrier that nothing ever

@@ -165,6 +165,9 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
+  // everything above touched only shared and tensor memory: it may run under the tail of
+  // the kernel before this one
+  launch_gate();
 
   if (warp == 0 && lane == 0) {
     // ---------------- TMA producer
@@ -467,12 +470,10 @@ cudaError_t launch_wgrad_tc(const GemmArgs& a, cudaStream_t s) {
     up.sync = a.upd.sync;
   }
   if (fused)
-    wgrad_tc_kernel<true><<<ctas, 320, smem, s>>>(ma, mb, mo, mu, num_kb, n_stages, n_tiles, m_tiles,
-                                                  chunks, a.Nb, up, a.status);
-  else
-    wgrad_tc_kernel<false><<<ctas, kThreads, smem, s>>>(ma, mb, mo, mu, num_kb, n_stages, n_tiles,
-                                                        m_tiles, chunks, a.Nb, up, a.status);
-  return cudaGetLastError();
+    return launch_chained(wgrad_tc_kernel<true>, dim3(ctas), dim3(320), smem, s, ma, mb, mo, mu, num_kb,
+                          n_stages, n_tiles, m_tiles, chunks, a.Nb, up, a.status);
+  return launch_chained(wgrad_tc_kernel<false>, dim3(ctas), dim3(kThreads), smem, s, ma, mb, mo, mu,
+                        num_kb, n_stages, n_tiles, m_tiles, chunks, a.Nb, up, a.status);
 }
 
 }  // namespace olsgd

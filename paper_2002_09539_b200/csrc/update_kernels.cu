@@ -37,6 +37,7 @@ fused_update_kernel(const float* __restrict__ x_in, float* __restrict__ x_out,
                     const float* __restrict__ z, __nv_bfloat16* __restrict__ shadow, int64_t P,
                     int64_t n4, int64_t ld, int64_t ldg, int m, int wpt, bool gvec, float gamma,
                     float mu, float alpha) {
+  launch_gate();
   const int64_t col4 = (int64_t)blockIdx.x * kUpdateThreads + threadIdx.x;
   if (col4 >= n4) return;
   const int i0 = blockIdx.y * wpt;
@@ -158,6 +159,7 @@ worker_mean_anchor_kernel(const float* __restrict__ x, float* __restrict__ z,
 __global__ void __launch_bounds__(kUpdateThreads)
 worker_mean_broadcast_kernel(float* __restrict__ x, __nv_bfloat16* __restrict__ shadow,
                              float* __restrict__ z, int64_t n4, int64_t ld, int m, float m_f) {
+  launch_gate();
   const int64_t col4 = (int64_t)blockIdx.x * kUpdateThreads + threadIdx.x;
   if (col4 >= n4) return;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -275,11 +277,11 @@ cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t s) {
   const bool mom = a.u != nullptr && a.mu != 0.f;
   const bool shadow = a.shadow != nullptr;
   dim3 grid((unsigned)gx, (unsigned)gy), block(kUpdateThreads);
-#define OLSGD_LAUNCH_UPD(MOM, SYNC, SH)                                                        \
-  fused_update_kernel<MOM, SYNC, SH><<<grid, block, 0, s>>>(a.x_in, a.x_out, a.g, a.u, a.z,    \
-                                                           a.shadow, a.P, n4, a.ld, a.ldg,    \
-                                                           a.m, wpt, gvec, a.gamma, a.mu,     \
-                                                           a.alpha)
+  cudaError_t err = cudaSuccess;
+#define OLSGD_LAUNCH_UPD(MOM, SYNC, SH)                                                          \
+  err = launch_chained(fused_update_kernel<MOM, SYNC, SH>, grid, block, 0, s, a.x_in, a.x_out,   \
+                       a.g, a.u, a.z, a.shadow, a.P, n4, a.ld, a.ldg, a.m, wpt, gvec, a.gamma,   \
+                       a.mu, a.alpha)
   if (mom) {
     if (a.sync) { if (shadow) OLSGD_LAUNCH_UPD(true, true, true); else OLSGD_LAUNCH_UPD(true, true, false); }
     else        { if (shadow) OLSGD_LAUNCH_UPD(true, false, true); else OLSGD_LAUNCH_UPD(true, false, false); }
@@ -288,7 +290,7 @@ cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t s) {
     else        { if (shadow) OLSGD_LAUNCH_UPD(false, false, true); else OLSGD_LAUNCH_UPD(false, false, false); }
   }
 #undef OLSGD_LAUNCH_UPD
-  return cudaGetLastError();
+  return err;
 }
 
 template <int SLICES>
@@ -315,9 +317,9 @@ cudaError_t launch_worker_mean_anchor(const AnchorArgs& a, cudaStream_t s) {
 cudaError_t launch_worker_mean_broadcast(float* x, __nv_bfloat16* shadow, float* z, int64_t P,
                                          int64_t ld, int m, cudaStream_t s) {
   const int64_t n4 = (P + 3) / 4;
-  worker_mean_broadcast_kernel<<<(unsigned)((n4 + kUpdateThreads - 1) / kUpdateThreads),
-                                 kUpdateThreads, 0, s>>>(x, shadow, z, n4, ld, m, (float)m);
-  return cudaGetLastError();
+  return launch_chained(worker_mean_broadcast_kernel,
+                        dim3((unsigned)((n4 + kUpdateThreads - 1) / kUpdateThreads)),
+                        dim3(kUpdateThreads), 0, s, x, shadow, z, n4, ld, m, (float)m);
 }
 
 cudaError_t launch_anchor_from_sum(const float* sum, float* z, float* v, int64_t P, float beta,

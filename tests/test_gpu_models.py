@@ -271,3 +271,47 @@ def test_run_with_replayed_graph_equals_single_steps(kind, dims, gemm, tau, epoc
     assert np.array_equal(xa, xb) and np.array_equal(za, zb) and np.array_equal(va, vb)
     assert np.array_equal(la[1:].cpu().numpy(), lb[1:].cpu().numpy())
     assert a.launch_count >= b.launch_count      # the replayed launches are counted too
+
+
+@pytest.mark.parametrize("kind,dims,gemm,tau", [("softmax", [100, 7], 0, 2),
+                                                ("mlp", [128, 256, 128, 10], 1, 3),
+                                                ("linreg", [24], 0, 2)])
+def test_overlapped_launches_give_the_bits_of_plain_stream_order(kind, dims, gemm, tau):
+    # with olsgd_set_launch_overlap(1) a kernel may become resident under the tail of its
+    # predecessor but touches global memory only once the predecessor has completed: the
+    # trajectory must not change by a bit, on the replayed graph and call by call
+    from paper_2002_09539_b200 import OverlapLocalSGD, set_launch_overlap
+    m, n, batch, iters = 3, 96, 64, 60
+    if kind == "linreg":
+        X, y, _ = si.linreg_data(15, m, n, dims[0])
+        x0 = np.zeros(dims[0], np.float32)
+    else:
+        X, y = si.mixture_data(15, m, n, dims[0])
+        y = (y % dims[-1]).astype(np.int32)
+        x0 = (si.model_init(15, "mlp", dims) if kind == "mlp" else
+              (0.1 * np.random.default_rng(15).standard_normal(models.n_params(kind, dims))).astype(np.float32))
+    kw = dict(dims=dims, gemm_bf16=gemm, m=m, tau=tau, batch=batch, gamma=0.02, alpha=0.5, beta=0.7,
+              mu=0.9, seed=15, x0=x0, X=to_dev(X), y=to_dev(y))
+    got = {}
+    before = set_launch_overlap(True)
+    try:
+        for on in (True, False):
+            set_launch_overlap(on)
+            stream = torch.cuda.Stream()
+            stream.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(stream):
+                a = OverlapLocalSGD(kind, **kw)
+                la = torch.zeros((iters, m), device="cuda")
+                a.run(iters, la)
+                assert a.graph_replays >= 1
+                for k in range(iters, iters + 5):
+                    a.local_step()
+                    if (k + 1) % tau == 0:
+                        a.period_sync()
+                a.join()
+            torch.cuda.synchronize()
+            got[on] = a.state() + (la.cpu().numpy(),)
+    finally:
+        set_launch_overlap(before)
+    for p, q in zip(got[True], got[False]):
+        assert np.array_equal(p, q)
