@@ -52,7 +52,7 @@ __device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
 }
 
 constexpr int kHeadThreads = 128;
-constexpr int kHeadSmallGrid = 2 * 148;
+constexpr int kHeadSmallGrid = 4 * 148;
 
 // Forward, loss and input gradient of the output layer for R batch rows of one worker.
 //

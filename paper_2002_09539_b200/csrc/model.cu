@@ -288,10 +288,19 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
     gw.out_f = io.g + mb.w_off[l - 1];
     gw.ldo = spec.dims[l - 1];
     gw.out_batch = io.ld;
-    if (io.upd.enabled && mb.fused_layer[l - 1]) {
+    const bool fused = io.upd.enabled && mb.fused_layer[l - 1];
+    if (fused) {
       // the update of W_l happens in this GEMM's epilogue: no gradient is stored
       gw.upd = io.upd;
       gw.upd.w_off = mb.w_off[l - 1];
+    }
+    // the tensor-core weight-gradient kernel also adds up the rows of dA_l^T: the bias gradient
+    const bool rowsum_in_gemm = tensor_path(spec) && wgrad_tc_supported(gw);
+    if (rowsum_in_gemm) {
+      gw.rowsum_out = io.g + mb.b_off[l - 1];
+      gw.rowsum_batch = io.ld;
+    }
+    if (fused) {
       if (io.wait_before_update && !waited) {
         OLSGD_TRY(cudaStreamWaitEvent(s, io.wait_before_update, 0));
         waited = true;
@@ -302,7 +311,7 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
       Scope sc(hook, OLSGD_KC_BACKWARD, s);
       OLSGD_TRY(run_gemm(spec, gw, io.status, s));
     }
-    {
+    if (!rowsum_in_gemm) {
       Scope sc(hook, OLSGD_KC_BACKWARD, s);
       OLSGD_TRY(launch_bias_grad(mb.dat[l], io.g, io.ld, mb.b_off[l - 1], m, spec.dims[l], B, s));
     }

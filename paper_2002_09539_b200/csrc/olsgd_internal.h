@@ -212,6 +212,10 @@ struct GemmArgs {
   int64_t ldo, out_batch;
   int* status;               // device word that receives OLSGD_ETIMEOUT if a bounded wait gives up
   FusedUpdateArgs upd;       // weight-gradient kernel only
+  // weight-gradient kernel only, or null: rowsum_out[i * rowsum_batch + row] = sum_k A[i][row][k],
+  // the bias gradient of the layer (A = dA^T), summed in the order of the bias-gradient kernel
+  float* rowsum_out;
+  int64_t rowsum_batch;
 };
 // Plain CUDA-core version, used to validate the tensor-core kernel.
 cudaError_t launch_gemm_simt(const GemmArgs& a, cudaStream_t s);

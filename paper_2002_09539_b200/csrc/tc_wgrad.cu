@@ -12,11 +12,11 @@
 // is double-buffered in tensor memory so that the MMAs of unit j+1 run under
 // the epilogue of unit j.
 //
-// Plain variant (192 threads): warp 0 TMA loads, warp 1 MMA issue + TMEM owner,
+// Plain variant (224 threads): warp 0 TMA loads, warp 1 MMA issue + TMEM owner,
 // warps 2-5 epilogue, which moves 32 x 32 blocks from TMEM through swizzled
 // shared memory to global memory with TMA stores (whole 128-byte lines).
 //
-// FUSED variant (320 threads, eight epilogue warps): the gradient never goes to
+// FUSED variant (352 threads, eight epilogue warps): the gradient never goes to
 // memory.  Each 32 x 32 block of dW is turned, through a swizzled shared-memory
 // buffer, from "one accumulator row per thread" into "one 16-byte row segment
 // per thread", and the same thread then applies the parameter update to that
@@ -26,6 +26,10 @@
 // are prefetched by TMA two blocks ahead into a per-warp ring, which is what
 // keeps enough bytes in flight; results leave as whole 128-byte row segments.
 // That removes the 4-byte write and the 4-byte read of G_k per parameter.
+//
+// One more warp in either variant adds up the rows of the resident A operand, which is the
+// layer's bias gradient, in the first CTA of every slab: lane l takes the columns l, l + 32,
+// ... in order and a fixed shuffle tree combines the lanes.
 //
 // Every mbarrier wait is bounded (see tc_common.cuh).
 #include "tc_common.cuh"
@@ -115,12 +119,15 @@ struct WgradCtl {
 constexpr uint32_t kXuTile = 32 * 32 * 4;        // one fp32 tile of x or u
 constexpr uint32_t kXuPerWarp = 2 * 2 * kXuTile; // two buffers of (x, u)
 
+constexpr int kFusedThreads = 352;   // TMA, MMA, eight epilogue warps, row sums
+constexpr int kPlainThreads = 224;   // TMA, MMA, four epilogue warps, row sums
+
 template <bool FUSED>
-__global__ void __launch_bounds__(FUSED ? 320 : kThreads, 1)
+__global__ void __launch_bounds__(FUSED ? kFusedThreads : kPlainThreads, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_u,
                 int num_kb, int n_stages, int n_tiles, int m_tiles, int chunks, int ldw,
-                WgradUpd up, int* status) {
+                WgradUpd up, float* rowsum, int64_t rowsum_batch, int* status) {
   constexpr uint32_t kABlock = kBM * kBK * 2;   // one k-block of the A slab, 16 KB
   constexpr uint32_t kBBlock = kWN * kBK * 2;   // one k-block of a B tile, 16 KB
   constexpr uint32_t kEpiBuf = 32 * 32 * 4;     // one 32 x 32 fp32 block, 4 KB
@@ -169,7 +176,43 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   // the kernel before this one
   launch_gate();
 
-  if (warp == 0 && lane == 0) {
+  constexpr int kRowsumWarp = FUSED ? 10 : 6;
+  if (warp == kRowsumWarp) {
+    // ---------------- row sums of the resident A operand (the layer's bias gradient)
+    if (rowsum && my_first == 0 && n_units > 0 &&
+        mbar_wait(smem_u32(&ctl->a_full), 0u, abort_flag)) {
+      const int worker = my_slab / m_tiles, m0 = (my_slab - worker * m_tiles) * kBM;
+      float* dst = rowsum + (int64_t)worker * rowsum_batch + m0;
+      // One thread per row.  The sum keeps the order of the bias-gradient kernel (partial l
+      // takes the columns l, l + 32, ... in order; the partials are combined by the tree of
+      // an xor-shuffle reduction), so both give the same bits.  Row r of a k-block is 128
+      // bytes whose 16-byte chunks are permuted by the 128-byte swizzle (chunk j at j ^ (r % 8)).
+      for (int rr = 0; rr < kBM / 32; ++rr) {
+        const int row = rr * 32 + lane;
+        float part[32];
+#pragma unroll
+        for (int l = 0; l < 32; ++l) part[l] = 0.f;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          const uint8_t* rowp = a_smem + kb * kABlock + row * 128;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint4 q = *reinterpret_cast<const uint4*>(rowp + ((j ^ (row & 7)) << 4));
+            const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              part[8 * (j & 3) + 2 * e] += __uint_as_float(w[e] << 16);
+              part[8 * (j & 3) + 2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
+            }
+          }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+          for (int l = 0; l < o; ++l) part[l] += part[l + o];
+        dst[row] = part[0];
+      }
+    }
+  } else if (warp == 0 && lane == 0) {
     // ---------------- TMA producer
     const uint32_t a_full = smem_u32(&ctl->a_full);
     int issued = 0, visit = -1, cur_slab = -1;
@@ -470,10 +513,12 @@ cudaError_t launch_wgrad_tc(const GemmArgs& a, cudaStream_t s) {
     up.sync = a.upd.sync;
   }
   if (fused)
-    return launch_chained(wgrad_tc_kernel<true>, dim3(ctas), dim3(320), smem, s, ma, mb, mo, mu, num_kb,
-                          n_stages, n_tiles, m_tiles, chunks, a.Nb, up, a.status);
-  return launch_chained(wgrad_tc_kernel<false>, dim3(ctas), dim3(kThreads), smem, s, ma, mb, mo, mu,
-                        num_kb, n_stages, n_tiles, m_tiles, chunks, a.Nb, up, a.status);
+    return launch_chained(wgrad_tc_kernel<true>, dim3(ctas), dim3(kFusedThreads), smem, s, ma, mb, mo,
+                          mu, num_kb, n_stages, n_tiles, m_tiles, chunks, a.Nb, up, a.rowsum_out,
+                          a.rowsum_batch, a.status);
+  return launch_chained(wgrad_tc_kernel<false>, dim3(ctas), dim3(kPlainThreads), smem, s, ma, mb, mo,
+                        mu, num_kb, n_stages, n_tiles, m_tiles, chunks, a.Nb, up, a.rowsum_out,
+                        a.rowsum_batch, a.status);
 }
 
 }  // namespace olsgd
