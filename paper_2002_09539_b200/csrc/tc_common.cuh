@@ -85,6 +85,18 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+// 16-byte global load whose lines are kept in L2 in preference to lines of normal priority
+// (for data that many CTAs read again while a stream of read-once data passes through L2).
+__device__ __forceinline__ float4 ld_global_keep_l2(const float* p) {
+  uint64_t policy;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
+  float4 v;
+  asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "l"(p), "l"(policy));
+  return v;
+}
+
 // Store one box from shared memory to global memory; completion is tracked by
 // the issuing thread's bulk async-group.
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1,

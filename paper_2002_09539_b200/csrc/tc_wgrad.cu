@@ -313,9 +313,11 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       if (n_blocks > 0) issue(0);
       if (n_blocks > 1) issue(1);
     }
-    // The anchor strip of a block comes straight from global memory (the anchor is shared
-    // by all workers and mostly served by L2) into registers, one block ahead, so that its
-    // latency is hidden behind the update of the block before.
+    // The anchor strip of a block comes straight from global memory into registers, one
+    // block ahead, so that its latency is hidden behind the update of the block before.  The
+    // anchor is shared by all workers, whose CTAs reach the same strip at different times
+    // while a gigabyte of read-once x and u tiles passes through L2: the loads ask L2 to
+    // evict the anchor's lines last.
     float4 zs[8], zn[8];
 #pragma unroll
     for (int t = 0; t < 8; ++t) zs[t] = zn[t] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -324,7 +326,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const float* zp = up.z + up.w_off + (int64_t)(pz.m0 + lane_group * 32 + (lane >> 3)) * ldw +
                         pz.col + (half + 2 * (nn & 1)) * 32 + (lane & 7) * 4;
 #pragma unroll
-      for (int t = 0; t < 8; ++t) dst[t] = *reinterpret_cast<const float4*>(zp + (int64_t)(t * 4) * ldw);
+      for (int t = 0; t < 8; ++t) dst[t] = ld_global_keep_l2(zp + (int64_t)(t * 4) * ldw);
     };
     if (up.sync && n_blocks > 0) load_z(0, zs);
     bool ok = true;
