@@ -277,9 +277,13 @@ def run_ours(args, rank, world):
     n, B, d0 = c["n"], c["batch"], c["dims"][0]
     rng = np.random.default_rng(seed + 77)
     Xh, yh = [], []
+    # a model whose GEMM operands are bf16 takes its rows in bf16 (the host data set is kept
+    # in the operand type; rounding to nearest even on the host gives the bits the device's
+    # own rounding of fp32 rows gives), any other model in fp32
+    host_dtype = torch.bfloat16 if c["gemm_bf16"] else torch.float32
     for _ in range(pool):
         idx = rng.integers(0, n, size=(m, B))
-        Xh.append(torch.from_numpy(np.stack([X[i][idx[i]] for i in range(m)])).pin_memory())
+        Xh.append(torch.from_numpy(np.stack([X[i][idx[i]] for i in range(m)])).to(host_dtype).pin_memory())
         yh.append(torch.from_numpy(np.stack([y[i][idx[i]] for i in range(m)])).pin_memory())
     loss_h = torch.zeros((K + W, m), dtype=torch.float32).pin_memory()
 
@@ -300,9 +304,12 @@ def run_ours(args, rank, world):
     e2e_ms = max_over_ranks(e2e_ms, world, "cuda")
     assert np.isfinite(loss_h[W:].numpy()).all()
     e2e = dict(value=round(world * m * K / (e2e_ms * 1e-3), 1), unit=UNIT,
-               h2d_bytes_per_step=int(m * B * d0 * 4 + m * B * 4), d2h_bytes_per_step=int(m * 4),
-               ms_per_step=round(e2e_ms / K, 4),
-               api="olsgd_local_step_host + olsgd_period_sync, pinned host minibatches")
+               h2d_bytes_per_step=int(Xh[0].numel() * Xh[0].element_size() +
+                                      yh[0].numel() * yh[0].element_size()),
+               d2h_bytes_per_step=int(m * 4), ms_per_step=round(e2e_ms / K, 4),
+               api="%s + olsgd_period_sync, pinned host minibatches (%s rows, int32 labels)"
+                   % ("olsgd_local_step_host_bf16" if c["gemm_bf16"] else "olsgd_local_step_host",
+                      "bf16" if c["gemm_bf16"] else "fp32"))
 
     out = None
     if rank == 0:

@@ -159,6 +159,19 @@ olsgd_status olsgd_local_step(olsgd_ctx* ctx, float* loss_device);
 olsgd_status olsgd_local_step_host(olsgd_ctx* ctx, const float* Xb_host, const void* yb_host,
                                    float* loss_host);
 
+/* olsgd_local_step_host for models whose GEMM operands are bf16 (OLSGD_MLP with
+ * gemm_bf16 != 0): the caller hands over the rows already rounded to bf16
+ * (round-to-nearest-even, the rounding the device applies to fp32 rows), which
+ * halves the host-to-device bytes of a step.  The result has the bits of
+ * olsgd_local_step_host on the fp32 rows they were rounded from.
+ *   Xb_host_bf16  bf16 (uint16 storage) [m][batch][dims[0]], host, same lifetime
+ *                 rule as Xb_host above
+ *   yb_host       int32 [m][batch]
+ *   loss_host     as above
+ * Returns OLSGD_ESTATE for any other model.                                  */
+olsgd_status olsgd_local_step_host_bf16(olsgd_ctx* ctx, const void* Xb_host_bf16,
+                                        const void* yb_host, float* loss_host);
+
 /* Block the host until every stream of the context is idle.                 */
 olsgd_status olsgd_join(olsgd_ctx* ctx);
 

@@ -64,6 +64,7 @@ def load_library():
         "olsgd_local_step": (i32, [vp, vp]),
         "olsgd_local_step_with_grads": (i32, [vp, vp]),
         "olsgd_local_step_host": (i32, [vp, vp, vp, vp]),
+        "olsgd_local_step_host_bf16": (i32, [vp, vp, vp, vp]),
         "olsgd_join": (i32, [vp]),
         "olsgd_selftest_wait_timeout": (i32, [vp, i32]),
         "olsgd_clear_status": (i32, [vp]),
@@ -193,13 +194,16 @@ class OverlapLocalSGD:
         _check(self.lib, self.lib.olsgd_local_step_with_grads(self.ctx, g.data_ptr()), self.ctx)
 
     def local_step_host(self, Xb, yb, loss=None):
-        """Xb, yb (and loss) are HOST tensors, ideally pinned."""
+        """Xb, yb (and loss) are HOST tensors, ideally pinned.  Xb is float32, or bfloat16 for
+        a model whose GEMM operands are bf16 (olsgd_local_step_host_bf16)."""
         assert not Xb.is_cuda and not yb.is_cuda and Xb.is_contiguous() and yb.is_contiguous()
-        assert Xb.dtype == torch.float32 and Xb.numel() == self.m * self.batch * self.spec.dims[0]
+        assert Xb.dtype in (torch.float32, torch.bfloat16)
+        assert Xb.numel() == self.m * self.batch * self.spec.dims[0]
         assert yb.numel() == self.m * self.batch and yb.element_size() == 4
-        _check(self.lib, self.lib.olsgd_local_step_host(
-            self.ctx, Xb.data_ptr(), yb.data_ptr(), loss.data_ptr() if loss is not None else None),
-            self.ctx)
+        fn = (self.lib.olsgd_local_step_host if Xb.dtype == torch.float32
+              else self.lib.olsgd_local_step_host_bf16)
+        _check(self.lib, fn(self.ctx, Xb.data_ptr(), yb.data_ptr(),
+                            loss.data_ptr() if loss is not None else None), self.ctx)
 
     def join(self):
         _check(self.lib, self.lib.olsgd_join(self.ctx), self.ctx)

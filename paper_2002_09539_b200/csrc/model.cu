@@ -185,7 +185,12 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
   // softmax regression in fp32 reads its rows straight from the data set (gather fused into
   // the two output-layer kernels); every other model stages the minibatch
   const bool fused_gather = !bf && L == 1;
-  if (!fused_gather) {
+  const bool rows_in_bf16 = bf && io.xb16_in != nullptr;
+  if (rows_in_bf16) {
+    Scope sc(hook, OLSGD_KC_GATHER, s);
+    OLSGD_TRY(launch_transpose_bf16(io.xb16_in, static_cast<const int32_t*>(data.y), mb.xb16t, mb.yb,
+                                    m, B, d0, s));
+  } else if (!fused_gather) {
     Scope sc(hook, OLSGD_KC_GATHER, s);
     OLSGD_TRY(launch_gather(X, static_cast<const int32_t*>(data.y), io.idx, bf ? nullptr : mb.xb32,
                             bf ? mb.xb16 : nullptr, bf ? mb.xb16t : nullptr, mb.yb, m, B, n, d0,
@@ -198,7 +203,7 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
     ga.A = io.shadow + mb.w_off[l - 1];
     ga.lda = spec.dims[l - 1];
     ga.a_batch = io.ld;
-    ga.B = (l == 1) ? mb.xb16 : mb.h[l - 1];
+    ga.B = (l == 1) ? (rows_in_bf16 ? io.xb16_in : mb.xb16) : mb.h[l - 1];
     ga.ldb = spec.dims[l - 1];
     ga.b_batch = (int64_t)B * spec.dims[l - 1];
     ga.m = m;

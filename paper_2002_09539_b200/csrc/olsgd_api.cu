@@ -366,8 +366,9 @@ cudaError_t draw_indices(olsgd_ctx* c, int64_t k) {
 // S2-S6 of one iteration on the main stream, reading the minibatch rows
 // idx[i][:] of `data`.  stage_slot >= 0 marks a host-fed staging slot to release.
 olsgd_status step_body(olsgd_ctx* c, const olsgd_data& data, const int32_t* idx,
-                       float* loss_device, int stage_slot) {
+                       float* loss_device, int stage_slot, const __nv_bfloat16* xb16_in = nullptr) {
   StepIO io;
+  io.xb16_in = xb16_in;
   io.x = c->x[c->cur];
   io.shadow = c->shadow;
   io.g = c->g;
@@ -578,19 +579,23 @@ olsgd_status olsgd_local_step(olsgd_ctx* c, float* loss_device) {
   return step_body(c, c->data, c->idx, loss_device, -1);
 }
 
-olsgd_status olsgd_local_step_host(olsgd_ctx* c, const float* Xb_host, const void* yb_host,
-                                   float* loss_host) {
+// Shared body of the two host-fed entry points; elem = bytes per input element (4 or 2).
+static olsgd_status local_step_host_impl(olsgd_ctx* c, const void* Xb_host, const void* yb_host,
+                                         float* loss_host, size_t elem) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
   if (c->spec.kind == OLSGD_FLAT)
     return fail(c, OLSGD_ESTATE, "OLSGD_FLAT contexts take olsgd_local_step_with_grads");
   if (!Xb_host || !yb_host) return fail(c, OLSGD_EINVAL, "host minibatch pointers are NULL");
+  if (elem == 2 && !(c->spec.kind == OLSGD_MLP && c->spec.gemm_bf16 != 0))
+    return fail(c, OLSGD_ESTATE, "bf16 minibatches are for models whose GEMM operands are bf16 "
+                                 "(OLSGD_MLP with gemm_bf16 != 0)");
   if (c->need_sync) return fail(c, OLSGD_ESTATE, "a period ended: call olsgd_period_sync first");
   const int slot = c->host_slot;
   c->host_slot ^= 1;
   const size_t rows = (size_t)c->hp.m * c->hp.batch;
   // the kernels that read this slot two steps ago must be done before it is refilled
   OLSGD_CUDA(c, cudaStreamWaitEvent(c->copy, c->stage_free[slot], 0));
-  OLSGD_CUDA(c, cudaMemcpyAsync(c->stage_x[slot], Xb_host, rows * c->spec.dims[0] * sizeof(float),
+  OLSGD_CUDA(c, cudaMemcpyAsync(c->stage_x[slot], Xb_host, rows * c->spec.dims[0] * elem,
                                 cudaMemcpyHostToDevice, c->copy));
   OLSGD_CUDA(c, cudaMemcpyAsync(c->stage_y[slot], yb_host, rows * 4, cudaMemcpyHostToDevice, c->copy));
   OLSGD_CUDA(c, cudaEventRecord(c->h2d_done[slot], c->copy));
@@ -599,12 +604,24 @@ olsgd_status olsgd_local_step_host(olsgd_ctx* c, const float* Xb_host, const voi
   staged.X = c->stage_x[slot];
   staged.y = c->stage_y[slot];
   staged.n_per_worker = c->hp.batch;
-  olsgd_status st = step_body(c, staged, c->ident, nullptr, slot);
+  const __nv_bfloat16* direct =
+      elem == 2 ? reinterpret_cast<const __nv_bfloat16*>(c->stage_x[slot]) : nullptr;
+  olsgd_status st = step_body(c, staged, c->ident, nullptr, slot, direct);
   if (st != OLSGD_OK) return st;
   if (loss_host)
     OLSGD_CUDA(c, cudaMemcpyAsync(loss_host, c->mb.loss, (size_t)c->hp.m * sizeof(float),
                                   cudaMemcpyDeviceToHost, c->main));
   return OLSGD_OK;
+}
+
+olsgd_status olsgd_local_step_host(olsgd_ctx* c, const float* Xb_host, const void* yb_host,
+                                   float* loss_host) {
+  return local_step_host_impl(c, Xb_host, yb_host, loss_host, sizeof(float));
+}
+
+olsgd_status olsgd_local_step_host_bf16(olsgd_ctx* c, const void* Xb_host_bf16, const void* yb_host,
+                                        float* loss_host) {
+  return local_step_host_impl(c, Xb_host_bf16, yb_host, loss_host, 2);
 }
 
 olsgd_status olsgd_selftest_wait_timeout(olsgd_ctx* c, int32_t limit_ms) {

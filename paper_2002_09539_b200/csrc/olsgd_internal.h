@@ -126,6 +126,10 @@ cudaError_t launch_linreg(const float* X, const float* y, const int32_t* idx, co
 //   xb32  float [m][B][d]   (or null)
 //   xb16  bf16  [m][B][d]   (or null), xb16t bf16 [m][d][B] (or null)
 //   yb    int32 [m][B]
+// bf16 minibatch rows [m][batch][d] -> their transposed copy [m][d][batch], and the labels
+// y[m][batch] -> yb (d % 64 == 0, batch % 8 == 0)
+cudaError_t launch_transpose_bf16(const __nv_bfloat16* xb16, const int32_t* y, __nv_bfloat16* xb16t,
+                                  int32_t* yb, int m, int batch, int d, cudaStream_t s);
 cudaError_t launch_gather(const float* X, const int32_t* y, const int32_t* idx, float* xb32,
                           __nv_bfloat16* xb16, __nv_bfloat16* xb16t, int32_t* yb, int m, int batch,
                           int64_t n, int d, cudaStream_t s);
@@ -262,6 +266,8 @@ struct StepIO {
   float* g;                      // out: [m][ld]
   int64_t ld;
   const int32_t* idx;            // [m][batch]
+  const __nv_bfloat16* xb16_in;  // if non-null: this step's rows, already bf16, [m][batch][dims[0]]
+                                 // (data.y then holds their labels [m][batch]); idx is unused
   float* loss;                   // out: [m] or null
   int* status;                   // device status word (see GemmArgs::status)
   FusedUpdateArgs upd;           // state pointers and factors for the fused epilogue (w_off unset)

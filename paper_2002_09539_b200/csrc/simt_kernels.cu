@@ -129,6 +129,43 @@ gather_vec_kernel(const float* __restrict__ X, const int32_t* __restrict__ y,
   }
 }
 
+// Minibatch rows that arrive in bf16 (host-fed steps): the [B][d] copy is the buffer itself,
+// only the [d][B] copy of the weight-gradient GEMM and the label copy are made.  A block turns
+// 32 rows x 64 columns; a thread loads 16 bytes of a row and stores eight consecutive batch
+// entries of a column.
+constexpr int kTrRows = 32, kTrCols = 64;
+
+__global__ void __launch_bounds__(256)
+transpose_bf16_kernel(const __nv_bfloat16* __restrict__ xb16, const int32_t* __restrict__ y,
+                      __nv_bfloat16* __restrict__ xb16t, int32_t* __restrict__ yb, int batch, int d) {
+  launch_gate();
+  __shared__ __align__(16) __nv_bfloat16 tile[kTrRows][kTrCols + 8];
+  const int i = blockIdx.z;
+  const int b0 = blockIdx.y * kTrRows, j0 = blockIdx.x * kTrCols;
+  {
+    const int bl = threadIdx.x >> 3, q = threadIdx.x & 7;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (b0 + bl < batch)
+      v = *reinterpret_cast<const uint4*>(xb16 + ((int64_t)i * batch + b0 + bl) * d + j0 + q * 8);
+    *reinterpret_cast<uint4*>(&tile[bl][q * 8]) = v;
+    if (blockIdx.x == 0 && q == 0 && b0 + bl < batch)
+      yb[(int64_t)i * batch + b0 + bl] = y[(int64_t)i * batch + b0 + bl];
+  }
+  __syncthreads();
+  const int jl = threadIdx.x >> 2, bq = threadIdx.x & 3;
+  if (b0 + bq * 8 < batch) {
+    uint32_t w[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const uint16_t lo = *reinterpret_cast<const uint16_t*>(&tile[bq * 8 + 2 * e][jl]);
+      const uint16_t hi = *reinterpret_cast<const uint16_t*>(&tile[bq * 8 + 2 * e + 1][jl]);
+      w[e] = (uint32_t)lo | ((uint32_t)hi << 16);
+    }
+    *reinterpret_cast<uint4*>(xb16t + ((int64_t)i * d + j0 + jl) * batch + b0 + bq * 8) =
+        make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
 // ------------------------------------------------------------------ linear regression
 
 __global__ void __launch_bounds__(128)
@@ -245,6 +282,13 @@ cudaError_t launch_gather(const float* X, const int32_t* y, const int32_t* idx, 
   dim3 grid((d + kGatherCols - 1) / kGatherCols, (batch + kGatherRows - 1) / kGatherRows, m);
   dim3 block(kGatherCols, 4);
   return launch_chained(gather_kernel, grid, block, 0, s, X, y, idx, xb32, xb16, xb16t, yb, batch, n, d);
+}
+
+cudaError_t launch_transpose_bf16(const __nv_bfloat16* xb16, const int32_t* y, __nv_bfloat16* xb16t,
+                                  int32_t* yb, int m, int batch, int d, cudaStream_t s) {
+  if (d % kTrCols != 0 || batch % 8 != 0) return cudaErrorInvalidValue;
+  dim3 grid(d / kTrCols, (batch + kTrRows - 1) / kTrRows, m);
+  return launch_chained(transpose_bf16_kernel, grid, dim3(256), 0, s, xb16, y, xb16t, yb, batch, d);
 }
 
 cudaError_t launch_linreg(const float* X, const float* y, const int32_t* idx, const float* x,
