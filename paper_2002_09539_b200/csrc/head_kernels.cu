@@ -4,6 +4,7 @@
 // and the layer's own weight and bias gradients.  All reductions have a fixed
 // order; nothing uses floating-point atomics.
 #include "olsgd_internal.h"
+#include "update_math.cuh"
 
 namespace olsgd {
 namespace {
@@ -361,7 +362,7 @@ head_forward_vec_kernel(HeadArgs a) {
 // barrier inside.
 template <int T>
 __device__ __forceinline__ void head_bias_and_loss(const HeadArgs& a, int i, int tid, float* scratch,
-                                                   float* gi, float* loss) {
+                                                   float* gi, float* loss, const FusedUpdateArgs& up) {
   const int C = a.C, B = a.batch;
   const float* dl = a.dlogits + (int64_t)i * B * C;
   __syncthreads();
@@ -377,7 +378,18 @@ __device__ __forceinline__ void head_bias_and_loss(const HeadArgs& a, int i, int
     float sum = scratch[tid];
 #pragma unroll
     for (int q = 1; q < NP; ++q) sum += scratch[q * 32 + tid];
-    gi[a.b_off + tid] = sum;
+    if (up.enabled) {
+      // Eq. 3 / Eq. 4 for bias entry tid of worker i
+      const int64_t e = a.b_off + tid, o = (int64_t)i * up.ld + e;
+      const bool mom = up.u != nullptr && up.mu != 0.f;
+      float x = up.x_in[o], u = mom ? up.u[o] : 0.f;
+      update_scalar_rt(x, u, sum, up.sync ? up.z[e] : 0.f, up.gamma, up.mu, up.alpha, mom, up.sync != 0);
+      up.x_out[o] = x;
+      if (mom) up.u[o] = u;
+      if (up.shadow) up.shadow[o] = __float2bfloat16_rn(x);
+    } else {
+      gi[a.b_off + tid] = sum;
+    }
   }
   if (loss && tid >= T - 32) {
     const int lane = tid % 32;
@@ -453,7 +465,8 @@ head_wgrad_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ loss) {
       gi[a.w_off + (int64_t)c * K + jj] = s;
     }
   }
-  if (blockIdx.x == 0) head_bias_and_loss<kWgCols * kWgSlices>(a, i, tid, &part[0][0][0], gi, loss);
+  FusedUpdateArgs none{};
+  if (blockIdx.x == 0) head_bias_and_loss<kWgCols * kWgSlices>(a, i, tid, &part[0][0][0], gi, loss, none);
 }
 
 // The same product for K % 4 == 0 and at most 16 classes: a thread owns FOUR adjacent input
@@ -464,7 +477,7 @@ constexpr int kWvCols = 16, kWvSlices = 8, kWvRows = 128, kWvFlight = 8;
 
 template <typename InT, int CMAX>
 __global__ void __launch_bounds__(kWvCols* kWvSlices)
-head_wgrad_vec_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ loss) {
+head_wgrad_vec_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ loss, FusedUpdateArgs up) {
   launch_gate();
   __shared__ float dsm[kWvRows][CMAX + 1];
   __shared__ __align__(16) float part[kWvSlices][CMAX][kWvCols * 4];
@@ -535,10 +548,29 @@ head_wgrad_vec_kernel(HeadArgs a, float* __restrict__ g, float* __restrict__ los
         s.z += p.z;
         s.w += p.w;
       }
-      *reinterpret_cast<float4*>(gi + a.w_off + (int64_t)c * K + jj) = s;
+      const int64_t e = a.w_off + (int64_t)c * K + jj;
+      if (up.enabled) {
+        // the gradient strip is consumed here: Eq. 3 (+ Nesterov) and, on sync steps, Eq. 4
+        const int64_t o = (int64_t)i * up.ld + e;
+        const bool mom = up.u != nullptr && up.mu != 0.f;
+        float4 x = *reinterpret_cast<const float4*>(up.x_in + o);
+        float4 u = mom ? *reinterpret_cast<const float4*>(up.u + o) : make_float4(0.f, 0.f, 0.f, 0.f);
+        const float4 z = up.sync ? *reinterpret_cast<const float4*>(up.z + e)
+                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+        const bool sync = up.sync != 0;
+        update_scalar_rt(x.x, u.x, s.x, z.x, up.gamma, up.mu, up.alpha, mom, sync);
+        update_scalar_rt(x.y, u.y, s.y, z.y, up.gamma, up.mu, up.alpha, mom, sync);
+        update_scalar_rt(x.z, u.z, s.z, z.z, up.gamma, up.mu, up.alpha, mom, sync);
+        update_scalar_rt(x.w, u.w, s.w, z.w, up.gamma, up.mu, up.alpha, mom, sync);
+        *reinterpret_cast<float4*>(up.x_out + o) = x;
+        if (mom) *reinterpret_cast<float4*>(up.u + o) = u;
+        if (up.shadow) *reinterpret_cast<uint2*>(up.shadow + o) = pack_bf16x4(x);
+      } else {
+        *reinterpret_cast<float4*>(gi + e) = s;
+      }
     }
   }
-  if (blockIdx.x == 0) head_bias_and_loss<kWvCols * kWvSlices>(a, i, tid, &part[0][0][0], gi, loss);
+  if (blockIdx.x == 0) head_bias_and_loss<kWvCols * kWvSlices>(a, i, tid, &part[0][0][0], gi, loss, up);
 }
 
 template <typename InT, int CMAX, int R>
@@ -574,17 +606,28 @@ cudaError_t launch_head_forward(const HeadArgs& a, cudaStream_t s) {
   return a.in32 ? launch_fwd_c<float>(a, s) : launch_fwd_c<__nv_bfloat16>(a, s);
 }
 
-cudaError_t launch_head_wgrad(const HeadArgs& a, float* g, float* loss, cudaStream_t s) {
+bool head_wgrad_can_update(const HeadArgs& a) {
+  // the four-column kernel; the bias update is scalar and has no alignment rule
+  return a.K % 4 == 0 && a.C <= 16 && a.w_off % 4 == 0 && a.ld % 4 == 0;
+}
+
+cudaError_t launch_head_wgrad(const HeadArgs& a, float* g, float* loss, const FusedUpdateArgs* upd,
+                              cudaStream_t s) {
   const bool f32 = a.in32 != nullptr;
   cudaError_t err = cudaSuccess;
-  if (a.K % 4 == 0 && a.C <= 16 && a.w_off % 4 == 0 && a.ld % 4 == 0) {
+  FusedUpdateArgs up{};
+  if (upd && upd->enabled) {
+    if (!head_wgrad_can_update(a)) return cudaErrorInvalidValue;
+    up = *upd;
+  }
+  if (head_wgrad_can_update(a)) {
     dim3 vgrid((a.K / 4 + kWvCols - 1) / kWvCols, a.m), vblock(kWvCols, kWvSlices);
     if (a.C <= 10) {
-      if (f32) err = launch_chained(head_wgrad_vec_kernel<float, 10>, vgrid, vblock, 0, s, a, g, loss);
-      else err = launch_chained(head_wgrad_vec_kernel<__nv_bfloat16, 10>, vgrid, vblock, 0, s, a, g, loss);
+      if (f32) err = launch_chained(head_wgrad_vec_kernel<float, 10>, vgrid, vblock, 0, s, a, g, loss, up);
+      else err = launch_chained(head_wgrad_vec_kernel<__nv_bfloat16, 10>, vgrid, vblock, 0, s, a, g, loss, up);
     } else {
-      if (f32) err = launch_chained(head_wgrad_vec_kernel<float, 16>, vgrid, vblock, 0, s, a, g, loss);
-      else err = launch_chained(head_wgrad_vec_kernel<__nv_bfloat16, 16>, vgrid, vblock, 0, s, a, g, loss);
+      if (f32) err = launch_chained(head_wgrad_vec_kernel<float, 16>, vgrid, vblock, 0, s, a, g, loss, up);
+      else err = launch_chained(head_wgrad_vec_kernel<__nv_bfloat16, 16>, vgrid, vblock, 0, s, a, g, loss, up);
     }
     return err;
   }

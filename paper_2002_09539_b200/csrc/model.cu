@@ -146,6 +146,14 @@ bool bind_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, const Mod
   for (int p = 0; p < L - 1; ++p)
     mb->fused_layer[p] = spec.gemm_bf16 == 1 && spec.dims[p + 1] % 128 == 0 &&
                          spec.dims[p] % 128 == 0 && hp.batch % 64 == 0 && hp.batch <= 128;
+  {
+    HeadArgs probe{};
+    probe.K = spec.dims[L - 1];
+    probe.C = spec.dims[L];
+    probe.w_off = mb->w_off[L - 1];
+    probe.ld = 4;   // every row pitch the context uses is a multiple of 64 floats
+    mb->fused_head = spec.gemm_bf16 == 1 && head_wgrad_can_update(probe);
+  }
   int64_t start = 0;
   mb->n_ranges = 0;
   auto close_range = [&](int64_t end) {
@@ -155,10 +163,12 @@ bool bind_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, const Mod
       mb->n_ranges++;
     }
   };
-  for (int p = 0; p < L - 1; ++p) {
-    if (mb->fused_layer[p]) {
+  // what is left for the update kernel: the layers that no weight-gradient kernel updates
+  for (int p = 0; p < L; ++p) {
+    const bool in_kernel = p < L - 1 ? mb->fused_layer[p] : mb->fused_head;
+    if (in_kernel) {
       close_range(mb->w_off[p]);
-      start = mb->b_off[p];
+      start = mb->b_off[p] + spec.dims[p + 1];
     }
   }
   close_range(P);
@@ -245,13 +255,22 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
     Scope sc(hook, OLSGD_KC_LOSS, s);
     OLSGD_TRY(launch_head_forward(ha, s));
   }
+  // From here on kernels may write x_{k+1} and, on sync steps, read the anchor: the anchor
+  // refresh of the previous period must have finished.
+  bool waited = false;
+  const bool head_updates = io.upd.enabled && mb.fused_head;
+  if (head_updates && io.wait_before_update) {
+    OLSGD_TRY(cudaStreamWaitEvent(s, io.wait_before_update, 0));
+    waited = true;
+  }
   {
+    FusedUpdateArgs hu = io.upd;
+    hu.b_off = -1;
     Scope sc(hook, OLSGD_KC_BACKWARD, s);
-    OLSGD_TRY(launch_head_wgrad(ha, io.g, loss, s));
+    OLSGD_TRY(launch_head_wgrad(ha, io.g, loss, head_updates ? &hu : nullptr, s));
   }
 
   // hidden layers, backward
-  bool waited = false;
   for (int l = L - 1; l >= 1; --l) {
     if (l >= 2) {
       // dA_{l-1}^T [d_{l-1}][B] = (W_l^T [d_{l-1}][d_l] * dA_l [B][d_l]^T) .* (H_{l-1}^T > 0).
@@ -298,10 +317,11 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
       // the update of W_l happens in this GEMM's epilogue: no gradient is stored
       gw.upd = io.upd;
       gw.upd.w_off = mb.w_off[l - 1];
+      gw.upd.b_off = mb.b_off[l - 1];   // and of its bias, from the row sums of dA_l^T
     }
     // the tensor-core weight-gradient kernel also adds up the rows of dA_l^T: the bias gradient
     const bool rowsum_in_gemm = tensor_path(spec) && wgrad_tc_supported(gw);
-    if (rowsum_in_gemm) {
+    if (rowsum_in_gemm && !fused) {
       gw.rowsum_out = io.g + mb.b_off[l - 1];
       gw.rowsum_batch = io.ld;
     }
@@ -321,6 +341,8 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
       OLSGD_TRY(launch_bias_grad(mb.dat[l], io.g, io.ld, mb.b_off[l - 1], m, spec.dims[l], B, s));
     }
   }
+  // no kernel above took the update: the update kernel that follows needs the same ordering
+  if (io.wait_before_update && !waited) OLSGD_TRY(cudaStreamWaitEvent(s, io.wait_before_update, 0));
   return cudaSuccess;
 }
 

@@ -166,7 +166,12 @@ cudaError_t launch_head_forward(const HeadArgs& a, cudaStream_t s);
 // Output layer weight/bias gradient and the mean loss:
 //   g[i][w_off + c*K + j] = sum_b dlogits[i][b][c] * in[i][b][j];  g[i][b_off + c] = sum_b dlogits
 //   loss[i] = mean_b rowloss[i][b]   (loss may be null)
-cudaError_t launch_head_wgrad(const HeadArgs& a, float* g, float* loss, cudaStream_t s);
+// With upd non-null and upd->enabled (only where head_wgrad_can_update says so) the gradient
+// is not stored: the kernel applies Eq. 3 / Eq. 4 to the layer's weights and bias on the spot.
+struct FusedUpdateArgs;
+bool head_wgrad_can_update(const HeadArgs& a);
+cudaError_t launch_head_wgrad(const HeadArgs& a, float* g, float* loss, const FusedUpdateArgs* upd,
+                              cudaStream_t s);
 
 // g[i][b_off + r] = sum_c dat[i][r][c]   (bias gradient of a hidden layer from dA^T [m][R][B])
 cudaError_t launch_bias_grad(const __nv_bfloat16* dat, float* g, int64_t ld, int64_t b_off, int m,
@@ -199,6 +204,10 @@ struct FusedUpdateArgs {
   int64_t ld, w_off;
   float gamma, mu, alpha;
   int sync;
+  // weight-gradient GEMM only: >= 0 makes the kernel update the layer's bias (parameters
+  // b_off .. b_off + Ma - 1 of every worker row) from the row sums it forms, instead of
+  // storing them as a gradient
+  int64_t b_off;
 };
 struct GemmArgs {
   const __nv_bfloat16* A;
@@ -254,8 +263,10 @@ struct ModelBuffers {
   __nv_bfloat16* da[OLSGD_MAX_DIMS] = {nullptr};
   __nv_bfloat16* dat[OLSGD_MAX_DIMS] = {nullptr};
   int64_t w_off[OLSGD_MAX_DIMS] = {0}, b_off[OLSGD_MAX_DIMS] = {0};
-  // weights of parameter layer p are updated inside their weight-gradient GEMM
+  // weights and bias of parameter layer p are updated inside their weight-gradient kernel
   bool fused_layer[OLSGD_MAX_DIMS] = {false};
+  // the output layer's weights and bias are updated inside its weight-gradient kernel
+  bool fused_head = false;
   // what is left for the stand-alone update kernel: ranges [off, off + len) of a worker row
   int n_ranges = 0;
   int64_t range_off[OLSGD_MAX_DIMS + 1] = {0}, range_len[OLSGD_MAX_DIMS + 1] = {0};

@@ -51,6 +51,7 @@ struct WgradUpd {
   const float* z;
   __nv_bfloat16* shadow;
   int64_t ld, w_off;
+  int64_t b_off;   // >= 0: the row-sum warp updates the layer's bias instead of storing its gradient
   float gamma, mu, alpha;
   int mom, sync;
 };
@@ -179,7 +180,8 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   constexpr int kRowsumWarp = FUSED ? 10 : 6;
   if (warp == kRowsumWarp) {
     // ---------------- row sums of the resident A operand (the layer's bias gradient)
-    if (rowsum && my_first == 0 && n_units > 0 &&
+    const bool bias_update = FUSED && up.b_off >= 0;
+    if ((rowsum || bias_update) && my_first == 0 && n_units > 0 &&
         mbar_wait(smem_u32(&ctl->a_full), 0u, abort_flag)) {
       const int worker = my_slab / m_tiles, m0 = (my_slab - worker * m_tiles) * kBM;
       float* dst = rowsum + (int64_t)worker * rowsum_batch + m0;
@@ -209,7 +211,19 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         for (int o = 16; o > 0; o >>= 1)
 #pragma unroll
           for (int l = 0; l < o; ++l) part[l] += part[l + o];
-        dst[row] = part[0];
+        if (bias_update) {
+          // Eq. 3 / Eq. 4 for bias entry m0 + row of this worker, with the arithmetic of the
+          // update kernel
+          const int64_t e = up.b_off + m0 + row, o = (int64_t)worker * up.ld + e;
+          float x = up.x_in[o], u = up.mom ? up.u[o] : 0.f;
+          update_scalar_rt(x, u, part[0], up.sync ? up.z[e] : 0.f, up.gamma, up.mu, up.alpha,
+                           up.mom != 0, up.sync != 0);
+          up.x_out[o] = x;
+          if (up.mom) up.u[o] = u;
+          up.shadow[o] = __float2bfloat16_rn(x);
+        } else {
+          dst[row] = part[0];
+        }
       }
     }
   } else if (warp == 0 && lane == 0) {
@@ -513,6 +527,9 @@ cudaError_t launch_wgrad_tc(const GemmArgs& a, cudaStream_t s) {
     up.alpha = a.upd.alpha;
     up.mom = (a.upd.u != nullptr && a.upd.mu != 0.f) ? 1 : 0;
     up.sync = a.upd.sync;
+    up.b_off = a.upd.b_off;
+  } else {
+    up.b_off = -1;
   }
   if (fused)
     return launch_chained(wgrad_tc_kernel<true>, dim3(ctas), dim3(kFusedThreads), smem, s, ma, mb, mo,

@@ -33,6 +33,19 @@ __device__ __forceinline__ void update4(float4& x, float4& u, const float4& g, c
   update_scalar<MOM, SYNC>(x.w, u.w, g.w, z.w, gamma, mu, alpha);
 }
 
+// The same arithmetic with the two switches taken at run time (kernels in which the update is
+// a small tail, not the main loop).
+__device__ __forceinline__ void update_scalar_rt(float& x, float& u, float g, float z, float gamma,
+                                                 float mu, float alpha, bool mom, bool sync) {
+  if (mom) {
+    if (sync) update_scalar<true, true>(x, u, g, z, gamma, mu, alpha);
+    else update_scalar<true, false>(x, u, g, z, gamma, mu, alpha);
+  } else {
+    if (sync) update_scalar<false, true>(x, u, g, z, gamma, mu, alpha);
+    else update_scalar<false, false>(x, u, g, z, gamma, mu, alpha);
+  }
+}
+
 // four floats -> four bf16 (round to nearest even), packed in 8 bytes
 __device__ __forceinline__ uint2 pack_bf16x4(const float4& v) {
   __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
