@@ -204,7 +204,7 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
     Scope sc(hook, OLSGD_KC_GATHER, s);
     OLSGD_TRY(launch_gather(X, static_cast<const int32_t*>(data.y), io.idx, bf ? nullptr : mb.xb32,
                             bf ? mb.xb16 : nullptr, bf ? mb.xb16t : nullptr, mb.yb, m, B, n, d0,
-                            s));
+                            io.rule, s));
   }
 
   // hidden layers, forward: H_l^T [d_l][B] = relu(W_l [d_l][d_{l-1}] * H_{l-1} [B][d_{l-1}]^T + b)
@@ -263,11 +263,28 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
     OLSGD_TRY(cudaStreamWaitEvent(s, io.wait_before_update, 0));
     waited = true;
   }
+  // The output layer's weight gradient (and update) depends only on the output-layer forward
+  // kernel, and nothing before the end of the backward pass depends on it: with hidden layers
+  // it runs on the second stream, beside the input-gradient and weight-gradient GEMMs.
+  const bool beside = io.aux != nullptr && L >= 2;
   {
     FusedUpdateArgs hu = io.upd;
     hu.b_off = -1;
-    Scope sc(hook, OLSGD_KC_BACKWARD, s);
-    OLSGD_TRY(launch_head_wgrad(ha, io.g, loss, head_updates ? &hu : nullptr, s));
+    cudaStream_t hs = s;
+    if (beside) {
+      OLSGD_TRY(cudaEventRecord(io.aux_fork, s));
+      OLSGD_TRY(cudaStreamWaitEvent(io.aux, io.aux_fork, 0));
+      hs = io.aux;
+      g_launch_plain = true;
+    }
+    cudaError_t he;
+    {
+      Scope sc(hook, OLSGD_KC_BACKWARD, hs);
+      he = launch_head_wgrad(ha, io.g, loss, head_updates ? &hu : nullptr, hs);
+    }
+    g_launch_plain = false;
+    OLSGD_TRY(he);
+    if (beside) OLSGD_TRY(cudaEventRecord(io.aux_join, io.aux));
   }
 
   // hidden layers, backward
@@ -341,6 +358,7 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
       OLSGD_TRY(launch_bias_grad(mb.dat[l], io.g, io.ld, mb.b_off[l - 1], m, spec.dims[l], B, s));
     }
   }
+  if (beside) OLSGD_TRY(cudaStreamWaitEvent(s, io.aux_join, 0));
   // no kernel above took the update: the update kernel that follows needs the same ordering
   if (io.wait_before_update && !waited) OLSGD_TRY(cudaStreamWaitEvent(s, io.wait_before_update, 0));
   return cudaSuccess;

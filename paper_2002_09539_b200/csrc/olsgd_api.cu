@@ -52,6 +52,8 @@ struct olsgd_ctx {
 
   cudaStream_t main = nullptr, side = nullptr;
   cudaStream_t copy = nullptr;       // owned: host-to-device staging copies
+  cudaStream_t aux = nullptr;        // owned: backward-pass work beside the critical path
+  cudaEvent_t aux_fork = nullptr, aux_join = nullptr;
   cudaEvent_t pullback_done = nullptr, reduce_done = nullptr;
   cudaEvent_t h2d_done[2] = {nullptr, nullptr}, stage_free[2] = {nullptr, nullptr};
   int host_slot = 0;
@@ -151,6 +153,9 @@ void free_host_side(olsgd_ctx* c) {
     if (c->stage_free[b]) cudaEventDestroy(c->stage_free[b]);
   }
   if (c->copy) cudaStreamDestroy(c->copy);
+  if (c->aux_fork) cudaEventDestroy(c->aux_fork);
+  if (c->aux_join) cudaEventDestroy(c->aux_join);
+  if (c->aux) cudaStreamDestroy(c->aux);
   if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
   delete c;
 }
@@ -365,10 +370,12 @@ cudaError_t draw_indices(olsgd_ctx* c, int64_t k) {
 
 // S2-S6 of one iteration on the main stream, reading the minibatch rows
 // idx[i][:] of `data`.  stage_slot >= 0 marks a host-fed staging slot to release.
-olsgd_status step_body(olsgd_ctx* c, const olsgd_data& data, const int32_t* idx,
-                       float* loss_device, int stage_slot, const __nv_bfloat16* xb16_in = nullptr) {
+olsgd_status step_body(olsgd_ctx* c, const olsgd_data& data, int32_t* idx,
+                       float* loss_device, int stage_slot, const __nv_bfloat16* xb16_in = nullptr,
+                       const IndexRule* rule = nullptr) {
   StepIO io;
   io.xb16_in = xb16_in;
+  io.rule = rule;
   io.x = c->x[c->cur];
   io.shadow = c->shadow;
   io.g = c->g;
@@ -378,6 +385,12 @@ olsgd_status step_body(olsgd_ctx* c, const olsgd_data& data, const int32_t* idx,
   io.status = c->dev_status;
   memset(&io.upd, 0, sizeof io.upd);
   io.wait_before_update = nullptr;
+  // with the two streams of the context serialised (side == main) nothing runs beside the
+  // main stream either
+  const bool beside = c->aux != nullptr && c->side != c->main;
+  io.aux = beside ? c->aux : nullptr;
+  io.aux_fork = c->aux_fork;
+  io.aux_join = c->aux_join;
   if (c->spec.kind == OLSGD_MLP && c->spec.gemm_bf16 == 1) {
     const bool sync = (c->k + 1) % c->hp.tau == 0 && c->hp.mode == OLSGD_MODE_OVERLAP;
     const int nxt = 1 - c->cur;
@@ -432,6 +445,7 @@ olsgd_status check_device_status(olsgd_ctx* c) {
 namespace olsgd {
 void set_thread_error(const char* text) { g_last_error = text ? text : ""; }
 int g_launch_overlap = 1;
+thread_local bool g_launch_plain = false;
 }  // namespace olsgd
 
 extern "C" {
@@ -520,6 +534,9 @@ olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const ols
   OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->reduce_done, cudaEventDisableTiming));
   if (pl.has_g) {
     OLSGD_INIT_CUDA(cudaStreamCreateWithFlags(&c->copy, cudaStreamNonBlocking));
+    OLSGD_INIT_CUDA(cudaStreamCreateWithFlags(&c->aux, cudaStreamNonBlocking));
+    OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->aux_fork, cudaEventDisableTiming));
+    OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->aux_join, cudaEventDisableTiming));
     for (int b = 0; b < 2; ++b) {
       OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->h2d_done[b], cudaEventDisableTiming));
       OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->stage_free[b], cudaEventDisableTiming));
@@ -571,7 +588,20 @@ olsgd_status olsgd_local_step(olsgd_ctx* c, float* loss_device) {
   if (c->spec.kind == OLSGD_FLAT)
     return fail(c, OLSGD_ESTATE, "OLSGD_FLAT contexts take olsgd_local_step_with_grads");
   if (c->need_sync) return fail(c, OLSGD_ESTATE, "a period ended: call olsgd_period_sync first");
-  // S1: minibatch indices xi_k^(i)
+  // S1: minibatch indices xi_k^(i).  Where the minibatch is staged by the gather kernel and
+  // the rule is the with-replacement one, that kernel draws them itself.
+  const bool staged = c->spec.kind == OLSGD_MLP && c->spec.gemm_bf16 != 0;
+  if (staged && c->hp.sampling == 0 && gather_draws_indices(c->hp.batch, c->spec.dims[0])) {
+    IndexRule rule;
+    rule.key0 = (uint32_t)(c->hp.seed & 0xFFFFFFFFu);
+    rule.key1 = (uint32_t)(c->hp.seed >> 32);
+    // while a graph is being captured: the offset inside the block, added on the device to
+    // the block's first iteration
+    rule.k_base = (uint64_t)(c->capturing ? c->k - c->capture_k0 : c->k);
+    rule.k_ptr = c->capturing ? reinterpret_cast<const long long*>(c->dev_k) : nullptr;
+    rule.worker_offset = (uint32_t)c->hp.worker_offset;
+    return step_body(c, c->data, c->idx, loss_device, -1, nullptr, &rule);
+  }
   {
     Launch l(c, OLSGD_KC_INDEX, c->main);
     OLSGD_CUDA(c, draw_indices(c, c->k));
@@ -644,6 +674,7 @@ olsgd_status olsgd_clear_status(olsgd_ctx* c) {
 olsgd_status olsgd_join(olsgd_ctx* c) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
   if (c->copy) OLSGD_CUDA(c, cudaStreamSynchronize(c->copy));
+  if (c->aux) OLSGD_CUDA(c, cudaStreamSynchronize(c->aux));
   OLSGD_CUDA(c, cudaStreamSynchronize(c->side));
   OLSGD_CUDA(c, cudaStreamSynchronize(c->main));
   c->reduce_pending = false;

@@ -19,6 +19,9 @@ namespace olsgd {
 // kernel after this one start its own launch.  A kernel launched the ordinary way passes
 // through the gate at once.
 extern int g_launch_overlap;   // olsgd_set_launch_overlap
+// Set around a launch that goes to a stream whose previous operation is an event wait, not a
+// kernel: such a launch is an ordinary one (its kernel passes the gate at once).
+extern thread_local bool g_launch_plain;
 
 #ifdef __CUDACC__
 __device__ __forceinline__ void launch_gate() {
@@ -38,7 +41,7 @@ cudaError_t launch_chained(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = g_launch_overlap ? 1 : 0;
+  cfg.numAttrs = (g_launch_overlap && !g_launch_plain) ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 #endif
@@ -130,9 +133,19 @@ cudaError_t launch_linreg(const float* X, const float* y, const int32_t* idx, co
 // y[m][batch] -> yb (d % 64 == 0, batch % 8 == 0)
 cudaError_t launch_transpose_bf16(const __nv_bfloat16* xb16, const int32_t* y, __nv_bfloat16* xb16t,
                                   int32_t* yb, int m, int batch, int d, cudaStream_t s);
-cudaError_t launch_gather(const float* X, const int32_t* y, const int32_t* idx, float* xb32,
+// With `rule` non-null (only where gather_draws_indices says so) the kernel draws the
+// with-replacement minibatch indices of iteration k itself (and stores them to idx) instead
+// of reading idx.
+struct IndexRule {
+  uint32_t key0, key1;        // seed, low and high word
+  uint64_t k_base;            // iteration number, or its offset from *k_ptr
+  const long long* k_ptr;     // device-resident iteration number of a captured graph, or null
+  uint32_t worker_offset;     // global id of local worker 0
+};
+bool gather_draws_indices(int batch, int d);
+cudaError_t launch_gather(const float* X, const int32_t* y, int32_t* idx, float* xb32,
                           __nv_bfloat16* xb16, __nv_bfloat16* xb16t, int32_t* yb, int m, int batch,
-                          int64_t n, int d, cudaStream_t s);
+                          int64_t n, int d, const IndexRule* rule, cudaStream_t s);
 
 // Output layer, forward + loss + backward to its input, one warp per batch row.
 //   in32 / in16   the layer's input [m][B][K], exactly one non-null
@@ -276,13 +289,18 @@ struct StepIO {
   const __nv_bfloat16* shadow;   // bf16 copy of x_k or null
   float* g;                      // out: [m][ld]
   int64_t ld;
-  const int32_t* idx;            // [m][batch]
+  int32_t* idx;                  // [m][batch]
+  const IndexRule* rule;         // if non-null, idx is an output: the gather draws the indices
   const __nv_bfloat16* xb16_in;  // if non-null: this step's rows, already bf16, [m][batch][dims[0]]
                                  // (data.y then holds their labels [m][batch]); idx is unused
   float* loss;                   // out: [m] or null
   int* status;                   // device status word (see GemmArgs::status)
   FusedUpdateArgs upd;           // state pointers and factors for the fused epilogue (w_off unset)
   cudaEvent_t wait_before_update;  // if non-null, the stream waits for it before x_out is written
+  // Optional second stream (with two events) for work that does not lie on the critical
+  // path of the backward pass; null: everything runs on the main stream.
+  cudaStream_t aux;
+  cudaEvent_t aux_fork, aux_join;
 };
 // Lets model.cu count and time its launches without knowing the context type.
 struct ProfHook {

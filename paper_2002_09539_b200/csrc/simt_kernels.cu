@@ -4,6 +4,7 @@
 // Every reduction runs in a fixed order (no floating-point atomics), so a step
 // is reproducible bit for bit from run to run.
 #include "olsgd_internal.h"
+#include "philox.cuh"
 
 namespace olsgd {
 namespace {
@@ -82,9 +83,9 @@ constexpr int kGvRows = 32, kGvCols = 128;
 
 __global__ void __launch_bounds__(256)
 gather_vec_kernel(const float* __restrict__ X, const int32_t* __restrict__ y,
-                  const int32_t* __restrict__ idx, float* __restrict__ xb32,
+                  int32_t* __restrict__ idx, float* __restrict__ xb32,
                   __nv_bfloat16* __restrict__ xb16, __nv_bfloat16* __restrict__ xb16t,
-                  int32_t* __restrict__ yb, int batch, int64_t n, int d) {
+                  int32_t* __restrict__ yb, int batch, int64_t n, int d, bool draw, IndexRule rule) {
   launch_gate();
   __shared__ __align__(16) __nv_bfloat16 tile[kGvRows][kGvCols + 8];
   __shared__ int32_t rows[kGvRows];
@@ -92,9 +93,19 @@ gather_vec_kernel(const float* __restrict__ X, const int32_t* __restrict__ y,
   const int b0 = blockIdx.y * kGvRows, j0 = blockIdx.x * kGvCols;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x < kGvRows) {
-    const int32_t r = idx[(int64_t)i * batch + b0 + threadIdx.x];
+    const int64_t slot = (int64_t)i * batch + b0 + threadIdx.x;
+    int32_t r;
+    if (draw) {
+      // S1 inside S2: the row of slot b0 + tid by the with-replacement index rule
+      const uint32_t k = (uint32_t)(rule.k_base + (rule.k_ptr ? (uint64_t)*rule.k_ptr : 0ull));
+      r = minibatch_index(rule.key0, rule.key1, k, (uint32_t)i + rule.worker_offset,
+                          b0 + (int)threadIdx.x, (uint32_t)n);
+      if (blockIdx.x == 0) idx[slot] = r;
+    } else {
+      r = idx[slot];
+    }
     rows[threadIdx.x] = r;
-    if (blockIdx.x == 0) yb[(int64_t)i * batch + b0 + threadIdx.x] = y[(int64_t)i * n + r];
+    if (blockIdx.x == 0) yb[slot] = y[(int64_t)i * n + r];
   }
   __syncthreads();
 #pragma unroll
@@ -271,13 +282,16 @@ cudaError_t launch_cast_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cu
   return cudaGetLastError();
 }
 
-cudaError_t launch_gather(const float* X, const int32_t* y, const int32_t* idx, float* xb32,
+bool gather_draws_indices(int batch, int d) { return d % kGvCols == 0 && batch % kGvRows == 0; }
+
+cudaError_t launch_gather(const float* X, const int32_t* y, int32_t* idx, float* xb32,
                           __nv_bfloat16* xb16, __nv_bfloat16* xb16t, int32_t* yb, int m, int batch,
-                          int64_t n, int d, cudaStream_t s) {
-  if (d % kGvCols == 0 && batch % kGvRows == 0) {
+                          int64_t n, int d, const IndexRule* rule, cudaStream_t s) {
+  if (rule && !gather_draws_indices(batch, d)) return cudaErrorInvalidValue;
+  if (gather_draws_indices(batch, d)) {
     dim3 grid(d / kGvCols, batch / kGvRows, m);
     return launch_chained(gather_vec_kernel, grid, dim3(256), 0, s, X, y, idx, xb32, xb16, xb16t, yb,
-                          batch, n, d);
+                          batch, n, d, rule != nullptr, rule ? *rule : IndexRule{});
   }
   dim3 grid((d + kGatherCols - 1) / kGatherCols, (batch + kGatherRows - 1) / kGatherRows, m);
   dim3 block(kGatherCols, 4);
