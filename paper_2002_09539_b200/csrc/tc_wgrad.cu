@@ -497,12 +497,14 @@ cudaError_t launch_wgrad_tc(const GemmArgs& a, cudaStream_t s) {
   if (n_stages > kWStages) n_stages = kWStages;
   if (n_stages < 2 || fused) n_stages = 2;
   const size_t smem = fixed + (size_t)n_stages * kWN * kBK * 2 + (fused ? 8 * kXuPerWarp : 0);
-  // `chunks` CTAs per slab, about four CTAs per SM in total (measured: the count hardly
-  // matters, the alignment to slabs and the joint sweep do)
+  // `chunks` CTAs share a slab and take its column tiles round-robin: about three tiles per
+  // CTA.  Measured on 16 workers x (1024 x 3072) and x (1024 x 1024), and on 64 workers x
+  // (512 x 3072): with fewer CTAs per slab the joint sweep over adjacent column tiles gets
+  // narrower and the last partial wave of CTAs weighs more; with one or two tiles per CTA its
+  // set-up (A slab, barriers, tensor memory) is no longer amortised.
   const int slabs = m_tiles * a.m;
-  int chunks = (4 * 148) / slabs;
+  int chunks = n_tiles / 3;
   if (chunks < 1) chunks = 1;
-  if (chunks > n_tiles) chunks = n_tiles;
   const int ctas = slabs * chunks;
   static size_t configured[2] = {0, 0};
   if (smem > configured[fused]) {
