@@ -56,7 +56,7 @@ bool plan_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, ModelPlan
   }
   const int L = n_layers(spec);
   const size_t d0 = spec.dims[0], C = spec.dims[L];
-  mp->off_yb = take(m * B * sizeof(int32_t));
+  mp->off_yb[0] = mp->off_yb[1] = take(m * B * sizeof(int32_t));
   mp->off_dlogits = take(m * B * C * sizeof(float));
   mp->off_rowloss = take(m * B * sizeof(float));
   if (!bf16_path(spec)) {
@@ -93,8 +93,11 @@ bool plan_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, ModelPlan
     return false;
   }
   const size_t e = sizeof(__nv_bfloat16);
-  mp->off_xb16 = take(m * B * d0 * e);
-  mp->off_xb16t = take(m * B * d0 * e);
+  mp->off_yb[1] = take(m * B * sizeof(int32_t));
+  for (int b = 0; b < 2; ++b) {
+    mp->off_xb16[b] = take(m * B * d0 * e);
+    mp->off_xb16t[b] = take(m * B * d0 * e);
+  }
   for (int l = 1; l < L; ++l) {
     const size_t w = spec.dims[l];
     mp->off_h[l] = take(m * B * w * e);
@@ -123,7 +126,7 @@ bool bind_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, const Mod
     mb->b_off[l] = off;
     off += spec.dims[l + 1];
   }
-  mb->yb = reinterpret_cast<int32_t*>(base + mp.off_yb);
+  for (int b = 0; b < 2; ++b) mb->yb[b] = reinterpret_cast<int32_t*>(base + mp.off_yb[b]);
   mb->dlogits = reinterpret_cast<float*>(base + mp.off_dlogits);
   mb->rowloss = reinterpret_cast<float*>(base + mp.off_rowloss);
   mb->range_len[0] = off;
@@ -132,8 +135,10 @@ bool bind_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, const Mod
     return true;
   }
   auto bp = [&](size_t o) { return reinterpret_cast<__nv_bfloat16*>(base + o); };
-  mb->xb16 = bp(mp.off_xb16);
-  mb->xb16t = bp(mp.off_xb16t);
+  for (int b = 0; b < 2; ++b) {
+    mb->xb16[b] = bp(mp.off_xb16[b]);
+    mb->xb16t[b] = bp(mp.off_xb16t[b]);
+  }
   for (int l = 1; l < L; ++l) {
     mb->h[l] = bp(mp.off_h[l]);
     mb->ht[l] = bp(mp.off_ht[l]);
@@ -196,15 +201,18 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
   // the two output-layer kernels); every other model stages the minibatch
   const bool fused_gather = !bf && L == 1;
   const bool rows_in_bf16 = bf && io.xb16_in != nullptr;
+  const int set = bf ? io.batch_set : 0;
   if (rows_in_bf16) {
     Scope sc(hook, OLSGD_KC_GATHER, s);
-    OLSGD_TRY(launch_transpose_bf16(io.xb16_in, static_cast<const int32_t*>(data.y), mb.xb16t, mb.yb,
-                                    m, B, d0, s));
+    OLSGD_TRY(launch_transpose_bf16(io.xb16_in, static_cast<const int32_t*>(data.y), mb.xb16t[set],
+                                    mb.yb[set], m, B, d0, s));
+  } else if (bf && io.batch_staged) {
+    // the rows of this iteration were staged ahead of time (model_stage_batch)
   } else if (!fused_gather) {
     Scope sc(hook, OLSGD_KC_GATHER, s);
     OLSGD_TRY(launch_gather(X, static_cast<const int32_t*>(data.y), io.idx, bf ? nullptr : mb.xb32,
-                            bf ? mb.xb16 : nullptr, bf ? mb.xb16t : nullptr, mb.yb, m, B, n, d0,
-                            io.rule, s));
+                            bf ? mb.xb16[set] : nullptr, bf ? mb.xb16t[set] : nullptr, mb.yb[set], m,
+                            B, n, d0, io.rule, s));
   }
 
   // hidden layers, forward: H_l^T [d_l][B] = relu(W_l [d_l][d_{l-1}] * H_{l-1} [B][d_{l-1}]^T + b)
@@ -213,7 +221,7 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
     ga.A = io.shadow + mb.w_off[l - 1];
     ga.lda = spec.dims[l - 1];
     ga.a_batch = io.ld;
-    ga.B = (l == 1) ? (rows_in_bf16 ? io.xb16_in : mb.xb16) : mb.h[l - 1];
+    ga.B = (l == 1) ? (rows_in_bf16 ? io.xb16_in : mb.xb16[set]) : mb.h[l - 1];
     ga.ldb = spec.dims[l - 1];
     ga.b_batch = (int64_t)B * spec.dims[l - 1];
     ga.m = m;
@@ -240,7 +248,7 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
   ha.ld = io.ld;
   ha.w_off = mb.w_off[L - 1];
   ha.b_off = mb.b_off[L - 1];
-  ha.yb = mb.yb;
+  ha.yb = mb.yb[set];
   ha.dlogits = mb.dlogits;
   ha.rowloss = mb.rowloss;
   ha.din32 = nullptr;
@@ -318,7 +326,7 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
     gw.A = mb.dat[l];
     gw.lda = B;
     gw.a_batch = (int64_t)spec.dims[l] * B;
-    gw.B = (l == 1) ? mb.xb16t : mb.ht[l - 1];
+    gw.B = (l == 1) ? mb.xb16t[set] : mb.ht[l - 1];
     gw.ldb = B;
     gw.b_batch = (int64_t)spec.dims[l - 1] * B;
     gw.m = m;
@@ -362,6 +370,16 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
   // no kernel above took the update: the update kernel that follows needs the same ordering
   if (io.wait_before_update && !waited) OLSGD_TRY(cudaStreamWaitEvent(s, io.wait_before_update, 0));
   return cudaSuccess;
+}
+
+cudaError_t model_stage_batch(const olsgd_model_spec& spec, const olsgd_hparams& hp,
+                              const olsgd_data& data, const ModelBuffers& mb, int32_t* idx,
+                              const IndexRule& rule, int set, cudaStream_t s, const ProfHook& hook) {
+  if (!bf16_path(spec)) return cudaErrorInvalidValue;
+  Scope sc(hook, OLSGD_KC_GATHER, s);
+  return launch_gather(static_cast<const float*>(data.X), static_cast<const int32_t*>(data.y), idx,
+                       nullptr, mb.xb16[set], mb.xb16t[set], mb.yb[set], hp.m, hp.batch,
+                       data.n_per_worker, spec.dims[0], &rule, s);
 }
 
 cudaError_t model_post_update(const olsgd_model_spec& spec, const olsgd_hparams& hp,

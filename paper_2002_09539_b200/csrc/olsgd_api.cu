@@ -42,6 +42,7 @@ struct olsgd_ctx {
   float* tmp = nullptr;              // [ld] scratch for olsgd_get_params
   __nv_bfloat16* shadow = nullptr;   // bf16 copy of x_k [m][ld] (tensor-core path)
   int32_t* idx = nullptr;            // [m][batch]
+  int32_t* idx_next = nullptr;       // [m][batch], indices of the minibatch staged ahead
   int32_t* ident = nullptr;          // [m][batch], ident[i][j] = j
   int* dev_status = nullptr;         // one word: a kernel's bounded wait gave up
   int64_t* dev_k = nullptr;          // iteration number read by the index kernel inside a graph
@@ -54,6 +55,13 @@ struct olsgd_ctx {
   cudaStream_t copy = nullptr;       // owned: host-to-device staging copies
   cudaStream_t aux = nullptr;        // owned: backward-pass work beside the critical path
   cudaEvent_t aux_fork = nullptr, aux_join = nullptr;
+  // Staging of the next iteration's minibatch beside the current iteration (bf16 path, index
+  // rule with replacement): the rows of iteration pre_k are, or are being, staged into set
+  // pre_k % 2 on stream `pre`; pre_pending: the main stream has not yet waited for pre_done.
+  cudaStream_t pre = nullptr;
+  cudaEvent_t pre_begin = nullptr, pre_done = nullptr;
+  bool pre_pending = false;
+  int64_t pre_k = -1;
   cudaEvent_t pullback_done = nullptr, reduce_done = nullptr;
   cudaEvent_t h2d_done[2] = {nullptr, nullptr}, stage_free[2] = {nullptr, nullptr};
   int host_slot = 0;
@@ -67,6 +75,8 @@ struct olsgd_ctx {
   int graph_block = 0;
   cudaGraphExec_t graph_exec = nullptr;
   int graph_cur = -1;            // c->cur at capture time
+  int graph_kpar = -1;           // parity of k at capture time (selects the staged-minibatch set)
+  bool graph_staged = false;     // the captured block starts from rows staged ahead
   bool graph_off = false;        // capture failed once: stay on the plain path
   bool capturing = false;        // the index kernel reads k from dev_k
   int64_t capture_k0 = 0;        // k at the start of the block being captured
@@ -156,6 +166,9 @@ void free_host_side(olsgd_ctx* c) {
   if (c->aux_fork) cudaEventDestroy(c->aux_fork);
   if (c->aux_join) cudaEventDestroy(c->aux_join);
   if (c->aux) cudaStreamDestroy(c->aux);
+  if (c->pre_begin) cudaEventDestroy(c->pre_begin);
+  if (c->pre_done) cudaEventDestroy(c->pre_done);
+  if (c->pre) cudaStreamDestroy(c->pre);
   if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
   delete c;
 }
@@ -180,7 +193,7 @@ int graph_block_len(int tau) {
 struct Plan {
   int64_t P = 0, ld = 0;
   size_t off_x0 = 0, off_x1 = 0, off_u = 0, off_g = 0, off_z = 0, off_v = 0, off_tmp = 0,
-         off_shadow = 0, off_idx = 0, off_ident = 0, off_status = 0, off_dev_k = 0,
+         off_shadow = 0, off_idx = 0, off_idx_next = 0, off_ident = 0, off_status = 0, off_dev_k = 0,
          off_loss_ring = 0, off_stage_x[2] = {0, 0},
          off_stage_y[2] = {0, 0}, off_model = 0, total = 0;
   bool has_u = false, has_g = false, has_shadow = false;
@@ -273,6 +286,7 @@ olsgd_status make_plan(const olsgd_model_spec* spec, const olsgd_hparams* hp, Pl
   pl->off_loss_ring = take((size_t)graph_block_len(hp->tau) * m * sizeof(float));
   pl->off_shadow = pl->has_shadow ? take((size_t)pl->ld * m * sizeof(__nv_bfloat16)) : 0;
   pl->off_idx = pl->has_g ? take((size_t)m * hp->batch * sizeof(int32_t)) : 0;
+  pl->off_idx_next = pl->has_g ? take((size_t)m * hp->batch * sizeof(int32_t)) : 0;
   if (pl->has_g) {
     pl->off_ident = take((size_t)m * hp->batch * sizeof(int32_t));
     for (int b = 0; b < 2; ++b) {
@@ -372,10 +386,12 @@ cudaError_t draw_indices(olsgd_ctx* c, int64_t k) {
 // idx[i][:] of `data`.  stage_slot >= 0 marks a host-fed staging slot to release.
 olsgd_status step_body(olsgd_ctx* c, const olsgd_data& data, int32_t* idx,
                        float* loss_device, int stage_slot, const __nv_bfloat16* xb16_in = nullptr,
-                       const IndexRule* rule = nullptr) {
+                       const IndexRule* rule = nullptr, bool batch_staged = false) {
   StepIO io;
   io.xb16_in = xb16_in;
   io.rule = rule;
+  io.batch_set = (int)(c->k & 1);
+  io.batch_staged = batch_staged;
   io.x = c->x[c->cur];
   io.shadow = c->shadow;
   io.g = c->g;
@@ -510,6 +526,7 @@ olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const ols
   c->graph_block = graph_block_len(hp->tau);
   c->shadow = pl.has_shadow ? reinterpret_cast<__nv_bfloat16*>(ws + pl.off_shadow) : nullptr;
   c->idx = pl.has_g ? reinterpret_cast<int32_t*>(ws + pl.off_idx) : nullptr;
+  c->idx_next = pl.has_g ? reinterpret_cast<int32_t*>(ws + pl.off_idx_next) : nullptr;
   if (pl.has_g) {
     c->ident = reinterpret_cast<int32_t*>(ws + pl.off_ident);
     for (int b = 0; b < 2; ++b) {
@@ -537,6 +554,14 @@ olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const ols
     OLSGD_INIT_CUDA(cudaStreamCreateWithFlags(&c->aux, cudaStreamNonBlocking));
     OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->aux_fork, cudaEventDisableTiming));
     OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->aux_join, cudaEventDisableTiming));
+    {
+      // staging ahead must not take SMs from the kernels on the critical path
+      int lo = 0, hi = 0;
+      OLSGD_INIT_CUDA(cudaDeviceGetStreamPriorityRange(&lo, &hi));
+      OLSGD_INIT_CUDA(cudaStreamCreateWithPriority(&c->pre, cudaStreamNonBlocking, lo));
+    }
+    OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->pre_begin, cudaEventDisableTiming));
+    OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->pre_done, cudaEventDisableTiming));
     for (int b = 0; b < 2; ++b) {
       OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->h2d_done[b], cudaEventDisableTiming));
       OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->stage_free[b], cudaEventDisableTiming));
@@ -592,15 +617,43 @@ olsgd_status olsgd_local_step(olsgd_ctx* c, float* loss_device) {
   // the rule is the with-replacement one, that kernel draws them itself.
   const bool staged = c->spec.kind == OLSGD_MLP && c->spec.gemm_bf16 != 0;
   if (staged && c->hp.sampling == 0 && gather_draws_indices(c->hp.batch, c->spec.dims[0])) {
-    IndexRule rule;
-    rule.key0 = (uint32_t)(c->hp.seed & 0xFFFFFFFFu);
-    rule.key1 = (uint32_t)(c->hp.seed >> 32);
-    // while a graph is being captured: the offset inside the block, added on the device to
-    // the block's first iteration
-    rule.k_base = (uint64_t)(c->capturing ? c->k - c->capture_k0 : c->k);
-    rule.k_ptr = c->capturing ? reinterpret_cast<const long long*>(c->dev_k) : nullptr;
-    rule.worker_offset = (uint32_t)c->hp.worker_offset;
-    return step_body(c, c->data, c->idx, loss_device, -1, nullptr, &rule);
+    auto rule_for = [&](int64_t k) {
+      IndexRule rule;
+      rule.key0 = (uint32_t)(c->hp.seed & 0xFFFFFFFFu);
+      rule.key1 = (uint32_t)(c->hp.seed >> 32);
+      // while a graph is being captured: the offset inside the block, added on the device to
+      // the block's first iteration
+      rule.k_base = (uint64_t)(c->capturing ? k - c->capture_k0 : k);
+      rule.k_ptr = c->capturing ? reinterpret_cast<const long long*>(c->dev_k) : nullptr;
+      rule.worker_offset = (uint32_t)c->hp.worker_offset;
+      return rule;
+    };
+    // Were this iteration's rows staged beside the previous one?
+    bool have = c->pre_k == c->k;
+    if (c->pre_pending) {
+      // also when they were not: the staging in flight must not outlive its buffers' next use
+      OLSGD_CUDA(c, cudaStreamWaitEvent(c->main, c->pre_done, 0));
+      c->pre_pending = false;
+    }
+    // Stage the rows of iteration k + 1 on the context's own stream while iteration k runs: its
+    // set (k + 1) % 2 was last read by iteration k - 1, which precedes pre_begin on the main
+    // stream.  Not with the two streams of the context serialised.
+    if (c->pre && c->side != c->main) {
+      OLSGD_CUDA(c, cudaEventRecord(c->pre_begin, c->main));
+      OLSGD_CUDA(c, cudaStreamWaitEvent(c->pre, c->pre_begin, 0));
+      const IndexRule next = rule_for(c->k + 1);
+      g_launch_plain = true;
+      const cudaError_t e = model_stage_batch(c->spec, c->hp, c->data, c->mb, c->idx_next, next,
+                                              (int)((c->k + 1) & 1), c->pre, make_hook(c));
+      g_launch_plain = false;
+      if (e != cudaSuccess)
+        return fail(c, OLSGD_ECUDA, "staging the next minibatch failed: %s", cudaGetErrorString(e));
+      OLSGD_CUDA(c, cudaEventRecord(c->pre_done, c->pre));
+      c->pre_pending = true;
+      c->pre_k = c->k + 1;
+    }
+    const IndexRule rule = rule_for(c->k);
+    return step_body(c, c->data, c->idx, loss_device, -1, nullptr, &rule, have);
   }
   {
     Launch l(c, OLSGD_KC_INDEX, c->main);
@@ -620,6 +673,12 @@ static olsgd_status local_step_host_impl(olsgd_ctx* c, const void* Xb_host, cons
     return fail(c, OLSGD_ESTATE, "bf16 minibatches are for models whose GEMM operands are bf16 "
                                  "(OLSGD_MLP with gemm_bf16 != 0)");
   if (c->need_sync) return fail(c, OLSGD_ESTATE, "a period ended: call olsgd_period_sync first");
+  // this step writes the staged-minibatch set of iteration k itself
+  if (c->pre_pending) {
+    OLSGD_CUDA(c, cudaStreamWaitEvent(c->main, c->pre_done, 0));
+    c->pre_pending = false;
+  }
+  if (c->pre_k == c->k) c->pre_k = -1;
   const int slot = c->host_slot;
   c->host_slot ^= 1;
   const size_t rows = (size_t)c->hp.m * c->hp.batch;
@@ -675,6 +734,7 @@ olsgd_status olsgd_join(olsgd_ctx* c) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
   if (c->copy) OLSGD_CUDA(c, cudaStreamSynchronize(c->copy));
   if (c->aux) OLSGD_CUDA(c, cudaStreamSynchronize(c->aux));
+  if (c->pre) OLSGD_CUDA(c, cudaStreamSynchronize(c->pre));
   OLSGD_CUDA(c, cudaStreamSynchronize(c->side));
   OLSGD_CUDA(c, cudaStreamSynchronize(c->main));
   c->reduce_pending = false;
@@ -778,7 +838,7 @@ static bool capture_block(olsgd_ctx* c) {
     cudaGraphExecDestroy(c->graph_exec);
     c->graph_exec = nullptr;
   }
-  const int64_t k0 = c->k, launches0 = c->launches;
+  const int64_t k0 = c->k, launches0 = c->launches, pre_k0 = c->pre_k;
   const int cur0 = c->cur;
   cudaGraph_t graph = nullptr;
   if (cudaStreamBeginCapture(c->main, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
@@ -795,6 +855,10 @@ static bool capture_block(olsgd_ctx* c) {
     ok = cudaStreamWaitEvent(c->main, c->reduce_done, 0) == cudaSuccess;
     c->reduce_pending = false;
   }
+  // the staging of the iteration after the block joins the main stream before the counter
+  // it reads is advanced (and every stream of a capture must rejoin its origin)
+  if (ok && c->pre_pending) ok = cudaStreamWaitEvent(c->main, c->pre_done, 0) == cudaSuccess;
+  c->pre_pending = false;
   if (ok) ok = launch_counter(c->dev_k, 0, c->graph_block, false, c->main) == cudaSuccess;
   c->capturing = false;
   const cudaError_t e = cudaStreamEndCapture(c->main, &graph);
@@ -803,6 +867,7 @@ static bool capture_block(olsgd_ctx* c) {
   c->launches = launches0;
   c->k = k0;
   c->cur = cur0;
+  c->pre_k = pre_k0;
   c->need_sync = false;
   c->reduce_pending = false;
   if (!ok || e != cudaSuccess || !graph) {
@@ -820,6 +885,8 @@ static bool capture_block(olsgd_ctx* c) {
     return false;
   }
   c->graph_cur = cur0;
+  c->graph_kpar = (int)(k0 & 1);
+  c->graph_staged = pre_k0 == k0;
   return true;
 }
 
@@ -854,7 +921,16 @@ olsgd_status olsgd_run(olsgd_ctx* c, int64_t n_iters, float* loss_device) {
     OLSGD_CUDA(c, cudaStreamWaitEvent(c->main, c->reduce_done, 0));
     c->reduce_pending = false;
   }
-  if ((!c->graph_exec || c->graph_cur != c->cur) && !capture_block(c)) return plain(n_iters - t);
+  // a minibatch staged ahead by the plain steps joins the main stream here, outside any
+  // capture: the block starts from "the rows of iteration k are staged" (or from "none are")
+  if (c->pre_pending) {
+    OLSGD_CUDA(c, cudaStreamWaitEvent(c->main, c->pre_done, 0));
+    c->pre_pending = false;
+  }
+  const bool staged_now = c->pre_k == c->k;
+  if ((!c->graph_exec || c->graph_cur != c->cur || c->graph_kpar != (int)(c->k & 1) ||
+       c->graph_staged != staged_now) && !capture_block(c))
+    return plain(n_iters - t);
   {
     Launch l(c, OLSGD_KC_INDEX, c->main);
     OLSGD_CUDA(c, launch_counter(c->dev_k, c->k, 0, true, c->main));
@@ -866,6 +942,7 @@ olsgd_status olsgd_run(olsgd_ctx* c, int64_t n_iters, float* loss_device) {
                                     (size_t)block * c->hp.m * sizeof(float),
                                     cudaMemcpyDeviceToDevice, c->main));
     c->k += block;
+    if (c->graph_staged) c->pre_k = c->k;   // the block's last iteration staged the next rows
     c->graph_replays += 1;
     c->launches += c->graph_launches;
     t += block;
@@ -1037,6 +1114,8 @@ const char* olsgd_last_error(const olsgd_ctx* c) {
 olsgd_status olsgd_destroy(olsgd_ctx* c) {
   if (!c) return OLSGD_OK;
   if (c->copy) cudaStreamSynchronize(c->copy);
+  if (c->aux) cudaStreamSynchronize(c->aux);
+  if (c->pre) cudaStreamSynchronize(c->pre);
   cudaStreamSynchronize(c->side);
   cudaStreamSynchronize(c->main);
   free_host_side(c);

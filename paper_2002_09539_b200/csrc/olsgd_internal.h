@@ -260,16 +260,19 @@ struct ModelPlan {
   size_t bytes = 0;
   char error[160] = {0};
   // offsets inside the model area
-  size_t off_yb = 0, off_xb32 = 0, off_xb16 = 0, off_xb16t = 0, off_dlogits = 0, off_rowloss = 0,
-         off_loss = 0;
+  size_t off_yb[2] = {0, 0}, off_xb32 = 0, off_xb16[2] = {0, 0}, off_xb16t[2] = {0, 0},
+         off_dlogits = 0, off_rowloss = 0, off_loss = 0;
   size_t off_h[OLSGD_MAX_DIMS] = {0}, off_ht[OLSGD_MAX_DIMS] = {0};    // hidden activations
   size_t off_da[OLSGD_MAX_DIMS] = {0}, off_dat[OLSGD_MAX_DIMS] = {0};  // their gradients
 };
 struct ModelBuffers {
   char error[160] = {0};
-  int32_t* yb = nullptr;
+  // The staged minibatch exists twice on the bf16 path (iteration k uses set k % 2), so that
+  // the rows of iteration k + 1 can be staged while iteration k still reads its own; every
+  // other model has one set and both entries point at it.
+  int32_t* yb[2] = {nullptr, nullptr};
   float* xb32 = nullptr;
-  __nv_bfloat16 *xb16 = nullptr, *xb16t = nullptr;
+  __nv_bfloat16 *xb16[2] = {nullptr, nullptr}, *xb16t[2] = {nullptr, nullptr};
   float *dlogits = nullptr, *rowloss = nullptr, *loss = nullptr;
   __nv_bfloat16* h[OLSGD_MAX_DIMS] = {nullptr};
   __nv_bfloat16* ht[OLSGD_MAX_DIMS] = {nullptr};
@@ -293,6 +296,8 @@ struct StepIO {
   const IndexRule* rule;         // if non-null, idx is an output: the gather draws the indices
   const __nv_bfloat16* xb16_in;  // if non-null: this step's rows, already bf16, [m][batch][dims[0]]
                                  // (data.y then holds their labels [m][batch]); idx is unused
+  int batch_set;                 // which staged-minibatch set this iteration uses (0 or 1)
+  bool batch_staged;             // the set already holds this iteration's rows: no gather
   float* loss;                   // out: [m] or null
   int* status;                   // device status word (see GemmArgs::status)
   FusedUpdateArgs upd;           // state pointers and factors for the fused epilogue (w_off unset)
@@ -314,6 +319,11 @@ bool bind_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, const Mod
 cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hparams& hp,
                                    const olsgd_data& data, const ModelBuffers& mb,
                                    const StepIO& io, cudaStream_t s, const ProfHook& hook);
+// S1 + S2 of the bf16 path for one iteration, by themselves: draws the indices by `rule` and
+// stages the rows into set `set` on stream s.
+cudaError_t model_stage_batch(const olsgd_model_spec& spec, const olsgd_hparams& hp,
+                              const olsgd_data& data, const ModelBuffers& mb, int32_t* idx,
+                              const IndexRule& rule, int set, cudaStream_t s, const ProfHook& hook);
 // Work that must follow every parameter update (none at present).
 cudaError_t model_post_update(const olsgd_model_spec& spec, const olsgd_hparams& hp,
                               const ModelBuffers& mb, const __nv_bfloat16* shadow, int64_t ld,
