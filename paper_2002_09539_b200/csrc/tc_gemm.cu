@@ -64,6 +64,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const int n0 = blockIdx.x * BN, m0 = blockIdx.y * kBM, worker = blockIdx.z;
 
   if (threadIdx.x == 0) {
+    prefetch_tensormap(&map_a);
+    prefetch_tensormap(&map_b);
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&ctl->full[s]), 1);
       mbar_init(smem_u32(&ctl->empty[s]), 1);
@@ -138,15 +140,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     umma_commit(smem_u32(&ctl->tmem_full));   // accumulator complete
   } else if (warp >= 2) {
     // ---------------- epilogue: TMEM lane r <-> row m0 + r, column j <-> col n0 + j
+    // what the epilogue needs besides the accumulator is fetched while the main loop runs:
+    // the row's bias, or the first 32 columns of its ReLU mask (the next 32 are fetched
+    // while the current ones are applied)
+    const int lane_group = warp & 3;
+    const int row = m0 + lane_group * 32 + lane;
+    const int64_t wk = worker;
+    float bias = 0.f;
+    if (ea.epilogue == GEMM_EPI_BIAS_RELU) bias = ea.bias[wk * ea.bias_batch + row];
+    uint4 mk[4], mk_next[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) mk[q] = mk_next[q] = make_uint4(0u, 0u, 0u, 0u);
+    const uint4* mask_row = nullptr;
+    if (ea.epilogue == GEMM_EPI_RELU_MASK) {
+      mask_row = reinterpret_cast<const uint4*>(ea.mask + (wk * ea.Ma + row) * ea.Nb + n0);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) mk[q] = mask_row[q];
+    }
     if (mbar_wait(smem_u32(&ctl->tmem_full), 0, abort_flag) && !*abort_flag) {
       tc_fence_after();
-      const int lane_group = warp & 3;
-      const int row = m0 + lane_group * 32 + lane;
-      const int64_t wk = worker;
-      float bias = 0.f;
-      if (ea.epilogue == GEMM_EPI_BIAS_RELU) bias = ea.bias[wk * ea.bias_batch + row];
 #pragma unroll 1
       for (int c = 0; c < BN / 32; ++c) {
+        if (ea.epilogue == GEMM_EPI_RELU_MASK && c + 1 < BN / 32) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) mk_next[q] = mask_row[(c + 1) * 4 + q];
+        }
         float v[32];
         tmem_ld32(tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)(c * 32), v);
         const int col0 = n0 + c * 32;
@@ -162,7 +180,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j] + bias, 0.f);
           } else {
-            const uint4* mk = reinterpret_cast<const uint4*>(ea.mask + t_off);
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
               const uint4 w = mk[q];
@@ -174,6 +191,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (!(lo != 0 && lo < 0x8000u)) v[q * 8 + e * 2] = 0.f;
                 if (!(hi != 0 && hi < 0x8000u)) v[q * 8 + e * 2 + 1] = 0.f;
               }
+              mk[q] = mk_next[q];
             }
           }
           uint32_t pk[16];
