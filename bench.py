@@ -132,7 +132,7 @@ NCU_TRAFFIC = {
     # (workload, gemm mode, kernel class)
     ("c3", 3, "update"): (1426.4e6, 1445.1e6),      # profiles/fused_update_c3_mlp.txt
     # profiles/wgrad_update_fused_c3_mlp.txt: mean of the two fused layers' launches
-    ("c3", 1, "wgrad_update"): ((256.8e6 + 869.0e6) / 2, (268.8e6 + 923.7e6) / 2),
+    ("c3", 1, "wgrad_update"): ((256.5e6 + 869.6e6) / 2, (262.3e6 + 885.3e6) / 2),
 }
 
 
