@@ -131,8 +131,6 @@ class ClockSampler:
 NCU_TRAFFIC = {
     # (workload, gemm mode, kernel class)
     ("c3", 3, "update"): (1426.4e6, 1445.1e6),      # profiles/fused_update_c3_mlp.txt
-    # profiles/wgrad_update_fused_c3_mlp.txt: mean of the two fused layers' launches
-    ("c3", 1, "wgrad_update"): ((256.5e6 + 869.6e6) / 2, (262.3e6 + 885.3e6) / 2),
 }
 
 
@@ -163,15 +161,15 @@ def algorithmic_bytes(c, kernel_class, P, sync_fraction):
     shadow = 2 if c.get("gemm_bf16") else 0
     fused = fused_weight_count(c)
     if kernel_class == "wgrad_update":
-        # per launch, averaged over the fused layers: x read+write, u read+write, bf16 shadow
-        # write per parameter per worker, the anchor once on sync steps, the bf16 operands once
+        # one launch covers all fused layers: x read+write, u read+write, bf16 shadow write
+        # per parameter per worker, the anchor once on sync steps, the bf16 operands once
         if not fused:
             return None
         d, B = c["dims"], c["batch"]
         layers = [p for p in range(len(d) - 2) if layer_is_fused(c, p)]
         per = (16 if mom else 8) + 2
         operands = sum(m * B * 2 * (d[p + 1] + d[p]) for p in layers)
-        return (m * fused * per + sync_fraction * 4 * fused + operands) / len(layers)
+        return m * fused * per + sync_fraction * 4 * fused + operands
     if kernel_class == "update":
         per = (20 if mom else 12) + shadow
         rest = P - fused

@@ -295,7 +295,23 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
     if (beside) OLSGD_TRY(cudaEventRecord(io.aux_join, io.aux));
   }
 
-  // hidden layers, backward
+  // hidden layers, backward.  The weight-gradient GEMMs that carry their own update are
+  // collected and launched together after the input-gradient chain (they depend on nothing
+  // else in it, and every input-gradient GEMM still reads its layer's bf16 shadow before the
+  // launch that overwrites it).
+  GemmArgs pending[OLSGD_MAX_DIMS];
+  int n_pending = 0;
+  auto flush = [&]() -> cudaError_t {
+    if (n_pending == 0) return cudaSuccess;
+    if (io.wait_before_update && !waited) {
+      OLSGD_TRY(cudaStreamWaitEvent(s, io.wait_before_update, 0));
+      waited = true;
+    }
+    Scope sc(hook, OLSGD_KC_WGRAD_UPDATE, s);
+    const cudaError_t e = launch_wgrad_tc_batch(pending, n_pending, s);
+    n_pending = 0;
+    return e;
+  };
   for (int l = L - 1; l >= 1; --l) {
     if (l >= 2) {
       // dA_{l-1}^T [d_{l-1}][B] = (W_l^T [d_{l-1}][d_l] * dA_l [B][d_l]^T) .* (H_{l-1}^T > 0).
@@ -351,12 +367,9 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
       gw.rowsum_batch = io.ld;
     }
     if (fused) {
-      if (io.wait_before_update && !waited) {
-        OLSGD_TRY(cudaStreamWaitEvent(s, io.wait_before_update, 0));
-        waited = true;
-      }
-      Scope sc(hook, OLSGD_KC_WGRAD_UPDATE, s);
-      OLSGD_TRY(run_gemm(spec, gw, io.status, s));
+      gw.status = io.status;
+      pending[n_pending++] = gw;
+      if (n_pending == wgrad_tc_batch_limit()) OLSGD_TRY(flush());
     } else {
       Scope sc(hook, OLSGD_KC_BACKWARD, s);
       OLSGD_TRY(run_gemm(spec, gw, io.status, s));
@@ -366,6 +379,7 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
       OLSGD_TRY(launch_bias_grad(mb.dat[l], io.g, io.ld, mb.b_off[l - 1], m, spec.dims[l], B, s));
     }
   }
+  OLSGD_TRY(flush());
   if (beside) OLSGD_TRY(cudaStreamWaitEvent(s, io.aux_join, 0));
   // no kernel above took the update: the update kernel that follows needs the same ordering
   if (io.wait_before_update && !waited) OLSGD_TRY(cudaStreamWaitEvent(s, io.wait_before_update, 0));

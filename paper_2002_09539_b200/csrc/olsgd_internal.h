@@ -254,6 +254,10 @@ cudaError_t launch_wait_selftest(int* status, uint64_t limit_ns, cudaStream_t s)
 // K in {64, 128, 192, 256}, epilogue GEMM_EPI_STORE_F32.
 bool wgrad_tc_supported(const GemmArgs& a);
 cudaError_t launch_wgrad_tc(const GemmArgs& a, cudaStream_t s);
+// The same for n <= wgrad_tc_batch_limit() layers in ONE launch (all fused or all plain, same
+// workers, same K, same status word); the layers must not depend on one another.
+int wgrad_tc_batch_limit();
+cudaError_t launch_wgrad_tc_batch(const GemmArgs* args, int n, cudaStream_t s);
 
 // ---- model.cu ------------------------------------------------------------------
 struct ModelPlan {

@@ -32,6 +32,8 @@
 // ... in order and a fixed shuffle tree combines the lanes.
 //
 // Every mbarrier wait is bounded (see tc_common.cuh).
+#include <cstring>
+
 #include "tc_common.cuh"
 #include "update_math.cuh"
 
@@ -123,12 +125,40 @@ constexpr uint32_t kXuPerWarp = 2 * 2 * kXuTile; // two buffers of (x, u)
 constexpr int kFusedThreads = 352;   // TMA, MMA, eight epilogue warps, row sums
 constexpr int kPlainThreads = 224;   // TMA, MMA, four epilogue warps, row sums
 
+// One launch covers the weight-gradient GEMMs of up to kMaxWgradLayers layers (same workers,
+// same K): the CTAs of layer l are blockIdx.x in [cta_begin[l], cta_begin[l + 1]).  The layers
+// do not depend on one another, and in one grid the CTAs of the next layer fill the SMs that
+// the last partial wave of the previous one leaves idle.
+constexpr int kMaxWgradLayers = 4;
+struct WgradLayer {
+  CUtensorMap map_a, map_b, map_out, map_u;
+  WgradUpd up;
+  float* rowsum;
+  int64_t rowsum_batch;
+  int n_tiles, m_tiles, chunks, ldw;
+  int cta_begin;
+};
+struct WgradBatch {
+  WgradLayer layer[kMaxWgradLayers];
+  int n_layers;
+};
+
 template <bool FUSED>
 __global__ void __launch_bounds__(FUSED ? kFusedThreads : kPlainThreads, 1)
-wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_u,
-                int num_kb, int n_stages, int n_tiles, int m_tiles, int chunks, int ldw,
-                WgradUpd up, float* rowsum, int64_t rowsum_batch, int* status) {
+wgrad_tc_kernel(const __grid_constant__ WgradBatch wb, int num_kb, int n_stages, int* status) {
+  int layer_id = 0;
+  for (int l = 1; l < wb.n_layers; ++l)
+    if ((int)blockIdx.x >= wb.layer[l].cta_begin) layer_id = l;
+  const WgradLayer& ly = wb.layer[layer_id];
+  const CUtensorMap& map_a = ly.map_a;
+  const CUtensorMap& map_b = ly.map_b;
+  const CUtensorMap& map_out = ly.map_out;
+  const CUtensorMap& map_u = ly.map_u;
+  const int n_tiles = ly.n_tiles, m_tiles = ly.m_tiles, chunks = ly.chunks, ldw = ly.ldw;
+  const WgradUpd up = ly.up;
+  float* const rowsum = ly.rowsum;
+  const int64_t rowsum_batch = ly.rowsum_batch;
+  const int cta = (int)blockIdx.x - ly.cta_begin;
   constexpr uint32_t kABlock = kBM * kBK * 2;   // one k-block of the A slab, 16 KB
   constexpr uint32_t kBBlock = kWN * kBK * 2;   // one k-block of a B tile, 16 KB
   constexpr uint32_t kEpiBuf = 32 * 32 * 4;     // one 32 x 32 fp32 block, 4 KB
@@ -147,7 +177,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   // this CTA's units: every `chunks`-th tile of one slab, so that the CTAs that share a
   // slab (neighbours in the grid, running at the same time) sweep adjacent column tiles
   // together and touch each DRAM page while it is open
-  const int my_slab = blockIdx.x / chunks, my_first = blockIdx.x - my_slab * chunks;
+  const int my_slab = cta / chunks, my_first = cta - my_slab * chunks;
   const int n_units = (n_tiles - my_first + chunks - 1) / chunks;
   auto unit_of = [&](int j) { return my_slab * n_tiles + my_first + j * chunks; };
 
@@ -470,25 +500,67 @@ bool wgrad_tc_supported(const GemmArgs& a) {
   return true;
 }
 
-cudaError_t launch_wgrad_tc(const GemmArgs& a, cudaStream_t s) {
-  if (!wgrad_tc_supported(a)) return cudaErrorInvalidValue;
-  const bool fused = a.upd.enabled != 0;
-  CUtensorMap ma, mb, mo;
-  if (!make_map(&ma, a.A, a.K, a.Ma, a.m, a.lda, a.a_batch, kBM)) return cudaErrorInvalidValue;
-  if (!make_map(&mb, a.B, a.K, a.Nb, a.m, a.ldb, a.b_batch, kWN)) return cudaErrorInvalidValue;
-  CUtensorMap mu = ma;
-  if (fused) {
-    // map_out covers x_k, map_u the momentum buffer: [m][Ma][Nb] fp32 views of the weight matrix
-    if (!make_map_f32(&mo, a.upd.x_in + a.upd.w_off, a.Nb, a.Ma, a.m, a.Nb, a.upd.ld, 32))
+cudaError_t launch_wgrad_tc_batch(const GemmArgs* args, int n, cudaStream_t s) {
+  if (n < 1 || n > kMaxWgradLayers) return cudaErrorInvalidValue;
+  const bool fused = args[0].upd.enabled != 0;
+  const int num_kb = args[0].K / kBK;
+  WgradBatch wb;
+  memset(&wb, 0, sizeof wb);
+  wb.n_layers = n;
+  int ctas = 0;
+  for (int l = 0; l < n; ++l) {
+    const GemmArgs& a = args[l];
+    if (!wgrad_tc_supported(a) || (a.upd.enabled != 0) != fused || a.K != args[0].K ||
+        a.m != args[0].m || a.status != args[0].status)
       return cudaErrorInvalidValue;
-    if (a.upd.u && a.upd.mu != 0.f &&
-        !make_map_f32(&mu, a.upd.u + a.upd.w_off, a.Nb, a.Ma, a.m, a.Nb, a.upd.ld, 32))
+    WgradLayer& ly = wb.layer[l];
+    if (!make_map(&ly.map_a, a.A, a.K, a.Ma, a.m, a.lda, a.a_batch, kBM)) return cudaErrorInvalidValue;
+    if (!make_map(&ly.map_b, a.B, a.K, a.Nb, a.m, a.ldb, a.b_batch, kWN)) return cudaErrorInvalidValue;
+    ly.map_u = ly.map_a;
+    if (fused) {
+      // map_out covers x_k, map_u the momentum buffer: [m][Ma][Nb] fp32 views of the weight matrix
+      if (!make_map_f32(&ly.map_out, a.upd.x_in + a.upd.w_off, a.Nb, a.Ma, a.m, a.Nb, a.upd.ld, 32))
+        return cudaErrorInvalidValue;
+      if (a.upd.u && a.upd.mu != 0.f &&
+          !make_map_f32(&ly.map_u, a.upd.u + a.upd.w_off, a.Nb, a.Ma, a.m, a.Nb, a.upd.ld, 32))
+        return cudaErrorInvalidValue;
+    } else if (!make_map_f32(&ly.map_out, a.out_f, a.Nb, a.Ma, a.m, a.ldo, a.out_batch, 32)) {
       return cudaErrorInvalidValue;
-  } else if (!make_map_f32(&mo, a.out_f, a.Nb, a.Ma, a.m, a.ldo, a.out_batch, 32)) {
-    return cudaErrorInvalidValue;
+    }
+    ly.n_tiles = a.Nb / kWN;
+    ly.m_tiles = a.Ma / kBM;
+    // `chunks` CTAs share a slab and take its column tiles round-robin: about three tiles per
+    // CTA.  Measured on 16 workers x (1024 x 3072) and x (1024 x 1024), and on 64 workers x
+    // (512 x 3072): with fewer CTAs per slab the joint sweep over adjacent column tiles gets
+    // narrower and the last partial wave of CTAs weighs more; with one or two tiles per CTA its
+    // set-up (A slab, barriers, tensor memory) is no longer amortised.
+    ly.chunks = ly.n_tiles / 3;
+    if (ly.chunks < 1) ly.chunks = 1;
+    ly.ldw = a.Nb;
+    ly.rowsum = a.rowsum_out;
+    ly.rowsum_batch = a.rowsum_batch;
+    ly.cta_begin = ctas;
+    const int64_t mine = (int64_t)ly.m_tiles * a.m * ly.chunks;
+    if (mine + ctas > 0x7FFFFFFF) return cudaErrorInvalidValue;
+    ctas += (int)mine;
+    WgradUpd& up = ly.up;
+    up.b_off = -1;
+    if (fused) {
+      up.x_in = a.upd.x_in;
+      up.x_out = a.upd.x_out;
+      up.u = a.upd.u;
+      up.z = a.upd.z;
+      up.shadow = a.upd.shadow;
+      up.ld = a.upd.ld;
+      up.w_off = a.upd.w_off;
+      up.gamma = a.upd.gamma;
+      up.mu = a.upd.mu;
+      up.alpha = a.upd.alpha;
+      up.mom = (a.upd.u != nullptr && a.upd.mu != 0.f) ? 1 : 0;
+      up.sync = a.upd.sync;
+      up.b_off = a.upd.b_off;
+    }
   }
-  const int num_kb = a.K / kBK;
-  const int n_tiles = a.Nb / kWN, m_tiles = a.Ma / kBM;
   // shared memory: the fused variant fills an SM by itself (x/u tile rings); the plain one
   // takes as many B stages as still let two CTAs share an SM's 227 KB
   const size_t fixed = (size_t)num_kb * kBM * kBK * 2 + 8 * 32 * 32 * 4 + sizeof(WgradCtl) + 1024;
@@ -497,15 +569,6 @@ cudaError_t launch_wgrad_tc(const GemmArgs& a, cudaStream_t s) {
   if (n_stages > kWStages) n_stages = kWStages;
   if (n_stages < 2 || fused) n_stages = 2;
   const size_t smem = fixed + (size_t)n_stages * kWN * kBK * 2 + (fused ? 8 * kXuPerWarp : 0);
-  // `chunks` CTAs share a slab and take its column tiles round-robin: about three tiles per
-  // CTA.  Measured on 16 workers x (1024 x 3072) and x (1024 x 1024), and on 64 workers x
-  // (512 x 3072): with fewer CTAs per slab the joint sweep over adjacent column tiles gets
-  // narrower and the last partial wave of CTAs weighs more; with one or two tiles per CTA its
-  // set-up (A slab, barriers, tensor memory) is no longer amortised.
-  const int slabs = m_tiles * a.m;
-  int chunks = n_tiles / 3;
-  if (chunks < 1) chunks = 1;
-  const int ctas = slabs * chunks;
   static size_t configured[2] = {0, 0};
   if (smem > configured[fused]) {
     cudaError_t e = fused ? cudaFuncSetAttribute(wgrad_tc_kernel<true>,
@@ -515,31 +578,15 @@ cudaError_t launch_wgrad_tc(const GemmArgs& a, cudaStream_t s) {
     if (e != cudaSuccess) return e;
     configured[fused] = smem;
   }
-  WgradUpd up{};
-  if (fused) {
-    up.x_in = a.upd.x_in;
-    up.x_out = a.upd.x_out;
-    up.u = a.upd.u;
-    up.z = a.upd.z;
-    up.shadow = a.upd.shadow;
-    up.ld = a.upd.ld;
-    up.w_off = a.upd.w_off;
-    up.gamma = a.upd.gamma;
-    up.mu = a.upd.mu;
-    up.alpha = a.upd.alpha;
-    up.mom = (a.upd.u != nullptr && a.upd.mu != 0.f) ? 1 : 0;
-    up.sync = a.upd.sync;
-    up.b_off = a.upd.b_off;
-  } else {
-    up.b_off = -1;
-  }
   if (fused)
-    return launch_chained(wgrad_tc_kernel<true>, dim3(ctas), dim3(kFusedThreads), smem, s, ma, mb, mo,
-                          mu, num_kb, n_stages, n_tiles, m_tiles, chunks, a.Nb, up, a.rowsum_out,
-                          a.rowsum_batch, a.status);
-  return launch_chained(wgrad_tc_kernel<false>, dim3(ctas), dim3(kPlainThreads), smem, s, ma, mb, mo,
-                        mu, num_kb, n_stages, n_tiles, m_tiles, chunks, a.Nb, up, a.rowsum_out,
-                        a.rowsum_batch, a.status);
+    return launch_chained(wgrad_tc_kernel<true>, dim3(ctas), dim3(kFusedThreads), smem, s, wb, num_kb,
+                          n_stages, args[0].status);
+  return launch_chained(wgrad_tc_kernel<false>, dim3(ctas), dim3(kPlainThreads), smem, s, wb, num_kb,
+                        n_stages, args[0].status);
 }
+
+cudaError_t launch_wgrad_tc(const GemmArgs& a, cudaStream_t s) { return launch_wgrad_tc_batch(&a, 1, s); }
+
+int wgrad_tc_batch_limit() { return kMaxWgradLayers; }
 
 }  // namespace olsgd
