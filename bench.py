@@ -131,6 +131,7 @@ class ClockSampler:
 NCU_TRAFFIC = {
     # (workload, gemm mode, kernel class)
     ("c3", 3, "update"): (1426.4e6, 1445.1e6),      # profiles/fused_update_c3_mlp.txt
+    ("c3", 1, "wgrad_update"): (1180.1e6, 1203.4e6),  # profiles/wgrad_update_fused_c3_mlp.txt
 }
 
 
