@@ -132,6 +132,15 @@ bool bind_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, const Mod
   mb->range_len[0] = off;
   if (!bf16_path(spec)) {
     mb->xb32 = reinterpret_cast<float*>(base + mp.off_xb32);
+    // softmax regression: where the output-layer weight-gradient kernel can apply the update
+    // itself, nothing is left for the update kernel
+    HeadArgs probe{};
+    probe.K = spec.dims[0];
+    probe.C = spec.dims[1];
+    probe.w_off = 0;
+    probe.ld = 4;
+    mb->fused_head = spec.kind == OLSGD_SOFTMAX && L == 1 && head_wgrad_can_update(probe);
+    if (mb->fused_head) mb->n_ranges = 0;
     return true;
   }
   auto bp = [&](size_t o) { return reinterpret_cast<__nv_bfloat16*>(base + o); };
