@@ -94,6 +94,13 @@ worker_mean_anchor_kernel(const float* __restrict__ x, float* __restrict__ z,
   const int64_t col4 = (int64_t)blockIdx.x * kMeanCols + threadIdx.x;
   const int slice = threadIdx.y;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  // slice 0 finishes the column: its anchor (and anchor momentum) strip is fetched together
+  // with the first worker rows, not after the sum
+  float4 z_old = make_float4(0.f, 0.f, 0.f, 0.f), v_old = z_old;
+  if (MOM && !partial && slice == 0 && col4 < n4) {
+    z_old = reinterpret_cast<const float4*>(z)[col4];
+    v_old = reinterpret_cast<const float4*>(v)[col4];
+  }
   if (col4 < n4) {
     for (int ib = slice; ib < m; ib += kMeanSlices * kUnroll) {
       float4 xv[kUnroll];
@@ -138,7 +145,7 @@ worker_mean_anchor_kernel(const float* __restrict__ x, float* __restrict__ z,
   if (MOM) {
     // Eq. 10: v <- beta v + (mean - z);  Eq. 11: z <- z + v
     float4* v4 = reinterpret_cast<float4*>(v) + col4;
-    float4 zz = *z4, vv = *v4;
+    float4 zz = z_old, vv = v_old;
     vv.x = fmaf(beta, vv.x, s.x - zz.x);
     vv.y = fmaf(beta, vv.y, s.y - zz.y);
     vv.z = fmaf(beta, vv.z, s.z - zz.z);
