@@ -213,6 +213,17 @@ head_forward_vec_kernel(HeadArgs a) {
 #pragma unroll
   for (int r = 0; r < R; ++r) rowp[r] = head_row<InT>(a, i, b0 + (r < rows ? r : 0));
 
+  // what the softmax step needs from global memory is fetched now, under the first sweep:
+  // lane c's bias entry and the labels of the rows this warp will finish
+  constexpr int kRowsPerWarp = (R + kHeadThreads / 32 - 1) / (kHeadThreads / 32);
+  const float bias_c = (lane < C) ? bias[lane] : 0.f;
+  int label_of[kRowsPerWarp];
+#pragma unroll
+  for (int j = 0; j < kRowsPerWarp; ++j) {
+    const int r = warp + j * (kHeadThreads / 32);
+    label_of[j] = (r < rows) ? head_label(a, i, b0 + r) : 0;
+  }
+
   float acc[R][CMAX];
 #pragma unroll
   for (int r = 0; r < R; ++r)
@@ -260,16 +271,19 @@ head_forward_vec_kernel(HeadArgs a) {
     if (lane == 0) lg[o] = sum;
   }
   __syncthreads();
-  for (int r = warp; r < R; r += kHeadThreads / 32) {
+#pragma unroll
+  for (int j = 0; j < kRowsPerWarp; ++j) {
+    const int r = warp + j * (kHeadThreads / 32);
+    if (r >= R) break;
     const int b = b0 + r;
     const bool live = r < rows;
-    const float logit = (lane < C) ? lg[r * CMAX + lane] + bias[lane] : -INFINITY;
+    const float logit = (lane < C) ? lg[r * CMAX + lane] + bias_c : -INFINITY;
     float mx = logit;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     const float e = (lane < C) ? expf(logit - mx) : 0.f;
     const float lse = mx + logf(warp_sum(e));
-    const int label = live ? head_label(a, i, b) : 0;
+    const int label = label_of[j];
     const float picked = __shfl_sync(0xffffffffu, logit, label);
     float dl = 0.f;
     if (lane < C) dl = (expf(logit - lse) - (lane == label ? 1.f : 0.f)) / (float)B;
