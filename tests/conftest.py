@@ -14,6 +14,13 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on the B200 box)")
 
 
+@pytest.fixture(scope="session", autouse=True)
+def _library_is_built():
+    """libolsgd.so is built in-tree before any test runs (a no-op when it is up to date)."""
+    from paper_2002_09539_b200.build import build
+    build()
+
+
 def pytest_collection_modifyitems(config, items):
     try:
         import torch
