@@ -211,7 +211,9 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
   const bool fused_gather = !bf && L == 1;
   const bool rows_in_bf16 = bf && io.xb16_in != nullptr;
   const int set = bf ? io.batch_set : 0;
-  if (rows_in_bf16) {
+  if (rows_in_bf16 && io.batch_staged) {
+    // transposed copy and labels were made on the copy stream (model_stage_host_rows)
+  } else if (rows_in_bf16) {
     Scope sc(hook, OLSGD_KC_GATHER, s);
     OLSGD_TRY(launch_transpose_bf16(io.xb16_in, static_cast<const int32_t*>(data.y), mb.xb16t[set],
                                     mb.yb[set], m, B, d0, s));
@@ -403,6 +405,15 @@ cudaError_t model_stage_batch(const olsgd_model_spec& spec, const olsgd_hparams&
   return launch_gather(static_cast<const float*>(data.X), static_cast<const int32_t*>(data.y), idx,
                        nullptr, mb.xb16[set], mb.xb16t[set], mb.yb[set], hp.m, hp.batch,
                        data.n_per_worker, spec.dims[0], &rule, s);
+}
+
+cudaError_t model_stage_host_rows(const olsgd_model_spec& spec, const olsgd_hparams& hp,
+                                  const __nv_bfloat16* rows, const int32_t* labels,
+                                  const ModelBuffers& mb, int set, cudaStream_t s,
+                                  const ProfHook& hook) {
+  if (!bf16_path(spec)) return cudaErrorInvalidValue;
+  Scope sc(hook, OLSGD_KC_GATHER, s);
+  return launch_transpose_bf16(rows, labels, mb.xb16t[set], mb.yb[set], hp.m, hp.batch, spec.dims[0], s);
 }
 
 cudaError_t model_post_update(const olsgd_model_spec& spec, const olsgd_hparams& hp,

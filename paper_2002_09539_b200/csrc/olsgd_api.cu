@@ -60,6 +60,9 @@ struct olsgd_ctx {
   // pre_k % 2 on stream `pre`; pre_pending: the main stream has not yet waited for pre_done.
   cudaStream_t pre = nullptr;
   cudaEvent_t pre_begin = nullptr, pre_done = nullptr;
+  // recorded on the main stream when an iteration has finished reading staged-minibatch set b
+  cudaEvent_t set_free[2] = {nullptr, nullptr};
+  bool set_free_valid[2] = {false, false};   // false: the event does not cover the set's last reader
   bool pre_pending = false;
   int64_t pre_k = -1;
   cudaEvent_t pullback_done = nullptr, reduce_done = nullptr;
@@ -168,6 +171,8 @@ void free_host_side(olsgd_ctx* c) {
   if (c->aux) cudaStreamDestroy(c->aux);
   if (c->pre_begin) cudaEventDestroy(c->pre_begin);
   if (c->pre_done) cudaEventDestroy(c->pre_done);
+  for (int b = 0; b < 2; ++b)
+    if (c->set_free[b]) cudaEventDestroy(c->set_free[b]);
   if (c->pre) cudaStreamDestroy(c->pre);
   if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
   delete c;
@@ -433,6 +438,10 @@ olsgd_status step_body(olsgd_ctx* c, const olsgd_data& data, int32_t* idx,
   if (e != cudaSuccess)
     return fail(c, OLSGD_ECUDA, "forward/backward failed: %s", cudaGetErrorString(e));
   if (stage_slot >= 0) OLSGD_CUDA(c, cudaEventRecord(c->stage_free[stage_slot], c->main));
+  if (c->set_free[0] && !c->capturing && c->spec.kind == OLSGD_MLP && c->spec.gemm_bf16 != 0) {
+    OLSGD_CUDA(c, cudaEventRecord(c->set_free[io.batch_set], c->main));
+    c->set_free_valid[io.batch_set] = true;
+  }
   // S5-S6
   olsgd_status st = apply_update(c, c->g, c->ld);
   if (st != OLSGD_OK) return st;
@@ -563,6 +572,8 @@ olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const ols
     }
     OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->pre_begin, cudaEventDisableTiming));
     OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->pre_done, cudaEventDisableTiming));
+    for (int b = 0; b < 2; ++b)
+      OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->set_free[b], cudaEventDisableTiming));
     for (int b = 0; b < 2; ++b) {
       OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->h2d_done[b], cudaEventDisableTiming));
       OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->stage_free[b], cudaEventDisableTiming));
@@ -674,9 +685,11 @@ static olsgd_status local_step_host_impl(olsgd_ctx* c, const void* Xb_host, cons
     return fail(c, OLSGD_ESTATE, "bf16 minibatches are for models whose GEMM operands are bf16 "
                                  "(OLSGD_MLP with gemm_bf16 != 0)");
   if (c->need_sync) return fail(c, OLSGD_ESTATE, "a period ended: call olsgd_period_sync first");
-  // this step writes the staged-minibatch set of iteration k itself
+  // this step writes the staged-minibatch set of iteration k itself (bf16 rows: on the copy
+  // stream)
   if (c->pre_pending) {
     OLSGD_CUDA(c, cudaStreamWaitEvent(c->main, c->pre_done, 0));
+    OLSGD_CUDA(c, cudaStreamWaitEvent(c->copy, c->pre_done, 0));
     c->pre_pending = false;
   }
   if (c->pre_k == c->k) c->pre_k = -1;
@@ -688,6 +701,26 @@ static olsgd_status local_step_host_impl(olsgd_ctx* c, const void* Xb_host, cons
   OLSGD_CUDA(c, cudaMemcpyAsync(c->stage_x[slot], Xb_host, rows * c->spec.dims[0] * elem,
                                 cudaMemcpyHostToDevice, c->copy));
   OLSGD_CUDA(c, cudaMemcpyAsync(c->stage_y[slot], yb_host, rows * 4, cudaMemcpyHostToDevice, c->copy));
+  // bf16 rows need only their transposed copy and the label copy: both are made on the copy
+  // stream, right behind the transfer, into the set of iteration k, once the last iteration
+  // that read that set (normally k - 2) is done.
+  const bool stage_on_copy = elem == 2 && c->side != c->main;
+  if (stage_on_copy) {
+    const int set = (int)(c->k & 1);
+    if (!c->set_free_valid[set]) {
+      // unknown (graph replays do not record it): everything issued so far
+      OLSGD_CUDA(c, cudaEventRecord(c->set_free[set], c->main));
+      c->set_free_valid[set] = true;
+    }
+    OLSGD_CUDA(c, cudaStreamWaitEvent(c->copy, c->set_free[set], 0));
+    g_launch_plain = true;
+    const cudaError_t e = model_stage_host_rows(
+        c->spec, c->hp, reinterpret_cast<const __nv_bfloat16*>(c->stage_x[slot]),
+        reinterpret_cast<const int32_t*>(c->stage_y[slot]), c->mb, set, c->copy, make_hook(c));
+    g_launch_plain = false;
+    if (e != cudaSuccess)
+      return fail(c, OLSGD_ECUDA, "staging the host rows failed: %s", cudaGetErrorString(e));
+  }
   OLSGD_CUDA(c, cudaEventRecord(c->h2d_done[slot], c->copy));
   OLSGD_CUDA(c, cudaStreamWaitEvent(c->main, c->h2d_done[slot], 0));
   olsgd_data staged;
@@ -696,7 +729,7 @@ static olsgd_status local_step_host_impl(olsgd_ctx* c, const void* Xb_host, cons
   staged.n_per_worker = c->hp.batch;
   const __nv_bfloat16* direct =
       elem == 2 ? reinterpret_cast<const __nv_bfloat16*>(c->stage_x[slot]) : nullptr;
-  olsgd_status st = step_body(c, staged, c->ident, nullptr, slot, direct);
+  olsgd_status st = step_body(c, staged, c->ident, nullptr, slot, direct, nullptr, stage_on_copy);
   if (st != OLSGD_OK) return st;
   if (loss_host)
     OLSGD_CUDA(c, cudaMemcpyAsync(loss_host, c->mb.loss, (size_t)c->hp.m * sizeof(float),
@@ -944,6 +977,7 @@ olsgd_status olsgd_run(olsgd_ctx* c, int64_t n_iters, float* loss_device) {
                                     cudaMemcpyDeviceToDevice, c->main));
     c->k += block;
     if (c->graph_staged) c->pre_k = c->k;   // the block's last iteration staged the next rows
+    c->set_free_valid[0] = c->set_free_valid[1] = false;
     c->graph_replays += 1;
     c->launches += c->graph_launches;
     t += block;

@@ -301,7 +301,8 @@ struct StepIO {
   const __nv_bfloat16* xb16_in;  // if non-null: this step's rows, already bf16, [m][batch][dims[0]]
                                  // (data.y then holds their labels [m][batch]); idx is unused
   int batch_set;                 // which staged-minibatch set this iteration uses (0 or 1)
-  bool batch_staged;             // the set already holds this iteration's rows: no gather
+  bool batch_staged;             // the set already holds this iteration's rows (or, with
+                                 // xb16_in, their transposed copy and labels): no staging kernel
   float* loss;                   // out: [m] or null
   int* status;                   // device status word (see GemmArgs::status)
   FusedUpdateArgs upd;           // state pointers and factors for the fused epilogue (w_off unset)
@@ -328,6 +329,11 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
 cudaError_t model_stage_batch(const olsgd_model_spec& spec, const olsgd_hparams& hp,
                               const olsgd_data& data, const ModelBuffers& mb, int32_t* idx,
                               const IndexRule& rule, int set, cudaStream_t s, const ProfHook& hook);
+// The staging of host-fed bf16 rows by itself: transposed copy and labels into set `set`.
+cudaError_t model_stage_host_rows(const olsgd_model_spec& spec, const olsgd_hparams& hp,
+                                  const __nv_bfloat16* rows, const int32_t* labels,
+                                  const ModelBuffers& mb, int set, cudaStream_t s,
+                                  const ProfHook& hook);
 // Work that must follow every parameter update (none at present).
 cudaError_t model_post_update(const olsgd_model_spec& spec, const olsgd_hparams& hp,
                               const ModelBuffers& mb, const __nv_bfloat16* shadow, int64_t ld,
