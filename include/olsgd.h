@@ -6,8 +6,13 @@
  * One context holds the m worker models x^(1..m), their local momentum
  * buffers, the anchor z and the anchor momentum buffer v, all resident in
  * device memory that the CALLER allocates and hands over as one workspace.
- * A context owns host memory, CUDA events and one stream for host-to-device
- * staging copies.  The library never allocates device memory, never throws,
+ * A context owns host memory, CUDA events and three small streams of its
+ * own: one for host-to-device staging copies, one on which the output layer's
+ * weight gradient runs beside the hidden layers' backward pass, and one
+ * (low priority) on which the next iteration's minibatch rows are staged
+ * while the current iteration computes; all of them are joined by
+ * olsgd_join and olsgd_destroy, and the borrowed data set must stay valid
+ * until then.  The library never allocates device memory, never throws,
  * never aborts: every call returns a status and `olsgd_last_error` gives the
  * reason as text.
  *
