@@ -92,3 +92,72 @@ def test_bf16_host_rows_are_refused_by_fp32_models():
         opt.local_step_host(Xb, yb)
     assert opt.iteration == 0
     opt.close()
+
+
+def _mixed_sequence(opt, ref, X, y, dtype):
+    """Device-sampled steps, host-fed steps, a long run (captured graph where the streams
+    allow one), a jump of the iteration counter and more steps, in one context."""
+    m, tau = opt.m, opt.tau
+    keep = []
+
+    def sync():
+        if opt.iteration % tau == 0:
+            opt.period_sync()
+
+    def device_steps(count):
+        for _ in range(count):
+            opt.local_step()
+            sync()
+
+    def host_steps(count):
+        for _ in range(count):
+            idx = ref.get_indices(opt.iteration)
+            Xb = torch.from_numpy(np.stack([X[i][idx[i]] for i in range(m)])).to(dtype).pin_memory()
+            yb = torch.from_numpy(np.stack([y[i][idx[i]] for i in range(m)])).pin_memory()
+            keep.append((Xb, yb))
+            opt.local_step_host(Xb, yb)
+            sync()
+
+    device_steps(3)
+    host_steps(2)
+    device_steps(1)
+    host_steps(1)
+    device_steps(tau - opt.iteration % tau if opt.iteration % tau else 0)   # to a period boundary
+    opt.run(40)
+    host_steps(1)
+    device_steps(2 * tau - 1)
+    opt.join()
+    opt.set_iteration(4 * tau)
+    device_steps(3)
+    opt.run(7)
+    opt.join()
+    return opt.state()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_staging_ahead_gives_the_bits_of_serial_streams(dtype):
+    """With overlap (rows of the next iteration staged on the context's own stream, host rows
+    staged on the copy stream, captured graphs) and with one serial stream the same mixed
+    sequence of calls must end in the same bits."""
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    dims, m, n, batch, tau, seed = [128, 256, 128, 10], 3, 96, 64, 2, 9
+    X, y = si.mixture_data(seed, m, n, dims[0])
+    y = (y % dims[-1]).astype(np.int32)
+    x0 = si.model_init(seed, "mlp", dims)
+    kw = dict(m=m, tau=tau, batch=batch, gamma=0.05, alpha=0.6, beta=0.9, mu=0.9, seed=seed,
+              dims=dims, gemm_bf16=1, x0=x0)
+    states = []
+    for overlap in (True, False):
+        stream = torch.cuda.Stream()
+        with torch.cuda.stream(stream):
+            new = lambda: OverlapLocalSGD("mlp", X=torch.from_numpy(X).cuda(),
+                                          y=torch.from_numpy(y).cuda(), overlap=overlap, **kw)
+            opt, ref = new(), new()
+            states.append(_mixed_sequence(opt, ref, X, y, dtype))
+            if overlap:
+                assert opt.graph_replays > 0
+            opt.close()
+            ref.close()
+        stream.synchronize()
+    for a, b in zip(states[0], states[1]):
+        assert np.array_equal(a, b)
