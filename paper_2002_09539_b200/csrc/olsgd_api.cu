@@ -391,8 +391,10 @@ cudaError_t draw_indices(olsgd_ctx* c, int64_t k) {
 // idx[i][:] of `data`.  stage_slot >= 0 marks a host-fed staging slot to release.
 olsgd_status step_body(olsgd_ctx* c, const olsgd_data& data, int32_t* idx,
                        float* loss_device, int stage_slot, const __nv_bfloat16* xb16_in = nullptr,
-                       const IndexRule* rule = nullptr, bool batch_staged = false) {
+                       const IndexRule* rule = nullptr, bool batch_staged = false,
+                       cudaEvent_t mid_event = nullptr) {
   StepIO io;
+  io.mid_event = mid_event;
   io.xb16_in = xb16_in;
   io.rule = rule;
   io.batch_set = (int)(c->k & 1);
@@ -647,25 +649,29 @@ olsgd_status olsgd_local_step(olsgd_ctx* c, float* loss_device) {
       OLSGD_CUDA(c, cudaStreamWaitEvent(c->main, c->pre_done, 0));
       c->pre_pending = false;
     }
-    // Stage the rows of iteration k + 1 on the context's own stream while iteration k runs: its
-    // set (k + 1) % 2 was last read by iteration k - 1, which precedes pre_begin on the main
-    // stream.  Not with the two streams of the context serialised.
-    if (c->pre && c->side != c->main) {
-      OLSGD_CUDA(c, cudaEventRecord(c->pre_begin, c->main));
+    // Stage the rows of iteration k + 1 on the context's own stream while iteration k runs,
+    // from the point where iteration k's forward GEMMs are launched (pre_begin, recorded on
+    // the main stream inside the step): set (k + 1) % 2 was last read by iteration k - 1,
+    // which precedes that point.  Not with the two streams of the context serialised.
+    const bool ahead = c->pre && c->side != c->main;
+    const int64_t k_now = c->k;
+    const IndexRule rule = rule_for(k_now), next = rule_for(k_now + 1);
+    olsgd_status st = step_body(c, c->data, c->idx, loss_device, -1, nullptr, &rule, have,
+                                ahead ? c->pre_begin : nullptr);
+    if (st != OLSGD_OK) return st;
+    if (ahead) {
       OLSGD_CUDA(c, cudaStreamWaitEvent(c->pre, c->pre_begin, 0));
-      const IndexRule next = rule_for(c->k + 1);
       g_launch_plain = true;
       const cudaError_t e = model_stage_batch(c->spec, c->hp, c->data, c->mb, c->idx_next, next,
-                                              (int)((c->k + 1) & 1), c->pre, make_hook(c));
+                                              (int)((k_now + 1) & 1), c->pre, make_hook(c));
       g_launch_plain = false;
       if (e != cudaSuccess)
         return fail(c, OLSGD_ECUDA, "staging the next minibatch failed: %s", cudaGetErrorString(e));
       OLSGD_CUDA(c, cudaEventRecord(c->pre_done, c->pre));
       c->pre_pending = true;
-      c->pre_k = c->k + 1;
+      c->pre_k = k_now + 1;
     }
-    const IndexRule rule = rule_for(c->k);
-    return step_body(c, c->data, c->idx, loss_device, -1, nullptr, &rule, have);
+    return OLSGD_OK;
   }
   {
     Launch l(c, OLSGD_KC_INDEX, c->main);

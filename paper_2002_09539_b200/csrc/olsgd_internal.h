@@ -311,6 +311,9 @@ struct StepIO {
   // path of the backward pass; null: everything runs on the main stream.
   cudaStream_t aux;
   cudaEvent_t aux_fork, aux_join;
+  // If non-null: recorded on the main stream once the forward GEMMs are launched, the point
+  // from which the next iteration's rows may be staged beside this iteration.
+  cudaEvent_t mid_event;
 };
 // Lets model.cu count and time its launches without knowing the context type.
 struct ProfHook {
