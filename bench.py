@@ -205,6 +205,8 @@ def run_ours(args, rank, world):
     if c["gemm_bf16"] and args.gemm_mode:
         c["gemm_bf16"] = args.gemm_mode
     local_sgd = args.method != "overlap"
+    if args.tau:
+        c["tau"] = args.tau          # a study of the sync cost, not the configuration's own period
     if args.method == "sync_sgd":
         c["tau"] = 1                 # fully synchronous SGD = Eq. 2 with tau = 1
     seed = rank                      # every rank is an independent replica
@@ -329,6 +331,7 @@ def run_ours(args, rank, world):
                        "batch": B, "dims": c["dims"], "P": P, "gamma": c["gamma"],
                        "alpha": c["alpha"], "beta": c["beta"], "mu": c["mu"],
                        "gemm_mode": c["gemm_bf16"], "method": args.method,
+                       "tau_overridden": bool(args.tau),
                        "l2": "no flush: resident inputs+state %.0f MB exceed the %d MB L2"
                              % (resident / 1e6, L2_BYTES >> 20) if resident > L2_BYTES else
                              "state fits in L2 (%.1f MB): steady-state training keeps it there"
@@ -633,6 +636,8 @@ def main():
     ap.add_argument("--shard-workers", action="store_true",
                     help="split the m workers of ONE job over the GPUs (strong scaling) instead of "
                          "running one replica of the job per GPU")
+    ap.add_argument("--tau", type=int, default=0,
+                    help="c1-c4: override the configuration's period (to measure what a sync costs)")
     ap.add_argument("--P", type=int, default=0, help="c5 only: one parameter count")
     ap.add_argument("--m", type=int, default=0, help="c5 only: one worker count")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
