@@ -240,6 +240,9 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
     ga.Ma = spec.dims[l];
     ga.Nb = B;
     ga.K = spec.dims[l - 1];
+    // W_1 is not read again in this iteration (no input gradient is formed for the data);
+    // the weights of the other layers are read again by their input-gradient GEMM
+    ga.a_read_once = (l == 1) ? 1 : 0;
     ga.epilogue = GEMM_EPI_BIAS_RELU;
     ga.bias = io.x + mb.b_off[l - 1];
     ga.bias_batch = io.ld;

@@ -228,6 +228,7 @@ struct GemmArgs {
   int64_t lda, a_batch, ldb, b_batch;
   int m, Ma, Nb, K;
   int a_mn_major;            // A is stored [K][Ma]
+  int a_read_once;           // nothing reads A again soon: L2 may give its lines up first
   int epilogue;
   const float* bias;         // BIAS_RELU: bias[i * bias_batch + row]
   int64_t bias_batch;

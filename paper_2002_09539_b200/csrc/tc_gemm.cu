@@ -24,6 +24,7 @@ namespace {
 using namespace tc;
 
 struct EpiArgs {
+  int once;      // A is read once: its TMA loads carry an evict-first policy
   int epilogue;
   int Ma, Nb;
   const float* bias;
@@ -98,7 +99,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         tma_load_3d(a_dst, &map_a, full, m0, kb * kBK, worker);
         tma_load_3d(a_dst + kABytes / 2, &map_a, full, m0 + 64, kb * kBK, worker);
       } else {
-        tma_load_3d(a_dst, &map_a, full, kb * kBK, m0, worker);
+        if (ea.once) tma_load_3d_once(a_dst, &map_a, full, kb * kBK, m0, worker);
+        else tma_load_3d(a_dst, &map_a, full, kb * kBK, m0, worker);
       }
       tma_load_3d(a_dst + kABytes, &map_b, full, kb * kBK, n0, worker);
       issued = kb + 1;
@@ -259,6 +261,7 @@ cudaError_t launch_one(const GemmArgs& a, const CUtensorMap& ma, const CUtensorM
   }
   EpiArgs ea;
   ea.epilogue = a.epilogue;
+  ea.once = a.a_read_once;
   ea.Ma = a.Ma;
   ea.Nb = a.Nb;
   ea.bias = a.bias;
