@@ -115,7 +115,10 @@ bool bind_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, const Mod
   mb->n_ranges = 1;
   mb->range_off[0] = 0;
   if (spec.kind == OLSGD_LINREG) {
+    // the model kernel applies the update itself: nothing is left for the update kernel
     mb->range_len[0] = spec.dims[0];
+    mb->fused_head = true;
+    mb->n_ranges = 0;
     return true;
   }
   const int L = n_layers(spec);
@@ -198,9 +201,12 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
   const float* X = static_cast<const float*>(data.X);
 
   if (spec.kind == OLSGD_LINREG) {
+    // the kernel writes x_{k+1} and, on sync steps, reads the anchor
+    if (io.upd.enabled && io.wait_before_update)
+      OLSGD_TRY(cudaStreamWaitEvent(s, io.wait_before_update, 0));
     Scope sc(hook, OLSGD_KC_FORWARD, s);
     return launch_linreg(X, static_cast<const float*>(data.y), io.idx, io.x, io.g, loss, m, B, n,
-                         spec.dims[0], io.ld, s);
+                         spec.dims[0], io.ld, io.upd.enabled ? &io.upd : nullptr, s);
   }
 
   const int L = n_layers(spec);

@@ -415,7 +415,7 @@ olsgd_status step_body(olsgd_ctx* c, const olsgd_data& data, int32_t* idx,
   io.aux_fork = c->aux_fork;
   io.aux_join = c->aux_join;
   if ((c->spec.kind == OLSGD_MLP && c->spec.gemm_bf16 == 1) ||
-      (c->spec.kind == OLSGD_SOFTMAX && c->mb.fused_head)) {
+      ((c->spec.kind == OLSGD_SOFTMAX || c->spec.kind == OLSGD_LINREG) && c->mb.fused_head)) {
     const bool sync = (c->k + 1) % c->hp.tau == 0 && c->hp.mode == OLSGD_MODE_OVERLAP;
     const int nxt = 1 - c->cur;
     io.upd.enabled = 1;

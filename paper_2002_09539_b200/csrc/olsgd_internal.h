@@ -120,10 +120,12 @@ constexpr int kMaxClasses = 32;  // the output layer is handled by one warp per 
 cudaError_t launch_cast_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t s);
 
 // Linear regression, one block per worker: r = X_b w - y_b, loss = sum r^2 / 2B,
-// g = X_b^T r / B, reading the batch rows straight from the worker's partition.
+// g = X_b^T r / B, reading the batch rows straight from the worker's partition.  With upd
+// non-null and enabled the gradient is not stored: the kernel applies Eq. 3 / Eq. 4 itself.
+struct FusedUpdateArgs;
 cudaError_t launch_linreg(const float* X, const float* y, const int32_t* idx, const float* x,
                           float* g, float* loss, int m, int batch, int64_t n, int d, int64_t ld,
-                          cudaStream_t s);
+                          const FusedUpdateArgs* upd, cudaStream_t s);
 
 // S2: copy the minibatch rows of every worker into contiguous staging.
 //   xb32  float [m][B][d]   (or null)

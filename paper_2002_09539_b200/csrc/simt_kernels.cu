@@ -5,6 +5,7 @@
 // is reproducible bit for bit from run to run.
 #include "olsgd_internal.h"
 #include "philox.cuh"
+#include "update_math.cuh"
 
 namespace olsgd {
 namespace {
@@ -182,7 +183,8 @@ transpose_bf16_kernel(const __nv_bfloat16* __restrict__ xb16, const int32_t* __r
 __global__ void __launch_bounds__(128)
 linreg_kernel(const float* __restrict__ X, const float* __restrict__ y,
               const int32_t* __restrict__ idx, const float* __restrict__ x, float* __restrict__ g,
-              float* __restrict__ loss, int batch, int64_t n, int d, int64_t ld) {
+              float* __restrict__ loss, int batch, int64_t n, int d, int64_t ld,
+              FusedUpdateArgs up) {
   launch_gate();
   extern __shared__ float sm[];  // residuals [batch]
   const int i = blockIdx.x;
@@ -205,7 +207,19 @@ linreg_kernel(const float* __restrict__ X, const float* __restrict__ y,
       const int32_t r = idx[(int64_t)i * batch + b];
       acc = fmaf(sm[b], Xi[(int64_t)r * d + j], acc);
     }
-    g[(int64_t)i * ld + j] = acc * inv_b;
+    const float gj = acc * inv_b;
+    if (up.enabled) {
+      // Eq. 3 / Eq. 4 for entry j of worker i, with the arithmetic of the update kernel
+      const int64_t o = (int64_t)i * up.ld + j;
+      const bool mom = up.u != nullptr && up.mu != 0.f;
+      float xv = up.x_in[o], uv = mom ? up.u[o] : 0.f;
+      update_scalar_rt(xv, uv, gj, up.sync ? up.z[j] : 0.f, up.gamma, up.mu, up.alpha, mom,
+                       up.sync != 0);
+      up.x_out[o] = xv;
+      if (mom) up.u[o] = uv;
+    } else {
+      g[(int64_t)i * ld + j] = gj;
+    }
   }
   if (loss && threadIdx.x == 0) {
     float s = 0.f;
@@ -307,9 +321,11 @@ cudaError_t launch_transpose_bf16(const __nv_bfloat16* xb16, const int32_t* y, _
 
 cudaError_t launch_linreg(const float* X, const float* y, const int32_t* idx, const float* x,
                           float* g, float* loss, int m, int batch, int64_t n, int d, int64_t ld,
-                          cudaStream_t s) {
+                          const FusedUpdateArgs* upd, cudaStream_t s) {
+  FusedUpdateArgs up{};
+  if (upd) up = *upd;
   return launch_chained(linreg_kernel, dim3(m), dim3(128), (size_t)batch * sizeof(float), s, X, y, idx,
-                        x, g, loss, batch, n, d, ld);
+                        x, g, loss, batch, n, d, ld, up);
 }
 
 cudaError_t launch_bias_grad(const __nv_bfloat16* dat, float* g, int64_t ld, int64_t b_off, int m,
