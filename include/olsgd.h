@@ -133,6 +133,9 @@ olsgd_status olsgd_workspace_bytes(const olsgd_model_spec* spec, const olsgd_hpa
  *   side_stream      cudaStream_t on which the anchor refresh runs; may equal
  *                    main_stream (then nothing overlaps)
  *   data             may be NULL for OLSGD_FLAT
+ * The context belongs to the CUDA device that is current during this call (the workspace,
+ * the data set and both streams must live there); every later call on it must be made with
+ * the same device current and returns OLSGD_ESTATE otherwise.
  * Checks: m, tau, batch >= 1; gamma > 0; 0 <= alpha <= 1; 0 <= beta < 1;
  * 0 <= mu < 1; pointers non-null and aligned.  On error *out is NULL.       */
 olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const olsgd_hparams* hp,
@@ -189,6 +192,12 @@ olsgd_status olsgd_join(olsgd_ctx* ctx);
  * stay usable throughout.  limit_ms must be in [1, 2000].                        */
 olsgd_status olsgd_selftest_wait_timeout(olsgd_ctx* ctx, int32_t limit_ms);
 olsgd_status olsgd_clear_status(olsgd_ctx* ctx);
+
+/* Host-only self-test of the table that remembers, per device ordinal, which dynamic
+ * shared-memory limit each kernel has been configured for (kernel attributes belong to a
+ * device: a process that opens contexts on two GPUs must configure both).  Launches
+ * nothing and needs no GPU.  OLSGD_OK, or OLSGD_ESTATE if the table misbehaves.          */
+olsgd_status olsgd_selftest_per_device_table(void);
 
 /* Same iteration for OLSGD_FLAT: the stacked gradients G_k (Eq. 7 without its
  * zero column) come from the caller.
@@ -275,6 +284,14 @@ olsgd_status olsgd_consensus_distance(olsgd_ctx* ctx, double* out_host);
  * (seed mod 2^32, seed div 2^32).  Computed on the device; blocks the host.
  *   dst  int32 [m][batch], host or device                                   */
 olsgd_status olsgd_get_indices(olsgd_ctx* ctx, int64_t k, int32_t* dst);
+
+/* h of the epoch minibatch rule (olsgd_hparams.sampling = 1) for a partition of n samples:
+ * the Feistel network permutes the 2^(2h) values of two h-bit halves, h = ceil(ceil(log2 n)
+ * / 2), so 2^(2h) < 4 n and a pass of the cycle walk succeeds with probability above 1/4.
+ * The device gives a slot up after 64 passes (probability below 1e-8 per draw), stores index
+ * 0 for it and raises the status word: the next joining call returns OLSGD_ETIMEOUT.
+ * Host only.  Returns -1 unless 1 <= n < 2^31.                                          */
+int32_t olsgd_epoch_rule_half_bits(int64_t n);
 
 /* Non-IID partition table: the two classes (of ten) each worker samples
  * from.  Class slots are concatenated seeded Fisher-Yates permutations of

@@ -142,19 +142,3 @@ def matrix_form_step(X, G, gamma, W):
     """Eq. 8: X, G are d x (m+1) with the anchor (resp. a zero) last."""
     return (X - gamma * G) @ W
 
-
-def run(x0, m, tau, gamma, alpha, beta, mu, n_iters, grad_fn, on_step=None):
-    """Drive the iteration; grad_fn(i, k, x_i) -> (loss, g_i(x_i; xi_k^(i))).
-
-    Returns the final state object and the [n_iters][m] minibatch losses.
-    """
-    st = OverlapLocalSGD(x0, m, tau, gamma, alpha, beta, mu)
-    losses = np.zeros((n_iters, m))
-    g = np.zeros_like(st.x)
-    for k in range(n_iters):
-        for i in range(m):
-            losses[k, i], g[i] = grad_fn(i, k, st.x[i])
-        st.step(g)
-        if on_step is not None:
-            on_step(st)
-    return st, losses

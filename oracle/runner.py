@@ -12,25 +12,31 @@ from . import models, olsgd, sampling
 
 def run_model(kind, dims, X, y, x0, *, m, tau, batch, gamma, alpha, beta, mu, seed,
               iters, bf16_operands=False, snapshots=(), local_sgd=False,
-              epoch_sampling=False):
+              epoch_sampling=False, state=None):
     """Run `iters` iterations; returns (state, losses[iters][m], {k: state copy}).
 
     X [m][n][d_in], y [m][n]; worker i only ever touches X[i], y[i] (Eq. 1).
     `snapshots` lists iteration counts k at which (x, z, v) are copied out.
+    `state`: continue from this state object (its x, u, z, v and k) instead of starting
+    from x0; the minibatch rule is a function of k, so a run can be resumed anywhere.
     """
     n = X.shape[1]
-    st = (olsgd.LocalSGD(x0, m, tau, gamma, mu) if local_sgd
-          else olsgd.OverlapLocalSGD(x0, m, tau, gamma, alpha, beta, mu))
+    if state is not None:
+        st = state
+    else:
+        st = (olsgd.LocalSGD(x0, m, tau, gamma, mu) if local_sgd
+              else olsgd.OverlapLocalSGD(x0, m, tau, gamma, alpha, beta, mu))
     losses = np.zeros((iters, m))
     g = np.zeros_like(st.x)
     snaps = {}
-    for k in range(iters):
+    for t in range(iters):
+        k = st.k
         idx = (sampling.minibatch_indices_epoch(seed, m, k, batch, n) if epoch_sampling
                else sampling.minibatch_indices(seed, m, k, batch, n))
         for i in range(m):
             Xb = X[i][idx[i]]
             yb = y[i][idx[i]]
-            losses[k, i], g[i] = models.loss_grad(kind, dims, st.x[i], Xb, yb,
+            losses[t, i], g[i] = models.loss_grad(kind, dims, st.x[i], Xb, yb,
                                                   bf16_operands=bf16_operands)
         st.step(g)
         if st.k in snapshots:

@@ -68,6 +68,8 @@ def load_library():
         "olsgd_join": (i32, [vp]),
         "olsgd_selftest_wait_timeout": (i32, [vp, i32]),
         "olsgd_clear_status": (i32, [vp]),
+        "olsgd_selftest_per_device_table": (i32, []),
+        "olsgd_epoch_rule_half_bits": (i32, [i64]),
         "olsgd_period_sync": (i32, [vp]),
         "olsgd_period_sync_begin": (i32, [vp, vp]),
         "olsgd_period_sync_finish": (i32, [vp, vp]),

@@ -53,7 +53,6 @@ __device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
 }
 
 constexpr int kHeadThreads = 128;
-constexpr int kHeadSmallGrid = 4 * 148;
 
 // Forward, loss and input gradient of the output layer for R batch rows of one worker.
 //
@@ -595,11 +594,10 @@ cudaError_t launch_fwd(const HeadArgs& a, cudaStream_t s) {
   constexpr int VC = CMAX <= 16 ? CMAX : 1;
   const bool vec = CMAX <= 16 && a.K % 4 == 0 && a.w_off % 4 == 0 && a.ld % 4 == 0;
   auto kern = vec ? head_forward_vec_kernel<InT, VC, R> : head_forward_kernel<InT, CMAX, R>;
-  static bool configured[2] = {false, false};
-  if (!configured[vec]) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  static PerDeviceSmem configured[2];
+  {
+    const cudaError_t e = ensure_dynamic_smem(configured[vec], kern, smem);
     if (e != cudaSuccess) return e;
-    configured[vec] = true;
   }
   dim3 grid((a.batch + R - 1) / R, a.m), block(kHeadThreads);
   return launch_chained(kern, grid, block, smem, s, a);
@@ -608,7 +606,7 @@ cudaError_t launch_fwd(const HeadArgs& a, cudaStream_t s) {
 template <typename InT>
 cudaError_t launch_fwd_c(const HeadArgs& a, cudaStream_t s) {
   // eight batch rows per block, or four where that leaves fewer than two blocks per SM
-  const bool small = (int64_t)((a.batch + 7) / 8) * a.m < kHeadSmallGrid;
+  const bool small = (int64_t)((a.batch + 7) / 8) * a.m < 4 * (int64_t)sm_count();
   if (a.C <= 10) return small ? launch_fwd<InT, 10, 4>(a, s) : launch_fwd<InT, 10, 8>(a, s);
   if (a.C <= 16) return small ? launch_fwd<InT, 16, 4>(a, s) : launch_fwd<InT, 16, 8>(a, s);
   return launch_fwd<InT, 32, 4>(a, s);

@@ -433,13 +433,4 @@ cudaError_t model_stage_host_rows(const olsgd_model_spec& spec, const olsgd_hpar
   return launch_transpose_bf16(rows, labels, mb.xb16t[set], mb.yb[set], hp.m, hp.batch, spec.dims[0], s);
 }
 
-cudaError_t model_post_update(const olsgd_model_spec& spec, const olsgd_hparams& hp,
-                              const ModelBuffers& mb, const __nv_bfloat16* shadow, int64_t ld,
-                              cudaStream_t s, const ProfHook& hook) {
-  // nothing is derived from the parameters any more: the input-gradient GEMM reads the
-  // bf16 shadow of W_l in place as an MN-major operand
-  (void)spec; (void)hp; (void)mb; (void)shadow; (void)ld; (void)s; (void)hook;
-  return cudaSuccess;
-}
-
 }  // namespace olsgd

@@ -86,6 +86,7 @@ struct olsgd_ctx {
   int64_t graph_launches = 0;    // kernel launches of one block
   int64_t graph_replays = 0;
 
+  int device = -1;              // ordinal of the device the context was created on
   int64_t k = 0;
   int64_t launches = 0;
   bool prof = false;
@@ -115,6 +116,21 @@ olsgd_status fail(olsgd_ctx* ctx, olsgd_status st, const char* fmt, ...) {
     if (e_ != cudaSuccess)                                                                \
       return fail(ctx, OLSGD_ECUDA, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(e_), \
                   __FILE__, __LINE__);                                                    \
+  } while (0)
+
+// A context belongs to the device that was current in olsgd_init: its workspace, streams and
+// events live there, and kernel attributes are configured per device.
+olsgd_status check_device(olsgd_ctx* c) {
+  const int dev = current_device();
+  if (dev != c->device)
+    return fail(c, OLSGD_ESTATE, "the context was created on device %d but device %d is current",
+                c->device, dev);
+  return OLSGD_OK;
+}
+#define OLSGD_ON_DEVICE(c)                          \
+  do {                                              \
+    olsgd_status ds_ = check_device(c);             \
+    if (ds_ != OLSGD_OK) return ds_;                \
   } while (0)
 
 // Brackets one kernel launch: counts it and, when profiling, times it with
@@ -309,6 +325,11 @@ olsgd_status make_plan(const olsgd_model_spec* spec, const olsgd_hparams* hp, Pl
 }
 
 olsgd_status drain_profile(olsgd_ctx* c) {
+  // launches are bracketed on every stream the context uses: all of them must be idle
+  // before the events are read, or the sample of a launch still in flight would be lost
+  if (c->copy) OLSGD_CUDA(c, cudaStreamSynchronize(c->copy));
+  if (c->aux) OLSGD_CUDA(c, cudaStreamSynchronize(c->aux));
+  if (c->pre) OLSGD_CUDA(c, cudaStreamSynchronize(c->pre));
   OLSGD_CUDA(c, cudaStreamSynchronize(c->main));
   OLSGD_CUDA(c, cudaStreamSynchronize(c->side));
   for (auto& r : c->prof_pending) {
@@ -382,7 +403,7 @@ cudaError_t draw_indices(olsgd_ctx* c, int64_t k) {
   if (c->hp.sampling == 1)
     return launch_minibatch_indices_epoch(c->idx, c->hp.seed, c->hp.m, k, c->hp.batch,
                                           c->data.n_per_worker, c->hp.worker_offset, k_ptr,
-                                          c->main);
+                                          c->dev_status, c->main);
   return launch_minibatch_indices(c->idx, c->hp.seed, c->hp.m, k, c->hp.batch,
                                   c->data.n_per_worker, c->hp.worker_offset, k_ptr, c->main);
 }
@@ -447,9 +468,6 @@ olsgd_status step_body(olsgd_ctx* c, const olsgd_data& data, int32_t* idx,
   // S5-S6
   olsgd_status st = apply_update(c, c->g, c->ld);
   if (st != OLSGD_OK) return st;
-  e = model_post_update(c->spec, c->hp, c->mb, c->shadow, c->ld, c->main, hook);
-  if (e != cudaSuccess)
-    return fail(c, OLSGD_ECUDA, "post-update failed: %s", cudaGetErrorString(e));
   return OLSGD_OK;
 }
 
@@ -474,6 +492,28 @@ namespace olsgd {
 void set_thread_error(const char* text) { g_last_error = text ? text : ""; }
 int g_launch_overlap = 1;
 thread_local bool g_launch_plain = false;
+
+int current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    cudaGetLastError();
+    return -1;
+  }
+  return dev;
+}
+
+int sm_count() {
+  static int cached[kMaxDevices] = {0};
+  const int dev = current_device();
+  if (dev >= 0 && dev < kMaxDevices && cached[dev] > 0) return cached[dev];
+  int n = 0;
+  if (dev < 0 || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+    cudaGetLastError();
+    return 1;
+  }
+  if (dev < kMaxDevices) cached[dev] = n;
+  return n;
+}
 }  // namespace olsgd
 
 extern "C" {
@@ -519,6 +559,7 @@ olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const ols
   if (!c) return fail(nullptr, OLSGD_ENOMEM, "host allocation failed");
   c->spec = *spec;
   c->hp = *hp;
+  c->device = current_device();
   if (data) c->data = *data; else memset(&c->data, 0, sizeof c->data);
   c->P = pl.P;
   c->ld = pl.ld;
@@ -601,10 +642,6 @@ olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const ols
       Launch l(c, OLSGD_KC_OTHER, c->main);
       OLSGD_INIT_CUDA(launch_cast_bf16(c->x[0], c->shadow, (int64_t)c->hp.m * c->ld, c->main));
     }
-    cudaError_t e = model_post_update(c->spec, c->hp, c->mb, c->shadow, c->ld, c->main,
-                                      make_hook(c));
-    if (e != cudaSuccess)
-      return bail(fail(c, OLSGD_ECUDA, "model set-up failed: %s", cudaGetErrorString(e)));
   }
   OLSGD_INIT_CUDA(cudaStreamSynchronize(c->main));
 #undef OLSGD_INIT_CUDA
@@ -614,6 +651,7 @@ olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const ols
 
 olsgd_status olsgd_local_step_with_grads(olsgd_ctx* c, const float* g_device) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  OLSGD_ON_DEVICE(c);
   if (c->spec.kind != OLSGD_FLAT)
     return fail(c, OLSGD_ESTATE, "olsgd_local_step_with_grads is for OLSGD_FLAT contexts");
   if (!g_device || (reinterpret_cast<uintptr_t>(g_device) & 3))
@@ -624,6 +662,7 @@ olsgd_status olsgd_local_step_with_grads(olsgd_ctx* c, const float* g_device) {
 
 olsgd_status olsgd_local_step(olsgd_ctx* c, float* loss_device) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  OLSGD_ON_DEVICE(c);
   if (c->spec.kind == OLSGD_FLAT)
     return fail(c, OLSGD_ESTATE, "OLSGD_FLAT contexts take olsgd_local_step_with_grads");
   if (c->need_sync) return fail(c, OLSGD_ESTATE, "a period ended: call olsgd_period_sync first");
@@ -684,6 +723,7 @@ olsgd_status olsgd_local_step(olsgd_ctx* c, float* loss_device) {
 static olsgd_status local_step_host_impl(olsgd_ctx* c, const void* Xb_host, const void* yb_host,
                                          float* loss_host, size_t elem) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  OLSGD_ON_DEVICE(c);
   if (c->spec.kind == OLSGD_FLAT)
     return fail(c, OLSGD_ESTATE, "OLSGD_FLAT contexts take olsgd_local_step_with_grads");
   if (!Xb_host || !yb_host) return fail(c, OLSGD_EINVAL, "host minibatch pointers are NULL");
@@ -755,6 +795,7 @@ olsgd_status olsgd_local_step_host_bf16(olsgd_ctx* c, const void* Xb_host_bf16, 
 
 olsgd_status olsgd_selftest_wait_timeout(olsgd_ctx* c, int32_t limit_ms) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  OLSGD_ON_DEVICE(c);
   if (limit_ms < 1 || limit_ms > 2000) return fail(c, OLSGD_EINVAL, "limit_ms must be in [1, 2000]");
   Launch l(c, OLSGD_KC_OTHER, c->main);
   OLSGD_CUDA(c, launch_wait_selftest(c->dev_status, (uint64_t)limit_ms * 1000000ull, c->main));
@@ -772,6 +813,7 @@ olsgd_status olsgd_clear_status(olsgd_ctx* c) {
 
 olsgd_status olsgd_join(olsgd_ctx* c) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  OLSGD_ON_DEVICE(c);
   if (c->copy) OLSGD_CUDA(c, cudaStreamSynchronize(c->copy));
   if (c->aux) OLSGD_CUDA(c, cudaStreamSynchronize(c->aux));
   if (c->pre) OLSGD_CUDA(c, cudaStreamSynchronize(c->pre));
@@ -783,6 +825,7 @@ olsgd_status olsgd_join(olsgd_ctx* c) {
 
 olsgd_status olsgd_period_sync(olsgd_ctx* c) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  OLSGD_ON_DEVICE(c);
   if (!c->need_sync || c->sync_begun)
     return fail(c, OLSGD_ESTATE, "olsgd_period_sync is legal once, right after a period ends (k=%lld, tau=%d)",
                 (long long)c->k, c->hp.tau);
@@ -814,6 +857,7 @@ olsgd_status olsgd_period_sync(olsgd_ctx* c) {
 
 olsgd_status olsgd_period_sync_begin(olsgd_ctx* c, float* partial_sum_device) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  OLSGD_ON_DEVICE(c);
   if (!partial_sum_device || (reinterpret_cast<uintptr_t>(partial_sum_device) & 15))
     return fail(c, OLSGD_EINVAL, "partial_sum_device must be non-null and 16-byte aligned");
   if (!c->need_sync || c->sync_begun)
@@ -841,6 +885,7 @@ olsgd_status olsgd_period_sync_begin(olsgd_ctx* c, float* partial_sum_device) {
 
 olsgd_status olsgd_period_sync_finish(olsgd_ctx* c, const float* total_sum_device) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  OLSGD_ON_DEVICE(c);
   if (!total_sum_device || (reinterpret_cast<uintptr_t>(total_sum_device) & 15))
     return fail(c, OLSGD_EINVAL, "total_sum_device must be non-null and 16-byte aligned");
   if (!c->sync_begun)
@@ -932,6 +977,7 @@ static bool capture_block(olsgd_ctx* c) {
 
 olsgd_status olsgd_run(olsgd_ctx* c, int64_t n_iters, float* loss_device) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  OLSGD_ON_DEVICE(c);
   if (n_iters < 0) return fail(c, OLSGD_EINVAL, "n_iters must be >= 0");
   if (c->spec.kind == OLSGD_FLAT)
     return fail(c, OLSGD_ESTATE, "OLSGD_FLAT contexts take olsgd_local_step_with_grads");
@@ -993,6 +1039,7 @@ olsgd_status olsgd_run(olsgd_ctx* c, int64_t n_iters, float* loss_device) {
 
 olsgd_status olsgd_get_params(olsgd_ctx* c, int32_t which, float* dst, size_t n_floats) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  OLSGD_ON_DEVICE(c);
   if (!dst) return fail(c, OLSGD_EINVAL, "dst is NULL");
   if (n_floats != (size_t)c->P)
     return fail(c, OLSGD_EINVAL, "n_floats is %zu but P is %lld", n_floats, (long long)c->P);
@@ -1023,6 +1070,7 @@ olsgd_status olsgd_get_params(olsgd_ctx* c, int32_t which, float* dst, size_t n_
 
 olsgd_status olsgd_set_params(olsgd_ctx* c, int32_t which, const float* src, size_t n_floats) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  OLSGD_ON_DEVICE(c);
   if (!src) return fail(c, OLSGD_EINVAL, "src is NULL");
   if (n_floats != (size_t)c->P)
     return fail(c, OLSGD_EINVAL, "n_floats is %zu but P is %lld", n_floats, (long long)c->P);
@@ -1057,6 +1105,7 @@ olsgd_status olsgd_set_iteration(olsgd_ctx* c, int64_t k) {
 
 olsgd_status olsgd_consensus_distance(olsgd_ctx* c, double* out_host) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  OLSGD_ON_DEVICE(c);
   if (!out_host) return fail(c, OLSGD_EINVAL, "out_host is NULL");
   OLSGD_CUDA(c, cudaStreamSynchronize(c->side));
   c->reduce_pending = false;
@@ -1076,6 +1125,7 @@ olsgd_status olsgd_consensus_distance(olsgd_ctx* c, double* out_host) {
 
 olsgd_status olsgd_get_indices(olsgd_ctx* c, int64_t k, int32_t* dst) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  OLSGD_ON_DEVICE(c);
   if (!dst) return fail(c, OLSGD_EINVAL, "dst is NULL");
   if (c->spec.kind == OLSGD_FLAT) return fail(c, OLSGD_ESTATE, "OLSGD_FLAT draws no minibatches");
   if (k < 0) return fail(c, OLSGD_EINVAL, "k must be >= 0");
@@ -1112,6 +1162,31 @@ olsgd_status olsgd_class_pairs(uint64_t seed, int32_t m, int32_t* dst, void* str
   if (e != cudaSuccess)
     return fail(nullptr, OLSGD_ECUDA, "class-pair kernel failed: %s", cudaGetErrorString(e));
   return OLSGD_OK;
+}
+
+olsgd_status olsgd_selftest_per_device_table(void) {
+  // host only: the table the launch wrappers consult, driven with made-up device ordinals
+  olsgd::PerDeviceSmem t;
+  bool ok = t.needs(0, 100);                  // nothing configured yet
+  t.set(0, 100);
+  ok = ok && !t.needs(0, 100) && !t.needs(0, 64);   // device 0 is configured for up to 100 bytes
+  ok = ok && t.needs(1, 100);                 // ... which says nothing about device 1
+  ok = ok && t.needs(0, 200);                 // a larger request configures again
+  t.set(0, 200);
+  t.set(0, 150);                              // and the table only ever grows
+  ok = ok && !t.needs(0, 200);
+  t.set(1, 100);
+  ok = ok && !t.needs(1, 100) && !t.needs(0, 200);
+  ok = ok && t.needs(-1, 1) && t.needs(olsgd::kMaxDevices, 1);   // unknown ordinals: always
+  t.set(olsgd::kMaxDevices, 1);
+  ok = ok && t.needs(olsgd::kMaxDevices, 1);
+  if (!ok) return fail(nullptr, OLSGD_ESTATE, "per-device attribute table is inconsistent");
+  return OLSGD_OK;
+}
+
+int32_t olsgd_epoch_rule_half_bits(int64_t n) {
+  if (n < 1 || n > 0x7FFFFFFF) return -1;
+  return olsgd::epoch_rule_half_bits(n);
 }
 
 int64_t olsgd_iteration(const olsgd_ctx* c) { return c ? c->k : -1; }

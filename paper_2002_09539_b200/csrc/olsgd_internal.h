@@ -50,6 +50,38 @@ cudaError_t launch_chained(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t
 // Records the text olsgd_last_error(NULL) returns for context-free calls of this thread.
 void set_thread_error(const char* text);
 
+// ---- per-device bookkeeping ---------------------------------------------------
+// Kernel attributes set with cudaFuncSetAttribute and the number of multiprocessors belong to
+// a device, not to the process: one process may drive several GPUs (one context each), so
+// "already configured" is remembered per device ordinal.
+constexpr int kMaxDevices = 64;
+struct PerDeviceSmem {
+  size_t bytes[kMaxDevices] = {0};   // largest dynamic shared-memory size configured so far
+  // does a launch with `smem` bytes on device `dev` need the attribute (re)set first?  An
+  // ordinal outside the table is never remembered: it is configured on every launch.
+  bool needs(int dev, size_t smem) const {
+    return dev < 0 || dev >= kMaxDevices || smem > bytes[dev];
+  }
+  void set(int dev, size_t smem) {
+    if (dev >= 0 && dev < kMaxDevices && smem > bytes[dev]) bytes[dev] = smem;
+  }
+};
+int current_device();   // ordinal of the current device, -1 if it cannot be read
+int sm_count();         // multiprocessors of the current device (cached per device; >= 1)
+#ifdef __CUDACC__
+// Raises the kernel's dynamic shared-memory limit on the current device when this launch
+// needs more than that device was configured for.  Not to be called inside a stream capture
+// for the first time (olsgd_run launches its first block outside the capture for this reason).
+template <typename Kern>
+cudaError_t ensure_dynamic_smem(PerDeviceSmem& table, Kern kern, size_t smem) {
+  const int dev = current_device();
+  if (!table.needs(dev, smem)) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e == cudaSuccess) table.set(dev, smem);
+  return e;
+}
+#endif
+
 // ---- update_kernels.cu ------------------------------------------------------
 // Eq. 3 (+ local Nesterov buffer) and, when `sync`, Eq. 4, for all m workers.
 // x_in/x_out/u/shadow rows have stride `ld` floats (multiple of 4, 16-byte
@@ -107,9 +139,12 @@ cudaError_t launch_minibatch_indices(int32_t* idx, uint64_t seed, int m, int64_t
 // *p = value (set) or *p += by
 cudaError_t launch_counter(int64_t* p, int64_t value, int64_t by, bool set, cudaStream_t s);
 // The epoch rule (one pass over the worker's samples per epoch, Feistel permutation).
+// status: device word that receives OLSGD_ETIMEOUT if the cycle walk of a slot runs out.
 cudaError_t launch_minibatch_indices_epoch(int32_t* idx, uint64_t seed, int m, int64_t k, int batch,
                                            int64_t n, int worker_offset, const int64_t* k_ptr,
-                                           cudaStream_t s);
+                                           int* status, cudaStream_t s);
+// h of the epoch rule: the Feistel network permutes 2^(2h) values, h = ceil(ceil(log2 n) / 2).
+int epoch_rule_half_bits(int64_t n);
 cudaError_t launch_class_pairs(int32_t* dst, uint64_t seed, int m, cudaStream_t s);
 // idx[i][j] = j: the "indices" of a minibatch that is already contiguous
 cudaError_t launch_identity_indices(int32_t* idx, int m, int batch, cudaStream_t s);
@@ -340,9 +375,5 @@ cudaError_t model_stage_host_rows(const olsgd_model_spec& spec, const olsgd_hpar
                                   const __nv_bfloat16* rows, const int32_t* labels,
                                   const ModelBuffers& mb, int set, cudaStream_t s,
                                   const ProfHook& hook);
-// Work that must follow every parameter update (none at present).
-cudaError_t model_post_update(const olsgd_model_spec& spec, const olsgd_hparams& hp,
-                              const ModelBuffers& mb, const __nv_bfloat16* shadow, int64_t ld,
-                              cudaStream_t s, const ProfHook& hook);
 
 }  // namespace olsgd

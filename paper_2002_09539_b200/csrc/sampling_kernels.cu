@@ -51,12 +51,17 @@ __global__ void class_pairs_kernel(int32_t* __restrict__ dst, uint32_t k0, uint3
 
 // Epoch rule, one thread per slot: draw t = k * batch + j belongs to epoch e = t / n and takes
 // sample pi(t % n); pi is a four-round balanced Feistel network on two h-bit halves whose
-// round function is a Philox word, applied again while the result is >= n (cycle walking;
-// at most a handful of passes since 2^(2h) < 4 n).
+// round function is a Philox word, applied again while the result is >= n (cycle walking).
+// The domain 2^(2h) is below 4 n, so a pass lands inside [0, n) with probability above 1/4
+// and the expected number of passes is below 4; kEpochWalkLimit passes all failing has
+// probability below (3/4)^64 = 1e-8 per draw of a random permutation.  Should it happen
+// anyway, no out-of-range index is stored: the slot gets 0 and the status word is raised, so
+// the next joining call reports OLSGD_ETIMEOUT.
+constexpr int kEpochWalkLimit = 64;
 __global__ void minibatch_indices_epoch_kernel(int32_t* __restrict__ idx, uint32_t k0, uint32_t k1,
                                                int m, uint64_t k_base, const long long* k_ptr,
                                                int batch, uint32_t n, int h,
-                                               uint32_t worker_offset) {
+                                               uint32_t worker_offset, int* status) {
   launch_gate();
   const uint64_t k = k_base + (k_ptr ? (uint64_t)*k_ptr : 0ull);
   const int t_id = blockIdx.x * blockDim.x + threadIdx.x;
@@ -66,7 +71,8 @@ __global__ void minibatch_indices_epoch_kernel(int32_t* __restrict__ idx, uint32
   const uint32_t e = (uint32_t)(t / n);
   uint32_t v = (uint32_t)(t % n);
   const uint32_t mask = (1u << h) - 1u;
-  for (int walk = 0; walk < 64; ++walk) {       // bounded; a valid value appears long before
+  bool found = false;
+  for (int walk = 0; walk < kEpochWalkLimit; ++walk) {
     uint32_t left = v >> h, right = v & mask;
 #pragma unroll
     for (uint32_t r = 0; r < 4; ++r) {
@@ -77,7 +83,14 @@ __global__ void minibatch_indices_epoch_kernel(int32_t* __restrict__ idx, uint32
       left = nl;
     }
     v = (left << h) | right;
-    if (v < n) break;
+    if (v < n) {
+      found = true;
+      break;
+    }
+  }
+  if (!found) {
+    v = 0;
+    if (status) atomicExch(status, (int)OLSGD_ETIMEOUT);
   }
   idx[t_id] = (int32_t)v;
 }
@@ -94,6 +107,12 @@ __global__ void identity_indices_kernel(int32_t* __restrict__ idx, int total, in
 }
 
 }  // namespace
+
+int epoch_rule_half_bits(int64_t n) {
+  int bits = 1;
+  while (((int64_t)1 << bits) < n) ++bits;       // ceil(log2 n), at least 1
+  return (bits + 1) / 2;
+}
 
 cudaError_t launch_identity_indices(int32_t* idx, int m, int batch, cudaStream_t s) {
   const int total = m * batch, threads = 256;
@@ -114,16 +133,14 @@ cudaError_t launch_minibatch_indices(int32_t* idx, uint64_t seed, int m, int64_t
 
 cudaError_t launch_minibatch_indices_epoch(int32_t* idx, uint64_t seed, int m, int64_t k, int batch,
                                            int64_t n, int worker_offset, const int64_t* k_ptr,
-                                           cudaStream_t s) {
-  int bits = 1;
-  while (((int64_t)1 << bits) < n) ++bits;       // ceil(log2 n), at least 1
-  const int h = (bits + 1) / 2;
+                                           int* status, cudaStream_t s) {
+  const int h = epoch_rule_half_bits(n);
   const int total = m * batch, threads = 128;
   return launch_chained(minibatch_indices_epoch_kernel, dim3((total + threads - 1) / threads),
                         dim3(threads), 0, s, idx, (uint32_t)(seed & 0xFFFFFFFFu),
                         (uint32_t)(seed >> 32), m, (uint64_t)k,
                         reinterpret_cast<const long long*>(k_ptr), batch, (uint32_t)n, h,
-                        (uint32_t)worker_offset);
+                        (uint32_t)worker_offset, status);
 }
 
 cudaError_t launch_counter(int64_t* p, int64_t value, int64_t by, bool set, cudaStream_t s) {

@@ -252,12 +252,11 @@ template <int BN, int STAGES>
 cudaError_t launch_one(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMap& mb,
                        cudaStream_t s) {
   constexpr size_t smem = (size_t)STAGES * (kBM * kBK * 2 + BN * kBK * 2) + sizeof(SharedCtl) + 1024;
-  static bool configured = false;
+  static PerDeviceSmem configured;
   auto kern = gemm_tc_kernel<BN, STAGES>;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  {
+    const cudaError_t e = ensure_dynamic_smem(configured, kern, smem);
     if (e != cudaSuccess) return e;
-    configured = true;
   }
   EpiArgs ea;
   ea.epilogue = a.epilogue;
@@ -329,7 +328,7 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, cudaStream_t s) {
       // whole grid is resident in one wave
       const int64_t ctas = (int64_t)(a.Nb / 64) * (a.Ma / kBM) * a.m;
       if (short_k) return launch_one<64, 2>(a, ma, mb, s);
-      return ctas > 148 ? launch_one<64, 4>(a, ma, mb, s) : launch_one<64, 8>(a, ma, mb, s);
+      return ctas > sm_count() ? launch_one<64, 4>(a, ma, mb, s) : launch_one<64, 8>(a, ma, mb, s);
     }
   }
 }

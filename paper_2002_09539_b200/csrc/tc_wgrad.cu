@@ -569,14 +569,11 @@ cudaError_t launch_wgrad_tc_batch(const GemmArgs* args, int n, cudaStream_t s) {
   if (n_stages > kWStages) n_stages = kWStages;
   if (n_stages < 2 || fused) n_stages = 2;
   const size_t smem = fixed + (size_t)n_stages * kWN * kBK * 2 + (fused ? 8 * kXuPerWarp : 0);
-  static size_t configured[2] = {0, 0};
-  if (smem > configured[fused]) {
-    cudaError_t e = fused ? cudaFuncSetAttribute(wgrad_tc_kernel<true>,
-                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-                          : cudaFuncSetAttribute(wgrad_tc_kernel<false>,
-                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  static PerDeviceSmem configured[2];
+  {
+    const cudaError_t e = fused ? ensure_dynamic_smem(configured[1], wgrad_tc_kernel<true>, smem)
+                                : ensure_dynamic_smem(configured[0], wgrad_tc_kernel<false>, smem);
     if (e != cudaSuccess) return e;
-    configured[fused] = smem;
   }
   if (fused)
     return launch_chained(wgrad_tc_kernel<true>, dim3(ctas), dim3(kFusedThreads), smem, s, wb, num_kb,

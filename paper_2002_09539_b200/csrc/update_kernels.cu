@@ -272,9 +272,9 @@ __global__ void virtual_sequence_kernel(const float* __restrict__ x, const float
 cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t s) {
   const int64_t n4 = (a.P + 3) / 4;
   const int64_t gx = (n4 + kUpdateThreads - 1) / kUpdateThreads;
-  // enough blocks for a few waves over 148 SMs; the rest of the worker
+  // enough blocks for a few waves over the multiprocessors; the rest of the worker
   // dimension is walked inside the thread so the anchor strip is reused
-  const int64_t target_blocks = 148 * 16;
+  const int64_t target_blocks = (int64_t)sm_count() * 16;
   int gy = (int)((target_blocks + gx - 1) / gx);
   if (gy < 1) gy = 1;
   if (gy > a.m) gy = a.m;

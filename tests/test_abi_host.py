@@ -96,3 +96,21 @@ def test_init_rejects_null_and_small_workspace_without_touching_the_device(lib):
     assert lib.olsgd_destroy(None) == 0
     assert lib.olsgd_local_step(None, None) == 1
     assert lib.olsgd_period_sync(None) == 1
+
+
+def test_kernel_attributes_are_remembered_per_device(lib):
+    # one process may open contexts on several GPUs; "this kernel's shared-memory limit is
+    # configured" must be remembered per device, which the library checks on its own table
+    assert lib.olsgd_selftest_per_device_table() == 0
+
+
+def test_epoch_rule_cycle_walk_domain_is_below_four_n(lib):
+    # the permutation's domain 2^(2h) must cover n and stay below 4 n: then a pass of the
+    # cycle walk lands in [0, n) with probability > 1/4 and fewer than 4 passes are expected,
+    # far from the 64 after which the device raises its status word
+    for n in list(range(1, 300)) + [1023, 1024, 1025, 5000, 65535, 65536, 65537, 10 ** 6,
+                                    2 ** 30 - 1, 2 ** 30, 2 ** 30 + 1, 2 ** 31 - 1]:
+        h = lib.olsgd_epoch_rule_half_bits(n)
+        assert h >= 1 and n <= 2 ** (2 * h) and (2 ** (2 * h) < 4 * n or n <= 2), (n, h)
+    assert lib.olsgd_epoch_rule_half_bits(0) == -1
+    assert lib.olsgd_epoch_rule_half_bits(2 ** 31) == -1

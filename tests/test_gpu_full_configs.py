@@ -139,6 +139,60 @@ def test_mlp_configs_full_length(name):
     assert abs(np.linalg.norm(xbar) - gold["norm2_mean_model"]) <= 0.02 * gold["norm2_mean_model"]
 
 
+def test_config3_late_regime_resynchronised_with_the_oracle():
+    """Config 3 beyond the point where its trajectory stops being reproducible: the small-loss,
+    large-momentum regime of iterations 300-1000.  Chaos cannot be followed over hundreds of
+    iterations, but ten can: at the period boundaries k0 the device's whole state (x_i, u_i, z,
+    v) is read back and handed to a fresh exact-fp64 oracle as ITS start, exactly as x0 is at
+    k = 0 (an input to both sides, no expected value comes from the device); both then run
+    ten iterations on the rule's own minibatches, and every per-worker minibatch loss of those
+    iterations is held to the 2e-2 bar, as are the parameters after them."""
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    c = si.CONFIGS["c3"]
+    m, steps = c["m"], 10
+    X, y = si.mixture_data(0, m, c["n"], c["dims"][0])
+    x0 = si.model_init(0, "mlp", c["dims"])
+    opt = OverlapLocalSGD("mlp", m=m, tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"],
+                          beta=c["beta"], mu=c["mu"], batch=c["batch"], seed=0, dims=c["dims"],
+                          gemm_bf16=c["gemm_bf16"], x0=x0, X=to_dev(X), y=to_dev(y))
+    first_loss = None
+    for k0 in (300, 600, 900):
+        warm = torch.zeros((k0 - opt.iteration, m), device="cuda")
+        opt.run(k0 - opt.iteration, warm)        # long run: replayed graph blocks, as bench.py
+        if first_loss is None:
+            first_loss = float(warm[0].mean())
+        assert opt.iteration == k0
+        st = olsgd.OverlapLocalSGD(x0, m, c["tau"], c["gamma"], c["alpha"], c["beta"], c["mu"])
+        st.x = np.stack([opt.get_params(i).copy() for i in range(m)]).astype(np.float64)
+        st.u = np.stack([opt.get_params(-5 - i).copy() for i in range(m)]).astype(np.float64)
+        st.z = opt.get_params(-1).astype(np.float64)
+        st.v = opt.get_params(-2).astype(np.float64)
+        st.k = k0
+        x_start, z_start = st.x.copy(), st.z.copy()
+        # the regime the test is about: trained far below the start, momentum buffers loaded
+        assert float(warm[-10:].mean()) < 0.5 * first_loss
+        assert np.abs(st.u).max() > 0 and np.abs(st.v).max() > 0
+        lg = torch.zeros((steps, m), device="cuda")
+        opt.run(steps, lg)
+        lg = lg.cpu().numpy()
+        st, lo, _ = runner.run_model("mlp", c["dims"], X, y, None, m=m, tau=c["tau"],
+                                     batch=c["batch"], gamma=c["gamma"], alpha=c["alpha"],
+                                     beta=c["beta"], mu=c["mu"], seed=0, iters=steps, state=st)
+        assert st.k == opt.iteration == k0 + steps
+        # every iteration, every worker: |loss_gpu - loss_oracle| <= 2e-2 of the iteration's scale
+        scale = np.abs(lo).max(axis=1, keepdims=True)
+        assert (np.abs(lg - lo) <= TOL_BF16_LOSS * scale).all(), (k0, np.abs(lg - lo).max(), scale.min())
+        mean_g, mean_o = lg.mean(axis=1), lo.mean(axis=1)
+        assert (np.abs(mean_g - mean_o) <= TOL_BF16_LOSS * mean_o).all(), (k0, mean_g, mean_o)
+        assert state_err(opt, st) <= TOL_BF16_LOSS, (k0, state_err(opt, st))
+        # the ten steps themselves (not the state they started from) agree as well
+        xg, zg, _ = opt.state()
+        moved_o = np.abs(st.x - x_start).max()
+        assert np.abs((xg - x_start) - (st.x - x_start)).max() <= 0.1 * moved_o, k0
+        assert np.abs((zg - z_start) - (st.z - z_start)).max() <= 0.1 * np.abs(st.z - z_start).max(), k0
+    opt.close()
+
+
 @pytest.mark.parametrize("m", [8, 16, 64])
 def test_config5_parity_size_point(m):
     from paper_2002_09539_b200 import OverlapLocalSGD

@@ -115,6 +115,70 @@ def test_bf16_mode_is_close_to_exact_and_not_identical():
     assert np.abs(g0 - g1).max() < 2e-2 * np.abs(g0).max()
 
 
+def test_bf16_rounding_points_worked_by_hand():
+    """Which operands `bf16_operands=True` rounds, pinned on a 2-2-2 network whose values sit on
+    bf16 ties, with the expected loss and gradient worked out by hand below (no oracle routine
+    is called to produce them).  bf16 keeps 8 significant bits; with e = 2^-8 the representable
+    numbers are e apart in [0.5, 1), 2e apart in [1, 2), 4e in [2, 4), and a tie goes to the
+    neighbour whose last kept bit is 0.
+
+    Roundings used:  1+e -> 1,  1+3e -> 1+4e,  2+2e -> 2,  0.5+e/2 would go to 0.5 and 64.125
+    to 64 (but biases are NOT rounded).
+
+    Forward.  q(X) = [[-1, 1], [1+4e, -0.5], [.75, .25]],  q(W1) = [[1, .5], [1+4e, -1]],
+    b1 = [0.5+e/2, 1].
+      sample 0: unit 0 = -1 + .5 + .5 + e/2 = e/2;                unit 1 = -(1+4e) - 1 + 1 < 0
+      sample 1: unit 0 = (1+4e) - .25 + .5 + e/2 = 1.25 + 4.5e;   unit 1 = (1+4e)^2 + .5 + 1
+      sample 2: unit 0 = .75 + .125 + .5 + e/2 = 1.375 + e/2;     unit 1 = .75(1+4e) - .25 + 1
+    rounded hidden activations: [[e/2, 0], [1.25+4e, 2.5+8e], [1.375, 1.5+4e]]
+    (1.5+3e is a tie: 1.5+2e ends in an odd bit, so it goes to 1.5+4e).
+    q(W2) = [[1, -(1+4e)], [3, 2]], b2 = [0, 64.125], so
+      logit_1 - logit_0 = h . [2, 3+4e] + 64.125  >= 64 for every sample:
+    softmax puts probability 1 (to 1e-27) on class 1.  Samples 0 and 1 carry label 0, so their
+    loss is that gap; sample 2 carries label 1 and contributes 0:
+      gap_0 = 2(e/2) + 64.125 = 64.125 + e
+      gap_1 = 2(1.25+4e) + (2.5+8e)(3+4e) + 64.125 = 74.125 + 42e + 32e^2
+      loss  = (gap_0 + gap_1) / 3.
+
+    Backward.  d loss / d logits = [-1/3, +1/3] for samples 0 and 1, zero for sample 2.
+      bias gradient of layer 2 (from the unrounded values): [-2/3, 2/3]
+      D = q(1/3): 1/3 = 1.0101010 1010..b x 2^-2 rounds up to 1.0101011b x 2^-2 = 171/512
+      dW2 = [-D, D]^T (h_0 + h_1) with h_0 + h_1 = [1.25 + 4.5e, 2.5 + 8e]
+      into the hidden layer: D * (q(W2)[1] - q(W2)[0]) = D [2, 3+4e], masked by h > 0:
+        sample 0: [2D, 0],   sample 1: [2D, D(3+4e)]
+      bias gradient of layer 1 (unrounded): [4D, D(3+4e)] = [171/128, 33003/32768]
+      rounded for the weight gradient: 2D = 171/256 is representable; D(3+4e) = 33003/32768,
+      33003 = 10000000 11101011b rounds up to 10000001b x 2^8, i.e. 129/128
+      dW1 row 0 = 2D (q(x_0) + q(x_1)) = 2D [4e, .5] = [8De, D]
+      dW1 row 1 = (129/128) q(x_1) = (129/128) [1+4e, -.5].
+
+    Leaving out any one rounding (input, weight, hidden activation, either back-propagated
+    gradient), rounding a bias, or summing the bias gradient from rounded values changes the
+    loss by >= 2.8e-5 relative or a gradient entry by >= 6.5e-4.
+    """
+    e = 2.0 ** -8
+    X = np.array([[-(1 + e), 1 + e], [1 + 3 * e, -0.5], [0.75, 0.25]])
+    labels = np.array([0, 0, 1])
+    W1, b1 = np.array([[1 + e, 0.5], [1 + 3 * e, -1.0]]), np.array([0.5 + e / 2, 1.0])
+    W2, b2 = np.array([[1 + e, -(1 + 3 * e)], [3.0, 2 + 2 * e]]), np.array([0.0, 64.125])
+    params = np.concatenate([W1.ravel(), b1, W2.ravel(), b2])
+    loss, g = models.mlp_loss_grad([2, 2, 2], params, X, labels, bf16_operands=True)
+
+    D = 171.0 / 512.0
+    want_loss = ((64.125 + e) + (74.125 + 42 * e + 32 * e * e)) / 3.0
+    want = np.array([8 * D * e, D,                                  # dW1 row 0
+                     129.0 / 128.0 * (1 + 4 * e), -129.0 / 256.0,   # dW1 row 1
+                     171.0 / 128.0, 33003.0 / 32768.0,              # db1
+                     -D * (1.25 + 4.5 * e), -D * (2.5 + 8 * e),     # dW2 row 0
+                     D * (1.25 + 4.5 * e), D * (2.5 + 8 * e),       # dW2 row 1
+                     -2.0 / 3.0, 2.0 / 3.0])                        # db2
+    assert loss == pytest.approx(want_loss, rel=1e-13)
+    assert np.abs(g - want).max() <= 1e-13, np.abs(g - want)
+    # the same network without operand rounding is visibly different on both
+    l_exact, g_exact = models.mlp_loss_grad([2, 2, 2], params, X, labels)
+    assert abs(l_exact - want_loss) > 1e-5 * want_loss and np.abs(g_exact - want).max() > 1e-4
+
+
 def test_full_objective_is_mean_over_workers():
     rng = np.random.default_rng(7)
     X, y, w = rng.standard_normal((3, 9, 4)), rng.standard_normal((3, 9)), rng.standard_normal(4)

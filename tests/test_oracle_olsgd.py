@@ -322,6 +322,26 @@ def test_brute_force_tiny_problem_with_real_minibatches():
     assert np.allclose(st.z, np.array(z), rtol=1e-12, atol=1e-14)
 
 
+def test_runner_resumed_from_a_copied_state_continues_the_same_trajectory():
+    # the minibatch rule is a function of k alone, so a run split at a period boundary and
+    # resumed from copies of (x, u, z, v, k) must give the bits of the unsplit run
+    from oracle import runner
+    rng = np.random.default_rng(19)
+    m, n, d = 3, 20, 4
+    X, y = rng.standard_normal((m, n, d)), rng.standard_normal((m, n))
+    kw = dict(m=m, tau=2, batch=5, gamma=0.05, alpha=0.6, beta=0.7, mu=0.9, seed=3)
+    whole, l_whole, _ = runner.run_model("linreg", [d], X, y, np.zeros(d), iters=10, **kw)
+    first, l_a, _ = runner.run_model("linreg", [d], X, y, np.zeros(d), iters=6, **kw)
+    again = olsgd.OverlapLocalSGD(np.zeros(d), m, 2, 0.05, 0.6, 0.7, 0.9)
+    again.x, again.u, again.z, again.v, again.k = (first.x.copy(), first.u.copy(), first.z.copy(),
+                                                   first.v.copy(), first.k)
+    second, l_b, _ = runner.run_model("linreg", [d], X, y, None, iters=4, state=again, **kw)
+    assert second.k == 10
+    assert np.array_equal(second.x, whole.x) and np.array_equal(second.z, whole.z)
+    assert np.array_equal(second.v, whole.v) and np.array_equal(second.u, whole.u)
+    assert np.array_equal(np.concatenate([l_a, l_b]), l_whole)
+
+
 # ------------------------------------------------------------ Eq. 2, Local SGD
 
 def test_local_sgd_tau_one_is_sgd_on_the_averaged_gradient():
