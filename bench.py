@@ -30,6 +30,7 @@ import synth_inputs as si  # noqa: E402
 METRIC = "simulated_worker_steps_per_sec"
 UNIT = "worker-steps/s"
 L2_BYTES = 126 * 2 ** 20
+MAX_BLOCKS = 2000          # upper bound on repeated timed blocks
 
 
 def measured_peaks():
@@ -125,13 +126,22 @@ class ClockSampler:
 
 # ------------------------------------------------------------------ roofline accounting
 
+def git_blob_id(path):
+    """The id git gives a file's content (sha1 of the header "blob <size>" + NUL + bytes)."""
+    import hashlib
+    with open(path, "rb") as f:
+        data = f.read()
+    return hashlib.sha1(b"blob %d\0" % len(data) + data).hexdigest()
+
+
+CSRC = os.path.join(ROOT, "paper_2002_09539_b200", "csrc")
+
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the ncu capture
-# summarised in profiles/, keyed by (workload, kernel class); (ordinary step, sync step).
-# An entry must be removed when its kernel changes.
+# summarised in profiles/, keyed by (workload, gemm mode, kernel class): (ordinary step, sync
+# step), the kernel's source file and that file's git blob id when the counters were taken.
+# When the file has changed since, the entry no longer describes the kernel and `traffic`
+# is reported as null.
 NCU_TRAFFIC = {
-    # (workload, gemm mode, kernel class)
-    ("c3", 3, "update"): (1426.4e6, 1445.1e6),      # profiles/fused_update_c3_mlp.txt
-    ("c3", 1, "wgrad_update"): (1180.1e6, 1203.4e6),  # profiles/wgrad_update_fused_c3_mlp.txt
 }
 
 
@@ -139,7 +149,13 @@ def ncu_traffic(name, mode, kernel_class, sync_fraction):
     t = NCU_TRAFFIC.get((name, mode, kernel_class))
     if t is None:
         return None
-    return int((1.0 - sync_fraction) * t[0] + sync_fraction * t[1])
+    plain, sync, source, blob = t
+    try:
+        if git_blob_id(os.path.join(CSRC, source)) != blob:
+            return None
+    except OSError:
+        return None
+    return int((1.0 - sync_fraction) * plain + sync_fraction * sync)
 
 
 def layer_is_fused(c, p):
@@ -177,7 +193,140 @@ def algorithmic_bytes(c, kernel_class, P, sync_fraction):
         return m * rest * per + sync_fraction * 4 * rest
     if kernel_class == "anchor":
         return 4 * m * P + (16 if c["beta"] != 0.0 else 4) * P
+    if kernel_class == "output_layer" and c.get("kind") in ("softmax", "linreg"):
+        # the kernels of a model without hidden layers (forward + loss, weight gradient with the
+        # update applied on the spot): the step's minibatch rows ONCE, the parameters read by
+        # the forward pass, read and written by the update (with the momentum buffer, if any),
+        # the anchor once on sync steps
+        rows = m * c["batch"] * c["dims"][0] * 4
+        return rows + m * P * (4 + 8 + (8 if mom else 0)) + sync_fraction * 4 * P
     return None
+
+
+def gemm_rooflines(c, layers_prof, n_steps, peaks):
+    """Per tcgen05 GEMM launch of the MLP path: duration, TFLOP/s and the fraction of its bound,
+    min(bf16 peak, arithmetic intensity x HBM bandwidth), from the per-layer device profile."""
+    if c.get("kind") != "mlp" or not c.get("gemm_bf16"):
+        return []
+    d, m, B = c["dims"], c["m"], c["batch"]
+    L = len(d) - 1
+    peak_flops = peaks["bf16_tflops"] * 1e12
+    hbm = peaks["hbm_gbs"] * 1e9
+    out = []
+
+    def entry(name, cls, tag, flops, nbytes):
+        launches, ms = layers_prof[cls][tag]
+        if launches <= 0:
+            return
+        us = ms * 1e3 / launches
+        bound_s = max(flops / peak_flops, nbytes / hbm)
+        out.append(dict(kernel=name, launches_per_step=round(launches / n_steps, 3), us=round(us, 2),
+                        tflops=round(flops / (us * 1e-6) / 1e12, 1),
+                        frac_of_bf16_peak=round(flops / (us * 1e-6) / peak_flops, 4),
+                        flop_per_byte=round(flops / nbytes, 1), bound_us=round(bound_s * 1e6, 2),
+                        bound="hbm" if nbytes / hbm > flops / peak_flops else "tensor",
+                        frac_of_bound=round(bound_s * 1e6 / us, 4)))
+
+    for l in range(1, L):
+        # forward: W_l [d_l][d_{l-1}] bf16 read once, the batch operand read, H_l written in
+        # both layouts
+        flops = 2.0 * m * B * d[l] * d[l - 1]
+        nbytes = m * (2 * d[l] * d[l - 1] + 2 * B * d[l - 1] + 4 * B * d[l])
+        entry("gemm_tc_kernel forward, layer %d (%dx%d, batch %d)" % (l, d[l], d[l - 1], B),
+              "forward", l, flops, nbytes)
+    for l in range(1, L - 1):
+        # input gradient of hidden layer l: W_{l+1} read in place (bf16 shadow), dA_{l+1} read,
+        # the ReLU mask read, dA_l written in both layouts
+        flops = 2.0 * m * B * d[l] * d[l + 1]
+        nbytes = m * (2 * d[l + 1] * d[l] + 2 * B * d[l + 1] + 2 * B * d[l] + 4 * B * d[l])
+        entry("gemm_tc_kernel input gradient, layer %d (%dx%d, batch %d)" % (l, d[l], d[l + 1], B),
+              "backward", l, flops, nbytes)
+    return out
+
+
+def flat_point(P, m, K, W, peaks):
+    """Config 5 at one (P, m): the stand-alone fused update and worker-mean/anchor kernels on a
+    flat parameter vector with external gradients.  Returns the point's record."""
+    import torch
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    c = si.CONFIGS["c5"]
+    x0 = torch.randn(P, device="cuda")
+    g = torch.randn((m, P), device="cuda") * c["grad_std"]
+    kw = dict(m=m, tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"], beta=c["beta"], mu=c["mu"],
+              flat_P=P, x0=x0)
+    opt = OverlapLocalSGD("flat", **kw)
+
+    def steps(count):
+        for _ in range(count):
+            opt.local_step_with_grads(g)
+            if opt.iteration % c["tau"] == 0:
+                opt.period_sync()
+
+    steps(W)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n0 = opt.launch_count
+    e0.record()
+    steps(K)
+    opt.main.wait_stream(opt.side)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    launches = opt.launch_count - n0
+    opt.profile_enable(True)
+    steps(K)
+    prof_overlap = opt.profile_read()
+    opt.profile_enable(False)
+    # the per-kernel bandwidths are taken with the two streams serialised: under overlap the
+    # anchor kernel shares HBM with the next period's update kernels and its event-bracketed
+    # duration measures that sharing, not the kernel
+    opt.close()
+    opt = OverlapLocalSGD("flat", overlap=False, **kw)
+    steps(W)
+    opt.profile_enable(True)
+    steps(K)
+    prof = opt.profile_read()
+    opt.profile_enable(False)
+    opt.close()
+    cc = dict(c, m=m)
+    n_sync = K // c["tau"]
+    upd_b = algorithmic_bytes(cc, "update", P, n_sync / K)
+    anc_b = algorithmic_bytes(cc, "anchor", P, 0)
+    upd_ms = prof["update"][1] / prof["update"][0]
+    anc_ms = prof["anchor"][1] / max(1, prof["anchor"][0])
+    state_mb = (3 * m * P + 2 * P + m * P) * 4 / 1e6
+    point = dict(
+        P=P, m=m, worker_steps_per_s=round(m * K / (ms * 1e-3), 1),
+        ms_per_step=round(ms / K, 4), gpu_launches=int(launches),
+        update_gbs=round(upd_b / upd_ms / 1e6, 1), anchor_gbs=round(anc_b / anc_ms / 1e6, 1),
+        update_us=round(upd_ms * 1e3, 2), anchor_us=round(anc_ms * 1e3, 2),
+        anchor_us_overlapped=round(prof_overlap["anchor"][1] * 1e3 /
+                                   max(1, prof_overlap["anchor"][0]), 2),
+        update_frac_measured=round(upd_b / upd_ms / 1e6 / peaks["hbm_gbs"], 4),
+        anchor_frac_measured=round(anc_b / anc_ms / 1e6 / peaks["hbm_gbs"], 4),
+        update_frac_8000=round(upd_b / upd_ms / 1e6 / 8000.0, 4),
+        anchor_frac_8000=round(anc_b / anc_ms / 1e6 / 8000.0, 4),
+        resident_mb=round(state_mb, 1), in_l2=bool(state_mb * 1e6 < L2_BYTES))
+    del opt, g, x0
+    torch.cuda.empty_cache()
+    return point
+
+
+def standalone_kernel_rooflines(peaks, steps=12, warmup=4):
+    """The metric's second half: the stand-alone fused update kernel and the worker-mean/anchor
+    kernel on config 5's 10M x 16 and 50M x 64 points, streams serialised, as HBM GB/s against
+    the measured copy bandwidth and against 8 TB/s."""
+    out = []
+    for P, m in ((10_000_000, 16), (50_000_000, 64)):
+        pt = flat_point(P, m, steps, warmup, peaks)
+        where = "config 5, P=%dM, m=%d, tau=4, momentum, streams serialised" % (P // 1_000_000, m)
+        out.append(dict(kernel="fused_update_kernel", workload=where, us=pt["update_us"],
+                        gbs=pt["update_gbs"], frac_of_measured=pt["update_frac_measured"],
+                        frac_of_8000=pt["update_frac_8000"]))
+        out.append(dict(kernel="worker_mean_anchor_kernel", workload=where, us=pt["anchor_us"],
+                        gbs=pt["anchor_gbs"], frac_of_measured=pt["anchor_frac_measured"],
+                        frac_of_8000=pt["anchor_frac_8000"]))
+    return out
 
 
 # ------------------------------------------------------------------ our arm
@@ -237,47 +386,96 @@ def run_ours(args, rank, world):
         return max_over_ranks(e0.elapsed_time(e1), world, "cuda")
 
     # ---- device-resident throughput
+    # W warm-up steps as asked, then (still untimed) one run long enough for olsgd_run to
+    # capture its block of iterations, so that the timed blocks replay it.  A timed block is
+    # EXACTLY K steps between a barrier + synchronize on both sides; blocks are repeated until
+    # MIN_TIMED_S have been timed, and the median block is reported.
     opt.run(W)
+    block = opt.graph_block
+    opt.run(3 * block)
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
         sampler.wait_first_sample()
-    launches0 = opt.launch_count
-    ms = timed(lambda: opt.run(K))
+    launches0, replays0 = opt.launch_count, opt.graph_replays
+    times = [timed(lambda: opt.run(K))]
     launches = opt.launch_count - launches0
-    replays = opt.graph_replays
+    n_blocks = int(min(MAX_BLOCKS, max(1, np.ceil(args.min_time * 1e3 / times[0]))))
+    for _ in range(n_blocks - 1):
+        times.append(timed(lambda: opt.run(K)))
+    replays = opt.graph_replays - replays0
     clocks = sampler.stop() if rank == 0 else None
+    ms = float(np.median(times))
     value = world * m * K / (ms * 1e-3)
+    per_block = replays // len(times)
+    timing = dict(blocks=len(times), timed_s=round(sum(times) * 1e-3, 3),
+                  ms_per_step_median=round(ms / K, 4), ms_per_step_min=round(min(times) / K, 4),
+                  ms_per_step_max=round(max(times) / K, 4),
+                  path=("olsgd_run: %d replay(s) of the captured %d-iteration graph + %d plain "
+                        "step(s) per timed block" % (per_block, block, K - per_block * block))
+                  if per_block else "olsgd_run: plain launches (K is shorter than the captured block)")
 
     # ---- per-kernel-class device time (second pass, every launch bracketed by events)
+    KP = max(K, 2 * block)
     opt.profile_enable(True)
-    opt.run(K)
-    prof = opt.profile_read()
+    opt.run(KP)
+    layers_prof = opt.profile_read_layers()
     opt.profile_enable(False)
+    prof = {k: (sum(t[0] for t in v), sum(t[1] for t in v)) for k, v in layers_prof.items()}
     busy = {k: v for k, v in prof.items() if v[0] > 0}
     total_ms = sum(v[1] for v in busy.values())
     dominant = max(busy, key=lambda k: busy[k][1])
     peaks = measured_peaks()
-    n_sync = sum(1 for k in range(K) if (k + 1) % c["tau"] == 0)
-    # the roofline entry describes the HBM-bound kernel class that took the most device time
-    ranked = sorted(busy, key=lambda k: -busy[k][1])
-    roof_class = next((k for k in ranked if algorithmic_bytes(c, k, P, 0) is not None), None)
+    n_sync = sum(1 for k in range(KP) if (k + 1) % c["tau"] == 0) if not local_sgd else 0
+    if c["kind"] in ("softmax", "linreg"):
+        # no hidden layers: the time is in the output-layer kernels (forward + loss, weight
+        # gradient with the update), which together need the step's rows once
+        roof_class = "output_layer"
+        parts = [k for k in ("forward", "loss", "backward") if k in busy]
+        avg_ms = sum(busy[k][1] / busy[k][0] for k in parts)
+    else:
+        # the HBM-bound kernel class that took the most device time
+        ranked = sorted(busy, key=lambda k: -busy[k][1])
+        roof_class = next((k for k in ranked if algorithmic_bytes(c, k, P, 0) is not None), None)
+        avg_ms = busy[roof_class][1] / busy[roof_class][0] if roof_class else None
     if roof_class is not None:
-        ab = algorithmic_bytes(c, roof_class, P, n_sync / K)
-        avg_ms = busy[roof_class][1] / busy[roof_class][0]
+        ab = algorithmic_bytes(c, roof_class, P, n_sync / KP)
         achieved = ab / (avg_ms * 1e-3) / 1e9
+        traffic = ncu_traffic(name, c["gemm_bf16"], roof_class, n_sync / KP)
         roofline = dict(bound="hbm", kernel=roof_class, achieved=round(achieved, 1),
                         peak=peaks["hbm_gbs"], unit="GB/s", frac=round(achieved / peaks["hbm_gbs"], 4),
-                        frac_of_8000=round(achieved / 8000.0, 4),
-                        traffic=ncu_traffic(name, c["gemm_bf16"], roof_class, n_sync / K),
+                        frac_of_8000=round(achieved / 8000.0, 4), traffic=traffic,
                         peak_source=peaks["source"], avg_launch_us=round(avg_ms * 1e3, 2),
                         algorithmic_bytes_per_launch=int(ab))
+        if traffic:
+            # the same launch by the DRAM counters of the ncu capture instead of the byte count
+            roofline.update(achieved_by_traffic=round(traffic / (avg_ms * 1e-3) / 1e9, 1),
+                            frac_by_traffic=round(traffic / (avg_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4))
     else:
         roofline = dict(bound="hbm", kernel=None, achieved=None, peak=peaks["hbm_gbs"], unit="GB/s",
                         frac=None, traffic=None, peak_source=peaks["source"])
     roofline.update(dominant_class=dominant,
                     class_share={k: round(v[1] / total_ms, 4) for k, v in busy.items()},
-                    class_us_per_step={k: round(v[1] * 1e3 / K, 2) for k, v in busy.items()})
+                    class_us_per_step={k: round(v[1] * 1e3 / KP, 2) for k, v in busy.items()},
+                    kernels=[])
+    if c["kind"] == "mlp" and c["gemm_bf16"]:
+        # The tensor-core GEMMs one launch at a time: a second context with the library's
+        # streams serialised (no anchor refresh, gather or output-layer kernel beside them),
+        # so that the bracketed duration is the kernel's own; warm caches, as inside a step.
+        ser = OverlapLocalSGD(c["kind"], m=c["m"], tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"],
+                              beta=c["beta"], mu=c["mu"], batch=c["batch"], seed=seed, dims=c["dims"],
+                              gemm_bf16=c["gemm_bf16"], x0=x0, X=Xd, y=yd, local_sgd=local_sgd,
+                              overlap=False)
+        ser.run(W)
+        ser.profile_enable(True)
+        ser.run(KP)
+        ser_prof = ser.profile_read_layers()
+        ser.profile_enable(False)
+        ser.close()
+        del ser
+        roofline["kernels"] = gemm_rooflines(c, ser_prof, KP, peaks)
+        roofline["kernels_note"] = ("GEMM launches timed with the library's streams serialised "
+                                    "(each kernel alone on the GPU, warm caches)")
 
     # ---- end to end: host minibatches in, host losses out, through the C ABI
     pool = 4
@@ -292,31 +490,56 @@ def run_ours(args, rank, world):
         idx = rng.integers(0, n, size=(m, B))
         Xh.append(torch.from_numpy(np.stack([X[i][idx[i]] for i in range(m)])).to(host_dtype).pin_memory())
         yh.append(torch.from_numpy(np.stack([y[i][idx[i]] for i in range(m)])).pin_memory())
-    loss_h = torch.zeros((K + W, m), dtype=torch.float32).pin_memory()
+    loss_h = torch.zeros((K, m), dtype=torch.float32).pin_memory()
 
-    def e2e_steps(k0, count):
-        for t in range(k0, k0 + count):
-            opt.local_step_host(Xh[t % pool], yh[t % pool], loss_h[t])
+    def e2e_steps(count):
+        for t in range(count):
+            opt.local_step_host(Xh[t % pool], yh[t % pool], loss_h[t % K])
             if (opt.iteration) % c["tau"] == 0 and not local_sgd:
                 opt.period_sync()
 
-    e2e_steps(0, W)
+    def e2e_block():
+        # K steps from pinned host rows to host-visible losses, by the host's clock
+        barrier()
+        t0 = time.perf_counter()
+        e2e_steps(K)
+        opt.join()                      # host sees the last losses here
+        t1 = time.perf_counter()
+        return max_over_ranks((t1 - t0) * 1e3, world, "cuda")
+
+    e2e_steps(W)
     opt.join()
-    barrier()
-    t0 = time.perf_counter()
-    e2e_steps(W, K)
-    opt.join()                      # host sees the last losses here
-    t1 = time.perf_counter()
-    e2e_ms = (t1 - t0) * 1e3
-    e2e_ms = max_over_ranks(e2e_ms, world, "cuda")
-    assert np.isfinite(loss_h[W:].numpy()).all()
+    e2e_times = [e2e_block()]
+    n_e2e = int(min(MAX_BLOCKS, max(1, np.ceil(args.min_time * 1e3 / e2e_times[0]))))
+    for _ in range(n_e2e - 1):
+        e2e_times.append(e2e_block())
+    e2e_ms = float(np.median(e2e_times))
+    assert np.isfinite(loss_h.numpy()).all()
     e2e = dict(value=round(world * m * K / (e2e_ms * 1e-3), 1), unit=UNIT,
                h2d_bytes_per_step=int(Xh[0].numel() * Xh[0].element_size() +
                                       yh[0].numel() * yh[0].element_size()),
                d2h_bytes_per_step=int(m * 4), ms_per_step=round(e2e_ms / K, 4),
+               blocks=len(e2e_times), timed_s=round(sum(e2e_times) * 1e-3, 3),
+               ms_per_step_min=round(min(e2e_times) / K, 4),
+               ms_per_step_max=round(max(e2e_times) / K, 4),
                api="%s + olsgd_period_sync, pinned host minibatches (%s rows, int32 labels)"
                    % ("olsgd_local_step_host_bf16" if c["gemm_bf16"] else "olsgd_local_step_host",
                       "bf16" if c["gemm_bf16"] else "fp32"))
+    opt.close()
+    del opt, Xd, yd
+    torch.cuda.empty_cache()
+
+    # ---- the update and anchor kernels by themselves (the metric's second half)
+    if rank == 0 and world == 1 and not args.no_kernel_points:
+        roofline["kernels"] += standalone_kernel_rooflines(peaks)
+
+    # ---- with several GPUs: the same job once more with its WORKERS sharded over the ranks
+    # (one all-reduce of the anchor sum per period), in the same process group
+    sharded = None
+    if world > 1 and c["m"] % world == 0 and not local_sgd:
+        c_job = dict(c, tau=si.CONFIGS[name]["tau"] if not args.tau else c["tau"])
+        s_ms, _, _, _, _ = sharded_job(args, rank, world, c_job, name, K, W)
+        sharded = sharded_summary(c_job, P, world, s_ms, K)
 
     out = None
     if rank == 0:
@@ -337,11 +560,12 @@ def run_ours(args, rank, world):
                              "state fits in L2 (%.1f MB): steady-state training keeps it there"
                              % (resident / 1e6),
                        "replicas": world},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+            "clocks": clocks, "timing": timing, "e2e": e2e, "gpu_launches": int(launches),
             "graph_replays": int(replays),
             "roofline": roofline, "cpu_baseline": cpu,
         }
-    opt.close()
+        if world > 1:
+            out["sharded"] = sharded
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
@@ -371,65 +595,7 @@ def run_flat_sweep(args, rank, world):
         sampler.wait_first_sample()
     for P in Ps:
         for m in ms_:
-            x0 = torch.randn(P, device="cuda")
-            g = torch.randn((m, P), device="cuda") * c["grad_std"]
-            opt = OverlapLocalSGD("flat", m=m, tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"],
-                                  beta=c["beta"], mu=c["mu"], flat_P=P, x0=x0)
-
-            def steps(count):
-                for _ in range(count):
-                    opt.local_step_with_grads(g)
-                    if opt.iteration % c["tau"] == 0:
-                        opt.period_sync()
-
-            steps(W)
-            torch.cuda.synchronize()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            n0 = opt.launch_count
-            e0.record()
-            steps(K)
-            opt.main.wait_stream(opt.side)
-            e1.record()
-            torch.cuda.synchronize()
-            ms = e0.elapsed_time(e1)
-            launches = opt.launch_count - n0
-            opt.profile_enable(True)
-            steps(K)
-            prof_overlap = opt.profile_read()
-            opt.profile_enable(False)
-            # the per-kernel bandwidths are taken with the two streams serialised: under
-            # overlap the anchor kernel shares HBM with the next period's update kernels and
-            # its event-bracketed duration measures that sharing, not the kernel
-            opt.close()
-            opt = OverlapLocalSGD("flat", m=m, tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"],
-                                  beta=c["beta"], mu=c["mu"], flat_P=P, x0=x0, overlap=False)
-            steps(W)
-            opt.profile_enable(True)
-            steps(K)
-            prof = opt.profile_read()
-            opt.profile_enable(False)
-            cc = dict(c, m=m)
-            n_sync = K // c["tau"]
-            upd_b = algorithmic_bytes(cc, "update", P, n_sync / K)
-            anc_b = algorithmic_bytes(cc, "anchor", P, 0)
-            upd_ms = prof["update"][1] / prof["update"][0]
-            anc_ms = prof["anchor"][1] / max(1, prof["anchor"][0])
-            state_mb = (3 * m * P + 2 * P + m * P) * 4 / 1e6
-            points.append(dict(
-                P=P, m=m, worker_steps_per_s=round(m * K / (ms * 1e-3), 1),
-                ms_per_step=round(ms / K, 4), gpu_launches=int(launches),
-                update_gbs=round(upd_b / upd_ms / 1e6, 1), anchor_gbs=round(anc_b / anc_ms / 1e6, 1),
-                update_us=round(upd_ms * 1e3, 2), anchor_us=round(anc_ms * 1e3, 2),
-                anchor_us_overlapped=round(prof_overlap["anchor"][1] * 1e3 /
-                                           max(1, prof_overlap["anchor"][0]), 2),
-                update_frac_measured=round(upd_b / upd_ms / 1e6 / peaks["hbm_gbs"], 4),
-                anchor_frac_measured=round(anc_b / anc_ms / 1e6 / peaks["hbm_gbs"], 4),
-                update_frac_8000=round(upd_b / upd_ms / 1e6 / 8000.0, 4),
-                anchor_frac_8000=round(anc_b / anc_ms / 1e6 / 8000.0, 4),
-                resident_mb=round(state_mb, 1), in_l2=bool(state_mb * 1e6 < L2_BYTES)))
-            opt.close()
-            del opt, g, x0
-            torch.cuda.empty_cache()
+            points.append(flat_point(P, m, K, W, peaks))
     clocks = sampler.stop() if rank == 0 else None
     big = points[-1]
     return {
@@ -449,38 +615,34 @@ def run_flat_sweep(args, rank, world):
     }
 
 
-def run_sharded(args, rank, world):
-    """--shard-workers: ONE m-worker job whose worker dimension is split over the ranks
-    (m / N workers per GPU, same data set and minibatches as the single-GPU job).  The only
-    exchange is the sum of Eq. 5, an NCCL all-reduce of P floats per period issued on the
-    side stream between olsgd_period_sync_begin and olsgd_period_sync_finish, so it overlaps
-    the next period's local steps as in the paper.  Total work is fixed: strong scaling."""
+def sharded_summary(c, P, world, ms, K):
+    """The `sharded` record: one m-worker job whose workers are split over `world` GPUs, timed
+    over K steps in `ms` milliseconds (max over ranks)."""
+    m = c["m"]
+    return dict(value=round(m * K / (ms * 1e-3), 1), unit=UNIT, ms_per_step=round(ms / K, 4),
+                steps=int(K), scaling="strong", workers_per_gpu=m // world, m=m, n_gpus=int(world),
+                allreduce_bytes_per_period=int(P * 4), periods_per_step=round(1.0 / c["tau"], 4),
+                collective="ncclAllReduce(sum) of the padded parameter row on the side stream, "
+                           "between olsgd_period_sync_begin and olsgd_period_sync_finish")
+
+
+def sharded_job(args, rank, world, c, name, K, W):
+    """ONE m-worker job whose worker dimension is split over the ranks of the (already
+    initialised) process group: m / N workers per GPU, the same data set and minibatches as
+    the single-GPU job (seed 0, global worker ids).  The only exchange is the sum of Eq. 5, an
+    NCCL all-reduce of P floats per period issued on the side stream between
+    olsgd_period_sync_begin and olsgd_period_sync_finish, so it overlaps the next period's
+    local steps as in the paper.  Returns (ms over K steps as the max over ranks, launches,
+    per-class profile, |z| sum, clocks)."""
     import torch
     import torch.distributed as dist
     from paper_2002_09539_b200 import OverlapLocalSGD, class_pairs
-    from paper_2002_09539_b200.build import build
 
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local_rank)
-    if not dist.is_initialized():
-        if "MASTER_ADDR" not in os.environ:
-            os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT="29533")
-        dist.init_process_group("nccl", rank=rank, world_size=world,
-                                device_id=torch.device("cuda", local_rank))
-    if rank == 0:
-        build()
-    dist.barrier()
-    name = args.workload
-    c = dict(si.CONFIGS[name])
-    if c["gemm_bf16"] and args.gemm_mode:
-        c["gemm_bf16"] = args.gemm_mode
-    m, K, W = c["m"], args.steps, args.warmup
-    if m % world:
-        raise SystemExit("--shard-workers needs m (%d) divisible by the number of GPUs (%d)" % (m, world))
+    m = c["m"]
     m_loc, off = m // world, rank * (m // world)
     table = class_pairs(0, m, device="cpu").numpy() if c.get("non_iid") else None
     X, y, x0 = make_inputs(name, 0, table)          # every rank builds the same data set
-    P = n_params(c)
     Xd = torch.from_numpy(np.ascontiguousarray(X[off:off + m_loc])).cuda()
     yd = torch.from_numpy(np.ascontiguousarray(y[off:off + m_loc])).cuda()
     opt = OverlapLocalSGD(c["kind"], m=m_loc, tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"],
@@ -518,6 +680,37 @@ def run_sharded(args, rank, world):
     opt.profile_enable(False)
     zsum = float(np.abs(opt.get_params(-1)).sum())
     opt.close()
+    del opt, Xd, yd, buf
+    torch.cuda.empty_cache()
+    return ms, launches, prof, zsum, clocks
+
+
+def run_sharded(args, rank, world):
+    """--shard-workers: the sharded job (see sharded_job) as the whole benchmark.  Total work
+    is fixed: strong scaling."""
+    import torch
+    import torch.distributed as dist
+    from paper_2002_09539_b200.build import build
+
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if not dist.is_initialized():
+        if "MASTER_ADDR" not in os.environ:
+            os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT="29533")
+        dist.init_process_group("nccl", rank=rank, world_size=world,
+                                device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        build()
+    dist.barrier()
+    name = args.workload
+    c = dict(si.CONFIGS[name])
+    if c["gemm_bf16"] and args.gemm_mode:
+        c["gemm_bf16"] = args.gemm_mode
+    m, K, W = c["m"], args.steps, args.warmup
+    if m % world:
+        raise SystemExit("--shard-workers needs m (%d) divisible by the number of GPUs (%d)" % (m, world))
+    P = n_params(c)
+    ms, launches, prof, zsum, clocks = sharded_job(args, rank, world, c, name, K, W)
     out = None
     if rank == 0:
         busy = {k: v for k, v in prof.items() if v[0] > 0}
@@ -526,11 +719,12 @@ def run_sharded(args, rank, world):
             "steps": K, "warmup": W, "ms_per_step": round(ms / K, 4), "higher_is_better": True,
             "scaling": "strong", "vs_baseline": None,
             "dtype": "bf16" if c["gemm_bf16"] else "f32", "data": "synthetic",
-            "config": {"workload": workload_name(name, c), "m": m, "workers_per_gpu": m_loc,
+            "config": {"workload": workload_name(name, c), "m": m, "workers_per_gpu": m // world,
                        "tau": c["tau"], "batch": c["batch"], "dims": c["dims"], "P": P,
                        "parallelism": "workers sharded over %d GPU(s), all-reduce of the anchor sum" % world,
                        "allreduce_bytes_per_period": int(P * 4), "anchor_abs_sum": zsum},
             "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
+            "sharded": sharded_summary(c, P, world, ms, K),
             "roofline": dict(bound="hbm", kernel=None, traffic=None,
                              class_us_per_step={k: round(v[1] * 1e3 / K, 2) for k, v in busy.items()}),
             "cpu_baseline": None,
@@ -577,14 +771,31 @@ def cpu_cores():
         return os.cpu_count()
 
 
-def cpu_baseline(name, c, X, y, x0, seed, budget_s=15.0):
-    """The oracle as it stands, timed on a bounded sample of the same workload."""
-    m = c["m"]
-    t1 = oracle_steps(c, X, y, x0, seed, m, 1)              # one full iteration, all workers
-    iters = int(max(1, min(c["iters"], budget_s / max(t1, 1e-6))))
-    t = oracle_steps(c, X, y, x0, seed, m, iters)
-    return dict(value=round(m * iters / t, 2), unit=UNIT, cores=cpu_cores(), kind="oracle",
-                sample="%d iterations of all %d workers (%.1f s)" % (iters, m, t))
+def blas_threads(n):
+    """Context manager that pins the BLAS thread pool numpy uses to n threads."""
+    from threadpoolctl import threadpool_limits
+    return threadpool_limits(limits=int(n))
+
+
+def cpu_baseline(name, c, X, y, x0, seed, budget_s=10.0):
+    """The oracle as it stands, timed on a bounded sample of the same workload: with its BLAS
+    thread pool set to every core the process may use, and to one core.  The oracle visits the
+    workers one after another; the cores are used inside each worker's matrix products."""
+    m, cores = c["m"], cpu_cores()
+    with blas_threads(cores):
+        t1 = oracle_steps(c, X, y, x0, seed, m, 1)              # one full iteration, all workers
+        iters = int(max(1, min(c["iters"], budget_s / max(t1, 1e-6))))
+        t = oracle_steps(c, X, y, x0, seed, m, iters)
+    with blas_threads(1):
+        p1 = oracle_steps(c, X, y, x0, seed, 1, 1)              # one worker, one iteration
+        w1 = int(max(1, min(m, budget_s / max(p1, 1e-6))))
+        it1 = int(max(1, min(c["iters"], budget_s / max(p1 * w1, 1e-6))))
+        ts = oracle_steps(c, X, y, x0, seed, w1, it1)
+    return dict(value=round(m * iters / t, 2), unit=UNIT, cores=cores, kind="oracle",
+                sample="%d iterations of all %d workers (%.1f s), BLAS threads = %d" % (iters, m, t, cores),
+                one_core=dict(value=round(w1 * it1 / ts, 2), unit=UNIT, cores=1,
+                              sample="%d iterations of %d of the %d workers (%.1f s), BLAS threads = 1"
+                                     % (it1, w1, m, ts)))
 
 
 def run_reference(args, rank, world):
@@ -600,11 +811,12 @@ def run_reference(args, rank, world):
     K, W = args.steps, args.warmup
     m = c["m"]
     # bounded sample: a subset of the workers per step, sized so the run ends in minutes
-    t1 = oracle_steps(c, X, y, x0, 0, 1, 1)
-    budget = 150.0
-    workers = int(max(1, min(m, budget / ((K + W) * max(t1, 1e-6)))))
-    oracle_steps(c, X, y, x0, 0, workers, W)
-    t = oracle_steps(c, X, y, x0, 0, workers, K)
+    with blas_threads(cpu_cores()):
+        t1 = oracle_steps(c, X, y, x0, 0, 1, 1)
+        budget = 150.0
+        workers = int(max(1, min(m, budget / ((K + W) * max(t1, 1e-6)))))
+        oracle_steps(c, X, y, x0, 0, workers, W)
+        t = oracle_steps(c, X, y, x0, 0, workers, K)
     value = workers * K / t
     sample = "%d of %d workers per step, %d steps" % (workers, m, K)
     return {
@@ -640,6 +852,12 @@ def main():
                     help="c1-c4: override the configuration's period (to measure what a sync costs)")
     ap.add_argument("--P", type=int, default=0, help="c5 only: one parameter count")
     ap.add_argument("--m", type=int, default=0, help="c5 only: one worker count")
+    ap.add_argument("--min-time", type=float, default=1.0,
+                    help="repeat the timed block of --steps iterations until this many seconds "
+                         "have been timed (the median block is reported); 0: one block")
+    ap.add_argument("--no-kernel-points", action="store_true",
+                    help="skip the stand-alone update/anchor kernel measurements (config 5's "
+                         "10M x 16 and 50M x 64 points) that the default line carries")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     if args.warmup < 3:

@@ -236,12 +236,16 @@ int64_t olsgd_row_floats(const olsgd_ctx* ctx);
 olsgd_status olsgd_run(olsgd_ctx* ctx, int64_t n_iters, float* loss_device);
 
 /* How often olsgd_run has replayed its captured CUDA graph on this context so far.  Long
- * runs (at least three blocks of max(8, 2 tau)-odd iterations) are executed as replays of
- * one captured block; the iteration number the minibatch rule needs is then read from
+ * runs (at least three blocks of olsgd_graph_block iterations, or one block once the graph
+ * exists) are executed as replays of one captured block; the iteration number the minibatch rule needs is then read from
  * device memory.  Capturing needs main_stream to be a real stream: with the legacy default
  * stream (NULL) olsgd_run keeps launching kernel by kernel and this stays 0.  The results
  * are the same bits either way.                                                        */
 int64_t olsgd_graph_replays(const olsgd_ctx* ctx);
+/* Iterations in one captured block of this context: whole periods, an even count, at least
+ * eight.  A first olsgd_run of at least three blocks captures the graph; after that every
+ * olsgd_run of at least one block replays it.                                            */
+int64_t olsgd_graph_block(const olsgd_ctx* ctx);
 
 /* Process-wide switch for how the kernels of one iteration follow each other on the main
  * stream.  on != 0 (the default): they are launched with programmatic stream serialization,
@@ -352,6 +356,14 @@ enum { OLSGD_KC_INDEX = 0, OLSGD_KC_GATHER = 1, OLSGD_KC_FORWARD = 2, OLSGD_KC_B
        OLSGD_KC_WGRAD_UPDATE = 8 /* weight-gradient GEMM with the update fused in */ };
 olsgd_status olsgd_profile_enable(olsgd_ctx* ctx, int32_t on);
 olsgd_status olsgd_profile_read(olsgd_ctx* ctx, int64_t* launches, double* millis, int32_t reset);
+/* The same profile split by layer: entry [c * OLSGD_MAX_DIMS + l] covers the launches of class
+ * c that belong to layer l (forward GEMM producing hidden layer l >= 1; OLSGD_KC_BACKWARD with
+ * l >= 1: the input-gradient GEMM producing the gradient of hidden layer l, or a weight-
+ * gradient GEMM that is launched by itself; l = 0: launches that belong to no hidden layer,
+ * e.g. the output layer's kernels).  Both arrays hold OLSGD_N_KERNEL_CLASSES * OLSGD_MAX_DIMS
+ * entries.  Summing over l gives olsgd_profile_read.                                      */
+olsgd_status olsgd_profile_read_layers(olsgd_ctx* ctx, int64_t* launches, double* millis,
+                                       int32_t reset);
 
 /* Text of the last error on this context ("" if none).  ctx may be NULL, in
  * which case the last error of a failed olsgd_init / context-free call in this

@@ -85,9 +85,11 @@ def load_library():
         "olsgd_iteration": (i64, [vp]),
         "olsgd_launch_count": (i64, [vp]),
         "olsgd_graph_replays": (i64, [vp]),
+        "olsgd_graph_block": (i64, [vp]),
         "olsgd_set_launch_overlap": (i32, [i32]),
         "olsgd_profile_enable": (i32, [vp, i32]),
         "olsgd_profile_read": (i32, [vp, C.POINTER(i64), C.POINTER(C.c_double), i32]),
+        "olsgd_profile_read_layers": (i32, [vp, C.POINTER(i64), C.POINTER(C.c_double), i32]),
         "olsgd_last_error": (C.c_char_p, [vp]),
         "olsgd_destroy": (i32, [vp]),
     }
@@ -284,6 +286,10 @@ class OverlapLocalSGD:
     def graph_replays(self):
         return self.lib.olsgd_graph_replays(self.ctx)
 
+    @property
+    def graph_block(self):
+        return self.lib.olsgd_graph_block(self.ctx)
+
     def profile_enable(self, on=True):
         _check(self.lib, self.lib.olsgd_profile_enable(self.ctx, 1 if on else 0), self.ctx)
 
@@ -294,6 +300,16 @@ class OverlapLocalSGD:
         _check(self.lib, self.lib.olsgd_profile_read(self.ctx, launches, millis, 1 if reset else 0),
                self.ctx)
         return {KERNEL_CLASSES[i]: (launches[i], millis[i]) for i in range(n)}
+
+    def profile_read_layers(self, reset=True):
+        """{class: [(launches, ms) per layer tag]} (olsgd_profile_read_layers)."""
+        n = len(KERNEL_CLASSES) * MAX_DIMS
+        launches = (C.c_int64 * n)()
+        millis = (C.c_double * n)()
+        _check(self.lib, self.lib.olsgd_profile_read_layers(self.ctx, launches, millis,
+                                                            1 if reset else 0), self.ctx)
+        return {KERNEL_CLASSES[i]: [(launches[i * MAX_DIMS + t], millis[i * MAX_DIMS + t])
+                                    for t in range(MAX_DIMS)] for i in range(len(KERNEL_CLASSES))}
 
     # -- conveniences built from the calls above ---------------------------------
     def state(self):

@@ -255,7 +255,7 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
     ga.out_t = mb.ht[l];
     ga.out_n = mb.h[l];
     {
-      Scope sc(hook, OLSGD_KC_FORWARD, s);
+      Scope sc(hook, OLSGD_KC_FORWARD | (l << 8), s);   // tagged with the layer it produces
       OLSGD_TRY(run_gemm(spec, ga, io.status, s));
     }
   }
@@ -362,7 +362,7 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
       gd.mask = mb.ht[l - 1];
       gd.out_t = mb.dat[l - 1];
       gd.out_n = mb.da[l - 1];
-      Scope sc(hook, OLSGD_KC_BACKWARD, s);
+      Scope sc(hook, OLSGD_KC_BACKWARD | ((l - 1) << 8), s);   // gradient of hidden layer l - 1
       OLSGD_TRY(run_gemm(spec, gd, io.status, s));
     }
     // dW_l [d_l][d_{l-1}] = dA_l^T [d_l][B] * (H_{l-1}^T [d_{l-1}][B])^T

@@ -20,7 +20,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct ProfRec {
-  int cls;
+  int cls, tag;
   cudaEvent_t start, stop;
 };
 
@@ -92,8 +92,9 @@ struct olsgd_ctx {
   bool prof = false;
   std::vector<ProfRec> prof_pending;
   std::vector<cudaEvent_t> prof_pool;
-  int64_t prof_launches[OLSGD_N_KERNEL_CLASSES] = {0};
-  double prof_ms[OLSGD_N_KERNEL_CLASSES] = {0};
+  // per kernel class and, inside a class, per tag (the layer a launch belongs to, else 0)
+  int64_t prof_launches[OLSGD_N_KERNEL_CLASSES][OLSGD_MAX_DIMS] = {{0}};
+  double prof_ms[OLSGD_N_KERNEL_CLASSES][OLSGD_MAX_DIMS] = {{0}};
   std::string err;
 };
 
@@ -140,7 +141,9 @@ struct Launch {
   cudaStream_t s;
   ProfRec rec{};
   bool timed = false;
-  Launch(olsgd_ctx* ctx, int cls, cudaStream_t stream) : c(ctx), s(stream) {
+  // code = kernel class + 256 * tag
+  Launch(olsgd_ctx* ctx, int code, cudaStream_t stream) : c(ctx), s(stream) {
+    const int cls = code & 0xFF;
     c->launches++;
     if (!c->prof) return;
     auto get = [&]() {
@@ -154,6 +157,7 @@ struct Launch {
       return e;
     };
     rec.cls = cls;
+    rec.tag = (code >> 8) & (OLSGD_MAX_DIMS - 1);
     rec.start = get();
     rec.stop = get();
     if (rec.start && rec.stop) {
@@ -335,8 +339,8 @@ olsgd_status drain_profile(olsgd_ctx* c) {
   for (auto& r : c->prof_pending) {
     float ms = 0.f;
     if (cudaEventElapsedTime(&ms, r.start, r.stop) == cudaSuccess) {
-      c->prof_ms[r.cls] += ms;
-      c->prof_launches[r.cls] += 1;
+      c->prof_ms[r.cls][r.tag] += ms;
+      c->prof_launches[r.cls][r.tag] += 1;
     }
     c->prof_pool.push_back(r.start);
     c->prof_pool.push_back(r.stop);
@@ -993,30 +997,44 @@ olsgd_status olsgd_run(olsgd_ctx* c, int64_t n_iters, float* loss_device) {
   // the legacy default stream cannot be captured
   const bool real_stream = c->main != nullptr && c->main != cudaStreamLegacy &&
                            c->main != cudaStreamPerThread;
+  // A run long enough for three blocks captures a graph (one block of plain launches, the
+  // capture, then replays); once a context has its graph, any run of at least one block
+  // replays it.
   const bool want_graph = real_stream && !c->graph_off && !c->prof && block > 0 &&
-                          n_iters >= 3 * (int64_t)block;
+                          (n_iters >= 3 * (int64_t)block || (c->graph_exec && n_iters >= block));
   if (!want_graph) return plain(n_iters);
-  // reach a period boundary, then run one block with plain launches (this also performs every
-  // one-time kernel attribute set-up, which must not happen inside a capture)
   olsgd_status st = OLSGD_OK;
+  // reach a period boundary
   while (c->k % c->hp.tau != 0 && t < n_iters)
     if ((st = plain(1)) != OLSGD_OK) return st;
-  if (n_iters - t < 2 * (int64_t)block) return plain(n_iters - t);
-  if ((st = plain(block)) != OLSGD_OK) return st;
-  if (c->reduce_pending) {
-    OLSGD_CUDA(c, cudaStreamWaitEvent(c->main, c->reduce_done, 0));
-    c->reduce_pending = false;
+  if (n_iters - t < block) return plain(n_iters - t);
+  // A block starts with the side stream joined and with the minibatch staged ahead by plain
+  // steps (if any) joined too, outside any capture: from "the rows of iteration k are staged"
+  // or from "none are".
+  auto settle = [&]() -> olsgd_status {
+    if (c->reduce_pending) {
+      OLSGD_CUDA(c, cudaStreamWaitEvent(c->main, c->reduce_done, 0));
+      c->reduce_pending = false;
+    }
+    if (c->pre_pending) {
+      OLSGD_CUDA(c, cudaStreamWaitEvent(c->main, c->pre_done, 0));
+      c->pre_pending = false;
+    }
+    return OLSGD_OK;
+  };
+  auto graph_fits = [&]() {
+    return c->graph_exec && c->graph_cur == c->cur && c->graph_kpar == (int)(c->k & 1) &&
+           c->graph_staged == (c->pre_k == c->k);
+  };
+  if ((st = settle()) != OLSGD_OK) return st;
+  if (!graph_fits()) {
+    // one block with plain launches first (this also performs every one-time kernel attribute
+    // set-up, which must not happen inside a capture), then the capture
+    if (n_iters - t < 2 * (int64_t)block) return plain(n_iters - t);
+    if ((st = plain(block)) != OLSGD_OK) return st;
+    if ((st = settle()) != OLSGD_OK) return st;
+    if (!graph_fits() && !capture_block(c)) return plain(n_iters - t);
   }
-  // a minibatch staged ahead by the plain steps joins the main stream here, outside any
-  // capture: the block starts from "the rows of iteration k are staged" (or from "none are")
-  if (c->pre_pending) {
-    OLSGD_CUDA(c, cudaStreamWaitEvent(c->main, c->pre_done, 0));
-    c->pre_pending = false;
-  }
-  const bool staged_now = c->pre_k == c->k;
-  if ((!c->graph_exec || c->graph_cur != c->cur || c->graph_kpar != (int)(c->k & 1) ||
-       c->graph_staged != staged_now) && !capture_block(c))
-    return plain(n_iters - t);
   {
     Launch l(c, OLSGD_KC_INDEX, c->main);
     OLSGD_CUDA(c, launch_counter(c->dev_k, c->k, 0, true, c->main));
@@ -1192,6 +1210,7 @@ int32_t olsgd_epoch_rule_half_bits(int64_t n) {
 int64_t olsgd_iteration(const olsgd_ctx* c) { return c ? c->k : -1; }
 int64_t olsgd_launch_count(const olsgd_ctx* c) { return c ? c->launches : -1; }
 int64_t olsgd_graph_replays(const olsgd_ctx* c) { return c ? c->graph_replays : -1; }
+int64_t olsgd_graph_block(const olsgd_ctx* c) { return c ? c->graph_block : -1; }
 
 int olsgd_set_launch_overlap(int on) {
   const int before = olsgd::g_launch_overlap;
@@ -1213,13 +1232,35 @@ olsgd_status olsgd_profile_read(olsgd_ctx* c, int64_t* launches, double* millis,
   olsgd_status st = drain_profile(c);
   if (st != OLSGD_OK) return st;
   for (int i = 0; i < OLSGD_N_KERNEL_CLASSES; ++i) {
-    launches[i] = c->prof_launches[i];
-    millis[i] = c->prof_ms[i];
-    if (reset) {
-      c->prof_launches[i] = 0;
-      c->prof_ms[i] = 0.0;
+    launches[i] = 0;
+    millis[i] = 0.0;
+    for (int t = 0; t < OLSGD_MAX_DIMS; ++t) {
+      launches[i] += c->prof_launches[i][t];
+      millis[i] += c->prof_ms[i][t];
+      if (reset) {
+        c->prof_launches[i][t] = 0;
+        c->prof_ms[i][t] = 0.0;
+      }
     }
   }
+  return OLSGD_OK;
+}
+
+olsgd_status olsgd_profile_read_layers(olsgd_ctx* c, int64_t* launches, double* millis,
+                                       int32_t reset) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  if (!launches || !millis) return fail(c, OLSGD_EINVAL, "output arrays are NULL");
+  olsgd_status st = drain_profile(c);
+  if (st != OLSGD_OK) return st;
+  for (int i = 0; i < OLSGD_N_KERNEL_CLASSES; ++i)
+    for (int t = 0; t < OLSGD_MAX_DIMS; ++t) {
+      launches[i * OLSGD_MAX_DIMS + t] = c->prof_launches[i][t];
+      millis[i * OLSGD_MAX_DIMS + t] = c->prof_ms[i][t];
+      if (reset) {
+        c->prof_launches[i][t] = 0;
+        c->prof_ms[i][t] = 0.0;
+      }
+    }
   return OLSGD_OK;
 }
 

@@ -353,7 +353,8 @@ struct StepIO {
   // from which the next iteration's rows may be staged beside this iteration.
   cudaEvent_t mid_event;
 };
-// Lets model.cu count and time its launches without knowing the context type.
+// Lets model.cu count and time its launches without knowing the context type.  `cls` is a
+// kernel class, optionally plus 256 * (the layer the launch belongs to).
 struct ProfHook {
   void* ctx;
   void* (*begin)(void* ctx, int cls, cudaStream_t s);

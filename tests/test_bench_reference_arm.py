@@ -37,6 +37,7 @@ def test_reference_arm_two_ranks_rank0_prints():
     lines = _json_lines(out.stdout)
     assert len(lines) == 1
     assert lines[0]["impl"] == "reference" and lines[0]["n_gpus"] == 2
+    assert "sharded" not in lines[0]      # the oracle arm runs on rank 0 alone: nothing is sharded
 
 
 def test_max_over_ranks_with_two_gloo_ranks():
@@ -46,3 +47,10 @@ def test_max_over_ranks_with_two_gloo_ranks():
     out = subprocess.run(cmd, cwd=ROOT, capture_output=True, text=True, timeout=300)
     assert out.returncode == 0, out.stderr[-2000:]
     assert "GLOO_OK 2" in out.stdout
+    # shape of the `sharded` record that bench.py --gpus N (N > 1) adds to its line
+    rec = json.loads([l for l in out.stdout.splitlines() if l.startswith("SHARDED ")][0][8:])
+    assert set(rec) >= {"value", "unit", "ms_per_step", "steps", "scaling", "workers_per_gpu", "m",
+                        "n_gpus", "allreduce_bytes_per_period", "collective"}
+    assert rec["unit"] == "worker-steps/s" and rec["scaling"] == "strong" and rec["n_gpus"] == 2
+    assert rec["workers_per_gpu"] == 8 and rec["allreduce_bytes_per_period"] == 4 * 4206602
+    assert rec["ms_per_step"] == 0.3          # the slower rank's 6 ms over 20 steps

@@ -143,10 +143,19 @@ def test_config3_late_regime_resynchronised_with_the_oracle():
     """Config 3 beyond the point where its trajectory stops being reproducible: the small-loss,
     large-momentum regime of iterations 300-1000.  Chaos cannot be followed over hundreds of
     iterations, but ten can: at the period boundaries k0 the device's whole state (x_i, u_i, z,
-    v) is read back and handed to a fresh exact-fp64 oracle as ITS start, exactly as x0 is at
-    k = 0 (an input to both sides, no expected value comes from the device); both then run
-    ten iterations on the rule's own minibatches, and every per-worker minibatch loss of those
-    iterations is held to the 2e-2 bar, as are the parameters after them."""
+    v) is read back and handed to a fresh oracle as ITS start, exactly as x0 is at k = 0 (an
+    input to both sides, no expected value comes from the device); both then run ten
+    iterations on the rule's own minibatches.
+
+    Held to the 2e-2 bar of the bf16 paths: against the EXACT fp64 oracle, every iteration's
+    worker-mean loss (relative) and every per-worker loss (on the scale of the window's
+    largest loss, the yardstick of the first-iterations test above); against the oracle with
+    the configuration's own operand rounding, every single per-worker loss relative to
+    itself.  The last is not asked of the exact oracle because the two ORACLES already differ
+    by up to 2.2 % on single entries there (measured: 1.1 %, 1.0 %, 2.2 % at k0 = 300, 600,
+    900, against 0.6 %, 0.9 %, 1.1 % between the device and the rounded oracle): that is the
+    operand rounding acting on one worker's small minibatch loss, not the kernels."""
+    import copy
     from paper_2002_09539_b200 import OverlapLocalSGD
     c = si.CONFIGS["c3"]
     m, steps = c["m"], 10
@@ -155,6 +164,8 @@ def test_config3_late_regime_resynchronised_with_the_oracle():
     opt = OverlapLocalSGD("mlp", m=m, tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"],
                           beta=c["beta"], mu=c["mu"], batch=c["batch"], seed=0, dims=c["dims"],
                           gemm_bf16=c["gemm_bf16"], x0=x0, X=to_dev(X), y=to_dev(y))
+    kw = dict(m=m, tau=c["tau"], batch=c["batch"], gamma=c["gamma"], alpha=c["alpha"],
+              beta=c["beta"], mu=c["mu"], seed=0, iters=steps)
     first_loss = None
     for k0 in (300, 600, 900):
         warm = torch.zeros((k0 - opt.iteration, m), device="cuda")
@@ -168,6 +179,7 @@ def test_config3_late_regime_resynchronised_with_the_oracle():
         st.z = opt.get_params(-1).astype(np.float64)
         st.v = opt.get_params(-2).astype(np.float64)
         st.k = k0
+        st_rounded = copy.deepcopy(st)
         x_start, z_start = st.x.copy(), st.z.copy()
         # the regime the test is about: trained far below the start, momentum buffers loaded
         assert float(warm[-10:].mean()) < 0.5 * first_loss
@@ -175,16 +187,20 @@ def test_config3_late_regime_resynchronised_with_the_oracle():
         lg = torch.zeros((steps, m), device="cuda")
         opt.run(steps, lg)
         lg = lg.cpu().numpy()
-        st, lo, _ = runner.run_model("mlp", c["dims"], X, y, None, m=m, tau=c["tau"],
-                                     batch=c["batch"], gamma=c["gamma"], alpha=c["alpha"],
-                                     beta=c["beta"], mu=c["mu"], seed=0, iters=steps, state=st)
+        st, lo, _ = runner.run_model("mlp", c["dims"], X, y, None, state=st, **kw)
+        st_rounded, lr, _ = runner.run_model("mlp", c["dims"], X, y, None, state=st_rounded,
+                                             bf16_operands=True, **kw)
         assert st.k == opt.iteration == k0 + steps
-        # every iteration, every worker: |loss_gpu - loss_oracle| <= 2e-2 of the iteration's scale
-        scale = np.abs(lo).max(axis=1, keepdims=True)
-        assert (np.abs(lg - lo) <= TOL_BF16_LOSS * scale).all(), (k0, np.abs(lg - lo).max(), scale.min())
+        # exact oracle: worker-mean loss of every iteration, relative
         mean_g, mean_o = lg.mean(axis=1), lo.mean(axis=1)
         assert (np.abs(mean_g - mean_o) <= TOL_BF16_LOSS * mean_o).all(), (k0, mean_g, mean_o)
+        # exact oracle: every per-worker loss on the scale of the window, and none far off
+        assert np.abs(lg - lo).max() <= TOL_BF16_LOSS * np.abs(lo).max(), (k0, np.abs(lg - lo).max())
+        assert (np.abs(lg - lo) <= 5e-2 * lo).all(), (k0, (np.abs(lg - lo) / lo).max())
+        # oracle with the operand rounding of the configuration: every per-worker loss, relative
+        assert (np.abs(lg - lr) <= TOL_BF16_LOSS * lr).all(), (k0, (np.abs(lg - lr) / lr).max())
         assert state_err(opt, st) <= TOL_BF16_LOSS, (k0, state_err(opt, st))
+        assert state_err(opt, st_rounded) <= TOL_BF16_LOSS, (k0, state_err(opt, st_rounded))
         # the ten steps themselves (not the state they started from) agree as well
         xg, zg, _ = opt.state()
         moved_o = np.abs(st.x - x_start).max()
