@@ -30,7 +30,7 @@ import synth_inputs as si  # noqa: E402
 METRIC = "simulated_worker_steps_per_sec"
 UNIT = "worker-steps/s"
 L2_BYTES = 126 * 2 ** 20
-MAX_BLOCKS = 2000          # upper bound on repeated timed blocks
+MAX_BLOCKS = 20000         # upper bound on repeated timed blocks
 
 
 def measured_peaks():
@@ -186,7 +186,10 @@ def algorithmic_bytes(c, kernel_class, P, sync_fraction):
         layers = [p for p in range(len(d) - 2) if layer_is_fused(c, p)]
         per = (16 if mom else 8) + 2
         operands = sum(m * B * 2 * (d[p + 1] + d[p]) for p in layers)
-        return m * fused * per + sync_fraction * 4 * fused + operands
+        # sync steps: the anchor read once, and (worker sum formed in the launch) one row of
+        # partial sums written per slice
+        slices = c.get("sum_slices", 0)
+        return m * fused * per + sync_fraction * 4 * (1 + slices) * fused + operands
     if kernel_class == "update":
         per = (20 if mom else 12) + shadow
         rest = P - fused
@@ -368,6 +371,8 @@ def run_ours(args, rank, world):
     opt = OverlapLocalSGD(c["kind"], m=c["m"], tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"],
                           beta=c["beta"], mu=c["mu"], batch=c["batch"], seed=seed, dims=c["dims"],
                           gemm_bf16=c["gemm_bf16"], x0=x0, X=Xd, y=yd, local_sgd=local_sgd)
+    if args.no_anchor_fusion:
+        opt.set_anchor_fusion(False)
     m, K, W = c["m"], args.steps, args.warmup
 
     def barrier():
@@ -400,8 +405,8 @@ def run_ours(args, rank, world):
     launches0, replays0 = opt.launch_count, opt.graph_replays
     times = [timed(lambda: opt.run(K))]
     launches = opt.launch_count - launches0
-    n_blocks = int(min(MAX_BLOCKS, max(1, np.ceil(args.min_time * 1e3 / times[0]))))
-    for _ in range(n_blocks - 1):
+    # (the block times are maxima over the ranks, so every rank takes the same decision)
+    while sum(times) < args.min_time * 1e3 and len(times) < MAX_BLOCKS:
         times.append(timed(lambda: opt.run(K)))
     replays = opt.graph_replays - replays0
     clocks = sampler.stop() if rank == 0 else None
@@ -416,6 +421,7 @@ def run_ours(args, rank, world):
                   if per_block else "olsgd_run: plain launches (K is shorter than the captured block)")
 
     # ---- per-kernel-class device time (second pass, every launch bracketed by events)
+    anchor_fusion_on = opt.anchor_fusion
     KP = max(K, 2 * block)
     opt.profile_enable(True)
     opt.run(KP)
@@ -439,6 +445,8 @@ def run_ours(args, rank, world):
         roof_class = next((k for k in ranked if algorithmic_bytes(c, k, P, 0) is not None), None)
         avg_ms = busy[roof_class][1] / busy[roof_class][0] if roof_class else None
     if roof_class is not None:
+        if anchor_fusion_on:
+            c = dict(c, sum_slices=4 if c["m"] >= 64 else 2 if c["m"] >= 8 else 1)
         ab = algorithmic_bytes(c, roof_class, P, n_sync / KP)
         achieved = ab / (avg_ms * 1e-3) / 1e9
         traffic = ncu_traffic(name, c["gemm_bf16"], roof_class, n_sync / KP)
@@ -510,8 +518,7 @@ def run_ours(args, rank, world):
     e2e_steps(W)
     opt.join()
     e2e_times = [e2e_block()]
-    n_e2e = int(min(MAX_BLOCKS, max(1, np.ceil(args.min_time * 1e3 / e2e_times[0]))))
-    for _ in range(n_e2e - 1):
+    while sum(e2e_times) < args.min_time * 1e3 and len(e2e_times) < MAX_BLOCKS:
         e2e_times.append(e2e_block())
     e2e_ms = float(np.median(e2e_times))
     assert np.isfinite(loss_h.numpy()).all()
@@ -525,6 +532,7 @@ def run_ours(args, rank, world):
                api="%s + olsgd_period_sync, pinned host minibatches (%s rows, int32 labels)"
                    % ("olsgd_local_step_host_bf16" if c["gemm_bf16"] else "olsgd_local_step_host",
                       "bf16" if c["gemm_bf16"] else "fp32"))
+    anchor_fusion = opt.anchor_fusion
     opt.close()
     del opt, Xd, yd
     torch.cuda.empty_cache()
@@ -554,6 +562,7 @@ def run_ours(args, rank, world):
                        "batch": B, "dims": c["dims"], "P": P, "gamma": c["gamma"],
                        "alpha": c["alpha"], "beta": c["beta"], "mu": c["mu"],
                        "gemm_mode": c["gemm_bf16"], "method": args.method,
+                       "anchor_fusion": bool(anchor_fusion),
                        "tau_overridden": bool(args.tau),
                        "l2": "no flush: resident inputs+state %.0f MB exceed the %d MB L2"
                              % (resident / 1e6, L2_BYTES >> 20) if resident > L2_BYTES else
@@ -858,6 +867,9 @@ def main():
     ap.add_argument("--no-kernel-points", action="store_true",
                     help="skip the stand-alone update/anchor kernel measurements (config 5's "
                          "10M x 16 and 50M x 64 points) that the default line carries")
+    ap.add_argument("--no-anchor-fusion", action="store_true",
+                    help="MLP workloads: form the worker sum of Eq. 5 / Eq. 10-11 in the worker-mean "
+                         "kernel only (olsgd_set_anchor_fusion(0)), to measure what the fusion buys")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     if args.warmup < 3:

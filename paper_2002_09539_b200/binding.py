@@ -71,6 +71,8 @@ def load_library():
         "olsgd_selftest_per_device_table": (i32, []),
         "olsgd_epoch_rule_half_bits": (i32, [i64]),
         "olsgd_period_sync": (i32, [vp]),
+        "olsgd_set_anchor_fusion": (i32, [vp, i32]),
+        "olsgd_anchor_fusion": (i32, [vp]),
         "olsgd_period_sync_begin": (i32, [vp, vp]),
         "olsgd_period_sync_finish": (i32, [vp, vp]),
         "olsgd_row_floats": (i64, [vp]),
@@ -220,6 +222,13 @@ class OverlapLocalSGD:
 
     def period_sync(self):
         _check(self.lib, self.lib.olsgd_period_sync(self.ctx), self.ctx)
+
+    def set_anchor_fusion(self, on):
+        _check(self.lib, self.lib.olsgd_set_anchor_fusion(self.ctx, 1 if on else 0), self.ctx)
+
+    @property
+    def anchor_fusion(self):
+        return bool(self.lib.olsgd_anchor_fusion(self.ctx))
 
     def period_sync_begin(self, partial_sum):
         assert partial_sum.is_cuda and partial_sum.dtype == torch.float32

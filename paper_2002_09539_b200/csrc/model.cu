@@ -32,6 +32,13 @@ inline bool tensor_path(const olsgd_model_spec& s) {
   return s.kind == OLSGD_MLP && (s.gemm_bf16 == 1 || s.gemm_bf16 == 3);
 }
 
+// Is the update of parameter layer p (a hidden layer's weights and bias) applied inside its
+// weight-gradient GEMM?
+bool layer_update_is_fused(const olsgd_model_spec& spec, const olsgd_hparams& hp, int p) {
+  return spec.gemm_bf16 == 1 && spec.dims[p + 1] % 128 == 0 && spec.dims[p] % 128 == 0 &&
+         hp.batch % 64 == 0 && hp.batch <= 128;
+}
+
 cudaError_t run_gemm(const olsgd_model_spec& spec, GemmArgs ga, int* status, cudaStream_t s) {
   ga.status = status;
   if (tensor_path(spec))
@@ -105,6 +112,18 @@ bool plan_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, ModelPlan
     mp->off_da[l] = take(m * B * w * e);
     mp->off_dat[l] = take(m * B * w * e);
   }
+  // scratch of the worker sum that the sync-step weight-gradient launch forms (Overlap mode,
+  // all workers in this context, at least one layer whose update is fused)
+  if (spec.gemm_bf16 == 1 && hp.mode == OLSGD_MODE_OVERLAP && (hp.m_total == 0 || hp.m_total == hp.m)) {
+    bool any = false;
+    for (int p = 0; p < L - 1; ++p) any = any || layer_update_is_fused(spec, hp, p);
+    if (any) {
+      size_t P = 0;
+      for (int l = 0; l < L; ++l) P += (size_t)spec.dims[l + 1] * spec.dims[l] + spec.dims[l + 1];
+      mp->off_sum_part = take((size_t)worker_sum_slices(hp.m) * align_up(P, 64) * sizeof(float));
+      mp->has_sum_part = true;
+    }
+  }
   mp->bytes = off;
   return true;
 }
@@ -160,9 +179,7 @@ bool bind_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, const Mod
   // gemm_bf16 == 1: hidden-layer weight matrices whose shape the weight-gradient kernel
   // takes are updated in its epilogue; everything else goes to the update kernel
   int64_t P = off;
-  for (int p = 0; p < L - 1; ++p)
-    mb->fused_layer[p] = spec.gemm_bf16 == 1 && spec.dims[p + 1] % 128 == 0 &&
-                         spec.dims[p] % 128 == 0 && hp.batch % 64 == 0 && hp.batch <= 128;
+  for (int p = 0; p < L - 1; ++p) mb->fused_layer[p] = layer_update_is_fused(spec, hp, p);
   {
     HeadArgs probe{};
     probe.K = spec.dims[L - 1];
@@ -189,6 +206,29 @@ bool bind_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, const Mod
     }
   }
   close_range(P);
+  // the worker sum inside the sync-step launch covers the fused layers' weight matrices; what
+  // is left for the worker-mean kernel are the ranges between them (biases, output layer)
+  if (mp.has_sum_part) {
+    mb->sum_part = reinterpret_cast<float*>(base + mp.off_sum_part);
+    int64_t from = 0;
+    mb->n_anchor_ranges = mb->n_summed = 0;
+    auto close_anchor = [&](int64_t end) {
+      if (end > from) {
+        mb->anchor_off[mb->n_anchor_ranges] = from;
+        mb->anchor_len[mb->n_anchor_ranges] = end - from;
+        mb->n_anchor_ranges++;
+      }
+    };
+    for (int p = 0; p < L - 1; ++p) {
+      if (!mb->fused_layer[p]) continue;
+      mb->summed_off[mb->n_summed] = mb->w_off[p];
+      mb->summed_len[mb->n_summed] = mb->b_off[p] - mb->w_off[p];
+      mb->n_summed++;
+      close_anchor(mb->w_off[p]);
+      from = mb->b_off[p];
+    }
+    close_anchor(P);
+  }
   return true;
 }
 
@@ -249,6 +289,10 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
     // W_1 is not read again in this iteration (no input gradient is formed for the data);
     // the weights of the other layers are read again by their input-gradient GEMM
     ga.a_read_once = (l == 1) ? 1 : 0;
+    // the weights' bf16 copy is written by the update at the end of an iteration: the kernel
+    // ahead of the first layer's GEMM may be that update, the one ahead of any later layer's
+    // GEMM is the previous layer's GEMM
+    ga.a_ready_early = (l >= 2) ? 1 : 0;
     ga.epilogue = GEMM_EPI_BIAS_RELU;
     ga.bias = io.x + mb.b_off[l - 1];
     ga.bias_batch = io.ld;
@@ -349,6 +393,8 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
       GemmArgs gd{};
       gd.A = io.shadow + mb.w_off[l - 1];
       gd.a_mn_major = 1;
+      gd.a_ready_early = 1;   // ahead of it runs the output-layer forward kernel or an input-
+                              // gradient GEMM; the launch that rewrites the bf16 copy comes later
       gd.lda = spec.dims[l - 1];
       gd.a_batch = io.ld;
       gd.B = mb.da[l];

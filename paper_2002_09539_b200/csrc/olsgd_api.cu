@@ -70,6 +70,8 @@ struct olsgd_ctx {
   int host_slot = 0;
   bool reduce_pending = false;  // an anchor refresh was launched and not yet waited for
   int reduce_reads = -1;        // which x buffer that refresh reads
+  bool anchor_fusion = false;   // sync steps form the worker sum inside the weight-gradient launch
+  bool last_sync_summed = false;  // ... and the sync step that closed this period did
   bool need_sync = false;       // a period ended; olsgd_period_sync is due
   bool sync_begun = false;      // olsgd_period_sync_begin ran; _finish is due
 
@@ -454,6 +456,16 @@ olsgd_status step_body(olsgd_ctx* c, const olsgd_data& data, int32_t* idx,
     io.upd.mu = c->hp.mu;
     io.upd.alpha = c->hp.alpha;
     io.upd.sync = sync ? 1 : 0;
+    if (sync) {
+      // the worker sums of the weight matrices whose update is fused are formed by the same
+      // launch; olsgd_period_sync finishes Eq. 5 / Eq. 10-11 from them
+      const bool summed = c->anchor_fusion && c->mb.sum_part != nullptr;
+      c->last_sync_summed = summed;
+      if (summed) {
+        io.upd.sum_part = c->mb.sum_part;
+        io.upd.sum_slices = worker_sum_slices(c->hp.m);
+      }
+    }
     // same rule as in apply_update, applied before the first kernel that writes x[nxt]
     if (c->reduce_pending && (sync || c->reduce_reads == nxt)) {
       io.wait_before_update = c->reduce_done;
@@ -646,6 +658,7 @@ olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const ols
       Launch l(c, OLSGD_KC_OTHER, c->main);
       OLSGD_INIT_CUDA(launch_cast_bf16(c->x[0], c->shadow, (int64_t)c->hp.m * c->ld, c->main));
     }
+    c->anchor_fusion = c->mb.sum_part != nullptr;
   }
   OLSGD_INIT_CUDA(cudaStreamSynchronize(c->main));
 #undef OLSGD_INIT_CUDA
@@ -848,7 +861,28 @@ olsgd_status olsgd_period_sync(olsgd_ctx* c) {
   if (c->hp.m_total != 0 && c->hp.m_total != c->hp.m)
     return fail(c, OLSGD_ESTATE, "this context holds a shard of the workers: use "
                                  "olsgd_period_sync_begin / olsgd_period_sync_finish");
-  {
+  if (c->last_sync_summed) {
+    // the weight matrices were summed over the workers by the sync step's own weight-gradient
+    // launch: their anchor only needs the S rows of partial sums, not the m worker models;
+    // the rest of the row (biases, output layer) goes through the worker-mean kernel
+    for (int r = 0; r < c->mb.n_summed; ++r) {
+      const int64_t off = c->mb.summed_off[r];
+      Launch l(c, OLSGD_KC_ANCHOR, c->side);
+      OLSGD_CUDA(c, launch_anchor_from_slices(c->mb.sum_part + off, worker_sum_slices(c->hp.m), c->ld,
+                                              c->z + off, c->v + off, c->mb.summed_len[r],
+                                              c->hp.beta, c->hp.m, c->side));
+    }
+    for (int r = 0; r < c->mb.n_anchor_ranges; ++r) {
+      AnchorArgs b = a;
+      const int64_t off = c->mb.anchor_off[r];
+      b.x = a.x + off;
+      b.z = a.z + off;
+      b.v = a.v + off;
+      b.P = c->mb.anchor_len[r];
+      Launch l(c, OLSGD_KC_ANCHOR, c->side);
+      OLSGD_CUDA(c, launch_worker_mean_anchor(b, c->side));
+    }
+  } else {
     Launch l(c, OLSGD_KC_ANCHOR, c->side);
     OLSGD_CUDA(c, launch_worker_mean_anchor(a, c->side));
   }
@@ -858,6 +892,24 @@ olsgd_status olsgd_period_sync(olsgd_ctx* c) {
   c->need_sync = false;
   return OLSGD_OK;
 }
+
+olsgd_status olsgd_set_anchor_fusion(olsgd_ctx* c, int32_t on) {
+  if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
+  if (c->need_sync || c->sync_begun)
+    return fail(c, OLSGD_ESTATE, "a period ended: call olsgd_period_sync first");
+  const bool want = on != 0 && c->mb.sum_part != nullptr;
+  if (want != c->anchor_fusion) {
+    c->anchor_fusion = want;
+    // a captured block carries the old choice
+    if (c->graph_exec) {
+      cudaGraphExecDestroy(c->graph_exec);
+      c->graph_exec = nullptr;
+    }
+  }
+  return OLSGD_OK;
+}
+
+int32_t olsgd_anchor_fusion(const olsgd_ctx* c) { return c && c->anchor_fusion ? 1 : 0; }
 
 olsgd_status olsgd_period_sync_begin(olsgd_ctx* c, float* partial_sum_device) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");

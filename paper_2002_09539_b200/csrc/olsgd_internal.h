@@ -111,9 +111,18 @@ struct AnchorArgs {
   float* partial;   // non-null: only write the undivided column sums there (sharded sync)
 };
 cudaError_t launch_worker_mean_anchor(const AnchorArgs& a, cudaStream_t s);
+// The number S of interleaved slices the worker sum is formed in (slice s adds the workers
+// s, s + S, ... in order, the slices are combined in order): a function of m alone, used by
+// every kernel that forms the sum so that all of them give the same bits.
+int worker_sum_slices(int m);
 // Eq. 5 / Eq. 10-11 from column sums over all m_total workers (sum is padded like a state row).
 cudaError_t launch_anchor_from_sum(const float* sum, float* z, float* v, int64_t P, float beta,
                                    int m_total, cudaStream_t s);
+// Eq. 5 / Eq. 10-11 for P entries from `slices` rows of partial worker sums (row pitch ld):
+// the rows are added in slice order, which completes the summation order of the worker-mean
+// kernel, then divided by m.
+cudaError_t launch_anchor_from_slices(const float* part, int slices, int64_t ld, float* z, float* v,
+                                      int64_t P, float beta, int m, cudaStream_t s);
 
 // Eq. 2 on a sync step: every worker row of x (and of its bf16 shadow, if any) and z are
 // replaced by the worker mean, summed in worker order.
@@ -258,6 +267,12 @@ struct FusedUpdateArgs {
   // b_off .. b_off + Ma - 1 of every worker row) from the row sums it forms, instead of
   // storing them as a gradient
   int64_t b_off;
+  // weight-gradient GEMM on sync steps only, sum_slices > 0: the launch also adds up
+  // x_{k+1} over the workers, in the order of the worker-mean kernel (sum_slices interleaved
+  // slices, each in worker order), and leaves slice s's sums of the layer's weight matrix in
+  // row s of sum_part; launch_anchor_from_slices finishes the anchor refresh from there.
+  float* sum_part;     // [sum_slices][ld] floats of scratch
+  int sum_slices;      // worker_sum_slices(m), or 0: no sum
 };
 struct GemmArgs {
   const __nv_bfloat16* A;
@@ -266,6 +281,10 @@ struct GemmArgs {
   int m, Ma, Nb, K;
   int a_mn_major;            // A is stored [K][Ma]
   int a_read_once;           // nothing reads A again soon: L2 may give its lines up first
+  // A was last written by a kernel that had completed before the kernel launched just ahead
+  // of this one started: with chained launches the first A tiles may then be loaded while
+  // that kernel still drains
+  int a_ready_early;
   int epilogue;
   const float* bias;         // BIAS_RELU: bias[i * bias_batch + row]
   int64_t bias_batch;
@@ -306,6 +325,9 @@ struct ModelPlan {
          off_dlogits = 0, off_rowloss = 0, off_loss = 0;
   size_t off_h[OLSGD_MAX_DIMS] = {0}, off_ht[OLSGD_MAX_DIMS] = {0};    // hidden activations
   size_t off_da[OLSGD_MAX_DIMS] = {0}, off_dat[OLSGD_MAX_DIMS] = {0};  // their gradients
+  // worker sum inside the sync-step weight-gradient launch: partial sums [slices][ld]
+  bool has_sum_part = false;
+  size_t off_sum_part = 0;
 };
 struct ModelBuffers {
   char error[160] = {0};
@@ -328,6 +350,14 @@ struct ModelBuffers {
   // what is left for the stand-alone update kernel: ranges [off, off + len) of a worker row
   int n_ranges = 0;
   int64_t range_off[OLSGD_MAX_DIMS + 1] = {0}, range_len[OLSGD_MAX_DIMS + 1] = {0};
+  // Worker sum inside the sync-step weight-gradient launch (fused layers' weight matrices):
+  // the scratch matrix, the ranges of a row it covers, and the ranges that are left for the
+  // worker-mean kernel (biases, output layer).
+  float* sum_part = nullptr;
+  int n_summed = 0;
+  int64_t summed_off[OLSGD_MAX_DIMS] = {0}, summed_len[OLSGD_MAX_DIMS] = {0};
+  int n_anchor_ranges = 0;
+  int64_t anchor_off[OLSGD_MAX_DIMS + 1] = {0}, anchor_len[OLSGD_MAX_DIMS + 1] = {0};
 };
 struct StepIO {
   const float* x;                // x_k, [m][ld]

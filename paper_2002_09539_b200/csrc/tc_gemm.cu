@@ -24,6 +24,7 @@ namespace {
 using namespace tc;
 
 struct EpiArgs {
+  int a_early;   // A was complete before the kernel ahead of this one started (see GemmArgs)
   int once;      // A is read once: its TMA loads carry an evict-first policy
   int epilogue;
   int Ma, Nb;
@@ -80,30 +81,46 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
-  // everything above touched only shared and tensor memory: it may run under the tail of
-  // the kernel before this one
+  auto load_a = [&](int kb, uint32_t a_dst, uint32_t full) {
+    if (a_mn) {
+      // A is stored [K][Ma]: two boxes of 64 (Ma) x 64 (K rows)
+      tma_load_3d(a_dst, &map_a, full, m0, kb * kBK, worker);
+      tma_load_3d(a_dst + kABytes / 2, &map_a, full, m0 + 64, kb * kBK, worker);
+    } else if (ea.once) {
+      tma_load_3d_once(a_dst, &map_a, full, kb * kBK, m0, worker);
+    } else {
+      tma_load_3d(a_dst, &map_a, full, kb * kBK, m0, worker);
+    }
+  };
+  // Everything above touched only shared and tensor memory: it may run under the tail of
+  // the kernel before this one.  So may the first loads of an A operand (weights) that the
+  // kernel before this one does not write: the ring's first stages are filled with A while
+  // that kernel drains, and only the B operand (its output) waits for the gate.
+  const int n_early = ea.a_early ? (num_kb < STAGES ? num_kb : STAGES) : 0;
+  if (warp == 0 && lane == 0) {
+    for (int kb = 0; kb < n_early; ++kb) {
+      const uint32_t full = smem_u32(&ctl->full[kb]);
+      mbar_expect_tx(full, kStageBytes);
+      load_a(kb, smem_u32(tiles + kb * kStageBytes), full);
+    }
+  }
   launch_gate();
 
   if (warp == 0 && lane == 0) {
     // ---------------- TMA producer
-    int issued = 0;
+    int issued = n_early;
     for (int kb = 0; kb < num_kb; ++kb) {
       const int s = kb % STAGES;
       const uint32_t ph = (kb / STAGES) & 1;
-      if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1, abort_flag)) break;
       const uint32_t full = smem_u32(&ctl->full[s]);
-      mbar_expect_tx(full, kStageBytes);
       const uint32_t a_dst = smem_u32(tiles + s * kStageBytes);
-      if (a_mn) {
-        // A is stored [K][Ma]: two boxes of 64 (Ma) x 64 (K rows)
-        tma_load_3d(a_dst, &map_a, full, m0, kb * kBK, worker);
-        tma_load_3d(a_dst + kABytes / 2, &map_a, full, m0 + 64, kb * kBK, worker);
-      } else {
-        if (ea.once) tma_load_3d_once(a_dst, &map_a, full, kb * kBK, m0, worker);
-        else tma_load_3d(a_dst, &map_a, full, kb * kBK, m0, worker);
+      if (kb >= n_early) {
+        if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1, abort_flag)) break;
+        mbar_expect_tx(full, kStageBytes);
+        load_a(kb, a_dst, full);
       }
       tma_load_3d(a_dst + kABytes, &map_b, full, kb * kBK, n0, worker);
-      issued = kb + 1;
+      if (kb + 1 > issued) issued = kb + 1;
     }
     if (*abort_flag) {
       // drain: wait (bounded) for the copies this thread still has in flight
@@ -261,6 +278,7 @@ cudaError_t launch_one(const GemmArgs& a, const CUtensorMap& ma, const CUtensorM
   EpiArgs ea;
   ea.epilogue = a.epilogue;
   ea.once = a.a_read_once;
+  ea.a_early = a.a_ready_early;
   ea.Ma = a.Ma;
   ea.Nb = a.Nb;
   ea.bias = a.bias;

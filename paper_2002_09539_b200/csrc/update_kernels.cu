@@ -229,6 +229,50 @@ anchor_from_sum_kernel(const float* __restrict__ sum, float* __restrict__ z, flo
   }
 }
 
+// Anchor refresh from S rows of partial worker sums (row pitch ld): total in slice order,
+// mean, Eq. 5 or Eq. 10-11.  The arithmetic after the total is that of
+// worker_mean_anchor_kernel, so the two routes to the anchor give the same bits.
+template <bool MOM>
+__global__ void __launch_bounds__(kUpdateThreads)
+anchor_from_slices_kernel(const float* __restrict__ part, int slices, int64_t ld,
+                          float* __restrict__ z, float* __restrict__ v, int64_t n4, float beta,
+                          float m_f) {
+  const int64_t col4 = (int64_t)blockIdx.x * kUpdateThreads + threadIdx.x;
+  if (col4 >= n4) return;
+  float4 zz = make_float4(0.f, 0.f, 0.f, 0.f), vv = zz;
+  if (MOM) {
+    zz = reinterpret_cast<const float4*>(z)[col4];
+    vv = reinterpret_cast<const float4*>(v)[col4];
+  }
+  float4 s = __ldcs(reinterpret_cast<const float4*>(part) + col4);
+  for (int t = 1; t < slices; ++t) {
+    const float4 p = __ldcs(reinterpret_cast<const float4*>(part + (int64_t)t * ld) + col4);
+    s.x += p.x;
+    s.y += p.y;
+    s.z += p.z;
+    s.w += p.w;
+  }
+  s.x /= m_f;
+  s.y /= m_f;
+  s.z /= m_f;
+  s.w /= m_f;
+  float4* z4 = reinterpret_cast<float4*>(z) + col4;
+  if (MOM) {
+    vv.x = fmaf(beta, vv.x, s.x - zz.x);
+    vv.y = fmaf(beta, vv.y, s.y - zz.y);
+    vv.z = fmaf(beta, vv.z, s.z - zz.z);
+    vv.w = fmaf(beta, vv.w, s.w - zz.w);
+    zz.x += vv.x;
+    zz.y += vv.y;
+    zz.z += vv.z;
+    zz.w += vv.w;
+    reinterpret_cast<float4*>(v)[col4] = vv;
+    *z4 = zz;
+  } else {
+    *z4 = s;
+  }
+}
+
 // Stage 1: block b adds (x_i[j] - z[j])^2 over its strided share of the m * P entries, each
 // thread sequentially, then the threads in a fixed tree.  Stage 2: one thread adds the block
 // partials in order.  Double precision throughout.
@@ -313,12 +357,19 @@ cudaError_t launch_mean(const AnchorArgs& a, cudaStream_t s) {
   return cudaGetLastError();
 }
 
+int worker_sum_slices(int m) {
+  // Few slices: where the sync-step weight-gradient launch forms the sum, every slice costs
+  // a row of partial sums that is written and read once.  At least four workers per slice
+  // (every thread of the worker-mean kernel keeps four loads in flight), at most sixteen.
+  return m >= 64 ? 4 : m >= 8 ? 2 : 1;
+}
+
 cudaError_t launch_worker_mean_anchor(const AnchorArgs& a, cudaStream_t s) {
-  // about four workers per slice, so that every thread has four loads in flight
-  if (a.m >= 32) return launch_mean<8>(a, s);
-  if (a.m >= 16) return launch_mean<4>(a, s);
-  if (a.m >= 8) return launch_mean<2>(a, s);
-  return launch_mean<1>(a, s);
+  switch (worker_sum_slices(a.m)) {
+    case 4: return launch_mean<4>(a, s);
+    case 2: return launch_mean<2>(a, s);
+    default: return launch_mean<1>(a, s);
+  }
 }
 
 cudaError_t launch_worker_mean_broadcast(float* x, __nv_bfloat16* shadow, float* z, int64_t P,
@@ -337,6 +388,17 @@ cudaError_t launch_anchor_from_sum(const float* sum, float* z, float* v, int64_t
     anchor_from_sum_kernel<true><<<grid, kUpdateThreads, 0, s>>>(sum, z, v, n4, beta, (float)m_total);
   else
     anchor_from_sum_kernel<false><<<grid, kUpdateThreads, 0, s>>>(sum, z, v, n4, beta, (float)m_total);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_anchor_from_slices(const float* part, int slices, int64_t ld, float* z, float* v,
+                                      int64_t P, float beta, int m, cudaStream_t s) {
+  const int64_t n4 = (P + 3) / 4;
+  const unsigned grid = (unsigned)((n4 + kUpdateThreads - 1) / kUpdateThreads);
+  if (beta != 0.f)
+    anchor_from_slices_kernel<true><<<grid, kUpdateThreads, 0, s>>>(part, slices, ld, z, v, n4, beta, (float)m);
+  else
+    anchor_from_slices_kernel<false><<<grid, kUpdateThreads, 0, s>>>(part, slices, ld, z, v, n4, beta, (float)m);
   return cudaGetLastError();
 }
 

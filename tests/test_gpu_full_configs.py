@@ -139,6 +139,39 @@ def test_mlp_configs_full_length(name):
     assert abs(np.linalg.norm(xbar) - gold["norm2_mean_model"]) <= 0.02 * gold["norm2_mean_model"]
 
 
+@pytest.mark.parametrize("name", ["c3", "c4"])
+def test_anchor_fusion_at_full_size_gives_the_bits_of_the_worker_mean_kernel(name):
+    # configs 3 and 4 as bench.py runs them (replayed graph blocks), with the worker sum inside
+    # the sync-step weight-gradient launch and with the worker-mean kernel: identical bits
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    c = si.CONFIGS[name]
+    table = sampling.class_pairs(0, c["m"]) if name == "c4" else None
+    X, y = si.mixture_data(0, c["m"], c["n"], c["dims"][0], table)
+    x0 = si.model_init(0, "mlp", c["dims"])
+    Xd, yd = to_dev(X), to_dev(y)
+    iters = 5 * c["tau"] * (4 if c["tau"] == 2 else 1)
+    got = {}
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    for fused in (True, False):
+        with torch.cuda.stream(stream):
+            opt = OverlapLocalSGD("mlp", m=c["m"], tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"],
+                                  beta=c["beta"], mu=c["mu"], batch=c["batch"], seed=0, dims=c["dims"],
+                                  gemm_bf16=1, x0=x0, X=Xd, y=yd)
+            opt.set_anchor_fusion(fused)
+            loss = torch.zeros((iters, c["m"]), device="cuda")
+            opt.run(iters, loss)
+            assert opt.graph_replays >= 1
+            opt.join()
+        torch.cuda.synchronize()
+        z, v = opt.get_params(-1).copy(), opt.get_params(-2).copy()
+        xs = [opt.get_params(i).copy() for i in (0, c["m"] // 2, c["m"] - 1)]
+        got[fused] = [z, v, loss.cpu().numpy()] + xs
+        opt.close()
+    for a, b in zip(got[True], got[False]):
+        assert np.array_equal(a, b)
+
+
 def test_config3_late_regime_resynchronised_with_the_oracle():
     """Config 3 beyond the point where its trajectory stops being reproducible: the small-loss,
     large-momentum regime of iterations 300-1000.  Chaos cannot be followed over hundreds of
