@@ -142,6 +142,8 @@ CSRC = os.path.join(ROOT, "paper_2002_09539_b200", "csrc")
 # When the file has changed since, the entry no longer describes the kernel and `traffic`
 # is reported as null.
 NCU_TRAFFIC = {
+    # profiles/wgrad_update_fused_c3_mlp.txt
+    ("c3", 1, "wgrad_update"): (1180.1e6, 1298.9e6, "tc_wgrad.cu", "c14ee59c23c2b664c639ec6efbf8356c2f4850cf"),
 }
 
 
@@ -551,7 +553,7 @@ def run_ours(args, rank, world):
 
     out = None
     if rank == 0:
-        cpu = cpu_baseline(name, c, X, y, x0, seed)
+        cpu = None if args.no_cpu_baseline else cpu_baseline(name, c, X, y, x0, seed)
         resident = X.nbytes + (2 + (1 if c["mu"] else 0) + 1) * m * P * 4
         out = {
             "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world,
@@ -867,6 +869,8 @@ def main():
     ap.add_argument("--no-kernel-points", action="store_true",
                     help="skip the stand-alone update/anchor kernel measurements (config 5's "
                          "10M x 16 and 50M x 64 points) that the default line carries")
+    ap.add_argument("--no-cpu-baseline", action="store_true",
+                    help="skip the oracle timing on the host cores (profiling runs)")
     ap.add_argument("--no-anchor-fusion", action="store_true",
                     help="MLP workloads: form the worker sum of Eq. 5 / Eq. 10-11 in the worker-mean "
                          "kernel only (olsgd_set_anchor_fusion(0)), to measure what the fusion buys")

@@ -271,6 +271,16 @@ int64_t olsgd_graph_block(const olsgd_ctx* ctx);
  * no counterpart: this is launch plumbing.                                               */
 int olsgd_set_launch_overlap(int on);
 
+/* Process-wide switch for the forward and input-gradient GEMMs of the tensor-core path.
+ * on != 0: where a layer has an even number of 128-row tiles they run on CTA pairs
+ * (thread-block clusters of two, one tcgen05.mma of M = 256 for both, each CTA loading half
+ * of the batch operand).  on == 0 (the default: measured slightly faster on the benchmark
+ * configurations): one CTA per tile.  The accumulation order of every output element is the
+ * same, so the results are the same bits.  Applies to launches made after the call (a
+ * captured graph keeps the setting it was captured with).  Returns the previous setting.
+ * The paper has no counterpart: this is kernel plumbing.                                    */
+int olsgd_set_gemm_pairs(int on);
+
 /* Copy one vector of the state to the caller.  Joins both streams (blocks
  * the host).  which: 0..m-1 worker model x^(i); -1 anchor z; -2 anchor
  * momentum v; -3 virtual sequence y = (1-alpha) mean_i x^(i) + alpha z

@@ -89,6 +89,7 @@ def load_library():
         "olsgd_graph_replays": (i64, [vp]),
         "olsgd_graph_block": (i64, [vp]),
         "olsgd_set_launch_overlap": (i32, [i32]),
+        "olsgd_set_gemm_pairs": (i32, [i32]),
         "olsgd_profile_enable": (i32, [vp, i32]),
         "olsgd_profile_read": (i32, [vp, C.POINTER(i64), C.POINTER(C.c_double), i32]),
         "olsgd_profile_read_layers": (i32, [vp, C.POINTER(i64), C.POINTER(C.c_double), i32]),
@@ -130,6 +131,11 @@ def class_pairs(seed, m, device="cuda"):
 def set_launch_overlap(on):
     """olsgd_set_launch_overlap: process-wide; returns the previous setting."""
     return bool(load_library().olsgd_set_launch_overlap(1 if on else 0))
+
+
+def set_gemm_pairs(on):
+    """olsgd_set_gemm_pairs: process-wide; returns the previous setting."""
+    return bool(load_library().olsgd_set_gemm_pairs(1 if on else 0))
 
 
 NOALLOC_MAX_WORKERS = 16384

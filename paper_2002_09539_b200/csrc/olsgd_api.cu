@@ -507,6 +507,7 @@ olsgd_status check_device_status(olsgd_ctx* c) {
 namespace olsgd {
 void set_thread_error(const char* text) { g_last_error = text ? text : ""; }
 int g_launch_overlap = 1;
+int g_gemm_pairs = 0;
 thread_local bool g_launch_plain = false;
 
 int current_device() {
@@ -1267,6 +1268,12 @@ int64_t olsgd_graph_block(const olsgd_ctx* c) { return c ? c->graph_block : -1; 
 int olsgd_set_launch_overlap(int on) {
   const int before = olsgd::g_launch_overlap;
   olsgd::g_launch_overlap = on ? 1 : 0;
+  return before;
+}
+
+int olsgd_set_gemm_pairs(int on) {
+  const int before = olsgd::g_gemm_pairs;
+  olsgd::g_gemm_pairs = on ? 1 : 0;
   return before;
 }
 

@@ -19,6 +19,7 @@ namespace olsgd {
 // kernel after this one start its own launch.  A kernel launched the ordinary way passes
 // through the gate at once.
 extern int g_launch_overlap;   // olsgd_set_launch_overlap
+extern int g_gemm_pairs;       // olsgd_set_gemm_pairs: long-K GEMMs on CTA pairs (cta_group::2)
 // Set around a launch that goes to a stream whose previous operation is an event wait, not a
 // kernel: such a launch is an ordinary one (its kernel passes the gate at once).
 extern thread_local bool g_launch_plain;

@@ -46,6 +46,92 @@ struct SharedCtl {
   int abort_flag;
 };
 
+// The epilogue of one 128 x BN accumulator tile, run by the four warps 2-5 of a CTA: TMEM lane
+// r <-> row m0 + r, column j <-> col n0 + j.  What it needs besides the accumulator is
+// fetched while the main loop runs: the row's bias, or the first 32 columns of its ReLU mask
+// (the next 32 are fetched while the current ones are applied).
+template <int BN>
+__device__ __forceinline__ void gemm_epilogue(const EpiArgs& ea, uint32_t tmem_base, uint32_t tmem_full_bar,
+                                              volatile int* abort_flag, int warp, int lane, int m0,
+                                              int n0, int worker) {
+  const int lane_group = warp & 3;
+  const int row = m0 + lane_group * 32 + lane;
+  const int64_t wk = worker;
+  float bias = 0.f;
+  if (ea.epilogue == GEMM_EPI_BIAS_RELU) bias = ea.bias[wk * ea.bias_batch + row];
+  uint4 mk[4], mk_next[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) mk[q] = mk_next[q] = make_uint4(0u, 0u, 0u, 0u);
+  const uint4* mask_row = nullptr;
+  if (ea.epilogue == GEMM_EPI_RELU_MASK) {
+    mask_row = reinterpret_cast<const uint4*>(ea.mask + (wk * ea.Ma + row) * ea.Nb + n0);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) mk[q] = mask_row[q];
+  }
+  if (mbar_wait(tmem_full_bar, 0, abort_flag) && !*abort_flag) {
+    tc_fence_after();
+#pragma unroll 1
+    for (int c = 0; c < BN / 32; ++c) {
+      if (ea.epilogue == GEMM_EPI_RELU_MASK && c + 1 < BN / 32) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) mk_next[q] = mask_row[(c + 1) * 4 + q];
+      }
+      float v[32];
+      tmem_ld32(tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)(c * 32), v);
+      const int col0 = n0 + c * 32;
+      if (ea.epilogue == GEMM_EPI_STORE_F32) {
+        float4* dst = reinterpret_cast<float4*>(ea.out_f + wk * ea.out_batch +
+                                                  (int64_t)row * ea.ldo + col0);
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+      } else {
+        const int64_t t_off = (wk * ea.Ma + row) * ea.Nb + col0;
+        if (ea.epilogue == GEMM_EPI_BIAS_RELU) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j] + bias, 0.f);
+        } else {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint4 w = mk[q];
+            const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              // a bf16 is positive iff its sign bit is clear and it is not zero
+              const uint32_t lo = ws[e] & 0xFFFFu, hi = ws[e] >> 16;
+              if (!(lo != 0 && lo < 0x8000u)) v[q * 8 + e * 2] = 0.f;
+              if (!(hi != 0 && hi < 0x8000u)) v[q * 8 + e * 2 + 1] = 0.f;
+            }
+            mk[q] = mk_next[q];
+          }
+        }
+        uint32_t pk[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+          pk[j] = *reinterpret_cast<uint32_t*>(&b2);
+        }
+        if (ea.out_t) {
+          uint4* dst = reinterpret_cast<uint4*>(ea.out_t + t_off);
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            dst[q] = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+        }
+        if (ea.out_n) {
+          // [Nb][Ma]: for a fixed column the 32 lanes of the warp write 32 consecutive rows
+          __nv_bfloat16* dst = ea.out_n + (wk * ea.Nb + col0) * ea.Ma + row;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const uint32_t w = pk[j >> 1];
+            const uint16_t h = (j & 1) ? (uint16_t)(w >> 16) : (uint16_t)(w & 0xFFFFu);
+            *reinterpret_cast<uint16_t*>(dst + (int64_t)j * ea.Ma) = h;
+          }
+        }
+      }
+    }
+  }
+}
+
 template <int BN, int STAGES>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
@@ -158,86 +244,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
     umma_commit(smem_u32(&ctl->tmem_full));   // accumulator complete
   } else if (warp >= 2) {
-    // ---------------- epilogue: TMEM lane r <-> row m0 + r, column j <-> col n0 + j
-    // what the epilogue needs besides the accumulator is fetched while the main loop runs:
-    // the row's bias, or the first 32 columns of its ReLU mask (the next 32 are fetched
-    // while the current ones are applied)
-    const int lane_group = warp & 3;
-    const int row = m0 + lane_group * 32 + lane;
-    const int64_t wk = worker;
-    float bias = 0.f;
-    if (ea.epilogue == GEMM_EPI_BIAS_RELU) bias = ea.bias[wk * ea.bias_batch + row];
-    uint4 mk[4], mk_next[4];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) mk[q] = mk_next[q] = make_uint4(0u, 0u, 0u, 0u);
-    const uint4* mask_row = nullptr;
-    if (ea.epilogue == GEMM_EPI_RELU_MASK) {
-      mask_row = reinterpret_cast<const uint4*>(ea.mask + (wk * ea.Ma + row) * ea.Nb + n0);
-#pragma unroll
-      for (int q = 0; q < 4; ++q) mk[q] = mask_row[q];
-    }
-    if (mbar_wait(smem_u32(&ctl->tmem_full), 0, abort_flag) && !*abort_flag) {
-      tc_fence_after();
-#pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        if (ea.epilogue == GEMM_EPI_RELU_MASK && c + 1 < BN / 32) {
-#pragma unroll
-          for (int q = 0; q < 4; ++q) mk_next[q] = mask_row[(c + 1) * 4 + q];
-        }
-        float v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)(c * 32), v);
-        const int col0 = n0 + c * 32;
-        if (ea.epilogue == GEMM_EPI_STORE_F32) {
-          float4* dst = reinterpret_cast<float4*>(ea.out_f + wk * ea.out_batch +
-                                                  (int64_t)row * ea.ldo + col0);
-#pragma unroll
-          for (int j = 0; j < 8; ++j)
-            dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-        } else {
-          const int64_t t_off = (wk * ea.Ma + row) * ea.Nb + col0;
-          if (ea.epilogue == GEMM_EPI_BIAS_RELU) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j] + bias, 0.f);
-          } else {
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const uint4 w = mk[q];
-              const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                // a bf16 is positive iff its sign bit is clear and it is not zero
-                const uint32_t lo = ws[e] & 0xFFFFu, hi = ws[e] >> 16;
-                if (!(lo != 0 && lo < 0x8000u)) v[q * 8 + e * 2] = 0.f;
-                if (!(hi != 0 && hi < 0x8000u)) v[q * 8 + e * 2 + 1] = 0.f;
-              }
-              mk[q] = mk_next[q];
-            }
-          }
-          uint32_t pk[16];
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
-            pk[j] = *reinterpret_cast<uint32_t*>(&b2);
-          }
-          if (ea.out_t) {
-            uint4* dst = reinterpret_cast<uint4*>(ea.out_t + t_off);
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-              dst[q] = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
-          }
-          if (ea.out_n) {
-            // [Nb][Ma]: for a fixed column the 32 lanes of the warp write 32 consecutive rows
-            __nv_bfloat16* dst = ea.out_n + (wk * ea.Nb + col0) * ea.Ma + row;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const uint32_t w = pk[j >> 1];
-              const uint16_t h = (j & 1) ? (uint16_t)(w >> 16) : (uint16_t)(w & 0xFFFFu);
-              *reinterpret_cast<uint16_t*>(dst + (int64_t)j * ea.Ma) = h;
-            }
-          }
-        }
-      }
-    }
+    gemm_epilogue<BN>(ea, tmem_base, smem_u32(&ctl->tmem_full), abort_flag, warp, lane, m0, n0, worker);
   }
 
   // ---------------- teardown: every role arrives here, all waits above are bounded
@@ -252,6 +259,132 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
     __syncwarp();
     tmem_dealloc(tmem_base, kTmemCols);
+  }
+  if (threadIdx.x == 0 && *abort_flag && ea.status) atomicExch(ea.status, (int)OLSGD_ETIMEOUT);
+}
+
+// The same GEMM on CTA pairs: the two CTAs of a cluster take two adjacent 128-row tiles of
+// one worker's D and issue ONE tcgen05.mma.cta_group::2 of M = 256 per 16 K elements.  Each
+// CTA still loads its own 128 rows of A, but only HALF of the B tile (the batch operand, which
+// every tile of a worker needs): the operand bytes per SM and k-block drop from 16 + BN / 8 KB
+// to 16 + BN / 16 KB, and delivery of operands into the SM is what bounds this kernel.
+// Every CTA fetches what it holds with its own TMA loads (no multicast); the loads of both
+// CTAs are counted on the full-barrier of the pair's leader (even rank), which alone issues
+// the MMAs; its commits arrive on the empty- and accumulator-barriers of both CTAs.
+template <int BN, int STAGES>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                    int num_kb, int a_mn, EpiArgs ea) {
+  constexpr uint32_t kABytes = kBM * kBK * 2;
+  constexpr uint32_t kBBytes = (BN / 2) * kBK * 2;         // this CTA's half of the B tile
+  constexpr uint32_t kStageBytes = kABytes + kBBytes;
+  constexpr uint32_t kTmemCols = BN < 32 ? 32 : BN;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                              ~static_cast<uintptr_t>(1023));
+  SharedCtl* ctl = reinterpret_cast<SharedCtl*>(tiles + STAGES * kStageBytes);
+  volatile int* abort_flag = &ctl->abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // the pair lies along the grid's x dimension, which counts the 128-row tiles here
+  const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * BN, worker = blockIdx.z;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+
+  if (threadIdx.x == 0) {
+    prefetch_tensormap(&map_a);
+    prefetch_tensormap(&map_b);
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&ctl->full[s]), 1);
+      mbar_init(smem_u32(&ctl->empty[s]), 1);
+    }
+    mbar_init(smem_u32(&ctl->tmem_full), 1);
+    ctl->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // the same warp of both CTAs allocates the pair's tensor memory
+  if (warp == 1) tmem_alloc_pair(smem_u32(&ctl->tmem_base), kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  // the peer's barriers are signalled from here: they must be initialised first
+  cluster_barrier();
+  tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+  auto load_a = [&](int kb, uint32_t a_dst, uint32_t bar) {
+    if (a_mn) {
+      tma_load_3d_pair(a_dst, &map_a, bar, m0, kb * kBK, worker);
+      tma_load_3d_pair(a_dst + kABytes / 2, &map_a, bar, m0 + 64, kb * kBK, worker);
+    } else {
+      tma_load_3d_pair(a_dst, &map_a, bar, kb * kBK, m0, worker);
+    }
+  };
+  // weights that the kernel ahead of this one does not write are requested before the gate
+  // (see gemm_tc_kernel); the leader announces both CTAs' bytes of a stage
+  const int n_early = ea.a_early ? (num_kb < STAGES ? num_kb : STAGES) : 0;
+  if (warp == 0 && lane == 0) {
+    for (int kb = 0; kb < n_early; ++kb) {
+      if (leader) mbar_expect_tx(smem_u32(&ctl->full[kb]), 2 * kStageBytes);
+      load_a(kb, smem_u32(tiles + kb * kStageBytes), pair_leader_addr(smem_u32(&ctl->full[kb])));
+    }
+  }
+  launch_gate();
+
+  if (warp == 0 && lane == 0) {
+    // ---------------- TMA producer (both CTAs)
+    for (int kb = 0; kb < num_kb; ++kb) {
+      const int s = kb % STAGES;
+      const uint32_t ph = (kb / STAGES) & 1;
+      const uint32_t full = smem_u32(&ctl->full[s]);
+      const uint32_t a_dst = smem_u32(tiles + s * kStageBytes);
+      if (kb >= n_early) {
+        if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1, abort_flag)) break;
+        if (leader) mbar_expect_tx(full, 2 * kStageBytes);
+        load_a(kb, a_dst, pair_leader_addr(full));
+      }
+      tma_load_3d_pair(a_dst + kABytes, &map_b, pair_leader_addr(full), kb * kBK,
+                       n0 + (int)rank * (BN / 2), worker);
+    }
+    // a CTA that gave up leaves its copies to the bounded grace period below
+  } else if (warp == 1 && lane == 0 && leader) {
+    // ---------------- MMA issuer (leader only)
+    const uint32_t idesc = instr_desc_bf16_pair(BN) | (a_mn ? (1u << 15) : 0u);
+    bool ok = true;
+    for (int kb = 0; kb < num_kb && ok; ++kb) {
+      const int s = kb % STAGES;
+      const uint32_t ph = (kb / STAGES) & 1;
+      ok = mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t a_addr = smem_u32(tiles + s * kStageBytes);
+      const uint64_t a_desc = a_mn ? smem_desc_mn_sw128(a_addr) : smem_desc_k_sw128(a_addr);
+      const uint64_t a_step = a_mn ? 128u : 2u;
+      const uint64_t b_desc = smem_desc_k_sw128(a_addr + kABytes);
+#pragma unroll
+      for (int k = 0; k < kBK / kUmmaK; ++k)
+        umma_bf16_pair(tmem_base, a_desc + a_step * (uint64_t)k, b_desc + (uint64_t)(2 * k), idesc,
+                       (kb > 0 || k > 0) ? 1u : 0u);
+      umma_commit_pair(smem_u32(&ctl->empty[s]));   // the stage is free in both CTAs
+    }
+    umma_commit_pair(smem_u32(&ctl->tmem_full));    // both accumulators are complete
+  } else if (warp >= 2) {
+    gemm_epilogue<BN>(ea, tmem_base, smem_u32(&ctl->tmem_full), abort_flag, warp, lane, m0, n0, worker);
+  }
+
+  // ---------------- teardown: every role of both CTAs arrives here, all waits are bounded
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) {
+    // bounded grace period for copies and MMAs that may still be in flight in the pair
+    const uint64_t t0 = global_ns();
+    while (global_ns() - t0 < 1000000ull) {
+    }
+  }
+  // neither CTA's shared or tensor memory may go while the other can still reach it
+  cluster_barrier();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
   }
   if (threadIdx.x == 0 && *abort_flag && ea.status) atomicExch(ea.status, (int)OLSGD_ETIMEOUT);
 }
@@ -294,6 +427,47 @@ cudaError_t launch_one(const GemmArgs& a, const CUtensorMap& ma, const CUtensorM
   return launch_chained(kern, grid, dim3(kThreads), smem, s, ma, mb, a.K / kBK, a.a_mn_major ? 1 : 0, ea);
 }
 
+template <int BN, int STAGES>
+cudaError_t launch_pair(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMap& mb, cudaStream_t s) {
+  constexpr size_t smem = (size_t)STAGES * (kBM * kBK * 2 + (BN / 2) * kBK * 2) + sizeof(SharedCtl) + 1024;
+  static PerDeviceSmem configured;
+  auto kern = gemm_tc_pair_kernel<BN, STAGES>;
+  {
+    const cudaError_t e = ensure_dynamic_smem(configured, kern, smem);
+    if (e != cudaSuccess) return e;
+  }
+  EpiArgs ea;
+  ea.epilogue = a.epilogue;
+  ea.once = a.a_read_once;
+  ea.a_early = a.a_ready_early;
+  ea.Ma = a.Ma;
+  ea.Nb = a.Nb;
+  ea.bias = a.bias;
+  ea.bias_batch = a.bias_batch;
+  ea.mask = a.mask;
+  ea.out_t = a.out_t;
+  ea.out_n = a.out_n;
+  ea.out_f = a.out_f;
+  ea.ldo = a.ldo;
+  ea.out_batch = a.out_batch;
+  ea.status = a.status;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(a.Ma / kBM, a.Nb / BN, a.m);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;   // pairs of adjacent 128-row tiles
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = (g_launch_overlap && !g_launch_plain) ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, kern, ma, mb, a.K / kBK, a.a_mn_major ? 1 : 0, ea);
+}
+
 // Self-test of the bounded wait: one thread waits on an mbarrier that nothing ever
 // arrives on, gives up after `limit_ns` and reports OLSGD_ETIMEOUT exactly as the GEMM
 // kernels do.  The context stays usable.
@@ -334,6 +508,12 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, cudaStream_t s) {
     if (!make_map(&ma, a.A, a.Ma, a.K, a.m, a.lda, a.a_batch, 64)) return cudaErrorInvalidValue;
   } else if (!make_map(&ma, a.A, a.K, a.Ma, a.m, a.lda, a.a_batch, kBM)) {
     return cudaErrorInvalidValue;
+  }
+  // long K and an even number of 128-row tiles: CTA pairs, each CTA loading half of the B tile
+  const bool pairs = g_gemm_pairs && a.K / kBK > 2 && (a.Ma / kBM) % 2 == 0 && (bn == 128 || bn == 64);
+  if (pairs) {
+    if (!make_map(&mb, a.B, a.K, a.Nb, a.m, a.ldb, a.b_batch, bn / 2)) return cudaErrorInvalidValue;
+    return bn == 128 ? launch_pair<128, 8>(a, ma, mb, s) : launch_pair<64, 8>(a, ma, mb, s);
   }
   if (!make_map(&mb, a.B, a.K, a.Nb, a.m, a.ldb, a.b_batch, bn)) return cudaErrorInvalidValue;
   // short K (weight gradients, K = batch): few stages so several CTAs share an SM

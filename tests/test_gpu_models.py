@@ -156,6 +156,36 @@ def test_fused_weight_gradient_update_gives_the_bits_of_the_separate_kernel(dims
         assert np.array_equal(a.get_params(-5 - i), b.get_params(-5 - i))
 
 
+@pytest.mark.parametrize("dims,m,n,batch", [([192, 256, 128, 7], 3, 100, 64),
+                                            ([256, 512, 256, 10], 2, 150, 128),
+                                            ([128, 256, 256, 256, 10], 2, 96, 64)])
+def test_gemm_on_cta_pairs_gives_the_bits_of_one_cta_per_tile(dims, m, n, batch):
+    # forward and input-gradient GEMMs on CTA pairs (one tcgen05.mma of M = 256 for two adjacent
+    # 128-row tiles, each CTA loading half of the batch operand) against one CTA per tile: every
+    # output element sums the same products in the same order
+    from paper_2002_09539_b200 import OverlapLocalSGD, set_gemm_pairs
+    X, y = si.mixture_data(23, m, n, dims[0])
+    y = (y % dims[-1]).astype(np.int32)
+    x0 = si.model_init(23, "mlp", dims)
+    kw = dict(dims=dims, gemm_bf16=1, m=m, tau=2, batch=batch, gamma=0.05, alpha=0.6, beta=0.9, mu=0.9,
+              seed=23, x0=x0, X=to_dev(X), y=to_dev(y))
+    got = {}
+    before = set_gemm_pairs(True)
+    try:
+        for on in (True, False):
+            set_gemm_pairs(on)
+            opt = OverlapLocalSGD("mlp", **kw)
+            loss = torch.zeros((5, m), device="cuda")
+            opt.run(5, loss)
+            got[on] = opt.state() + (loss.cpu().numpy(),)
+            opt.close()
+    finally:
+        set_gemm_pairs(before)
+    assert np.isfinite(got[True][3]).all()
+    for a, b in zip(got[True], got[False]):
+        assert np.array_equal(a, b)
+
+
 @pytest.mark.parametrize("m,beta,tau", [(2, 0.9, 2), (8, 0.0, 2), (16, 0.9, 1), (17, 0.7, 3),
                                         (33, 0.9, 2), (64, 0.0, 2)])
 def test_anchor_fusion_gives_the_bits_of_the_worker_mean_kernel(m, beta, tau):
