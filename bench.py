@@ -399,7 +399,7 @@ def run_ours(args, rank, world):
     # MIN_TIMED_S have been timed, and the median block is reported.
     opt.run(W)
     block = opt.graph_block
-    opt.run(3 * block)
+    opt.run(K if block <= K <= 64 else 3 * block)
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
@@ -415,11 +415,13 @@ def run_ours(args, rank, world):
     ms = float(np.median(times))
     value = world * m * K / (ms * 1e-3)
     per_block = replays // len(times)
+    unit = c["tau"] if c["tau"] % 2 == 0 else 2 * c["tau"]
+    glen = K // unit * unit if block <= K <= 64 else block      # what olsgd_run captures for this K
     timing = dict(blocks=len(times), timed_s=round(sum(times) * 1e-3, 3),
                   ms_per_step_median=round(ms / K, 4), ms_per_step_min=round(min(times) / K, 4),
                   ms_per_step_max=round(max(times) / K, 4),
                   path=("olsgd_run: %d replay(s) of the captured %d-iteration graph + %d plain "
-                        "step(s) per timed block" % (per_block, block, K - per_block * block))
+                        "step(s) per timed block" % (per_block, glen, K - per_block * glen))
                   if per_block else "olsgd_run: plain launches (K is shorter than the captured block)")
 
     # ---- per-kernel-class device time (second pass, every launch bracketed by events)
@@ -484,6 +486,21 @@ def run_ours(args, rank, world):
         ser.close()
         del ser
         roofline["kernels"] = gemm_rooflines(c, ser_prof, KP, peaks)
+        # the weight-gradient/update launch on ordinary and on sync steps, from the same pass
+        for tag, what in ((0, "ordinary step"), (1, "sync step: pull-back" +
+                                                 (", worker sums" if anchor_fusion_on else ""))):
+            launches_t, ms_t = ser_prof["wgrad_update"][tag]
+            if launches_t > 0:
+                cc = dict(c, sum_slices=(4 if c["m"] >= 64 else 2 if c["m"] >= 8 else 1)
+                          if anchor_fusion_on else 0)
+                ab_t = algorithmic_bytes(cc, "wgrad_update", P, float(tag))
+                us_t = ms_t * 1e3 / launches_t
+                roofline["kernels"].append(dict(
+                    kernel="wgrad_tc_kernel<FUSED%s>, %s" % (", SUM" if tag and anchor_fusion_on else "", what),
+                    us=round(us_t, 2), gbs=round(ab_t / us_t / 1e3, 1),
+                    frac_of_measured=round(ab_t / us_t / 1e3 / peaks["hbm_gbs"], 4),
+                    frac_of_8000=round(ab_t / us_t / 1e3 / 8000.0, 4),
+                    algorithmic_bytes_per_launch=int(ab_t)))
         roofline["kernels_note"] = ("GEMM launches timed with the library's streams serialised "
                                     "(each kernel alone on the GPU, warm caches)")
 

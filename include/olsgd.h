@@ -249,16 +249,18 @@ int64_t olsgd_row_floats(const olsgd_ctx* ctx);
  *   loss_device  n_iters * m floats ([iteration][worker]), device; or NULL  */
 olsgd_status olsgd_run(olsgd_ctx* ctx, int64_t n_iters, float* loss_device);
 
-/* How often olsgd_run has replayed its captured CUDA graph on this context so far.  Long
- * runs (at least three blocks of olsgd_graph_block iterations, or one block once the graph
- * exists) are executed as replays of one captured block; the iteration number the minibatch rule needs is then read from
- * device memory.  Capturing needs main_stream to be a real stream: with the legacy default
- * stream (NULL) olsgd_run keeps launching kernel by kernel and this stays 0.  The results
- * are the same bits either way.                                                        */
+/* How often olsgd_run has replayed a captured CUDA graph on this context so far.  olsgd_run
+ * executes its iterations as replays of one captured block of whole periods (an even number
+ * of iterations); the iteration number the minibatch rule needs is then read from device
+ * memory.  A run of at least three default blocks (olsgd_graph_block) launches one block
+ * kernel by kernel, captures it and replays it; a run of 8 to 64 iterations on a context that
+ * has already launched an ordinary and a sync step kernel by kernel is captured whole, so
+ * that repeating olsgd_run(n) costs one graph launch per call.  Capturing needs main_stream
+ * to be a real stream: with the legacy default stream (NULL) olsgd_run keeps launching kernel
+ * by kernel and this stays 0.  The results are the same bits either way.                   */
 int64_t olsgd_graph_replays(const olsgd_ctx* ctx);
-/* Iterations in one captured block of this context: whole periods, an even count, at least
- * eight.  A first olsgd_run of at least three blocks captures the graph; after that every
- * olsgd_run of at least one block replays it.                                            */
+/* Iterations in the default captured block of this context: whole periods, an even count, at
+ * least eight.                                                                            */
 int64_t olsgd_graph_block(const olsgd_ctx* ctx);
 
 /* Process-wide switch for how the kernels of one iteration follow each other on the main
@@ -383,8 +385,9 @@ olsgd_status olsgd_profile_read(olsgd_ctx* ctx, int64_t* launches, double* milli
 /* The same profile split by layer: entry [c * OLSGD_MAX_DIMS + l] covers the launches of class
  * c that belong to layer l (forward GEMM producing hidden layer l >= 1; OLSGD_KC_BACKWARD with
  * l >= 1: the input-gradient GEMM producing the gradient of hidden layer l, or a weight-
- * gradient GEMM that is launched by itself; l = 0: launches that belong to no hidden layer,
- * e.g. the output layer's kernels).  Both arrays hold OLSGD_N_KERNEL_CLASSES * OLSGD_MAX_DIMS
+ * gradient GEMM that is launched by itself; OLSGD_KC_WGRAD_UPDATE: l = 0 ordinary steps, l = 1
+ * sync steps; otherwise l = 0: launches that belong to no hidden layer, e.g. the output
+ * layer's kernels).  Both arrays hold OLSGD_N_KERNEL_CLASSES * OLSGD_MAX_DIMS
  * entries.  Summing over l gives olsgd_profile_read.                                      */
 olsgd_status olsgd_profile_read_layers(olsgd_ctx* ctx, int64_t* launches, double* millis,
                                        int32_t reset);

@@ -379,7 +379,9 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
       OLSGD_TRY(cudaStreamWaitEvent(s, io.wait_before_update, 0));
       waited = true;
     }
-    Scope sc(hook, OLSGD_KC_WGRAD_UPDATE, s);
+    // tagged 1 on sync steps (the launch that also applies Eq. 4 and, with the worker sum
+    // inside, forms the partial sums), 0 on ordinary steps
+    Scope sc(hook, OLSGD_KC_WGRAD_UPDATE | ((pending[0].upd.sync ? 1 : 0) << 8), s);
     const cudaError_t e = launch_wgrad_tc_batch(pending, n_pending, s);
     n_pending = 0;
     return e;

@@ -75,6 +75,12 @@ struct olsgd_ctx {
   bool need_sync = false;       // a period ended; olsgd_period_sync is due
   bool sync_begun = false;      // olsgd_period_sync_begin ran; _finish is due
 
+  // graph_block: default length of a captured block; graph_len: length of the block that
+  // graph_exec holds (a short run that is repeated is captured whole, up to kMaxGraphBlock);
+  // plain_steps: iterations launched kernel by kernel so far (one-time kernel set-up happens
+  // there, never inside a capture).
+  int graph_len = 0;
+  int64_t plain_steps = 0, plain_syncs = 0;
   // olsgd_run replays a captured CUDA graph of `graph_block` iterations (a whole number of
   // periods, an even number of steps so that the ping-pong buffers return to their places)
   int graph_block = 0;
@@ -211,6 +217,7 @@ ProfHook make_hook(olsgd_ctx* c) {
 }
 
 // Iterations in one captured block: whole periods, an even count, at least eight steps.
+constexpr int kMaxGraphBlock = 64;   // iterations in one captured block, at most
 int graph_block_len(int tau) {
   int periods = (8 + tau - 1) / tau;
   if ((periods * tau) % 2) periods *= 2;
@@ -310,7 +317,10 @@ olsgd_status make_plan(const olsgd_model_spec* spec, const olsgd_hparams* hp, Pl
   pl->off_tmp = take(row);
   pl->off_status = take(sizeof(int));
   pl->off_dev_k = take(sizeof(int64_t));
-  pl->off_loss_ring = take((size_t)graph_block_len(hp->tau) * m * sizeof(float));
+  {
+    const int base = graph_block_len(hp->tau);
+    pl->off_loss_ring = take((size_t)(base > kMaxGraphBlock ? base : kMaxGraphBlock) * m * sizeof(float));
+  }
   pl->off_shadow = pl->has_shadow ? take((size_t)pl->ld * m * sizeof(__nv_bfloat16)) : 0;
   pl->off_idx = pl->has_g ? take((size_t)m * hp->batch * sizeof(int32_t)) : 0;
   pl->off_idx_next = pl->has_g ? take((size_t)m * hp->batch * sizeof(int32_t)) : 0;
@@ -967,7 +977,11 @@ int64_t olsgd_row_floats(const olsgd_ctx* c) { return c ? c->ld : -1; }
 static olsgd_status run_one(olsgd_ctx* c, float* loss) {
   olsgd_status st = olsgd_local_step(c, loss);
   if (st != OLSGD_OK) return st;
-  if (c->need_sync) st = olsgd_period_sync(c);
+  if (c->need_sync) {
+    st = olsgd_period_sync(c);
+    if (!c->capturing) c->plain_syncs += 1;
+  }
+  if (!c->capturing) c->plain_steps += 1;
   return st;
 }
 
@@ -975,7 +989,7 @@ static olsgd_status run_one(olsgd_ctx* c, float* loss) {
 // graph.  The block ends with the side stream joined and with the device counter advanced,
 // so that replaying it continues the run.  On any failure the context falls back to plain
 // launches for good; the run itself is never affected because a capture executes nothing.
-static bool capture_block(olsgd_ctx* c) {
+static bool capture_block(olsgd_ctx* c, int len) {
   if (c->graph_exec) {
     cudaGraphExecDestroy(c->graph_exec);
     c->graph_exec = nullptr;
@@ -991,7 +1005,7 @@ static bool capture_block(olsgd_ctx* c) {
   c->capturing = true;
   c->capture_k0 = k0;
   bool ok = true;
-  for (int j = 0; j < c->graph_block && ok; ++j)
+  for (int j = 0; j < len && ok; ++j)
     ok = run_one(c, c->loss_ring + (int64_t)j * c->hp.m) == OLSGD_OK;
   if (ok && c->reduce_pending) {
     ok = cudaStreamWaitEvent(c->main, c->reduce_done, 0) == cudaSuccess;
@@ -1001,7 +1015,7 @@ static bool capture_block(olsgd_ctx* c) {
   // it reads is advanced (and every stream of a capture must rejoin its origin)
   if (ok && c->pre_pending) ok = cudaStreamWaitEvent(c->main, c->pre_done, 0) == cudaSuccess;
   c->pre_pending = false;
-  if (ok) ok = launch_counter(c->dev_k, 0, c->graph_block, false, c->main) == cudaSuccess;
+  if (ok) ok = launch_counter(c->dev_k, 0, len, false, c->main) == cudaSuccess;
   c->capturing = false;
   const cudaError_t e = cudaStreamEndCapture(c->main, &graph);
   // nothing ran: put the host-side state back to the start of the block
@@ -1029,6 +1043,7 @@ static bool capture_block(olsgd_ctx* c) {
   c->graph_cur = cur0;
   c->graph_kpar = (int)(k0 & 1);
   c->graph_staged = pre_k0 == k0;
+  c->graph_len = len;
   return true;
 }
 
@@ -1046,21 +1061,35 @@ olsgd_status olsgd_run(olsgd_ctx* c, int64_t n_iters, float* loss_device) {
     }
     return OLSGD_OK;
   };
-  const int block = c->graph_block;
   // the legacy default stream cannot be captured
   const bool real_stream = c->main != nullptr && c->main != cudaStreamLegacy &&
                            c->main != cudaStreamPerThread;
-  // A run long enough for three blocks captures a graph (one block of plain launches, the
-  // capture, then replays); once a context has its graph, any run of at least one block
-  // replays it.
-  const bool want_graph = real_stream && !c->graph_off && !c->prof && block > 0 &&
-                          (n_iters >= 3 * (int64_t)block || (c->graph_exec && n_iters >= block));
-  if (!want_graph) return plain(n_iters);
+  // Which block this run is executed in.  A run of at most kMaxGraphBlock iterations, on a
+  // context that has already launched an ordinary and a sync step kernel by kernel, is
+  // captured whole (whole periods, an even count): a caller that repeats olsgd_run(n) with a
+  // small n then pays one graph launch per call.  A long run (three default blocks or more)
+  // uses the default block: one block of plain launches, the capture, then replays.  Anything
+  // else that is at least as long as the block of an existing graph replays that graph.
+  const int base = c->graph_block;
+  const int unit = (c->hp.tau % 2) ? 2 * c->hp.tau : c->hp.tau;
+  if (!real_stream || c->graph_off || c->prof || base <= 0 || n_iters < base) return plain(n_iters);
   olsgd_status st = OLSGD_OK;
   // reach a period boundary
   while (c->k % c->hp.tau != 0 && t < n_iters)
     if ((st = plain(1)) != OLSGD_OK) return st;
-  if (n_iters - t < block) return plain(n_iters - t);
+  const int64_t left = n_iters - t, whole = left / unit * unit;
+  const bool plain_seen = c->plain_syncs >= 1 && (c->hp.tau == 1 || c->plain_steps > c->plain_syncs);
+  int block = 0;
+  bool first_plain = true;     // run one block with plain launches before a capture
+  if (whole >= base && whole <= kMaxGraphBlock && plain_seen) {
+    block = (int)whole;
+    first_plain = false;       // every kernel of a period has been launched before
+  } else if (left >= 3 * (int64_t)base) {
+    block = base;
+  } else if (c->graph_exec && left >= c->graph_len) {
+    block = c->graph_len;
+  }
+  if (block <= 0) return plain(left);
   // A block starts with the side stream joined and with the minibatch staged ahead by plain
   // steps (if any) joined too, outside any capture: from "the rows of iteration k are staged"
   // or from "none are".
@@ -1076,17 +1105,19 @@ olsgd_status olsgd_run(olsgd_ctx* c, int64_t n_iters, float* loss_device) {
     return OLSGD_OK;
   };
   auto graph_fits = [&]() {
-    return c->graph_exec && c->graph_cur == c->cur && c->graph_kpar == (int)(c->k & 1) &&
-           c->graph_staged == (c->pre_k == c->k);
+    return c->graph_exec && c->graph_len == block && c->graph_cur == c->cur &&
+           c->graph_kpar == (int)(c->k & 1) && c->graph_staged == (c->pre_k == c->k);
   };
   if ((st = settle()) != OLSGD_OK) return st;
   if (!graph_fits()) {
-    // one block with plain launches first (this also performs every one-time kernel attribute
-    // set-up, which must not happen inside a capture), then the capture
-    if (n_iters - t < 2 * (int64_t)block) return plain(n_iters - t);
-    if ((st = plain(block)) != OLSGD_OK) return st;
-    if ((st = settle()) != OLSGD_OK) return st;
-    if (!graph_fits() && !capture_block(c)) return plain(n_iters - t);
+    if (first_plain) {
+      // one block with plain launches first (this also performs every one-time kernel attribute
+      // set-up, which must not happen inside a capture), then the capture
+      if (n_iters - t < 2 * (int64_t)block) return plain(n_iters - t);
+      if ((st = plain(block)) != OLSGD_OK) return st;
+      if ((st = settle()) != OLSGD_OK) return st;
+    }
+    if (!graph_fits() && !capture_block(c, block)) return plain(n_iters - t);
   }
   {
     Launch l(c, OLSGD_KC_INDEX, c->main);
