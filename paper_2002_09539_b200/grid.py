@@ -66,9 +66,10 @@ def grid_points(taus, alphas, beta):
     return pts
 
 
-def run_grid(c, X, y, x0, points, iters, out_dir=None, tag="grid", command=""):
+def run_grid(c, X, y, x0, points, iters, out_dir=None, tag="grid", command="", consensus_stride=10):
     """Runs the points, returns {(label, tau, alpha): dict(loss, consensus, wsps)} and, with
-    out_dir, writes the two CSV files and the table."""
+    out_dir, writes the two CSV files and the table.  The consensus file keeps every
+    max(1, consensus_stride // tau)-th anchor refresh of a point (all of them are returned)."""
     results = {}
     for label, tau, alpha, beta, local in points:
         n = (iters // tau) * tau
@@ -92,11 +93,13 @@ def run_grid(c, X, y, x0, points, iters, out_dir=None, tag="grid", command=""):
         with open(os.path.join(out_dir, "hyperparameter_grid_%s_consensus.csv" % tag), "w") as f:
             f.write(head)
             f.write("# consensus_distance: sum_i ||x_i - z||^2 after the anchor refresh that closes "
-                    "iteration `iteration`\n")
+                    "iteration `iteration` (every max(1, %d // tau)-th refresh is listed)\n" % consensus_stride)
             f.write("method,tau,alpha,beta,iteration,consensus_distance\n")
             for (label, tau, alpha), r in results.items():
+                keep = max(1, consensus_stride // tau)
                 for k, v in r["consensus"]:
-                    f.write("%s,%d,%g,%g,%d,%.6e\n" % (label, tau, alpha, r["beta"], k, v))
+                    if (k // tau) % keep == 0:
+                        f.write("%s,%d,%g,%g,%d,%.6e\n" % (label, tau, alpha, r["beta"], k, v))
         with open(os.path.join(out_dir, "hyperparameter_grid_%s.md" % tag), "w") as f:
             f.write(head.replace("# ", "").replace("\n", "  \n"))
             f.write("\nLoss = training minibatch loss, mean over the workers; throughput by wall clock, "
@@ -119,6 +122,8 @@ def main():
     ap.add_argument("--alphas", default="0.5,0.6")
     ap.add_argument("--beta", type=float, default=0.7)
     ap.add_argument("--out", default="profiles")
+    ap.add_argument("--consensus-stride", type=int, default=10,
+                    help="list the consensus distance about every this many iterations")
     args = ap.parse_args()
     c = dict(si.CONFIGS[args.workload])
     table = class_pairs(0, c["m"], device="cpu").numpy() if c.get("non_iid") else None
@@ -130,7 +135,7 @@ def main():
     command = "--workload %s --iters %d --taus %s --alphas %s --beta %g" % (
         args.workload, args.iters, args.taus, args.alphas, args.beta)
     res = run_grid(c, X, y, x0, grid_points(taus, alphas, args.beta), args.iters, args.out,
-                   args.workload, command)
+                   args.workload, command, args.consensus_stride)
     for (label, tau, alpha), r in res.items():
         print("%-28s tau %2d alpha %.2f  loss %.4f -> %.4f  consensus %.3e  %.0f worker-steps/s"
               % (label, tau, alpha, r["loss"][0], r["loss"][-50:].mean(),

@@ -27,7 +27,8 @@ def test_grid_writes_loss_and_consensus_curves_that_follow_the_oracle(tmp_path):
     X, y = si.mixture_data(31, m, n, dims[0])
     x0 = si.model_init(31, "mlp", dims)
     points = [("Overlap-Local-SGD", tau, alpha, beta, False), ("Local SGD (Eq. 2)", tau, 0.0, 0.0, True)]
-    res = grid.run_grid(c, to_dev(X), to_dev(y), x0, points, iters, str(tmp_path), "tiny")
+    res = grid.run_grid(c, to_dev(X), to_dev(y), x0, points, iters, str(tmp_path), "tiny",
+                        consensus_stride=1)
     assert set(res) == {("Overlap-Local-SGD", tau, alpha), ("Local SGD (Eq. 2)", tau, 0.0)}
     loss_rows = _rows(os.path.join(tmp_path, "hyperparameter_grid_tiny_loss.csv"))
     cons_rows = _rows(os.path.join(tmp_path, "hyperparameter_grid_tiny_consensus.csv"))
