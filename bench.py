@@ -193,9 +193,11 @@ def algorithmic_bytes(c, kernel_class, P, sync_fraction):
         slices = c.get("sum_slices", 0)
         return m * fused * per + sync_fraction * 4 * (1 + slices) * fused + operands
     if kernel_class == "update":
+        # sync steps: the anchor read once, and (worker sum formed in the launch, long rows
+        # only) one row of partial sums written per slice
         per = (20 if mom else 12) + shadow
         rest = P - fused
-        return m * rest * per + sync_fraction * 4 * rest
+        return m * rest * per + sync_fraction * 4 * (1 + c.get("update_sum_slices", 0)) * rest
     if kernel_class == "anchor":
         return 4 * m * P + (16 if c["beta"] != 0.0 else 4) * P
     if kernel_class == "output_layer" and c.get("kind") in ("softmax", "linreg"):
@@ -249,70 +251,112 @@ def gemm_rooflines(c, layers_prof, n_steps, peaks):
     return out
 
 
+def worker_sum_slices(m):
+    """Rows of partial sums the library forms the worker sum in (a function of m alone)."""
+    return 4 if m >= 64 else 2 if m >= 8 else 1
+
+
 def flat_point(P, m, K, W, peaks):
-    """Config 5 at one (P, m): the stand-alone fused update and worker-mean/anchor kernels on a
-    flat parameter vector with external gradients.  Returns the point's record."""
+    """Config 5 at one (P, m): a flat parameter vector with external gradients.  The whole
+    iteration is timed as the library runs it by default (on long rows the sync step's update
+    launch also forms the worker sums, and the anchor refresh starts from those few rows) and
+    with the worker sum left to the worker-mean kernel; the kernels are timed one by one with
+    the two streams serialised.  Returns the point's record."""
     import torch
     from paper_2002_09539_b200 import OverlapLocalSGD
     c = si.CONFIGS["c5"]
+    tau = c["tau"]
     x0 = torch.randn(P, device="cuda")
     g = torch.randn((m, P), device="cuda") * c["grad_std"]
-    kw = dict(m=m, tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"], beta=c["beta"], mu=c["mu"],
+    kw = dict(m=m, tau=tau, gamma=c["gamma"], alpha=c["alpha"], beta=c["beta"], mu=c["mu"],
               flat_P=P, x0=x0)
-    opt = OverlapLocalSGD("flat", **kw)
 
-    def steps(count):
+    def steps(opt, count):
         for _ in range(count):
             opt.local_step_with_grads(g)
-            if opt.iteration % c["tau"] == 0:
+            if opt.iteration % tau == 0:
                 opt.period_sync()
 
-    steps(W)
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    n0 = opt.launch_count
-    e0.record()
-    steps(K)
-    opt.main.wait_stream(opt.side)
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1)
-    launches = opt.launch_count - n0
-    opt.profile_enable(True)
-    steps(K)
-    prof_overlap = opt.profile_read()
-    opt.profile_enable(False)
-    # the per-kernel bandwidths are taken with the two streams serialised: under overlap the
-    # anchor kernel shares HBM with the next period's update kernels and its event-bracketed
-    # duration measures that sharing, not the kernel
-    opt.close()
-    opt = OverlapLocalSGD("flat", overlap=False, **kw)
-    steps(W)
-    opt.profile_enable(True)
-    steps(K)
-    prof = opt.profile_read()
-    opt.profile_enable(False)
-    opt.close()
+    def timed(fusion):
+        opt = OverlapLocalSGD("flat", **kw)
+        opt.set_anchor_fusion(fusion)
+        steps(opt, W)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n0 = opt.launch_count
+        e0.record()
+        steps(opt, K)
+        opt.main.wait_stream(opt.side)
+        e1.record()
+        torch.cuda.synchronize()
+        ms, launches, summed = e0.elapsed_time(e1), opt.launch_count - n0, opt.summed_floats
+        opt.profile_enable(True)
+        steps(opt, K)
+        prof = opt.profile_read()
+        opt.profile_enable(False)
+        opt.close()
+        return ms, launches, summed, prof
+
+    def per_kernel(fusion):
+        # with the two streams serialised: under overlap the anchor kernel shares HBM with the
+        # next period's update kernels and its event-bracketed duration measures that sharing
+        opt = OverlapLocalSGD("flat", overlap=False, **kw)
+        opt.set_anchor_fusion(fusion)
+        steps(opt, W)
+        opt.profile_enable(True)
+        steps(opt, K)
+        prof = opt.profile_read_layers()
+        opt.profile_enable(False)
+        opt.close()
+        return {(cls, tag): (prof[cls][tag][1] / prof[cls][tag][0] if prof[cls][tag][0] else None)
+                for cls in ("update", "anchor") for tag in (0, 1)}
+
+    ms, launches, summed, prof_overlap = timed(True)
+    ms_plain = timed(False)[0] if summed else ms
+    ref = per_kernel(False)          # the stand-alone update kernel and the worker-mean kernel
     cc = dict(c, m=m)
-    n_sync = K // c["tau"]
-    upd_b = algorithmic_bytes(cc, "update", P, n_sync / K)
+    S = worker_sum_slices(m)
+    mom_rows = 16 if c["beta"] != 0.0 else 4
+    upd_b = algorithmic_bytes(cc, "update", P, 0)
+    upd_sync_b = algorithmic_bytes(cc, "update", P, 1)
     anc_b = algorithmic_bytes(cc, "anchor", P, 0)
-    upd_ms = prof["update"][1] / prof["update"][0]
-    anc_ms = prof["anchor"][1] / max(1, prof["anchor"][0])
+    n_sync = K // tau
+    # one figure for the update kernel, as before: all its launches, sync steps included
+    upd_ms = (ref[("update", 0)] * (K - n_sync) + ref[("update", 1)] * n_sync) / K
+    upd_all_b = (upd_b * (K - n_sync) + upd_sync_b * n_sync) / K
+    anc_ms = ref[("anchor", 0)]
     state_mb = (3 * m * P + 2 * P + m * P) * 4 / 1e6
+    gbs = lambda nbytes, t_ms: round(nbytes / t_ms / 1e6, 1)
+    frac = lambda nbytes, t_ms, peak: round(nbytes / t_ms / 1e6 / peak, 4)
     point = dict(
         P=P, m=m, worker_steps_per_s=round(m * K / (ms * 1e-3), 1),
         ms_per_step=round(ms / K, 4), gpu_launches=int(launches),
-        update_gbs=round(upd_b / upd_ms / 1e6, 1), anchor_gbs=round(anc_b / anc_ms / 1e6, 1),
+        worker_sum_in_update_launch=bool(summed),
+        ms_per_step_worker_mean_kernel=round(ms_plain / K, 4),
+        update_gbs=gbs(upd_all_b, upd_ms), anchor_gbs=gbs(anc_b, anc_ms),
         update_us=round(upd_ms * 1e3, 2), anchor_us=round(anc_ms * 1e3, 2),
         anchor_us_overlapped=round(prof_overlap["anchor"][1] * 1e3 /
                                    max(1, prof_overlap["anchor"][0]), 2),
-        update_frac_measured=round(upd_b / upd_ms / 1e6 / peaks["hbm_gbs"], 4),
-        anchor_frac_measured=round(anc_b / anc_ms / 1e6 / peaks["hbm_gbs"], 4),
-        update_frac_8000=round(upd_b / upd_ms / 1e6 / 8000.0, 4),
-        anchor_frac_8000=round(anc_b / anc_ms / 1e6 / 8000.0, 4),
+        update_frac_measured=frac(upd_all_b, upd_ms, peaks["hbm_gbs"]),
+        anchor_frac_measured=frac(anc_b, anc_ms, peaks["hbm_gbs"]),
+        update_frac_8000=frac(upd_all_b, upd_ms, 8000.0),
+        anchor_frac_8000=frac(anc_b, anc_ms, 8000.0),
         resident_mb=round(state_mb, 1), in_l2=bool(state_mb * 1e6 < L2_BYTES))
-    del opt, g, x0
+    if summed:
+        fused = per_kernel(True)
+        sum_b = upd_sync_b + 4 * S * P           # the sync-step launch also writes S rows of sums
+        fin_b = (4 * S + mom_rows) * P           # and the refresh reads them, with z and v
+        point.update(
+            sum_slices=S,
+            sync_update_sum_us=round(fused[("update", 1)] * 1e3, 2),
+            sync_update_sum_gbs=gbs(sum_b, fused[("update", 1)]),
+            sync_update_sum_frac_measured=frac(sum_b, fused[("update", 1)], peaks["hbm_gbs"]),
+            sync_update_plain_us=round(ref[("update", 1)] * 1e3, 2),
+            anchor_from_sums_us=round(fused[("anchor", 1)] * 1e3, 2),
+            anchor_from_sums_gbs=gbs(fin_b, fused[("anchor", 1)]),
+            anchor_from_sums_frac_measured=frac(fin_b, fused[("anchor", 1)], peaks["hbm_gbs"]),
+            sync_bytes_saved_per_period=int(anc_b - fin_b - 4 * S * P))
+    del g, x0
     torch.cuda.empty_cache()
     return point
 
@@ -320,7 +364,8 @@ def flat_point(P, m, K, W, peaks):
 def standalone_kernel_rooflines(peaks, steps=12, warmup=4):
     """The metric's second half: the stand-alone fused update kernel and the worker-mean/anchor
     kernel on config 5's 10M x 16 and 50M x 64 points, streams serialised, as HBM GB/s against
-    the measured copy bandwidth and against 8 TB/s."""
+    the measured copy bandwidth and against 8 TB/s; and the two launches that replace them on
+    sync steps (update with the worker sum inside, anchor refresh from the partial sums)."""
     out = []
     for P, m in ((10_000_000, 16), (50_000_000, 64)):
         pt = flat_point(P, m, steps, warmup, peaks)
@@ -331,6 +376,14 @@ def standalone_kernel_rooflines(peaks, steps=12, warmup=4):
         out.append(dict(kernel="worker_mean_anchor_kernel", workload=where, us=pt["anchor_us"],
                         gbs=pt["anchor_gbs"], frac_of_measured=pt["anchor_frac_measured"],
                         frac_of_8000=pt["anchor_frac_8000"]))
+        if pt["worker_sum_in_update_launch"]:
+            out.append(dict(kernel="fused_update_kernel<SUM> (sync steps)", workload=where,
+                            us=pt["sync_update_sum_us"], gbs=pt["sync_update_sum_gbs"],
+                            frac_of_measured=pt["sync_update_sum_frac_measured"],
+                            us_without_the_sum=pt["sync_update_plain_us"]))
+            out.append(dict(kernel="anchor_from_slices_kernel", workload=where,
+                            us=pt["anchor_from_sums_us"], gbs=pt["anchor_from_sums_gbs"],
+                            frac_of_measured=pt["anchor_from_sums_frac_measured"]))
     return out
 
 
@@ -425,7 +478,8 @@ def run_ours(args, rank, world):
                   if per_block else "olsgd_run: plain launches (K is shorter than the captured block)")
 
     # ---- per-kernel-class device time (second pass, every launch bracketed by events)
-    anchor_fusion_on = opt.anchor_fusion
+    # (a refresh has run by now: summed_floats says whether any launch formed worker sums)
+    anchor_fusion_on = opt.anchor_fusion and opt.summed_floats > 0
     KP = max(K, 2 * block)
     opt.profile_enable(True)
     opt.run(KP)
@@ -450,7 +504,9 @@ def run_ours(args, rank, world):
         avg_ms = busy[roof_class][1] / busy[roof_class][0] if roof_class else None
     if roof_class is not None:
         if anchor_fusion_on:
-            c = dict(c, sum_slices=4 if c["m"] >= 64 else 2 if c["m"] >= 8 else 1)
+            c = dict(c, sum_slices=worker_sum_slices(c["m"]))
+            if fused_weight_count(c) == 0 and opt.summed_floats > 0:
+                c["update_sum_slices"] = c["sum_slices"]     # the stand-alone update kernel sums
         ab = algorithmic_bytes(c, roof_class, P, n_sync / KP)
         achieved = ab / (avg_ms * 1e-3) / 1e9
         traffic = ncu_traffic(name, c["gemm_bf16"], roof_class, n_sync / KP)
@@ -491,8 +547,7 @@ def run_ours(args, rank, world):
                                                  (", worker sums" if anchor_fusion_on else ""))):
             launches_t, ms_t = ser_prof["wgrad_update"][tag]
             if launches_t > 0:
-                cc = dict(c, sum_slices=(4 if c["m"] >= 64 else 2 if c["m"] >= 8 else 1)
-                          if anchor_fusion_on else 0)
+                cc = dict(c, sum_slices=worker_sum_slices(c["m"]) if anchor_fusion_on else 0)
                 ab_t = algorithmic_bytes(cc, "wgrad_update", P, float(tag))
                 us_t = ms_t * 1e3 / launches_t
                 roofline["kernels"].append(dict(
@@ -551,7 +606,7 @@ def run_ours(args, rank, world):
                api="%s + olsgd_period_sync, pinned host minibatches (%s rows, int32 labels)"
                    % ("olsgd_local_step_host_bf16" if c["gemm_bf16"] else "olsgd_local_step_host",
                       "bf16" if c["gemm_bf16"] else "fp32"))
-    anchor_fusion = opt.anchor_fusion
+    anchor_fusion, summed_floats = anchor_fusion_on, opt.summed_floats
     opt.close()
     del opt, Xd, yd
     torch.cuda.empty_cache()
@@ -582,6 +637,7 @@ def run_ours(args, rank, world):
                        "alpha": c["alpha"], "beta": c["beta"], "mu": c["mu"],
                        "gemm_mode": c["gemm_bf16"], "method": args.method,
                        "anchor_fusion": bool(anchor_fusion),
+                       "worker_sum_formed_by_sync_step_launches_floats": int(summed_floats),
                        "tau_overridden": bool(args.tau),
                        "l2": "no flush: resident inputs+state %.0f MB exceed the %d MB L2"
                              % (resident / 1e6, L2_BYTES >> 20) if resident > L2_BYTES else

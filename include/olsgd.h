@@ -212,19 +212,24 @@ olsgd_status olsgd_local_step_with_grads(olsgd_ctx* ctx, const float* g_device);
  * OLSGD_ESTATE.                                                             */
 olsgd_status olsgd_period_sync(olsgd_ctx* ctx);
 
-/* Where the worker sum of Eq. 5 / Eq. 10-11 is formed.  With hidden layers on the tensor
- * cores (gemm_bf16 = 1, OLSGD_MODE_OVERLAP, all workers in this context) the sync step's
- * weight-gradient launch, which writes x_{k+1} anyway, also adds it up over the workers (a few
- * rows of partial sums in the workspace): x_{k+1} is not read a second time.
- * olsgd_period_sync then finishes the refresh on the side stream from those rows, and runs
- * the worker-mean kernel only on the rest of a parameter row (biases, output layer).  The
- * one-period lag stated after Eq. 5 is untouched: the anchor is written on the side stream
- * and first read by the next sync step.  on == 0 moves the whole sum back to the worker-mean
- * kernel; both ways give the same bits (same summation order).  Default: on where available.
- * Legal between periods (not while olsgd_period_sync is due); olsgd_anchor_fusion reports the
- * setting.                                                                               */
+/* Where the worker sum of Eq. 5 / Eq. 10-11 is formed.  In OLSGD_MODE_OVERLAP a sync step
+ * writes x_{k+1} anyway, so the launches that write it also add it up over this context's
+ * workers (a few rows of partial sums in the workspace) and x_{k+1} is not read a second
+ * time: the weight-gradient launch of hidden layers on the tensor cores (gemm_bf16 = 1), and
+ * the stand-alone update kernel on every range of a parameter row, of four workers or more,
+ * that is long enough to give every multiprocessor work with one thread per 16 bytes
+ * (OLSGD_FLAT rows, gemm_bf16 = 2, 3).
+ * olsgd_period_sync, or olsgd_period_sync_begin in a sharded run, then finishes on the side
+ * stream from those rows, and runs the worker-mean kernel only on the rest of a parameter
+ * row (biases, output layer, short rows).  The one-period lag stated after Eq. 5 is
+ * untouched: the anchor is written on the side stream and first read by the next sync step.
+ * on == 0 moves the whole sum back to the worker-mean kernel; both ways give the same bits
+ * (same summation order).  Default: on.  Legal between periods (not while olsgd_period_sync
+ * is due); olsgd_anchor_fusion reports the setting, olsgd_summed_floats how many parameters
+ * of a row the most recent anchor refresh took from such partial sums (0: none).          */
 olsgd_status olsgd_set_anchor_fusion(olsgd_ctx* ctx, int32_t on);
 int32_t olsgd_anchor_fusion(const olsgd_ctx* ctx);
+int64_t olsgd_summed_floats(const olsgd_ctx* ctx);
 
 /* The anchor refresh split in two for a worker dimension that is sharded over several
  * contexts: the only exchange of the method is the sum in Eq. 5.

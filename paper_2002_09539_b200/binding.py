@@ -73,6 +73,7 @@ def load_library():
         "olsgd_period_sync": (i32, [vp]),
         "olsgd_set_anchor_fusion": (i32, [vp, i32]),
         "olsgd_anchor_fusion": (i32, [vp]),
+        "olsgd_summed_floats": (i64, [vp]),
         "olsgd_period_sync_begin": (i32, [vp, vp]),
         "olsgd_period_sync_finish": (i32, [vp, vp]),
         "olsgd_row_floats": (i64, [vp]),
@@ -235,6 +236,12 @@ class OverlapLocalSGD:
     @property
     def anchor_fusion(self):
         return bool(self.lib.olsgd_anchor_fusion(self.ctx))
+
+    @property
+    def summed_floats(self):
+        """Parameters of a row that the most recent anchor refresh took from partial sums
+        formed by the sync step's own launches."""
+        return int(self.lib.olsgd_summed_floats(self.ctx))
 
     def period_sync_begin(self, partial_sum):
         assert partial_sum.is_cuda and partial_sum.dtype == torch.float32

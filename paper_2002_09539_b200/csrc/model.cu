@@ -112,18 +112,6 @@ bool plan_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, ModelPlan
     mp->off_da[l] = take(m * B * w * e);
     mp->off_dat[l] = take(m * B * w * e);
   }
-  // scratch of the worker sum that the sync-step weight-gradient launch forms (Overlap mode,
-  // all workers in this context, at least one layer whose update is fused)
-  if (spec.gemm_bf16 == 1 && hp.mode == OLSGD_MODE_OVERLAP && (hp.m_total == 0 || hp.m_total == hp.m)) {
-    bool any = false;
-    for (int p = 0; p < L - 1; ++p) any = any || layer_update_is_fused(spec, hp, p);
-    if (any) {
-      size_t P = 0;
-      for (int l = 0; l < L; ++l) P += (size_t)spec.dims[l + 1] * spec.dims[l] + spec.dims[l + 1];
-      mp->off_sum_part = take((size_t)worker_sum_slices(hp.m) * align_up(P, 64) * sizeof(float));
-      mp->has_sum_part = true;
-    }
-  }
   mp->bytes = off;
   return true;
 }
@@ -206,28 +194,14 @@ bool bind_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, const Mod
     }
   }
   close_range(P);
-  // the worker sum inside the sync-step launch covers the fused layers' weight matrices; what
-  // is left for the worker-mean kernel are the ranges between them (biases, output layer)
-  if (mp.has_sum_part) {
-    mb->sum_part = reinterpret_cast<float*>(base + mp.off_sum_part);
-    int64_t from = 0;
-    mb->n_anchor_ranges = mb->n_summed = 0;
-    auto close_anchor = [&](int64_t end) {
-      if (end > from) {
-        mb->anchor_off[mb->n_anchor_ranges] = from;
-        mb->anchor_len[mb->n_anchor_ranges] = end - from;
-        mb->n_anchor_ranges++;
-      }
-    };
-    for (int p = 0; p < L - 1; ++p) {
-      if (!mb->fused_layer[p]) continue;
-      mb->summed_off[mb->n_summed] = mb->w_off[p];
-      mb->summed_len[mb->n_summed] = mb->b_off[p] - mb->w_off[p];
-      mb->n_summed++;
-      close_anchor(mb->w_off[p]);
-      from = mb->b_off[p];
-    }
-    close_anchor(P);
+  // the ranges of a row whose worker sums the sync-step weight-gradient launch can form: the
+  // fused layers' weight matrices
+  mb->n_summed = 0;
+  for (int p = 0; p < L - 1; ++p) {
+    if (!mb->fused_layer[p]) continue;
+    mb->summed_off[mb->n_summed] = mb->w_off[p];
+    mb->summed_len[mb->n_summed] = mb->b_off[p] - mb->w_off[p];
+    mb->n_summed++;
   }
   return true;
 }

@@ -1,11 +1,13 @@
 // C ABI of libolsgd: context, argument checks, workspace carving, stream and
 // event choreography of one Overlap-Local-SGD period.  No arithmetic of the
 // method happens on the host; every step is a kernel launch.
+#include <algorithm>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
 #include <new>
 #include <string>
+#include <utility>
 #include <vector>
 
 #include "olsgd_internal.h"
@@ -70,8 +72,15 @@ struct olsgd_ctx {
   int host_slot = 0;
   bool reduce_pending = false;  // an anchor refresh was launched and not yet waited for
   int reduce_reads = -1;        // which x buffer that refresh reads
-  bool anchor_fusion = false;   // sync steps form the worker sum inside the weight-gradient launch
-  bool last_sync_summed = false;  // ... and the sync step that closed this period did
+  // Sync steps form the worker sum inside the launches that write x_{k+1} (the fused
+  // weight-gradient launch, the stand-alone update kernel on long ranges): sum_part is the
+  // [S][ld] scratch of partial sums, `summed` the ranges (offset, length) of a row that the
+  // sync step which closed this period covered that way; the anchor refresh takes those from
+  // the partial sums and the rest of the row from the worker models.
+  bool anchor_fusion = false;
+  float* sum_part = nullptr;
+  std::vector<std::pair<int64_t, int64_t>> summed;
+  int64_t last_summed = 0;   // parameters per row the most recent refresh took from sum_part
   bool need_sync = false;       // a period ended; olsgd_period_sync is due
   bool sync_begun = false;      // olsgd_period_sync_begin ran; _finish is due
 
@@ -228,9 +237,9 @@ struct Plan {
   int64_t P = 0, ld = 0;
   size_t off_x0 = 0, off_x1 = 0, off_u = 0, off_g = 0, off_z = 0, off_v = 0, off_tmp = 0,
          off_shadow = 0, off_idx = 0, off_idx_next = 0, off_ident = 0, off_status = 0, off_dev_k = 0,
-         off_loss_ring = 0, off_stage_x[2] = {0, 0},
+         off_loss_ring = 0, off_sum_part = 0, off_stage_x[2] = {0, 0},
          off_stage_y[2] = {0, 0}, off_model = 0, total = 0;
-  bool has_u = false, has_g = false, has_shadow = false;
+  bool has_u = false, has_g = false, has_shadow = false, has_sum_part = false;
   ModelPlan mp;
 };
 
@@ -322,6 +331,9 @@ olsgd_status make_plan(const olsgd_model_spec* spec, const olsgd_hparams* hp, Pl
     pl->off_loss_ring = take((size_t)(base > kMaxGraphBlock ? base : kMaxGraphBlock) * m * sizeof(float));
   }
   pl->off_shadow = pl->has_shadow ? take((size_t)pl->ld * m * sizeof(__nv_bfloat16)) : 0;
+  // partial worker sums of the sync steps (Eq. 5's sum formed where x_{k+1} is written)
+  pl->has_sum_part = hp->mode == OLSGD_MODE_OVERLAP && m >= 2;
+  pl->off_sum_part = pl->has_sum_part ? take((size_t)worker_sum_slices(hp->m) * row) : 0;
   pl->off_idx = pl->has_g ? take((size_t)m * hp->batch * sizeof(int32_t)) : 0;
   pl->off_idx_next = pl->has_g ? take((size_t)m * hp->batch * sizeof(int32_t)) : 0;
   if (pl->has_g) {
@@ -380,14 +392,20 @@ olsgd_status apply_update(olsgd_ctx* c, const float* g, int64_t ldg) {
   const int n_ranges = model ? c->mb.n_ranges : 1;
   for (int r = 0; r < n_ranges; ++r) {
     const int64_t off = model ? c->mb.range_off[r] : 0;
+    const int64_t len = model ? c->mb.range_len[r] : c->P;
     UpdateArgs a;
+    if (sync && c->anchor_fusion && update_sums_workers(len, c->hp.m)) {
+      a.sum_part = c->sum_part + off;
+      a.sum_slices = worker_sum_slices(c->hp.m);
+      c->summed.emplace_back(off, len);
+    }
     a.x_in = c->x[c->cur] + off;
     a.x_out = c->x[nxt] + off;
     a.g = g + off;
     a.u = c->u ? c->u + off : nullptr;
     a.z = c->z + off;
     a.shadow = c->shadow ? c->shadow + off : nullptr;
-    a.P = model ? c->mb.range_len[r] : c->P;
+    a.P = len;
     a.ld = c->ld;
     a.ldg = ldg;
     a.m = c->hp.m;
@@ -395,7 +413,8 @@ olsgd_status apply_update(olsgd_ctx* c, const float* g, int64_t ldg) {
     a.mu = c->hp.mu;
     a.alpha = c->hp.alpha;
     a.sync = sync;
-    Launch l(c, OLSGD_KC_UPDATE, c->main);
+    // tagged 1 on sync steps (Eq. 4 applied too, and the worker sum where the range is long)
+    Launch l(c, OLSGD_KC_UPDATE | ((sync ? 1 : 0) << 8), c->main);
     OLSGD_CUDA(c, launch_fused_update(a, c->main));
   }
   if (period_end && local_sgd) {
@@ -466,15 +485,13 @@ olsgd_status step_body(olsgd_ctx* c, const olsgd_data& data, int32_t* idx,
     io.upd.mu = c->hp.mu;
     io.upd.alpha = c->hp.alpha;
     io.upd.sync = sync ? 1 : 0;
-    if (sync) {
+    if (sync && c->anchor_fusion && c->mb.n_summed > 0) {
       // the worker sums of the weight matrices whose update is fused are formed by the same
-      // launch; olsgd_period_sync finishes Eq. 5 / Eq. 10-11 from them
-      const bool summed = c->anchor_fusion && c->mb.sum_part != nullptr;
-      c->last_sync_summed = summed;
-      if (summed) {
-        io.upd.sum_part = c->mb.sum_part;
-        io.upd.sum_slices = worker_sum_slices(c->hp.m);
-      }
+      // launch; the anchor refresh finishes Eq. 5 / Eq. 10-11 from them
+      io.upd.sum_part = c->sum_part;
+      io.upd.sum_slices = worker_sum_slices(c->hp.m);
+      for (int r = 0; r < c->mb.n_summed; ++r)
+        c->summed.emplace_back(c->mb.summed_off[r], c->mb.summed_len[r]);
     }
     // same rule as in apply_update, applied before the first kernel that writes x[nxt]
     if (c->reduce_pending && (sync || c->reduce_reads == nxt)) {
@@ -605,6 +622,8 @@ olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const ols
   c->loss_ring = reinterpret_cast<float*>(ws + pl.off_loss_ring);
   c->graph_block = graph_block_len(hp->tau);
   c->shadow = pl.has_shadow ? reinterpret_cast<__nv_bfloat16*>(ws + pl.off_shadow) : nullptr;
+  c->sum_part = pl.has_sum_part ? reinterpret_cast<float*>(ws + pl.off_sum_part) : nullptr;
+  c->anchor_fusion = c->sum_part != nullptr;
   c->idx = pl.has_g ? reinterpret_cast<int32_t*>(ws + pl.off_idx) : nullptr;
   c->idx_next = pl.has_g ? reinterpret_cast<int32_t*>(ws + pl.off_idx_next) : nullptr;
   if (pl.has_g) {
@@ -669,7 +688,6 @@ olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const ols
       Launch l(c, OLSGD_KC_OTHER, c->main);
       OLSGD_INIT_CUDA(launch_cast_bf16(c->x[0], c->shadow, (int64_t)c->hp.m * c->ld, c->main));
     }
-    c->anchor_fusion = c->mb.sum_part != nullptr;
   }
   OLSGD_INIT_CUDA(cudaStreamSynchronize(c->main));
 #undef OLSGD_INIT_CUDA
@@ -851,52 +869,62 @@ olsgd_status olsgd_join(olsgd_ctx* c) {
   return check_device_status(c);
 }
 
+// S7 on the side stream for one row.  The ranges whose worker sums the sync step left in
+// sum_part are finished from those S rows; what lies between them (biases, output layer, or
+// the whole row when nothing was summed) goes through the worker-mean kernel.  With `partial`
+// non-null both only write this context's undivided column sums there (sharded sync).
+static olsgd_status launch_anchor_refresh(olsgd_ctx* c, float* partial) {
+  std::sort(c->summed.begin(), c->summed.end());
+  c->last_summed = 0;
+  // the long ranges first: the next sync step's launches wait for all of this anyway, and
+  // the short kernels then run in the shadow of the next period's first GEMMs
+  for (const auto& r : c->summed) {
+    // tagged 1: the refresh from partial sums (0: the worker-mean kernel)
+    Launch l(c, OLSGD_KC_ANCHOR | (1 << 8), c->side);
+    OLSGD_CUDA(c, launch_anchor_from_slices(c->sum_part + r.first, worker_sum_slices(c->hp.m),
+                                            c->ld, c->z + r.first, c->v + r.first, r.second,
+                                            c->hp.beta, c->hp.m,
+                                            partial ? partial + r.first : nullptr, c->side));
+    c->last_summed += r.second;
+  }
+  int64_t from = 0;
+  auto rest = [&](int64_t end) -> cudaError_t {
+    if (end <= from) return cudaSuccess;
+    AnchorArgs a;
+    a.x = c->x[c->cur] + from;
+    a.z = c->z + from;
+    a.v = c->v + from;
+    a.P = end - from;
+    a.ld = c->ld;
+    a.m = c->hp.m;
+    a.beta = c->hp.beta;
+    a.partial = partial ? partial + from : nullptr;
+    Launch l(c, OLSGD_KC_ANCHOR, c->side);
+    return launch_worker_mean_anchor(a, c->side);
+  };
+  for (const auto& r : c->summed) {
+    OLSGD_CUDA(c, rest(r.first));
+    from = r.first + r.second;
+  }
+  OLSGD_CUDA(c, rest(c->P));
+  c->summed.clear();
+  return OLSGD_OK;
+}
+
 olsgd_status olsgd_period_sync(olsgd_ctx* c) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
   OLSGD_ON_DEVICE(c);
   if (!c->need_sync || c->sync_begun)
     return fail(c, OLSGD_ESTATE, "olsgd_period_sync is legal once, right after a period ends (k=%lld, tau=%d)",
                 (long long)c->k, c->hp.tau);
-  // S7 on the side stream, ordered after the pull-back that closed the period
-  OLSGD_CUDA(c, cudaEventRecord(c->pullback_done, c->main));
-  OLSGD_CUDA(c, cudaStreamWaitEvent(c->side, c->pullback_done, 0));
-  AnchorArgs a;
-  a.x = c->x[c->cur];
-  a.z = c->z;
-  a.v = c->v;
-  a.P = c->P;
-  a.ld = c->ld;
-  a.m = c->hp.m;
-  a.beta = c->hp.beta;
-  a.partial = nullptr;
   if (c->hp.m_total != 0 && c->hp.m_total != c->hp.m)
     return fail(c, OLSGD_ESTATE, "this context holds a shard of the workers: use "
                                  "olsgd_period_sync_begin / olsgd_period_sync_finish");
-  if (c->last_sync_summed) {
-    // the weight matrices were summed over the workers by the sync step's own weight-gradient
-    // launch: their anchor only needs the S rows of partial sums, not the m worker models;
-    // the rest of the row (biases, output layer) goes through the worker-mean kernel
-    for (int r = 0; r < c->mb.n_summed; ++r) {
-      const int64_t off = c->mb.summed_off[r];
-      Launch l(c, OLSGD_KC_ANCHOR, c->side);
-      OLSGD_CUDA(c, launch_anchor_from_slices(c->mb.sum_part + off, worker_sum_slices(c->hp.m), c->ld,
-                                              c->z + off, c->v + off, c->mb.summed_len[r],
-                                              c->hp.beta, c->hp.m, c->side));
-    }
-    for (int r = 0; r < c->mb.n_anchor_ranges; ++r) {
-      AnchorArgs b = a;
-      const int64_t off = c->mb.anchor_off[r];
-      b.x = a.x + off;
-      b.z = a.z + off;
-      b.v = a.v + off;
-      b.P = c->mb.anchor_len[r];
-      Launch l(c, OLSGD_KC_ANCHOR, c->side);
-      OLSGD_CUDA(c, launch_worker_mean_anchor(b, c->side));
-    }
-  } else {
-    Launch l(c, OLSGD_KC_ANCHOR, c->side);
-    OLSGD_CUDA(c, launch_worker_mean_anchor(a, c->side));
-  }
+  // S7 on the side stream, ordered after the pull-back that closed the period
+  OLSGD_CUDA(c, cudaEventRecord(c->pullback_done, c->main));
+  OLSGD_CUDA(c, cudaStreamWaitEvent(c->side, c->pullback_done, 0));
+  const olsgd_status st = launch_anchor_refresh(c, nullptr);
+  if (st != OLSGD_OK) return st;
   OLSGD_CUDA(c, cudaEventRecord(c->reduce_done, c->side));
   c->reduce_pending = true;
   c->reduce_reads = c->cur;
@@ -908,7 +936,7 @@ olsgd_status olsgd_set_anchor_fusion(olsgd_ctx* c, int32_t on) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
   if (c->need_sync || c->sync_begun)
     return fail(c, OLSGD_ESTATE, "a period ended: call olsgd_period_sync first");
-  const bool want = on != 0 && c->mb.sum_part != nullptr;
+  const bool want = on != 0 && c->sum_part != nullptr;
   if (want != c->anchor_fusion) {
     c->anchor_fusion = want;
     // a captured block carries the old choice
@@ -921,6 +949,7 @@ olsgd_status olsgd_set_anchor_fusion(olsgd_ctx* c, int32_t on) {
 }
 
 int32_t olsgd_anchor_fusion(const olsgd_ctx* c) { return c && c->anchor_fusion ? 1 : 0; }
+int64_t olsgd_summed_floats(const olsgd_ctx* c) { return c ? c->last_summed : -1; }
 
 olsgd_status olsgd_period_sync_begin(olsgd_ctx* c, float* partial_sum_device) {
   if (!c) return fail(nullptr, OLSGD_EINVAL, "ctx is NULL");
@@ -931,19 +960,8 @@ olsgd_status olsgd_period_sync_begin(olsgd_ctx* c, float* partial_sum_device) {
     return fail(c, OLSGD_ESTATE, "olsgd_period_sync_begin is legal once, right after a period ends");
   OLSGD_CUDA(c, cudaEventRecord(c->pullback_done, c->main));
   OLSGD_CUDA(c, cudaStreamWaitEvent(c->side, c->pullback_done, 0));
-  AnchorArgs a;
-  a.x = c->x[c->cur];
-  a.z = c->z;
-  a.v = c->v;
-  a.P = c->P;
-  a.ld = c->ld;
-  a.m = c->hp.m;
-  a.beta = c->hp.beta;
-  a.partial = partial_sum_device;
-  {
-    Launch l(c, OLSGD_KC_ANCHOR, c->side);
-    OLSGD_CUDA(c, launch_worker_mean_anchor(a, c->side));
-  }
+  const olsgd_status st = launch_anchor_refresh(c, partial_sum_device);
+  if (st != OLSGD_OK) return st;
   // from here on the worker models are no longer read by the refresh, but z is not ready:
   // the main stream must still wait for reduce_done (recorded by _finish) before it reads z
   c->sync_begun = true;

@@ -98,8 +98,17 @@ struct UpdateArgs {
   int m;
   float gamma, mu, alpha;
   bool sync;
+  // sync steps only, sum_slices > 0: the launch also adds up x_{k+1} over the workers in the
+  // order of the worker-mean kernel and leaves slice s's column sums in row s of sum_part
+  // (row pitch ld); launch_anchor_from_slices finishes the anchor refresh from there.
+  float* sum_part = nullptr;
+  int sum_slices = 0;
 };
 cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t s);
+// Whether a sync-step update launch over P parameters of m workers should form the worker
+// sums itself: only when its one-thread-per-column-strip grid of worker_sum_slices(m) rows
+// still fills the GPU (the choice changes the launches, never the bits).
+bool update_sums_workers(int64_t P, int m);
 
 // Eq. 5 (beta == 0) or Eq. 10-11: worker mean in a fixed order, then z (and v).
 struct AnchorArgs {
@@ -121,9 +130,10 @@ cudaError_t launch_anchor_from_sum(const float* sum, float* z, float* v, int64_t
                                    int m_total, cudaStream_t s);
 // Eq. 5 / Eq. 10-11 for P entries from `slices` rows of partial worker sums (row pitch ld):
 // the rows are added in slice order, which completes the summation order of the worker-mean
-// kernel, then divided by m.
+// kernel, then divided by m.  With `partial` non-null only the undivided totals are written,
+// there, and z, v are left alone (sharded sync, as in AnchorArgs).
 cudaError_t launch_anchor_from_slices(const float* part, int slices, int64_t ld, float* z, float* v,
-                                      int64_t P, float beta, int m, cudaStream_t s);
+                                      int64_t P, float beta, int m, float* partial, cudaStream_t s);
 
 // Eq. 2 on a sync step: every worker row of x (and of its bf16 shadow, if any) and z are
 // replaced by the worker mean, summed in worker order.
@@ -327,8 +337,6 @@ struct ModelPlan {
   size_t off_h[OLSGD_MAX_DIMS] = {0}, off_ht[OLSGD_MAX_DIMS] = {0};    // hidden activations
   size_t off_da[OLSGD_MAX_DIMS] = {0}, off_dat[OLSGD_MAX_DIMS] = {0};  // their gradients
   // worker sum inside the sync-step weight-gradient launch: partial sums [slices][ld]
-  bool has_sum_part = false;
-  size_t off_sum_part = 0;
 };
 struct ModelBuffers {
   char error[160] = {0};
@@ -351,14 +359,10 @@ struct ModelBuffers {
   // what is left for the stand-alone update kernel: ranges [off, off + len) of a worker row
   int n_ranges = 0;
   int64_t range_off[OLSGD_MAX_DIMS + 1] = {0}, range_len[OLSGD_MAX_DIMS + 1] = {0};
-  // Worker sum inside the sync-step weight-gradient launch (fused layers' weight matrices):
-  // the scratch matrix, the ranges of a row it covers, and the ranges that are left for the
-  // worker-mean kernel (biases, output layer).
-  float* sum_part = nullptr;
+  // Worker sum inside the sync-step weight-gradient launch: the ranges of a row it covers
+  // (the fused layers' weight matrices).
   int n_summed = 0;
   int64_t summed_off[OLSGD_MAX_DIMS] = {0}, summed_len[OLSGD_MAX_DIMS] = {0};
-  int n_anchor_ranges = 0;
-  int64_t anchor_off[OLSGD_MAX_DIMS + 1] = {0}, anchor_len[OLSGD_MAX_DIMS + 1] = {0};
 };
 struct StepIO {
   const float* x;                // x_k, [m][ld]

@@ -30,27 +30,33 @@ __device__ __forceinline__ float4 load_g(const float* g_row, int64_t col4, int64
 
 // One thread owns a 16-byte column strip and walks over `wpt` workers, so the
 // anchor strip is read once per thread on sync steps.
-template <bool MOM, bool SYNC, bool SHADOW>
+// SUM (sync steps): blockIdx.y is a slice of the worker sum instead; the thread walks over
+// the workers s, s + S, s + 2S, ... (S = gridDim.y), adds up the x_{k+1} it writes in that
+// order, starting from zero as the worker-mean kernel does, and stores its column sums in
+// row s of `part`.
+template <bool MOM, bool SYNC, bool SHADOW, bool SUM>
 __global__ void __launch_bounds__(kUpdateThreads)
 fused_update_kernel(const float* __restrict__ x_in, float* __restrict__ x_out,
                     const float* __restrict__ g, float* __restrict__ u,
-                    const float* __restrict__ z, __nv_bfloat16* __restrict__ shadow, int64_t P,
-                    int64_t n4, int64_t ld, int64_t ldg, int m, int wpt, bool gvec, float gamma,
-                    float mu, float alpha) {
+                    const float* __restrict__ z, __nv_bfloat16* __restrict__ shadow,
+                    float* __restrict__ part, int64_t P, int64_t n4, int64_t ld, int64_t ldg,
+                    int m, int wpt, bool gvec, float gamma, float mu, float alpha) {
   launch_gate();
   const int64_t col4 = (int64_t)blockIdx.x * kUpdateThreads + threadIdx.x;
   if (col4 >= n4) return;
-  const int i0 = blockIdx.y * wpt;
-  const int i1 = min(m, i0 + wpt);
+  const int stride = SUM ? (int)gridDim.y : 1;
+  const int i0 = SUM ? (int)blockIdx.y : (int)blockIdx.y * wpt;
+  const int i1 = SUM ? m : min(m, i0 + wpt);
 
   float4 zz = make_float4(0.f, 0.f, 0.f, 0.f);
   if (SYNC) zz = reinterpret_cast<const float4*>(z)[col4];
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 
-  for (int ib = i0; ib < i1; ib += kUnroll) {
+  for (int ib = i0; ib < i1; ib += kUnroll * stride) {
     float4 xv[kUnroll], gv[kUnroll], uv[kUnroll];
 #pragma unroll
     for (int t = 0; t < kUnroll; ++t) {
-      const int i = ib + t;
+      const int i = ib + t * stride;
       if (i < i1) {
         xv[t] = reinterpret_cast<const float4*>(x_in + (int64_t)i * ld)[col4];
         gv[t] = load_g(g + (int64_t)i * ldg, col4, P, gvec);
@@ -59,7 +65,7 @@ fused_update_kernel(const float* __restrict__ x_in, float* __restrict__ x_out,
     }
 #pragma unroll
     for (int t = 0; t < kUnroll; ++t) {
-      const int i = ib + t;
+      const int i = ib + t * stride;
       if (i < i1) {
         float4 x = xv[t];
         float4 uu = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -68,9 +74,16 @@ fused_update_kernel(const float* __restrict__ x_in, float* __restrict__ x_out,
         if (MOM) reinterpret_cast<float4*>(u + (int64_t)i * ld)[col4] = uu;
         reinterpret_cast<float4*>(x_out + (int64_t)i * ld)[col4] = x;
         if (SHADOW) reinterpret_cast<uint2*>(shadow + (int64_t)i * ld)[col4] = pack_bf16x4(x);
+        if (SUM) {
+          acc.x += x.x;
+          acc.y += x.y;
+          acc.z += x.z;
+          acc.w += x.w;
+        }
       }
     }
   }
+  if (SUM) __stcs(reinterpret_cast<float4*>(part + (int64_t)blockIdx.y * ld) + col4, acc);
 }
 
 constexpr int kMeanThreads = 256;
@@ -235,12 +248,12 @@ anchor_from_sum_kernel(const float* __restrict__ sum, float* __restrict__ z, flo
 template <bool MOM>
 __global__ void __launch_bounds__(kUpdateThreads)
 anchor_from_slices_kernel(const float* __restrict__ part, int slices, int64_t ld,
-                          float* __restrict__ z, float* __restrict__ v, int64_t n4, float beta,
-                          float m_f) {
+                          float* __restrict__ z, float* __restrict__ v,
+                          float* __restrict__ partial, int64_t n4, float beta, float m_f) {
   const int64_t col4 = (int64_t)blockIdx.x * kUpdateThreads + threadIdx.x;
   if (col4 >= n4) return;
   float4 zz = make_float4(0.f, 0.f, 0.f, 0.f), vv = zz;
-  if (MOM) {
+  if (MOM && !partial) {
     zz = reinterpret_cast<const float4*>(z)[col4];
     vv = reinterpret_cast<const float4*>(v)[col4];
   }
@@ -251,6 +264,10 @@ anchor_from_slices_kernel(const float* __restrict__ part, int slices, int64_t ld
     s.y += p.y;
     s.z += p.z;
     s.w += p.w;
+  }
+  if (partial) {
+    reinterpret_cast<float4*>(partial)[col4] = s;
+    return;
   }
   s.x /= m_f;
   s.y /= m_f;
@@ -313,33 +330,60 @@ __global__ void virtual_sequence_kernel(const float* __restrict__ x, const float
 
 }  // namespace
 
+// blocks that give the update kernel a few waves over the multiprocessors
+static int64_t update_target_blocks() { return (int64_t)sm_count() * 16; }
+
+bool update_sums_workers(int64_t P, int m) {
+  // The grid of a summing launch has one row of blocks per slice, so it needs a row long
+  // enough to give every multiprocessor a couple of blocks; with fewer than four workers
+  // the worker-mean kernel has next to nothing to re-read.  (Measured from 250k x 64 to
+  // 50M x 64 parameters x workers: the iteration is 1-5 % shorter wherever this holds.)
+  const int64_t n4 = (P + 3) / 4;
+  const int64_t gx = (n4 + kUpdateThreads - 1) / kUpdateThreads;
+  return m >= 4 && gx * worker_sum_slices(m) >= (int64_t)sm_count() * 2;
+}
+
 cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t s) {
   const int64_t n4 = (a.P + 3) / 4;
   const int64_t gx = (n4 + kUpdateThreads - 1) / kUpdateThreads;
   // enough blocks for a few waves over the multiprocessors; the rest of the worker
   // dimension is walked inside the thread so the anchor strip is reused
-  const int64_t target_blocks = (int64_t)sm_count() * 16;
+  const int64_t target_blocks = update_target_blocks();
   int gy = (int)((target_blocks + gx - 1) / gx);
   if (gy < 1) gy = 1;
   if (gy > a.m) gy = a.m;
-  const int wpt = (a.m + gy - 1) / gy;
+  int wpt = (a.m + gy - 1) / gy;
   gy = (a.m + wpt - 1) / wpt;
+  const bool sum = a.sync && a.sum_slices > 0;
+  if (sum) {
+    if (a.sum_slices != worker_sum_slices(a.m) || !a.sum_part) return cudaErrorInvalidValue;
+    gy = a.sum_slices;
+    wpt = 0;
+  }
   const bool gvec = (a.ldg % 4 == 0) && ((reinterpret_cast<uintptr_t>(a.g) & 15) == 0);
   const bool mom = a.u != nullptr && a.mu != 0.f;
   const bool shadow = a.shadow != nullptr;
   dim3 grid((unsigned)gx, (unsigned)gy), block(kUpdateThreads);
   cudaError_t err = cudaSuccess;
-#define OLSGD_LAUNCH_UPD(MOM, SYNC, SH)                                                          \
-  err = launch_chained(fused_update_kernel<MOM, SYNC, SH>, grid, block, 0, s, a.x_in, a.x_out,   \
-                       a.g, a.u, a.z, a.shadow, a.P, n4, a.ld, a.ldg, a.m, wpt, gvec, a.gamma,   \
-                       a.mu, a.alpha)
+#define OLSGD_LAUNCH_UPD(MOM, SYNC, SH, SUM)                                                     \
+  err = launch_chained(fused_update_kernel<MOM, SYNC, SH, SUM>, grid, block, 0, s, a.x_in,       \
+                       a.x_out, a.g, a.u, a.z, a.shadow, a.sum_part, a.P, n4, a.ld, a.ldg, a.m,  \
+                       wpt, gvec, a.gamma, a.mu, a.alpha)
+#define OLSGD_LAUNCH_UPD_SH(MOM, SYNC, SUM)                                                      \
+  do {                                                                                           \
+    if (shadow) OLSGD_LAUNCH_UPD(MOM, SYNC, true, SUM);                                          \
+    else OLSGD_LAUNCH_UPD(MOM, SYNC, false, SUM);                                                \
+  } while (0)
   if (mom) {
-    if (a.sync) { if (shadow) OLSGD_LAUNCH_UPD(true, true, true); else OLSGD_LAUNCH_UPD(true, true, false); }
-    else        { if (shadow) OLSGD_LAUNCH_UPD(true, false, true); else OLSGD_LAUNCH_UPD(true, false, false); }
+    if (sum) OLSGD_LAUNCH_UPD_SH(true, true, true);
+    else if (a.sync) OLSGD_LAUNCH_UPD_SH(true, true, false);
+    else OLSGD_LAUNCH_UPD_SH(true, false, false);
   } else {
-    if (a.sync) { if (shadow) OLSGD_LAUNCH_UPD(false, true, true); else OLSGD_LAUNCH_UPD(false, true, false); }
-    else        { if (shadow) OLSGD_LAUNCH_UPD(false, false, true); else OLSGD_LAUNCH_UPD(false, false, false); }
+    if (sum) OLSGD_LAUNCH_UPD_SH(false, true, true);
+    else if (a.sync) OLSGD_LAUNCH_UPD_SH(false, true, false);
+    else OLSGD_LAUNCH_UPD_SH(false, false, false);
   }
+#undef OLSGD_LAUNCH_UPD_SH
 #undef OLSGD_LAUNCH_UPD
   return err;
 }
@@ -392,13 +436,14 @@ cudaError_t launch_anchor_from_sum(const float* sum, float* z, float* v, int64_t
 }
 
 cudaError_t launch_anchor_from_slices(const float* part, int slices, int64_t ld, float* z, float* v,
-                                      int64_t P, float beta, int m, cudaStream_t s) {
+                                      int64_t P, float beta, int m, float* partial,
+                                      cudaStream_t s) {
   const int64_t n4 = (P + 3) / 4;
   const unsigned grid = (unsigned)((n4 + kUpdateThreads - 1) / kUpdateThreads);
   if (beta != 0.f)
-    anchor_from_slices_kernel<true><<<grid, kUpdateThreads, 0, s>>>(part, slices, ld, z, v, n4, beta, (float)m);
+    anchor_from_slices_kernel<true><<<grid, kUpdateThreads, 0, s>>>(part, slices, ld, z, v, partial, n4, beta, (float)m);
   else
-    anchor_from_slices_kernel<false><<<grid, kUpdateThreads, 0, s>>>(part, slices, ld, z, v, n4, beta, (float)m);
+    anchor_from_slices_kernel<false><<<grid, kUpdateThreads, 0, s>>>(part, slices, ld, z, v, partial, n4, beta, (float)m);
   return cudaGetLastError();
 }
 

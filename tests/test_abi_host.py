@@ -80,8 +80,13 @@ def test_workspace_size_counts_the_resident_state(lib):
     s = binding._spec("flat", flat_P=1_000_000)
     hp = _hp(m=8, mu=0.9, beta=0.9)
     assert lib.olsgd_workspace_bytes(C.byref(s), C.byref(hp), C.byref(n)) == 0
-    # two x buffers + u, each [8][1M] fp32, plus z, v and one scratch row
-    assert 3 * 8 * 4_000_000 + 3 * 4_000_000 <= n.value <= 3 * 8 * 4_000_000 + 3 * 4_000_000 + 65536
+    # two x buffers + u, each [8][1M] fp32, plus z, v, one scratch row and the two rows of
+    # partial worker sums that eight workers are added up in
+    want = 3 * 8 * 4_000_000 + 5 * 4_000_000
+    assert want <= n.value <= want + 65536
+    hp_local = _hp(m=8, mu=0.9, beta=0.9, mode=1)   # Local SGD (Eq. 2): no anchor refresh to feed
+    assert lib.olsgd_workspace_bytes(C.byref(s), C.byref(hp_local), C.byref(n)) == 0
+    assert want - 2 * 4_000_000 <= n.value <= want - 2 * 4_000_000 + 65536
 
 
 def test_init_rejects_null_and_small_workspace_without_touching_the_device(lib):

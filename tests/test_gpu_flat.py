@@ -49,6 +49,47 @@ def test_flat_parity(P, m, tau, beta, mu):
     assert max_rel_err([xbar], [st.mean_model()]) <= TOL
 
 
+def _run_bits(P, m, tau, beta, mu, iters, fusion, grads, x0):
+    from paper_2002_09539_b200 import OverlapLocalSGD
+    opt = OverlapLocalSGD("flat", m=m, tau=tau, gamma=0.05, alpha=0.5, beta=beta, mu=mu, flat_P=P, x0=x0)
+    opt.set_anchor_fusion(fusion)
+    for k in range(iters):
+        opt.local_step_with_grads(grads[k])
+        if (k + 1) % tau == 0:
+            opt.period_sync()
+    return opt
+
+
+# rows long enough that the sync step's update launch forms the worker sums itself (one
+# thread per 16 bytes and slice must give every multiprocessor work): S = 1, 2, 2 and 4
+# slices, ragged tails and ragged slices
+@pytest.mark.parametrize("beta,mu", [(0.0, 0.0), (0.9, 0.9)])
+@pytest.mark.parametrize("P,m,tau", [(2_500_003, 5, 2), (1_300_003, 16, 4), (300_001, 37, 1),
+                                     (700_002, 64, 2)])
+def test_update_kernel_forms_the_worker_sum_on_long_rows(P, m, tau, beta, mu):
+    iters = 2 * tau + 1
+    x0 = si.flat_init(3, P)
+    host = [si.flat_grads(3, k, m, P, 0.1) for k in range(iters)]
+    grads = [to_dev(g) for g in host]
+    on = _run_bits(P, m, tau, beta, mu, iters, True, grads, x0)
+    off = _run_bits(P, m, tau, beta, mu, iters, False, grads, x0)
+    assert on.anchor_fusion and not off.anchor_fusion
+    assert on.summed_floats == P and off.summed_floats == 0
+    for a, b in zip(on.state(), off.state()):
+        assert np.array_equal(a, b)                      # same summation order, same bits
+    st = runner.run_flat(x0, host, m=m, tau=tau, gamma=0.05, alpha=0.5, beta=beta, mu=mu)
+    assert state_err(on, st) <= TOL
+
+
+@pytest.mark.parametrize("P,m", [(50021, 16), (2_000_001, 3)])
+def test_short_rows_and_few_workers_leave_the_worker_sum_to_the_anchor_kernel(P, m):
+    tau = 2
+    x0 = si.flat_init(4, P)
+    grads = [to_dev(si.flat_grads(4, k, m, P, 0.1)) for k in range(tau)]
+    opt = _run_bits(P, m, tau, 0.9, 0.9, tau, True, grads, x0)
+    assert opt.anchor_fusion and opt.summed_floats == 0
+
+
 def test_hundred_iterations_stay_within_tolerance():
     opt, st = _run_pair(50021, 16, 4, 0.05, 0.5, 0.9, 0.9, iters=100)
     assert state_err(opt, st) <= TOL

@@ -139,12 +139,15 @@ def test_mlp_configs_full_length(name):
     assert abs(np.linalg.norm(xbar) - gold["norm2_mean_model"]) <= 0.02 * gold["norm2_mean_model"]
 
 
-@pytest.mark.parametrize("name", ["c3", "c4"])
-def test_anchor_fusion_at_full_size_gives_the_bits_of_the_worker_mean_kernel(name):
+@pytest.mark.parametrize("name,gemm", [("c3", 1), ("c4", 1), ("c3", 3)])
+def test_anchor_fusion_at_full_size_gives_the_bits_of_the_worker_mean_kernel(name, gemm):
     # configs 3 and 4 as bench.py runs them (replayed graph blocks), with the worker sum inside
-    # the sync-step weight-gradient launch and with the worker-mean kernel: identical bits
+    # the sync-step weight-gradient launch (gemm_bf16 = 1) or inside the stand-alone update
+    # kernel (gemm_bf16 = 3), and with the worker-mean kernel: identical bits
     from paper_2002_09539_b200 import OverlapLocalSGD
     c = si.CONFIGS[name]
+    P = sum(o * i + o for i, o in zip(c["dims"][:-1], c["dims"][1:]))
+    weights = sum(o * i for i, o in zip(c["dims"][:-2], c["dims"][1:-1]))   # hidden layers
     table = sampling.class_pairs(0, c["m"]) if name == "c4" else None
     X, y = si.mixture_data(0, c["m"], c["n"], c["dims"][0], table)
     x0 = si.model_init(0, "mlp", c["dims"])
@@ -157,12 +160,13 @@ def test_anchor_fusion_at_full_size_gives_the_bits_of_the_worker_mean_kernel(nam
         with torch.cuda.stream(stream):
             opt = OverlapLocalSGD("mlp", m=c["m"], tau=c["tau"], gamma=c["gamma"], alpha=c["alpha"],
                                   beta=c["beta"], mu=c["mu"], batch=c["batch"], seed=0, dims=c["dims"],
-                                  gemm_bf16=1, x0=x0, X=Xd, y=yd)
+                                  gemm_bf16=gemm, x0=x0, X=Xd, y=yd)
             opt.set_anchor_fusion(fused)
             loss = torch.zeros((iters, c["m"]), device="cuda")
             opt.run(iters, loss)
             assert opt.graph_replays >= 1
             opt.join()
+            assert opt.summed_floats == ((weights if gemm == 1 else P) if fused else 0)
         torch.cuda.synchronize()
         z, v = opt.get_params(-1).copy(), opt.get_params(-2).copy()
         xs = [opt.get_params(i).copy() for i in (0, c["m"] // 2, c["m"] - 1)]
