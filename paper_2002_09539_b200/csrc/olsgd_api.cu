@@ -331,9 +331,6 @@ olsgd_status make_plan(const olsgd_model_spec* spec, const olsgd_hparams* hp, Pl
     pl->off_loss_ring = take((size_t)(base > kMaxGraphBlock ? base : kMaxGraphBlock) * m * sizeof(float));
   }
   pl->off_shadow = pl->has_shadow ? take((size_t)pl->ld * m * sizeof(__nv_bfloat16)) : 0;
-  // partial worker sums of the sync steps (Eq. 5's sum formed where x_{k+1} is written)
-  pl->has_sum_part = hp->mode == OLSGD_MODE_OVERLAP && m >= 2;
-  pl->off_sum_part = pl->has_sum_part ? take((size_t)worker_sum_slices(hp->m) * row) : 0;
   pl->off_idx = pl->has_g ? take((size_t)m * hp->batch * sizeof(int32_t)) : 0;
   pl->off_idx_next = pl->has_g ? take((size_t)m * hp->batch * sizeof(int32_t)) : 0;
   if (pl->has_g) {
@@ -348,6 +345,9 @@ olsgd_status make_plan(const olsgd_model_spec* spec, const olsgd_hparams* hp, Pl
     if (!plan_model(*spec, *hp, &pl->mp)) return fail(nullptr, OLSGD_EINVAL, "%s", pl->mp.error);
     off = align_up(off + pl->mp.bytes, kAlign);
   }
+  // partial worker sums of the sync steps (Eq. 5's sum formed where x_{k+1} is written)
+  pl->has_sum_part = hp->mode == OLSGD_MODE_OVERLAP && m >= 2;
+  pl->off_sum_part = pl->has_sum_part ? take((size_t)worker_sum_slices(hp->m) * row) : 0;
   pl->total = off;
   return OLSGD_OK;
 }
