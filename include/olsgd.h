@@ -66,7 +66,14 @@ typedef struct {
                                    gradient GEMM; 3 = the same GEMMs with the update as a
                                    separate kernel; 2 = the same bf16 data flow on CUDA
                                    cores (a check of the tensor-core kernels); 0 = fp32
-                                   (models without hidden layers)                     */
+                                   (models without hidden layers).  Any layer widths and
+                                   batch sizes are accepted; in modes 1 and 3 a GEMM whose
+                                   shape the tensor-core kernels do not take (they want
+                                   hidden widths in multiples of 128, input widths in
+                                   multiples of 64, a batch of 64, 128, 192 or 256, and
+                                   weights that start on a 16-byte boundary) runs on the
+                                   CUDA-core kernel of mode 2, and a layer whose update
+                                   cannot be fused goes through the update kernel       */
   int32_t reserved;
   int64_t flat_P;               /* FLAT only: number of parameters                    */
 } olsgd_model_spec;
@@ -176,7 +183,9 @@ olsgd_status olsgd_local_step_host(olsgd_ctx* ctx, const float* Xb_host, const v
  *                 rule as Xb_host above
  *   yb_host       int32 [m][batch]
  *   loss_host     as above
- * Returns OLSGD_ESTATE for any other model.                                  */
+ * Returns OLSGD_ESTATE for any other model, and where dims[0] is not a
+ * multiple of 64 or the batch not a multiple of 8 (the rows are moved in
+ * 16-byte pieces; olsgd_local_step_host takes every shape).                 */
 olsgd_status olsgd_local_step_host_bf16(olsgd_ctx* ctx, const void* Xb_host_bf16,
                                         const void* yb_host, float* loss_host);
 

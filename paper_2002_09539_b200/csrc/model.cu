@@ -35,14 +35,24 @@ inline bool tensor_path(const olsgd_model_spec& s) {
 // Is the update of parameter layer p (a hidden layer's weights and bias) applied inside its
 // weight-gradient GEMM?
 bool layer_update_is_fused(const olsgd_model_spec& spec, const olsgd_hparams& hp, int p) {
+  // the layer's weights must start on a 32-byte boundary of a parameter row (tensor maps over
+  // x, u and the bf16 copy): earlier layers of odd sizes can push them off it
+  int64_t w_off = 0;
+  for (int q = 0; q < p; ++q) w_off += (int64_t)spec.dims[q + 1] * spec.dims[q] + spec.dims[q + 1];
   return spec.gemm_bf16 == 1 && spec.dims[p + 1] % 128 == 0 && spec.dims[p] % 128 == 0 &&
-         hp.batch % 64 == 0 && hp.batch <= 128;
+         hp.batch % 64 == 0 && hp.batch <= 128 && w_off % 8 == 0;
 }
 
+// One GEMM of the bf16 path.  On the tensor-core modes a GEMM whose shape or alignment the
+// tcgen05 kernels do not take (widths that are not multiples of 128 / 64, batches other than
+// 64, 128, 192, 256, operands off a 16-byte boundary) runs on the CUDA-core kernel instead:
+// same operand rounding, fp32 accumulation in another order.
 cudaError_t run_gemm(const olsgd_model_spec& spec, GemmArgs ga, int* status, cudaStream_t s) {
   ga.status = status;
-  if (tensor_path(spec))
-    return wgrad_tc_supported(ga) ? launch_wgrad_tc(ga, s) : launch_gemm_tc(ga, s);
+  if (tensor_path(spec)) {
+    if (wgrad_tc_supported(ga)) return launch_wgrad_tc(ga, s);
+    if (gemm_tc_supported(ga)) return launch_gemm_tc(ga, s);
+  }
   return launch_gemm_simt(ga, s);
 }
 
@@ -78,25 +88,6 @@ bool plan_model(const olsgd_model_spec& spec, const olsgd_hparams& hp, ModelPlan
   }
   if (L < 2) {
     snprintf(mp->error, sizeof mp->error, "gemm_bf16 needs at least one hidden layer");
-    return false;
-  }
-  if (B % 8 != 0) {
-    snprintf(mp->error, sizeof mp->error, "the bf16 path needs batch %% 8 == 0");
-    return false;
-  }
-  for (int l = 0; l < L; ++l) {
-    // every hidden width is a GEMM M dimension, every layer input a GEMM K
-    if (l < L - 1 && spec.dims[l + 1] % 128 != 0) {
-      snprintf(mp->error, sizeof mp->error, "hidden width dims[%d] must be a multiple of 128", l + 1);
-      return false;
-    }
-    if (l < L - 1 && spec.dims[l] % 64 != 0) {
-      snprintf(mp->error, sizeof mp->error, "dims[%d] must be a multiple of 64", l);
-      return false;
-    }
-  }
-  if (tensor_path(spec) && (B % 64 != 0 || B > 256)) {
-    snprintf(mp->error, sizeof mp->error, "the tensor-core path needs batch in {64, 128, 192, 256}");
     return false;
   }
   const size_t e = sizeof(__nv_bfloat16);

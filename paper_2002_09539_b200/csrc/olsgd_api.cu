@@ -776,6 +776,9 @@ static olsgd_status local_step_host_impl(olsgd_ctx* c, const void* Xb_host, cons
   if (elem == 2 && !(c->spec.kind == OLSGD_MLP && c->spec.gemm_bf16 != 0))
     return fail(c, OLSGD_ESTATE, "bf16 minibatches are for models whose GEMM operands are bf16 "
                                  "(OLSGD_MLP with gemm_bf16 != 0)");
+  if (elem == 2 && (c->spec.dims[0] % 64 != 0 || c->hp.batch % 8 != 0))
+    return fail(c, OLSGD_ESTATE, "bf16 minibatches need dims[0] %% 64 == 0 and batch %% 8 == 0 "
+                                 "(16-byte pieces of a row are moved): use olsgd_local_step_host");
   if (c->need_sync) return fail(c, OLSGD_ESTATE, "a period ended: call olsgd_period_sync first");
   // this step writes the staged-minibatch set of iteration k itself (bf16 rows: on the copy
   // stream)

@@ -67,9 +67,14 @@ def test_bad_model_specs_are_rejected(lib):
     for s in [binding._spec("flat", flat_P=0), binding._spec("linreg", [0]),
               binding._spec("softmax", [10, 5, 3]), binding._spec("mlp", [10]),
               binding._spec("mlp", [64, 128, 64]),          # 64 classes > limit
-              binding._spec("mlp", [64, 100, 10], gemm_bf16=1),   # width not a multiple of 128
+              binding._spec("mlp", [64, 10], gemm_bf16=1),        # bf16 GEMMs without a hidden layer
               binding._spec("mlp", [64, 128, 10], gemm_bf16=0)]:  # fp32 hidden layers
         assert lib.olsgd_workspace_bytes(C.byref(s), C.byref(hp), C.byref(n)) == 1
+    # every width and batch is taken: what the tensor-core kernels cannot do runs on CUDA cores
+    for dims in ([64, 100, 10], [50, 37, 21, 7]):
+        for mode in (1, 2, 3):
+            s = binding._spec("mlp", dims, gemm_bf16=mode)
+            assert lib.olsgd_workspace_bytes(C.byref(s), C.byref(_hp(batch=7)), C.byref(n)) == 0
     bad_kind = binding._spec("flat", flat_P=5)
     bad_kind.kind = 9
     assert lib.olsgd_workspace_bytes(C.byref(bad_kind), C.byref(hp), C.byref(n)) == 1

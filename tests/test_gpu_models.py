@@ -135,6 +135,64 @@ def test_mlp_cuda_core_path_accepts_small_batches():
     assert state_err(opt, st) <= TOL_BF16_PARAM
 
 
+# Shapes the tensor-core kernels do not take, in whole or in part: odd widths and batches
+# (everything on the CUDA-core kernels, scalar output-layer kernels), a first layer that fits
+# and a second that does not, an input width off the 64 grid, and a layer whose own shape fits
+# but whose weights start off a 16-byte boundary because of the odd layers ahead of it.
+ODD_SHAPES = [([50, 37, 21, 7], 3, 40, 10, 2, 5),
+              ([200, 136, 72, 10], 2, 60, 24, 2, 5),
+              ([128, 256, 100, 10], 2, 80, 64, 2, 5),
+              ([100, 128, 128, 10], 2, 80, 64, 2, 5),
+              ([64, 3, 128, 128, 10], 2, 80, 64, 3, 7),
+              ([128, 128, 10], 2, 70, 63, 2, 5)]
+
+
+@pytest.mark.parametrize("dims,m,n,batch,tau,iters", ODD_SHAPES)
+@pytest.mark.parametrize("gemm_bf16", [2, 3, 1])
+def test_mlp_of_any_shape(dims, m, n, batch, tau, iters, gemm_bf16):
+    opt, st, lg, lo = _mlp_case(dims, m, n, batch, tau, iters, gemm_bf16)
+    assert np.isfinite(lg).all()
+    assert np.abs(lg - lo).max() <= TOL_BF16_LOSS * np.abs(lo).max()
+    assert state_err(opt, st) <= TOL_BF16_PARAM
+
+
+def test_odd_shapes_replay_as_graphs_and_take_host_rows():
+    from paper_2002_09539_b200 import OverlapLocalSGD, OlsgdError
+    dims, m, n, batch, tau, iters = [100, 128, 128, 10], 2, 80, 64, 2, 24
+    X, y = si.mixture_data(9, m, n, dims[0])
+    x0 = si.model_init(9, "mlp", dims)
+    kw = dict(dims=dims, gemm_bf16=1, m=m, tau=tau, batch=batch, gamma=0.05, alpha=0.6, beta=0.9,
+              mu=0.9, seed=9, x0=x0, X=to_dev(X), y=to_dev(y))
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(stream):
+        a = OverlapLocalSGD("mlp", **kw)
+        la = torch.zeros((iters, m), device="cuda")
+        a.run(iters, la)
+        a.join()
+        assert a.graph_replays >= 1
+    b = OverlapLocalSGD("mlp", **kw)
+    lb = torch.zeros((iters, m), device="cuda")
+    for k in range(iters):
+        b.local_step(lb[k])
+        if (k + 1) % tau == 0:
+            b.period_sync()
+    for u, w in zip(a.state(), b.state()):
+        assert np.array_equal(u, w)
+    assert np.array_equal(la.cpu().numpy(), lb.cpu().numpy())
+    # fp32 host rows are taken at any shape; bf16 host rows want 16-byte pieces
+    idx = b.get_indices(iters)
+    rows = np.stack([X[i][idx[i]] for i in range(m)])
+    labels = np.stack([y[i][idx[i]] for i in range(m)]).astype(np.int32)
+    loss_h = torch.zeros(m).pin_memory()
+    b.local_step_host(torch.from_numpy(rows).pin_memory(), torch.from_numpy(labels).pin_memory(), loss_h)
+    b.join()
+    assert np.isfinite(loss_h.numpy()).all()
+    with pytest.raises(OlsgdError):
+        b.local_step_host(torch.from_numpy(rows).to(torch.bfloat16).pin_memory(),
+                          torch.from_numpy(labels).pin_memory(), loss_h)
+
+
 def test_deep_mlp_loss_parity():
     opt, st, lg, lo = _mlp_case(*DEEP_SHAPE, 1)
     assert np.isfinite(lg).all()
