@@ -67,13 +67,16 @@ typedef struct {
                                    separate kernel; 2 = the same bf16 data flow on CUDA
                                    cores (a check of the tensor-core kernels); 0 = fp32
                                    (models without hidden layers).  Any layer widths and
-                                   batch sizes are accepted; in modes 1 and 3 a GEMM whose
-                                   shape the tensor-core kernels do not take (they want
-                                   hidden widths in multiples of 128, input widths in
-                                   multiples of 64, a batch of 64, 128, 192 or 256, and
-                                   weights that start on a 16-byte boundary) runs on the
-                                   CUDA-core kernel of mode 2, and a layer whose update
-                                   cannot be fused goes through the update kernel       */
+                                   batch sizes are accepted.  In modes 1 and 3 the
+                                   tensor-core kernels take a batch of 64, 128, 192 or 256
+                                   and layer widths in multiples of 8 (16-byte row pitches;
+                                   partial last tiles are padded with zeros by TMA and
+                                   clipped on the way out); any other GEMM runs on the
+                                   CUDA-core kernel of mode 2.  The update is fused into
+                                   the weight-gradient GEMM of layers whose two widths are
+                                   multiples of 128 at a batch of 64 or 128; the other
+                                   layers go through the update kernel.
+                                   olsgd_tensor_core_launches counts what ran where.   */
   int32_t reserved;
   int64_t flat_P;               /* FLAT only: number of parameters                    */
 } olsgd_model_spec;
@@ -296,6 +299,11 @@ int olsgd_set_launch_overlap(int on);
  * captured graph keeps the setting it was captured with).  Returns the previous setting.
  * The paper has no counterpart: this is kernel plumbing.                                    */
 int olsgd_set_gemm_pairs(int on);
+
+/* How many launches of the tensor-core (tcgen05) kernels this process has made so far:
+ * forward / input-gradient GEMMs and weight-gradient launches.  Lets a caller (or a test)
+ * see whether a model's GEMMs ran there or on the CUDA-core kernel they fall back to.      */
+int64_t olsgd_tensor_core_launches(void);
 
 /* Copy one vector of the state to the caller.  Joins both streams (blocks
  * the host).  which: 0..m-1 worker model x^(i); -1 anchor z; -2 anchor

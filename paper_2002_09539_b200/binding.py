@@ -91,6 +91,7 @@ def load_library():
         "olsgd_graph_block": (i64, [vp]),
         "olsgd_set_launch_overlap": (i32, [i32]),
         "olsgd_set_gemm_pairs": (i32, [i32]),
+        "olsgd_tensor_core_launches": (i64, []),
         "olsgd_profile_enable": (i32, [vp, i32]),
         "olsgd_profile_read": (i32, [vp, C.POINTER(i64), C.POINTER(C.c_double), i32]),
         "olsgd_profile_read_layers": (i32, [vp, C.POINTER(i64), C.POINTER(C.c_double), i32]),
@@ -137,6 +138,11 @@ def set_launch_overlap(on):
 def set_gemm_pairs(on):
     """olsgd_set_gemm_pairs: process-wide; returns the previous setting."""
     return bool(load_library().olsgd_set_gemm_pairs(1 if on else 0))
+
+
+def tensor_core_launches():
+    """olsgd_tensor_core_launches: launches of the tcgen05 kernels made by this process."""
+    return int(load_library().olsgd_tensor_core_launches())
 
 
 NOALLOC_MAX_WORKERS = 16384

@@ -535,6 +535,7 @@ namespace olsgd {
 void set_thread_error(const char* text) { g_last_error = text ? text : ""; }
 int g_launch_overlap = 1;
 int g_gemm_pairs = 0;
+int64_t g_tc_launches = 0;
 thread_local bool g_launch_plain = false;
 
 int current_device() {
@@ -1322,6 +1323,8 @@ int olsgd_set_launch_overlap(int on) {
   olsgd::g_launch_overlap = on ? 1 : 0;
   return before;
 }
+
+int64_t olsgd_tensor_core_launches(void) { return olsgd::g_tc_launches; }
 
 int olsgd_set_gemm_pairs(int on) {
   const int before = olsgd::g_gemm_pairs;

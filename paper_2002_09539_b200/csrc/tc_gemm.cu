@@ -56,14 +56,17 @@ __device__ __forceinline__ void gemm_epilogue(const EpiArgs& ea, uint32_t tmem_b
                                               int n0, int worker) {
   const int lane_group = warp & 3;
   const int row = m0 + lane_group * 32 + lane;
+  // the last tile of a band may reach past row Ma - 1: those rows were loaded as zeros and
+  // are neither looked up nor stored
+  const bool live = row < ea.Ma;
   const int64_t wk = worker;
   float bias = 0.f;
-  if (ea.epilogue == GEMM_EPI_BIAS_RELU) bias = ea.bias[wk * ea.bias_batch + row];
+  if (ea.epilogue == GEMM_EPI_BIAS_RELU && live) bias = ea.bias[wk * ea.bias_batch + row];
   uint4 mk[4], mk_next[4];
 #pragma unroll
   for (int q = 0; q < 4; ++q) mk[q] = mk_next[q] = make_uint4(0u, 0u, 0u, 0u);
   const uint4* mask_row = nullptr;
-  if (ea.epilogue == GEMM_EPI_RELU_MASK) {
+  if (ea.epilogue == GEMM_EPI_RELU_MASK && live) {
     mask_row = reinterpret_cast<const uint4*>(ea.mask + (wk * ea.Ma + row) * ea.Nb + n0);
 #pragma unroll
     for (int q = 0; q < 4; ++q) mk[q] = mask_row[q];
@@ -72,62 +75,68 @@ __device__ __forceinline__ void gemm_epilogue(const EpiArgs& ea, uint32_t tmem_b
     tc_fence_after();
 #pragma unroll 1
     for (int c = 0; c < BN / 32; ++c) {
-      if (ea.epilogue == GEMM_EPI_RELU_MASK && c + 1 < BN / 32) {
+      if (mask_row && c + 1 < BN / 32) {
 #pragma unroll
         for (int q = 0; q < 4; ++q) mk_next[q] = mask_row[(c + 1) * 4 + q];
       }
       float v[32];
+      __syncwarp();
       tmem_ld32(tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)(c * 32), v);
-      const int col0 = n0 + c * 32;
-      if (ea.epilogue == GEMM_EPI_STORE_F32) {
-        float4* dst = reinterpret_cast<float4*>(ea.out_f + wk * ea.out_batch +
-                                                  (int64_t)row * ea.ldo + col0);
+      // (the load above is collective: every lane takes part in it, and meets the others
+      // again at the end of the iteration)
+      if (live) {
+        const int col0 = n0 + c * 32;
+        if (ea.epilogue == GEMM_EPI_STORE_F32) {
+          float4* dst = reinterpret_cast<float4*>(ea.out_f + wk * ea.out_batch +
+                                                    (int64_t)row * ea.ldo + col0);
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-          dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-      } else {
-        const int64_t t_off = (wk * ea.Ma + row) * ea.Nb + col0;
-        if (ea.epilogue == GEMM_EPI_BIAS_RELU) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j] + bias, 0.f);
+          for (int j = 0; j < 8; ++j)
+            dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
         } else {
+          const int64_t t_off = (wk * ea.Ma + row) * ea.Nb + col0;
+          if (ea.epilogue == GEMM_EPI_BIAS_RELU) {
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const uint4 w = mk[q];
-            const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+            for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j] + bias, 0.f);
+          } else {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              // a bf16 is positive iff its sign bit is clear and it is not zero
-              const uint32_t lo = ws[e] & 0xFFFFu, hi = ws[e] >> 16;
-              if (!(lo != 0 && lo < 0x8000u)) v[q * 8 + e * 2] = 0.f;
-              if (!(hi != 0 && hi < 0x8000u)) v[q * 8 + e * 2 + 1] = 0.f;
+            for (int q = 0; q < 4; ++q) {
+              const uint4 w = mk[q];
+              const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                // a bf16 is positive iff its sign bit is clear and it is not zero
+                const uint32_t lo = ws[e] & 0xFFFFu, hi = ws[e] >> 16;
+                if (!(lo != 0 && lo < 0x8000u)) v[q * 8 + e * 2] = 0.f;
+                if (!(hi != 0 && hi < 0x8000u)) v[q * 8 + e * 2 + 1] = 0.f;
+              }
+              mk[q] = mk_next[q];
             }
-            mk[q] = mk_next[q];
           }
-        }
-        uint32_t pk[16];
+          uint32_t pk[16];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
-          pk[j] = *reinterpret_cast<uint32_t*>(&b2);
-        }
-        if (ea.out_t) {
-          uint4* dst = reinterpret_cast<uint4*>(ea.out_t + t_off);
+          for (int j = 0; j < 16; ++j) {
+            __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+            pk[j] = *reinterpret_cast<uint32_t*>(&b2);
+          }
+          if (ea.out_t) {
+            uint4* dst = reinterpret_cast<uint4*>(ea.out_t + t_off);
 #pragma unroll
-          for (int q = 0; q < 4; ++q)
-            dst[q] = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
-        }
-        if (ea.out_n) {
-          // [Nb][Ma]: for a fixed column the 32 lanes of the warp write 32 consecutive rows
-          __nv_bfloat16* dst = ea.out_n + (wk * ea.Nb + col0) * ea.Ma + row;
+            for (int q = 0; q < 4; ++q)
+              dst[q] = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+          }
+          if (ea.out_n) {
+            // [Nb][Ma]: for a fixed column the 32 lanes of the warp write 32 consecutive rows
+            __nv_bfloat16* dst = ea.out_n + (wk * ea.Nb + col0) * ea.Ma + row;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const uint32_t w = pk[j >> 1];
-            const uint16_t h = (j & 1) ? (uint16_t)(w >> 16) : (uint16_t)(w & 0xFFFFu);
-            *reinterpret_cast<uint16_t*>(dst + (int64_t)j * ea.Ma) = h;
+            for (int j = 0; j < 32; ++j) {
+              const uint32_t w = pk[j >> 1];
+              const uint16_t h = (j & 1) ? (uint16_t)(w >> 16) : (uint16_t)(w & 0xFFFFu);
+              *reinterpret_cast<uint16_t*>(dst + (int64_t)j * ea.Ma) = h;
+            }
           }
         }
       }
+      __syncwarp();
     }
   }
 }
@@ -423,8 +432,10 @@ cudaError_t launch_one(const GemmArgs& a, const CUtensorMap& ma, const CUtensorM
   ea.ldo = a.ldo;
   ea.out_batch = a.out_batch;
   ea.status = a.status;
-  dim3 grid(a.Nb / BN, a.Ma / kBM, a.m);
-  return launch_chained(kern, grid, dim3(kThreads), smem, s, ma, mb, a.K / kBK, a.a_mn_major ? 1 : 0, ea);
+  dim3 grid(a.Nb / BN, (a.Ma + kBM - 1) / kBM, a.m);
+  g_tc_launches += 1;
+  return launch_chained(kern, grid, dim3(kThreads), smem, s, ma, mb, (a.K + kBK - 1) / kBK,
+                        a.a_mn_major ? 1 : 0, ea);
 }
 
 template <int BN, int STAGES>
@@ -465,6 +476,7 @@ cudaError_t launch_pair(const GemmArgs& a, const CUtensorMap& ma, const CUtensor
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = (g_launch_overlap && !g_launch_plain) ? 2 : 1;
+  g_tc_launches += 1;
   return cudaLaunchKernelEx(&cfg, kern, ma, mb, a.K / kBK, a.a_mn_major ? 1 : 0, ea);
 }
 
@@ -487,7 +499,10 @@ __global__ void wait_selftest_kernel(int* status, uint64_t limit_ns) {
 
 bool gemm_tc_supported(const GemmArgs& a) {
   auto al16 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; };
-  if (a.Ma % kBM != 0 || a.K % kBK != 0 || a.K < kBK || pick_bn(a.Nb) == 0) return false;
+  // Ma and K need not fill their last 128-row tile or 64-wide k-block: TMA delivers zeros
+  // for what lies outside the operand, and the epilogue skips the rows past Ma.  What
+  // remains are the alignment rules of the tensor maps (16-byte row pitches) and the batch.
+  if (a.Ma < 1 || a.K < 1 || pick_bn(a.Nb) == 0) return false;
   if (a.lda % 8 || a.ldb % 8 || a.a_batch % 8 || a.b_batch % 8) return false;
   if (!al16(a.A) || !al16(a.B)) return false;
   if (a.epilogue == GEMM_EPI_STORE_F32) {
@@ -510,21 +525,22 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, cudaStream_t s) {
     return cudaErrorInvalidValue;
   }
   // long K and an even number of 128-row tiles: CTA pairs, each CTA loading half of the B tile
-  const bool pairs = g_gemm_pairs && a.K / kBK > 2 && (a.Ma / kBM) % 2 == 0 && (bn == 128 || bn == 64);
+  const bool pairs = g_gemm_pairs && a.K % kBK == 0 && a.K / kBK > 2 && a.Ma % (2 * kBM) == 0 &&
+                     (bn == 128 || bn == 64);
   if (pairs) {
     if (!make_map(&mb, a.B, a.K, a.Nb, a.m, a.ldb, a.b_batch, bn / 2)) return cudaErrorInvalidValue;
     return bn == 128 ? launch_pair<128, 8>(a, ma, mb, s) : launch_pair<64, 8>(a, ma, mb, s);
   }
   if (!make_map(&mb, a.B, a.K, a.Nb, a.m, a.ldb, a.b_batch, bn)) return cudaErrorInvalidValue;
   // short K (weight gradients, K = batch): few stages so several CTAs share an SM
-  const bool short_k = a.K / kBK <= 2;
+  const bool short_k = (a.K + kBK - 1) / kBK <= 2;
   switch (bn) {
     case 256: return short_k ? launch_one<256, 2>(a, ma, mb, s) : launch_one<256, 4>(a, ma, mb, s);
     case 128: return short_k ? launch_one<128, 2>(a, ma, mb, s) : launch_one<128, 6>(a, ma, mb, s);
     default: {
       // more tiles than SMs: four stages (96 KB) so that two CTAs share an SM and the
       // whole grid is resident in one wave
-      const int64_t ctas = (int64_t)(a.Nb / 64) * (a.Ma / kBM) * a.m;
+      const int64_t ctas = (int64_t)(a.Nb / 64) * ((a.Ma + kBM - 1) / kBM) * a.m;
       if (short_k) return launch_one<64, 2>(a, ma, mb, s);
       return ctas > sm_count() ? launch_one<64, 4>(a, ma, mb, s) : launch_one<64, 8>(a, ma, mb, s);
     }

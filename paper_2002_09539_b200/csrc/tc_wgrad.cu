@@ -218,6 +218,7 @@ struct WgradLayer {
   float* rowsum;
   int64_t rowsum_batch;
   int n_tiles, m_tiles, chunks, ldw;
+  int rows;      // Ma: the last 128-row band may reach past it (plain variant only)
   int cta_begin;
 };
 struct WgradBatch {
@@ -372,7 +373,7 @@ wgrad_tc_kernel(const __grid_constant__ WgradBatch wb, int num_kb, int n_stages,
         const int row = rr * 32 + lane;
         const float sum = slab_row_sum_smem(a_smem, kABlock, num_kb, row);
         if (bias_update) update_bias_entry(up, work.worker, up.b_off + work.m0 + row, sum);
-        else dst[row] = sum;
+        else if (work.m0 + row < ly.rows) dst[row] = sum;
       }
     }
   } else if (warp == 0 && lane == 0) {
@@ -595,7 +596,10 @@ wgrad_tc_kernel(const __grid_constant__ WgradBatch wb, int num_kb, int n_stages,
         fence_async_smem();
         __syncwarp();
         if (lane == 0) {
-          tma_store_3d(&map_out, smem_u32(stage), p.col + c * 32, p.m0 + lane_group * 32, p.worker);
+          // a box that reaches past the matrix is clipped by the copy; one that lies outside
+          // it altogether is not issued
+          if (p.col + c * 32 < ldw && p.m0 + lane_group * 32 < ly.rows)
+            tma_store_3d(&map_out, smem_u32(stage), p.col + c * 32, p.m0 + lane_group * 32, p.worker);
           bulk_commit();
         }
         ++store_count;
@@ -631,13 +635,16 @@ wgrad_tc_kernel(const __grid_constant__ WgradBatch wb, int num_kb, int n_stages,
 bool wgrad_tc_supported(const GemmArgs& a) {
   auto al16 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; };
   if (a.epilogue != GEMM_EPI_STORE_F32) return false;
-  if (a.Ma % kBM != 0 || a.Nb % kWN != 0 || a.K % kBK != 0 || a.K < kBK || a.K > kMaxKB * kBK)
-    return false;
+  if (a.Ma < 1 || a.Nb < 1 || a.K % kBK != 0 || a.K < kBK || a.K > kMaxKB * kBK) return false;
   if (a.lda % 8 || a.ldb % 8 || a.a_batch % 8 || a.b_batch % 8) return false;
   if (!al16(a.A) || !al16(a.B)) return false;
-  if ((int64_t)(a.Ma / kBM) * a.m * (a.Nb / kWN) > 0x7FFFFFFF) return false;
+  if ((int64_t)((a.Ma + kBM - 1) / kBM) * a.m * ((a.Nb + kWN - 1) / kWN) > 0x7FFFFFFF) return false;
   if (a.upd.enabled) {
     const FusedUpdateArgs& u = a.upd;
+    // the fused epilogue writes whole tiles with plain stores: no partial bands or tiles
+    // (the variant that stores the gradient clips them: rows and columns past the matrix
+    // are loaded as zeros and its TMA stores drop what lies outside)
+    if (a.Ma % kBM != 0 || a.Nb % kWN != 0) return false;
     if (a.K > 2 * kBK) return false;   // the x/u tile ring needs the shared memory
     if (!al16(u.x_in) || !al16(u.x_out) || !al16(u.shadow) || (u.u && !al16(u.u)) ||
         (u.sync && !al16(u.z)))
@@ -681,9 +688,10 @@ cudaError_t launch_wgrad_tc_batch(const GemmArgs* args, int n, cudaStream_t s) {
     } else if (!make_map_f32(&ly.map_out, a.out_f, a.Nb, a.Ma, a.m, a.ldo, a.out_batch, 32)) {
       return cudaErrorInvalidValue;
     }
-    ly.n_tiles = a.Nb / tile_n;
-    ly.m_tiles = a.Ma / kBM;
+    ly.n_tiles = (a.Nb + tile_n - 1) / tile_n;
+    ly.m_tiles = (a.Ma + kBM - 1) / kBM;
     ly.ldw = a.Nb;
+    ly.rows = a.Ma;
     ly.rowsum = a.rowsum_out;
     ly.rowsum_batch = a.rowsum_batch;
     ly.cta_begin = ctas;
@@ -753,6 +761,7 @@ cudaError_t launch_wgrad_tc_batch(const GemmArgs* args, int n, cudaStream_t s) {
                                   : ensure_dynamic_smem(configured[0], wgrad_tc_kernel<false, false>, smem);
     if (e != cudaSuccess) return e;
   }
+  g_tc_launches += 1;
   if (sum)
     return launch_chained(wgrad_tc_kernel<true, true>, dim3(ctas), dim3(kSumThreads), smem, s, wb,
                           num_kb, n_stages, args[0].status);
