@@ -68,11 +68,11 @@ typedef struct {
                                    cores (a check of the tensor-core kernels); 0 = fp32
                                    (models without hidden layers).  Any layer widths and
                                    batch sizes are accepted.  In modes 1 and 3 the
-                                   tensor-core kernels take a batch of 64, 128, 192 or 256
-                                   and layer widths in multiples of 8 (16-byte row pitches;
-                                   partial last tiles are padded with zeros by TMA and
-                                   clipped on the way out); any other GEMM runs on the
-                                   CUDA-core kernel of mode 2.  The update is fused into
+                                   tensor-core kernels take batches and layer widths in
+                                   multiples of 8 (16-byte row pitches; partial last tiles
+                                   are padded with zeros by TMA and clipped on the way
+                                   out); any other GEMM runs on the CUDA-core kernel of
+                                   mode 2.  The update is fused into
                                    the weight-gradient GEMM of layers whose two widths are
                                    multiples of 128 at a batch of 64 or 128; the other
                                    layers go through the update kernel.

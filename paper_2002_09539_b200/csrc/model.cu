@@ -45,9 +45,8 @@ bool layer_update_is_fused(const olsgd_model_spec& spec, const olsgd_hparams& hp
 
 // One GEMM of the bf16 path.  On the tensor-core modes a GEMM whose shape or alignment the
 // tcgen05 kernels do not take (row pitches that are not multiples of 16 bytes, i.e. widths
-// off the grid of 8, batches other than 64, 128, 192, 256, operands off a 16-byte boundary)
-// runs on the CUDA-core kernel instead: same operand rounding, fp32 accumulation in another
-// order.
+// or batches off the grid of 8, operands off a 16-byte boundary) runs on the CUDA-core kernel
+// instead: same operand rounding, fp32 accumulation in another order.
 cudaError_t run_gemm(const olsgd_model_spec& spec, GemmArgs ga, int* status, cudaStream_t s) {
   ga.status = status;
   if (tensor_path(spec)) {

@@ -28,6 +28,7 @@ struct EpiArgs {
   int once;      // A is read once: its TMA loads carry an evict-first policy
   int epilogue;
   int Ma, Nb;
+  int full;      // no partial tiles in this launch
   const float* bias;
   int64_t bias_batch;
   const __nv_bfloat16* mask;
@@ -50,7 +51,9 @@ struct SharedCtl {
 // r <-> row m0 + r, column j <-> col n0 + j.  What it needs besides the accumulator is
 // fetched while the main loop runs: the row's bias, or the first 32 columns of its ReLU mask
 // (the next 32 are fetched while the current ones are applied).
-template <int BN>
+// FULL: every tile of the launch lies inside the matrix (Ma a multiple of 128, Nb of BN), so
+// the row and column tests are compiled out.
+template <int BN, bool FULL>
 __device__ __forceinline__ void gemm_epilogue(const EpiArgs& ea, uint32_t tmem_base, uint32_t tmem_full_bar,
                                               volatile int* abort_flag, int warp, int lane, int m0,
                                               int n0, int worker) {
@@ -58,7 +61,7 @@ __device__ __forceinline__ void gemm_epilogue(const EpiArgs& ea, uint32_t tmem_b
   const int row = m0 + lane_group * 32 + lane;
   // the last tile of a band may reach past row Ma - 1: those rows were loaded as zeros and
   // are neither looked up nor stored
-  const bool live = row < ea.Ma;
+  const bool live = FULL || row < ea.Ma;
   const int64_t wk = worker;
   float bias = 0.f;
   if (ea.epilogue == GEMM_EPI_BIAS_RELU && live) bias = ea.bias[wk * ea.bias_batch + row];
@@ -66,10 +69,13 @@ __device__ __forceinline__ void gemm_epilogue(const EpiArgs& ea, uint32_t tmem_b
 #pragma unroll
   for (int q = 0; q < 4; ++q) mk[q] = mk_next[q] = make_uint4(0u, 0u, 0u, 0u);
   const uint4* mask_row = nullptr;
+  // likewise the last column tile may reach past column Nb - 1 (Nb is a multiple of 8, the
+  // width of one 16-byte piece of a row): pieces past it are neither looked up nor stored
   if (ea.epilogue == GEMM_EPI_RELU_MASK && live) {
     mask_row = reinterpret_cast<const uint4*>(ea.mask + (wk * ea.Ma + row) * ea.Nb + n0);
 #pragma unroll
-    for (int q = 0; q < 4; ++q) mk[q] = mask_row[q];
+    for (int q = 0; q < 4; ++q)
+      if (FULL || n0 + 8 * q < ea.Nb) mk[q] = mask_row[q];
   }
   if (mbar_wait(tmem_full_bar, 0, abort_flag) && !*abort_flag) {
     tc_fence_after();
@@ -77,21 +83,23 @@ __device__ __forceinline__ void gemm_epilogue(const EpiArgs& ea, uint32_t tmem_b
     for (int c = 0; c < BN / 32; ++c) {
       if (mask_row && c + 1 < BN / 32) {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) mk_next[q] = mask_row[(c + 1) * 4 + q];
+        for (int q = 0; q < 4; ++q)
+          if (FULL || n0 + (c + 1) * 32 + 8 * q < ea.Nb) mk_next[q] = mask_row[(c + 1) * 4 + q];
       }
       float v[32];
-      __syncwarp();
+      if (!FULL) __syncwarp();
       tmem_ld32(tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)(c * 32), v);
       // (the load above is collective: every lane takes part in it, and meets the others
       // again at the end of the iteration)
-      if (live) {
-        const int col0 = n0 + c * 32;
+      const int col0 = n0 + c * 32;
+      const int ncols = FULL ? 32 : ea.Nb - col0;   // columns of this block inside the matrix (>= 32: all)
+      if (live && ncols > 0) {
         if (ea.epilogue == GEMM_EPI_STORE_F32) {
           float4* dst = reinterpret_cast<float4*>(ea.out_f + wk * ea.out_batch +
                                                     (int64_t)row * ea.ldo + col0);
 #pragma unroll
           for (int j = 0; j < 8; ++j)
-            dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            if (4 * j < ncols) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
         } else {
           const int64_t t_off = (wk * ea.Ma + row) * ea.Nb + col0;
           if (ea.epilogue == GEMM_EPI_BIAS_RELU) {
@@ -122,7 +130,7 @@ __device__ __forceinline__ void gemm_epilogue(const EpiArgs& ea, uint32_t tmem_b
             uint4* dst = reinterpret_cast<uint4*>(ea.out_t + t_off);
 #pragma unroll
             for (int q = 0; q < 4; ++q)
-              dst[q] = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+              if (8 * q < ncols) dst[q] = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
           }
           if (ea.out_n) {
             // [Nb][Ma]: for a fixed column the 32 lanes of the warp write 32 consecutive rows
@@ -131,12 +139,12 @@ __device__ __forceinline__ void gemm_epilogue(const EpiArgs& ea, uint32_t tmem_b
             for (int j = 0; j < 32; ++j) {
               const uint32_t w = pk[j >> 1];
               const uint16_t h = (j & 1) ? (uint16_t)(w >> 16) : (uint16_t)(w & 0xFFFFu);
-              *reinterpret_cast<uint16_t*>(dst + (int64_t)j * ea.Ma) = h;
+              if (j < ncols) *reinterpret_cast<uint16_t*>(dst + (int64_t)j * ea.Ma) = h;
             }
           }
         }
       }
-      __syncwarp();
+      if (!FULL) __syncwarp();
     }
   }
 }
@@ -253,7 +261,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
     umma_commit(smem_u32(&ctl->tmem_full));   // accumulator complete
   } else if (warp >= 2) {
-    gemm_epilogue<BN>(ea, tmem_base, smem_u32(&ctl->tmem_full), abort_flag, warp, lane, m0, n0, worker);
+    if (ea.full) gemm_epilogue<BN, true>(ea, tmem_base, smem_u32(&ctl->tmem_full), abort_flag, warp, lane, m0, n0, worker);
+    else gemm_epilogue<BN, false>(ea, tmem_base, smem_u32(&ctl->tmem_full), abort_flag, warp, lane, m0, n0, worker);
   }
 
   // ---------------- teardown: every role arrives here, all waits above are bounded
@@ -377,7 +386,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     }
     umma_commit_pair(smem_u32(&ctl->tmem_full));    // both accumulators are complete
   } else if (warp >= 2) {
-    gemm_epilogue<BN>(ea, tmem_base, smem_u32(&ctl->tmem_full), abort_flag, warp, lane, m0, n0, worker);
+    if (ea.full) gemm_epilogue<BN, true>(ea, tmem_base, smem_u32(&ctl->tmem_full), abort_flag, warp, lane, m0, n0, worker);
+    else gemm_epilogue<BN, false>(ea, tmem_base, smem_u32(&ctl->tmem_full), abort_flag, warp, lane, m0, n0, worker);
   }
 
   // ---------------- teardown: every role of both CTAs arrives here, all waits are bounded
@@ -400,11 +410,13 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 
 // ------------------------------------------------------------------ host side
 
+// The column-tile width for Nb columns (a multiple of 8): the widest that divides Nb, else 64
+// with a partial last tile.
 int pick_bn(int Nb) {
+  if (Nb % 8 != 0 || Nb < 8) return 0;
   if (Nb % 256 == 0) return 256;
   if (Nb % 128 == 0) return 128;
-  if (Nb % 64 == 0) return 64;
-  return 0;
+  return 64;
 }
 
 template <int BN, int STAGES>
@@ -423,6 +435,7 @@ cudaError_t launch_one(const GemmArgs& a, const CUtensorMap& ma, const CUtensorM
   ea.a_early = a.a_ready_early;
   ea.Ma = a.Ma;
   ea.Nb = a.Nb;
+  ea.full = (a.Ma % kBM == 0 && a.Nb % BN == 0) ? 1 : 0;
   ea.bias = a.bias;
   ea.bias_batch = a.bias_batch;
   ea.mask = a.mask;
@@ -432,7 +445,7 @@ cudaError_t launch_one(const GemmArgs& a, const CUtensorMap& ma, const CUtensorM
   ea.ldo = a.ldo;
   ea.out_batch = a.out_batch;
   ea.status = a.status;
-  dim3 grid(a.Nb / BN, (a.Ma + kBM - 1) / kBM, a.m);
+  dim3 grid((a.Nb + BN - 1) / BN, (a.Ma + kBM - 1) / kBM, a.m);
   g_tc_launches += 1;
   return launch_chained(kern, grid, dim3(kThreads), smem, s, ma, mb, (a.K + kBK - 1) / kBK,
                         a.a_mn_major ? 1 : 0, ea);
@@ -453,6 +466,7 @@ cudaError_t launch_pair(const GemmArgs& a, const CUtensorMap& ma, const CUtensor
   ea.a_early = a.a_ready_early;
   ea.Ma = a.Ma;
   ea.Nb = a.Nb;
+  ea.full = (a.Ma % kBM == 0 && a.Nb % BN == 0) ? 1 : 0;
   ea.bias = a.bias;
   ea.bias_batch = a.bias_batch;
   ea.mask = a.mask;
@@ -499,9 +513,10 @@ __global__ void wait_selftest_kernel(int* status, uint64_t limit_ns) {
 
 bool gemm_tc_supported(const GemmArgs& a) {
   auto al16 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; };
-  // Ma and K need not fill their last 128-row tile or 64-wide k-block: TMA delivers zeros
-  // for what lies outside the operand, and the epilogue skips the rows past Ma.  What
-  // remains are the alignment rules of the tensor maps (16-byte row pitches) and the batch.
+  // Ma, Nb and K need not fill their last 128-row tile, column tile or 64-wide k-block: TMA
+  // delivers zeros for what lies outside the operands, and the epilogue skips the rows past
+  // Ma and the 16-byte pieces past Nb.  What remains are the alignment rules of the tensor
+  // maps (16-byte row pitches) and Nb % 8 == 0.
   if (a.Ma < 1 || a.K < 1 || pick_bn(a.Nb) == 0) return false;
   if (a.lda % 8 || a.ldb % 8 || a.a_batch % 8 || a.b_batch % 8) return false;
   if (!al16(a.A) || !al16(a.B)) return false;
@@ -526,7 +541,7 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, cudaStream_t s) {
   }
   // long K and an even number of 128-row tiles: CTA pairs, each CTA loading half of the B tile
   const bool pairs = g_gemm_pairs && a.K % kBK == 0 && a.K / kBK > 2 && a.Ma % (2 * kBM) == 0 &&
-                     (bn == 128 || bn == 64);
+                     a.Nb % bn == 0 && (bn == 128 || bn == 64);
   if (pairs) {
     if (!make_map(&mb, a.B, a.K, a.Nb, a.m, a.ldb, a.b_batch, bn / 2)) return cudaErrorInvalidValue;
     return bn == 128 ? launch_pair<128, 8>(a, ma, mb, s) : launch_pair<64, 8>(a, ma, mb, s);
@@ -540,7 +555,7 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, cudaStream_t s) {
     default: {
       // more tiles than SMs: four stages (96 KB) so that two CTAs share an SM and the
       // whole grid is resident in one wave
-      const int64_t ctas = (int64_t)(a.Nb / 64) * ((a.Ma + kBM - 1) / kBM) * a.m;
+      const int64_t ctas = (int64_t)((a.Nb + 63) / 64) * ((a.Ma + kBM - 1) / kBM) * a.m;
       if (short_k) return launch_one<64, 2>(a, ma, mb, s);
       return ctas > sm_count() ? launch_one<64, 4>(a, ma, mb, s) : launch_one<64, 8>(a, ma, mb, s);
     }
