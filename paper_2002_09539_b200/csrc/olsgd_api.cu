@@ -535,7 +535,7 @@ namespace olsgd {
 void set_thread_error(const char* text) { g_last_error = text ? text : ""; }
 int g_launch_overlap = 1;
 int g_gemm_pairs = 0;
-int64_t g_tc_launches = 0;
+std::atomic<int64_t> g_tc_launches{0};
 thread_local bool g_launch_plain = false;
 
 int current_device() {
@@ -1324,7 +1324,7 @@ int olsgd_set_launch_overlap(int on) {
   return before;
 }
 
-int64_t olsgd_tensor_core_launches(void) { return olsgd::g_tc_launches; }
+int64_t olsgd_tensor_core_launches(void) { return olsgd::g_tc_launches.load(); }
 
 int olsgd_set_gemm_pairs(int on) {
   const int before = olsgd::g_gemm_pairs;

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "olsgd.h"
 
 namespace olsgd {
@@ -20,7 +22,8 @@ namespace olsgd {
 // through the gate at once.
 extern int g_launch_overlap;   // olsgd_set_launch_overlap
 extern int g_gemm_pairs;       // olsgd_set_gemm_pairs: long-K GEMMs on CTA pairs (cta_group::2)
-extern int64_t g_tc_launches;  // launches of the tcgen05 kernels so far (olsgd_tensor_core_launches)
+extern std::atomic<int64_t> g_tc_launches;  // launches of the tcgen05 kernels so far
+                                            // (olsgd_tensor_core_launches)
 // Set around a launch that goes to a stream whose previous operation is an event wait, not a
 // kernel: such a launch is an ordinary one (its kernel passes the gate at once).
 extern thread_local bool g_launch_plain;
