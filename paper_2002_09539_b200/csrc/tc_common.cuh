@@ -15,7 +15,7 @@ namespace tc {
 constexpr int kBM = 128;          // rows of A per tile = MMA M = TMEM lanes
 constexpr int kBK = 64;           // K elements per stage = one 128-byte swizzle row
 constexpr int kUmmaK = 16;        // K per tcgen05.mma for 16-bit operands
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;       // TMA, MMA and eight epilogue warps (GEMM kernels)
 constexpr uint32_t kSpinLimit = 1u << 22;          // iterations, for the drain loops
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // wall-clock bound of one barrier wait
 

@@ -5,12 +5,14 @@
 // elements (128 bytes per row) are brought in by TMA with the 128-byte swizzle
 // into a ring of shared-memory stages; one elected thread issues tcgen05.mma
 // (M = 128, N = BN, K = 16 per instruction) with the accumulator in tensor
-// memory; four warps read the accumulator back with tcgen05.ld and run the
+// memory; eight warps read the accumulator back with tcgen05.ld and run the
 // epilogue (bias + ReLU, ReLU mask, or fp32 store).
 //
-// Warp roles (192 threads): warp 0 TMA producer, warp 1 MMA issuer and owner
-// of the tensor-memory allocation, warps 2-5 epilogue (warp w reads the 32
-// TMEM lanes of group w % 4).
+// Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer and owner
+// of the tensor-memory allocation, warps 2-9 epilogue (warp w reads the 32
+// TMEM lanes of group w % 4; warps 2-5 take the left half of the tile's
+// columns, warps 6-9 the right half: the epilogue is the serial tail of a
+// CTA with one tile, and two warps per lane group halve it).
 //
 // Every wait on an mbarrier is bounded.  A wait that runs out raises a flag in
 // shared memory that all roles poll, records OLSGD_ETIMEOUT in the status word
@@ -47,7 +49,7 @@ struct SharedCtl {
   int abort_flag;
 };
 
-// The epilogue of one 128 x BN accumulator tile, run by the four warps 2-5 of a CTA: TMEM lane
+// The epilogue of one 128 x BN accumulator tile, run by the eight warps 2-9 of a CTA: TMEM lane
 // r <-> row m0 + r, column j <-> col n0 + j.  What it needs besides the accumulator is
 // fetched while the main loop runs: the row's bias, or the first 32 columns of its ReLU mask
 // (the next 32 are fetched while the current ones are applied).
@@ -57,7 +59,11 @@ template <int BN, bool FULL>
 __device__ __forceinline__ void gemm_epilogue(const EpiArgs& ea, uint32_t tmem_base, uint32_t tmem_full_bar,
                                               volatile int* abort_flag, int warp, int lane, int m0,
                                               int n0, int worker) {
-  const int lane_group = warp & 3;
+  // eight warps, two per TMEM lane group (a warp reads the lanes of group warp % 4): the
+  // first four take the left half of the tile's 32-column blocks, the others the right half
+  const int lane_group = warp & 3, half = (warp - 2) >> 2;
+  constexpr int kBlocksPerWarp = BN / 64;
+  const int c_begin = half * kBlocksPerWarp, c_end = c_begin + kBlocksPerWarp;
   const int row = m0 + lane_group * 32 + lane;
   // the last tile of a band may reach past row Ma - 1: those rows were loaded as zeros and
   // are neither looked up nor stored
@@ -75,13 +81,13 @@ __device__ __forceinline__ void gemm_epilogue(const EpiArgs& ea, uint32_t tmem_b
     mask_row = reinterpret_cast<const uint4*>(ea.mask + (wk * ea.Ma + row) * ea.Nb + n0);
 #pragma unroll
     for (int q = 0; q < 4; ++q)
-      if (FULL || n0 + 8 * q < ea.Nb) mk[q] = mask_row[q];
+      if (FULL || n0 + c_begin * 32 + 8 * q < ea.Nb) mk[q] = mask_row[c_begin * 4 + q];
   }
   if (mbar_wait(tmem_full_bar, 0, abort_flag) && !*abort_flag) {
     tc_fence_after();
 #pragma unroll 1
-    for (int c = 0; c < BN / 32; ++c) {
-      if (mask_row && c + 1 < BN / 32) {
+    for (int c = c_begin; c < c_end; ++c) {
+      if (mask_row && c + 1 < c_end) {
 #pragma unroll
         for (int q = 0; q < 4; ++q)
           if (FULL || n0 + (c + 1) * 32 + 8 * q < ea.Nb) mk_next[q] = mask_row[(c + 1) * 4 + q];
