@@ -144,6 +144,8 @@ CSRC = os.path.join(ROOT, "paper_2002_09539_b200", "csrc")
 NCU_TRAFFIC = {
     # profiles/wgrad_update_fused_c3_mlp.txt
     ("c3", 1, "wgrad_update"): (1179.9e6, 1294.8e6, "tc_wgrad.cu", "3aed0e701941734c2348052d213ea589fb019b40"),
+    # profiles/wgrad_update_fused_c4_mlp.txt
+    ("c4", 1, "wgrad_update"): (1787.0e6, 1897.0e6, "tc_wgrad.cu", "3aed0e701941734c2348052d213ea589fb019b40"),
 }
 
 
