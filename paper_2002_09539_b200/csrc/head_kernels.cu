@@ -4,6 +4,7 @@
 // and the layer's own weight and bias gradients.  All reductions have a fixed
 // order; nothing uses floating-point atomics.
 #include "olsgd_internal.h"
+#include "philox.cuh"
 #include "update_math.cuh"
 
 namespace olsgd {
@@ -28,7 +29,19 @@ __device__ __forceinline__ float load_in<__nv_bfloat16>(const __nv_bfloat16* p) 
   return __bfloat162float(*p);
 }
 
-// Row b of worker i of the layer's input, and its label, with or without the fused gather.
+// With the fused gather: which row of worker i's partition batch slot b holds, read from the
+// index buffer or (forward kernel, a.draw) drawn on the spot by the with-replacement rule.
+__device__ __forceinline__ int32_t head_slot_row(const HeadArgs& a, int i, int b) {
+  if (a.draw) {
+    const uint32_t k = (uint32_t)(a.rule.k_base + (a.rule.k_ptr ? (uint64_t)*a.rule.k_ptr : 0ull));
+    return minibatch_index(a.rule.key0, a.rule.key1, k, (uint32_t)i + a.rule.worker_offset, b,
+                           (uint32_t)a.n_rows);
+  }
+  return a.row_idx[(int64_t)i * a.batch + b];
+}
+
+// Row b of worker i of the layer's input, with or without the fused gather (weight-gradient
+// kernels: the rows of the batch slots are in the index buffer by then).
 template <typename InT>
 __device__ __forceinline__ const InT* head_row(const HeadArgs& a, int i, int b) {
   if (sizeof(InT) == 4) {
@@ -38,8 +51,30 @@ __device__ __forceinline__ const InT* head_row(const HeadArgs& a, int i, int b) 
   }
   return reinterpret_cast<const InT*>(a.in16) + ((int64_t)i * a.batch + b) * a.K;
 }
-__device__ __forceinline__ int head_label(const HeadArgs& a, int i, int b) {
-  if (a.row_idx) return a.y_all[(int64_t)i * a.n_rows + a.row_idx[(int64_t)i * a.batch + b]];
+// Forward kernels with the fused gather: thread r < R looks up (or draws, and leaves in idx_out
+// for the weight-gradient kernel) the row of batch slot b0 + r once, for the whole block.
+template <int R>
+__device__ __forceinline__ void head_block_rows(const HeadArgs& a, int i, int b0, int rows,
+                                                int32_t* slot_row) {
+  if (!a.row_idx) return;
+  if ((int)threadIdx.x < R) {
+    const int r = threadIdx.x;
+    const int32_t row = head_slot_row(a, i, b0 + (r < rows ? r : 0));
+    slot_row[r] = row;
+    if (a.draw && r < rows) a.idx_out[(int64_t)i * a.batch + b0 + r] = row;
+  }
+  __syncthreads();
+}
+template <typename InT>
+__device__ __forceinline__ const InT* head_row_of(const HeadArgs& a, int i, int b, int32_t slot_row) {
+  if (sizeof(InT) == 4) {
+    const int64_t row = a.row_idx ? (int64_t)i * a.n_rows + slot_row : (int64_t)i * a.batch + b;
+    return reinterpret_cast<const InT*>(a.in32) + row * a.K;
+  }
+  return reinterpret_cast<const InT*>(a.in16) + ((int64_t)i * a.batch + b) * a.K;
+}
+__device__ __forceinline__ int head_label_of(const HeadArgs& a, int i, int b, int32_t slot_row) {
+  if (a.row_idx) return a.y_all[(int64_t)i * a.n_rows + slot_row];
   return a.yb[(int64_t)i * a.batch + b];
 }
 
@@ -77,9 +112,11 @@ head_forward_kernel(HeadArgs a) {
   const float* W = a.x + (int64_t)i * a.ld + a.w_off;
   const float* bias = a.x + (int64_t)i * a.ld + a.b_off;
   const int rows = min(R, B - b0);
+  __shared__ int32_t slot_row[R];
+  head_block_rows<R>(a, i, b0, rows, slot_row);
   const InT* rowp[R];
 #pragma unroll
-  for (int r = 0; r < R; ++r) rowp[r] = head_row<InT>(a, i, b0 + (r < rows ? r : 0));
+  for (int r = 0; r < R; ++r) rowp[r] = head_row_of<InT>(a, i, b0 + (r < rows ? r : 0), slot_row[r]);
 
   float acc[R][CMAX];
 #pragma unroll
@@ -129,7 +166,7 @@ head_forward_kernel(HeadArgs a) {
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     const float e = (lane < C) ? expf(logit - mx) : 0.f;
     const float lse = mx + logf(warp_sum(e));
-    const int label = live ? head_label(a, i, b) : 0;
+    const int label = live ? head_label_of(a, i, b, slot_row[r]) : 0;
     const float picked = __shfl_sync(0xffffffffu, logit, label);
     float dl = 0.f;
     if (lane < C) dl = (expf(logit - lse) - (lane == label ? 1.f : 0.f)) / (float)B;
@@ -208,9 +245,11 @@ head_forward_vec_kernel(HeadArgs a) {
   const float* W = a.x + (int64_t)i * a.ld + a.w_off;
   const float* bias = a.x + (int64_t)i * a.ld + a.b_off;
   const int rows = min(R, B - b0);
+  __shared__ int32_t slot_row[R];
+  head_block_rows<R>(a, i, b0, rows, slot_row);
   const InT* rowp[R];
 #pragma unroll
-  for (int r = 0; r < R; ++r) rowp[r] = head_row<InT>(a, i, b0 + (r < rows ? r : 0));
+  for (int r = 0; r < R; ++r) rowp[r] = head_row_of<InT>(a, i, b0 + (r < rows ? r : 0), slot_row[r]);
 
   // what the softmax step needs from global memory is fetched now, under the first sweep:
   // lane c's bias entry and the labels of the rows this warp will finish
@@ -220,7 +259,7 @@ head_forward_vec_kernel(HeadArgs a) {
 #pragma unroll
   for (int j = 0; j < kRowsPerWarp; ++j) {
     const int r = warp + j * (kHeadThreads / 32);
-    label_of[j] = (r < rows) ? head_label(a, i, b0 + r) : 0;
+    label_of[j] = (r < rows) ? head_label_of(a, i, b0 + r, slot_row[r]) : 0;
   }
 
   float acc[R][CMAX];

@@ -211,7 +211,7 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
       OLSGD_TRY(cudaStreamWaitEvent(s, io.wait_before_update, 0));
     Scope sc(hook, OLSGD_KC_FORWARD, s);
     return launch_linreg(X, static_cast<const float*>(data.y), io.idx, io.x, io.g, loss, m, B, n,
-                         spec.dims[0], io.ld, io.upd.enabled ? &io.upd : nullptr, s);
+                         spec.dims[0], io.ld, io.upd.enabled ? &io.upd : nullptr, io.rule, s);
   }
 
   const int L = n_layers(spec);
@@ -296,8 +296,16 @@ cudaError_t model_forward_backward(const olsgd_model_spec& spec, const olsgd_hpa
   ha.C = C;
   ha.round_w_bf16 = bf;
   {
+    // with the fused gather and the with-replacement rule the forward kernel draws the rows
+    // of the minibatch itself and leaves them in io.idx for the weight-gradient kernel
+    HeadArgs fwd = ha;
+    if (fused_gather && io.rule) {
+      fwd.draw = 1;
+      fwd.rule = *io.rule;
+      fwd.idx_out = io.idx;
+    }
     Scope sc(hook, OLSGD_KC_LOSS, s);
-    OLSGD_TRY(launch_head_forward(ha, s));
+    OLSGD_TRY(launch_head_forward(fwd, s));
   }
 
   // From here on kernels may write x_{k+1} and, on sync steps, read the anchor: the anchor

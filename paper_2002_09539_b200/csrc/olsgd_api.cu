@@ -716,18 +716,18 @@ olsgd_status olsgd_local_step(olsgd_ctx* c, float* loss_device) {
   // S1: minibatch indices xi_k^(i).  Where the minibatch is staged by the gather kernel and
   // the rule is the with-replacement one, that kernel draws them itself.
   const bool staged = c->spec.kind == OLSGD_MLP && c->spec.gemm_bf16 != 0;
+  auto rule_for = [&](int64_t k) {
+    IndexRule rule;
+    rule.key0 = (uint32_t)(c->hp.seed & 0xFFFFFFFFu);
+    rule.key1 = (uint32_t)(c->hp.seed >> 32);
+    // while a graph is being captured: the offset inside the block, added on the device to
+    // the block's first iteration
+    rule.k_base = (uint64_t)(c->capturing ? k - c->capture_k0 : k);
+    rule.k_ptr = c->capturing ? reinterpret_cast<const long long*>(c->dev_k) : nullptr;
+    rule.worker_offset = (uint32_t)c->hp.worker_offset;
+    return rule;
+  };
   if (staged && c->hp.sampling == 0 && gather_draws_indices(c->hp.batch, c->spec.dims[0])) {
-    auto rule_for = [&](int64_t k) {
-      IndexRule rule;
-      rule.key0 = (uint32_t)(c->hp.seed & 0xFFFFFFFFu);
-      rule.key1 = (uint32_t)(c->hp.seed >> 32);
-      // while a graph is being captured: the offset inside the block, added on the device to
-      // the block's first iteration
-      rule.k_base = (uint64_t)(c->capturing ? k - c->capture_k0 : k);
-      rule.k_ptr = c->capturing ? reinterpret_cast<const long long*>(c->dev_k) : nullptr;
-      rule.worker_offset = (uint32_t)c->hp.worker_offset;
-      return rule;
-    };
     // Were this iteration's rows staged beside the previous one?
     bool have = c->pre_k == c->k;
     if (c->pre_pending) {
@@ -758,6 +758,12 @@ olsgd_status olsgd_local_step(olsgd_ctx* c, float* loss_device) {
       c->pre_k = k_now + 1;
     }
     return OLSGD_OK;
+  }
+  if (!staged && c->hp.sampling == 0) {
+    // linear and softmax regression read their rows straight from the data set: their first
+    // kernel draws the indices of the with-replacement rule itself
+    const IndexRule rule = rule_for(c->k);
+    return step_body(c, c->data, c->idx, loss_device, -1, nullptr, &rule);
   }
   {
     Launch l(c, OLSGD_KC_INDEX, c->main);

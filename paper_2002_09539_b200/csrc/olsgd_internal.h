@@ -181,10 +181,13 @@ cudaError_t launch_cast_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cu
 // Linear regression, one block per worker: r = X_b w - y_b, loss = sum r^2 / 2B,
 // g = X_b^T r / B, reading the batch rows straight from the worker's partition.  With upd
 // non-null and enabled the gradient is not stored: the kernel applies Eq. 3 / Eq. 4 itself.
+// With rule non-null the kernel draws the minibatch indices itself (S1 inside the model kernel,
+// the with-replacement rule) and writes them to idx; otherwise it reads them from idx.
 struct FusedUpdateArgs;
-cudaError_t launch_linreg(const float* X, const float* y, const int32_t* idx, const float* x,
+struct IndexRule;
+cudaError_t launch_linreg(const float* X, const float* y, int32_t* idx, const float* x,
                           float* g, float* loss, int m, int batch, int64_t n, int d, int64_t ld,
-                          const FusedUpdateArgs* upd, cudaStream_t s);
+                          const FusedUpdateArgs* upd, const IndexRule* rule, cudaStream_t s);
 
 // S2: copy the minibatch rows of every worker into contiguous staging.
 //   xb32  float [m][B][d]   (or null)
@@ -234,6 +237,12 @@ struct HeadArgs {
   const int32_t* row_idx;
   int64_t n_rows;
   const int32_t* y_all;
+  // Forward kernel only, with the fused gather: draw != 0 makes the kernel compute the rows
+  // of its batch slots by the with-replacement index rule (S1 inside the kernel) instead of
+  // reading row_idx, and write them to idx_out for the weight-gradient kernel that follows.
+  int draw;
+  IndexRule rule;
+  int32_t* idx_out;
 };
 cudaError_t launch_head_forward(const HeadArgs& a, cudaStream_t s);
 

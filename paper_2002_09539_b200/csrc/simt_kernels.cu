@@ -182,17 +182,32 @@ transpose_bf16_kernel(const __nv_bfloat16* __restrict__ xb16, const int32_t* __r
 
 __global__ void __launch_bounds__(128)
 linreg_kernel(const float* __restrict__ X, const float* __restrict__ y,
-              const int32_t* __restrict__ idx, const float* __restrict__ x, float* __restrict__ g,
+              int32_t* __restrict__ idx, const float* __restrict__ x, float* __restrict__ g,
               float* __restrict__ loss, int batch, int64_t n, int d, int64_t ld,
-              FusedUpdateArgs up) {
+              FusedUpdateArgs up, bool draw, IndexRule rule) {
   launch_gate();
-  extern __shared__ float sm[];  // residuals [batch]
+  extern __shared__ float sm[];  // residuals [batch], then the batch's row numbers [batch]
+  int32_t* rows = reinterpret_cast<int32_t*>(sm + batch);
   const int i = blockIdx.x;
   const float* w = x + (int64_t)i * ld;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32, nwarp = blockDim.x / 32;
   const float* Xi = X + (int64_t)i * n * d;
+  // S1: the rows of this worker's minibatch, drawn here by the with-replacement rule (and left
+  // in idx for whoever wants to see them) or taken from idx
+  for (int b = threadIdx.x; b < batch; b += blockDim.x) {
+    int32_t r;
+    if (draw) {
+      const uint32_t k = (uint32_t)(rule.k_base + (rule.k_ptr ? (uint64_t)*rule.k_ptr : 0ull));
+      r = minibatch_index(rule.key0, rule.key1, k, (uint32_t)i + rule.worker_offset, b, (uint32_t)n);
+      idx[(int64_t)i * batch + b] = r;
+    } else {
+      r = idx[(int64_t)i * batch + b];
+    }
+    rows[b] = r;
+  }
+  __syncthreads();
   for (int b = warp; b < batch; b += nwarp) {
-    const int32_t r = idx[(int64_t)i * batch + b];
+    const int32_t r = rows[b];
     const float* row = Xi + (int64_t)r * d;
     float acc = 0.f;
     for (int j = lane; j < d; j += 32) acc = fmaf(row[j], w[j], acc);
@@ -203,10 +218,7 @@ linreg_kernel(const float* __restrict__ X, const float* __restrict__ y,
   const float inv_b = 1.0f / (float)batch;
   for (int j = threadIdx.x; j < d; j += blockDim.x) {
     float acc = 0.f;
-    for (int b = 0; b < batch; ++b) {
-      const int32_t r = idx[(int64_t)i * batch + b];
-      acc = fmaf(sm[b], Xi[(int64_t)r * d + j], acc);
-    }
+    for (int b = 0; b < batch; ++b) acc = fmaf(sm[b], Xi[(int64_t)rows[b] * d + j], acc);
     const float gj = acc * inv_b;
     if (up.enabled) {
       // Eq. 3 / Eq. 4 for entry j of worker i, with the arithmetic of the update kernel
@@ -319,13 +331,14 @@ cudaError_t launch_transpose_bf16(const __nv_bfloat16* xb16, const int32_t* y, _
   return launch_chained(transpose_bf16_kernel, grid, dim3(256), 0, s, xb16, y, xb16t, yb, batch, d);
 }
 
-cudaError_t launch_linreg(const float* X, const float* y, const int32_t* idx, const float* x,
+cudaError_t launch_linreg(const float* X, const float* y, int32_t* idx, const float* x,
                           float* g, float* loss, int m, int batch, int64_t n, int d, int64_t ld,
-                          const FusedUpdateArgs* upd, cudaStream_t s) {
+                          const FusedUpdateArgs* upd, const IndexRule* rule, cudaStream_t s) {
   FusedUpdateArgs up{};
   if (upd) up = *upd;
-  return launch_chained(linreg_kernel, dim3(m), dim3(128), (size_t)batch * sizeof(float), s, X, y, idx,
-                        x, g, loss, batch, n, d, ld, up);
+  return launch_chained(linreg_kernel, dim3(m), dim3(128),
+                        (size_t)batch * (sizeof(float) + sizeof(int32_t)), s, X, y, idx, x, g, loss,
+                        batch, n, d, ld, up, rule != nullptr, rule ? *rule : IndexRule{});
 }
 
 cudaError_t launch_bias_grad(const __nv_bfloat16* dat, float* g, int64_t ld, int64_t b_off, int m,
