@@ -69,6 +69,11 @@ struct olsgd_ctx {
   int64_t pre_k = -1;
   cudaEvent_t pullback_done = nullptr, reduce_done = nullptr;
   cudaEvent_t h2d_done[2] = {nullptr, nullptr}, stage_free[2] = {nullptr, nullptr};
+  // host-fed steps hand their losses to the host on stream `pre`, off the main stream (a copy
+  // between two steps' kernels would hold up the next step's first launch): loss_read marks
+  // the end of that copy, which the next kernel that writes the loss buffer must wait for
+  cudaEvent_t loss_read = nullptr;
+  bool loss_read_pending = false;
   int host_slot = 0;
   bool reduce_pending = false;  // an anchor refresh was launched and not yet waited for
   int reduce_reads = -1;        // which x buffer that refresh reads
@@ -208,6 +213,7 @@ void free_host_side(olsgd_ctx* c) {
   if (c->aux) cudaStreamDestroy(c->aux);
   if (c->pre_begin) cudaEventDestroy(c->pre_begin);
   if (c->pre_done) cudaEventDestroy(c->pre_done);
+  if (c->loss_read) cudaEventDestroy(c->loss_read);
   for (int b = 0; b < 2; ++b)
     if (c->set_free[b]) cudaEventDestroy(c->set_free[b]);
   if (c->pre) cudaStreamDestroy(c->pre);
@@ -449,6 +455,12 @@ olsgd_status step_body(olsgd_ctx* c, const olsgd_data& data, int32_t* idx,
                        float* loss_device, int stage_slot, const __nv_bfloat16* xb16_in = nullptr,
                        const IndexRule* rule = nullptr, bool batch_staged = false,
                        cudaEvent_t mid_event = nullptr) {
+  if (c->loss_read_pending && !c->capturing) {
+    // the losses of the last host-fed step are still being copied out of the buffer this
+    // step's kernels write again
+    OLSGD_CUDA(c, cudaStreamWaitEvent(c->main, c->loss_read, 0));
+    c->loss_read_pending = false;
+  }
   StepIO io;
   io.mid_event = mid_event;
   io.xb16_in = xb16_in;
@@ -662,6 +674,7 @@ olsgd_status olsgd_init(olsgd_ctx** out, const olsgd_model_spec* spec, const ols
     }
     OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->pre_begin, cudaEventDisableTiming));
     OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->pre_done, cudaEventDisableTiming));
+    OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->loss_read, cudaEventDisableTiming));
     for (int b = 0; b < 2; ++b)
       OLSGD_INIT_CUDA(cudaEventCreateWithFlags(&c->set_free[b], cudaEventDisableTiming));
     for (int b = 0; b < 2; ++b) {
@@ -833,9 +846,14 @@ static olsgd_status local_step_host_impl(olsgd_ctx* c, const void* Xb_host, cons
       elem == 2 ? reinterpret_cast<const __nv_bfloat16*>(c->stage_x[slot]) : nullptr;
   olsgd_status st = step_body(c, staged, c->ident, nullptr, slot, direct, nullptr, stage_on_copy);
   if (st != OLSGD_OK) return st;
-  if (loss_host)
+  if (loss_host) {
+    // stage_free[slot] was recorded on the main stream behind the kernel that wrote the losses
+    OLSGD_CUDA(c, cudaStreamWaitEvent(c->pre, c->stage_free[slot], 0));
     OLSGD_CUDA(c, cudaMemcpyAsync(loss_host, c->mb.loss, (size_t)c->hp.m * sizeof(float),
-                                  cudaMemcpyDeviceToHost, c->main));
+                                  cudaMemcpyDeviceToHost, c->pre));
+    OLSGD_CUDA(c, cudaEventRecord(c->loss_read, c->pre));
+    c->loss_read_pending = true;
+  }
   return OLSGD_OK;
 }
 
@@ -1081,6 +1099,11 @@ olsgd_status olsgd_run(olsgd_ctx* c, int64_t n_iters, float* loss_device) {
   if (n_iters < 0) return fail(c, OLSGD_EINVAL, "n_iters must be >= 0");
   if (c->spec.kind == OLSGD_FLAT)
     return fail(c, OLSGD_ESTATE, "OLSGD_FLAT contexts take olsgd_local_step_with_grads");
+  if (c->loss_read_pending) {
+    // (a replayed graph cannot wait for an event from outside it: settle this one first)
+    OLSGD_CUDA(c, cudaStreamWaitEvent(c->main, c->loss_read, 0));
+    c->loss_read_pending = false;
+  }
   int64_t t = 0;
   auto plain = [&](int64_t count) -> olsgd_status {
     for (int64_t j = 0; j < count; ++j, ++t) {
